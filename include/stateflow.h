@@ -1,0 +1,206 @@
+/*
+ * stateflow.h - C ABI of the B200 (sm_100a) segment kernels for the chunkwise
+ * gated linear recurrence
+ *
+ *     S_t = exp(g_t) * S_{t-1} + k_t^T v_t ,      o_t = q_t S_t
+ *
+ * (paper Eq. 1 with the scalar-identity transition of Section 2.1), run over one
+ * sequence segment with an incoming boundary state S_in and an outgoing S_out
+ * (paper Eq. 4-5), and its backward, which takes dO and the downstream
+ * boundary-state gradient dS_out and returns dq, dk, dv, dg and dS_in (paper
+ * Eq. 6-7).  A "segment" is the paper's sequence chunk C_i, the scheduling unit;
+ * a "chunk" is its kernel-level chunk of T_C tokens (Section 3.1, last paragraph).
+ *
+ * Conventions for every entry point
+ *  - All data pointers are DEVICE pointers unless a comment says "host".  The
+ *    caller owns every buffer, including the workspace; the library allocates no
+ *    device memory (the one exception is documented at its declaration).
+ *  - Work is enqueued on the given stream and the call returns without
+ *    synchronising.  Outputs are valid once the stream reaches that point; all
+ *    buffers must stay alive and unmodified until then.
+ *  - Layout (row-major, strides in ELEMENTS of the tensor's type):
+ *      q, k, dq, dk : [B, T, H, d_k]       v, o, dO, dv : [B, T, H, d_v]
+ *      g, dg        : [B, T, H]  float32   (log-decay, g <= 0 expected, not checked)
+ *      states       : [B, H, d_k, d_v] float32, contiguous
+ *    A segment is a view: the pointer addresses its first token, consecutive
+ *    tokens are tok_stride_* apart, batches batch_stride_* apart, head h starts
+ *    h*d (resp. h) elements after the token base.  Passing the strides of the
+ *    full sequence lets segments be chained without copies.
+ *  - q, k, v, dO and o, dq, dk, dv have type desc->dtype; g, dg and all states
+ *    are float32.  Arithmetic accumulates in float32.
+ *  - Validation happens on the host before anything is launched.  A call that
+ *    returns an error has enqueued nothing.  The library never throws, aborts,
+ *    prints or traps the device.
+ *  - Pointers must be 16-byte aligned; for SF_BF16 the token and batch strides
+ *    must be multiples of 8 elements (16 bytes).
+ */
+#ifndef STATEFLOW_H
+#define STATEFLOW_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque here so that the header needs no CUDA include; pass a cudaStream_t. */
+typedef struct CUstream_st* sf_stream_t;
+
+typedef enum {
+    SF_OK = 0,
+    SF_ERR_INVALID_ARG = 1,   /* NULL where required, bad shape, seg_len % chunk != 0, misalignment, aliasing */
+    SF_ERR_UNSUPPORTED = 2,   /* (dtype, d_k, d_v, chunk) outside the supported set */
+    SF_ERR_WORKSPACE = 3,     /* workspace NULL or smaller than sf_workspace_bytes() */
+    SF_ERR_CUDA = 4,          /* a CUDA runtime/driver call or a launch failed (cudaGetLastError, no sync) */
+    SF_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out (see sf_device_status) */
+} sf_status_t;
+
+typedef enum { SF_BF16 = 0, SF_F32 = 1 } sf_dtype_t;
+
+/*
+ * Shape of one segment.  Supported sets:
+ *   SF_F32  : d_k, d_v in {32, 64, 128}, chunk in {16, 32, 64}          (CUDA-core kernels)
+ *   SF_BF16 : d_k = d_v = 128, chunk = 64                               (tcgen05 / TMEM / TMA kernels)
+ *             d_k, d_v in {32, 64}, chunk in {16, 32, 64}               (CUDA-core kernels)
+ * seg_len must be a positive multiple of chunk (the paper rounds boundaries to multiples of 128,
+ * Section 3.2).  chunks_per_block sets how many chunks form one block, the only granularity
+ * whose states are written to the workspace; 0 picks the default (16).  Heads are independent.
+ */
+typedef struct {
+    int32_t B, H, d_k, d_v;
+    int32_t seg_len, chunk;
+    int32_t dtype;                 /* sf_dtype_t */
+    int32_t chunks_per_block;      /* 0 = default */
+    int64_t tok_stride_qk, tok_stride_v, tok_stride_g;
+    int64_t batch_stride_qk, batch_stride_v, batch_stride_g;
+} sf_seg_desc_t;
+
+const char* sf_status_string(sf_status_t s);
+
+/* Number of blocks of the segment: ceil((seg_len / chunk) / chunks_per_block).  0 on an invalid descriptor. */
+int32_t sf_num_blocks(const sf_seg_desc_t* desc);
+
+/*
+ * Bytes of workspace a call needs (host function; 0 on an invalid descriptor).
+ *   backward == 0 : sf_segment_fwd
+ *   backward == 1 : sf_segment_bwd given the forward's workspace as fwd_saved
+ *   backward == 2 : sf_segment_bwd with fwd_saved == NULL (block states are replayed)
+ * The workspace must be 256-byte aligned.
+ */
+size_t sf_workspace_bytes(const sf_seg_desc_t* desc, int backward);
+
+/*
+ * Forward of one segment, (C_out, S_out) = Fwd(C_in, S_in) (paper Eq. 4) with C_in = (q, k, v, g),
+ * C_out = o.  Internally the three stages of paper Eq. 2: block aggregates (Pre), state scan over
+ * blocks (ST), chunk outputs (Out).
+ *   S_in  : nullable, NULL means the zero state (the paper's S_0 = 0)
+ *   S_out : required, must not alias S_in
+ *   workspace : sf_workspace_bytes(desc, 0) bytes; after the call it holds the block-entering
+ *               states, which sf_segment_bwd can reuse (fwd_saved) as long as it is left unchanged
+ */
+sf_status_t sf_segment_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v,
+                           const float* g, const float* S_in, void* o, float* S_out,
+                           void* workspace, size_t workspace_bytes, sf_stream_t stream);
+
+/*
+ * Backward of one segment, (dC_in, dS_in) = Bwd(C_in, S_in, dC_out, dS_out) (paper Eq. 6) with
+ * dC_out = dO and dC_in = (dq, dk, dv, dg).  Stages: state replay (SR, skipped when fwd_saved is
+ * given), backward block aggregates and reverse state scan (STB), output gradient (OG -> dq),
+ * preparation gradient (PG -> dk, dv), and the log-decay gradient dg assembled from both
+ * (Section 3.4, backward pass).
+ *   S_in      : the state the forward of this segment started from (nullable = zero)
+ *   dS_out    : nullable, NULL means zero
+ *   dS_in     : required, must not alias dS_out
+ *   fwd_saved : nullable; the workspace sf_segment_fwd filled for this same segment and descriptor
+ *   workspace : sf_workspace_bytes(desc, fwd_saved ? 1 : 2) bytes, distinct from fwd_saved
+ */
+sf_status_t sf_segment_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v,
+                           const float* g, const float* S_in, const void* dO, const float* dS_out,
+                           void* dq, void* dk, void* dv, float* dg, float* dS_in,
+                           const void* fwd_saved, void* workspace, size_t workspace_bytes,
+                           sf_stream_t stream);
+
+/*
+ * The ST stage alone (paper Eq. 2, second line; Eq. 5 / Eq. 7 across boundaries): the first-order
+ * linear recurrence over the n = sf_num_blocks(desc) blocks of a segment, element-wise over
+ * B*H*d_k*d_v lanes.  B, H, d_k, d_v, seg_len, chunk come from desc; chunks_per_block overrides
+ * desc->chunks_per_block when > 0.
+ *   forward (reverse == 0): X_0 = S_boundary_in; states[j] = X_j (state ENTERING block j);
+ *                           X_{j+1} = exp(log_decay[j]) X_j + U[j];  S_boundary_out = X_n
+ *   reverse (reverse != 0): X_n = S_boundary_in; states[j] = X_{j+1} (gradient LEAVING block j);
+ *                           X_j = exp(log_decay[j]) X_{j+1} + U[j];  S_boundary_out = X_0
+ *   log_decay [B,H,n] float32 block totals of g;  U, states [B,H,n,d_k,d_v] float32 (states may
+ *   alias U);  S_boundary_in nullable = zero;  S_boundary_out required, must not alias the input.
+ */
+sf_status_t sf_state_scan(const sf_seg_desc_t* desc, int32_t chunks_per_block, int32_t reverse,
+                          const float* log_decay, const float* U, const float* S_boundary_in,
+                          float* states, float* S_boundary_out, sf_stream_t stream);
+
+/*
+ * Segment-chaining driver (paper Eq. 5 and Eq. 7; the single-device part of the partial order of
+ * Eq. 8: F_{i-1} before F_i, F_i before B_i, B_{i+1} before B_i).  seg_lens is a HOST array of
+ * n_seg segment lengths (each a positive multiple of desc->chunk; desc->seg_len is ignored);
+ * q, k, v, g, o, ... address token 0 of the whole sequence of T = sum(seg_lens) tokens.
+ *
+ * sf_chain_fwd runs Fwd on segments 0..n_seg-1 with S_{i+1}^in = S_i^out.
+ *   S_init   : nullable = zero
+ *   S_bounds : [n_seg+1][B,H,d_k,d_v] float32; on return S_bounds[i] = S_i^in and
+ *              S_bounds[n_seg] = the final state.  Kept by the caller for sf_chain_bwd.
+ *   workspace: sf_chain_workspace_bytes(..., 0) bytes; holds every segment's saved block states.
+ * sf_chain_bwd runs Bwd on segments n_seg-1..0 with dS_i^out = dS_{i+1}^in.
+ *   dS_final : nullable = zero;   dS_init : required, receives dS_0^in
+ *   fwd_workspace : the workspace sf_chain_fwd filled, or NULL to replay block states
+ *   workspace: sf_chain_workspace_bytes(..., fwd_workspace ? 1 : 2) bytes
+ * overlap != 0 lets the driver run state-independent stages of neighbouring segments on internal
+ * side streams concurrently with the state scans (the split-and-overlap idea of Section 3.4,
+ * Eq. 17-18); the result is bit-identical to overlap == 0.  The side streams are joined back
+ * into `stream` before the call returns, so later work on `stream` sees all outputs.
+ */
+size_t sf_chain_workspace_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg,
+                                int backward);
+
+sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg,
+                         const void* q, const void* k, const void* v, const float* g,
+                         const float* S_init, void* o, float* S_bounds,
+                         void* workspace, size_t workspace_bytes, int32_t overlap, sf_stream_t stream);
+
+sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg,
+                         const void* q, const void* k, const void* v, const float* g,
+                         const float* S_bounds, const void* dO, const float* dS_final,
+                         void* dq, void* dk, void* dv, float* dg, float* dS_init,
+                         const void* fwd_workspace, void* workspace, size_t workspace_bytes,
+                         int32_t overlap, sf_stream_t stream);
+
+/*
+ * Host-memory convenience wrappers around the chain driver (the "end-to-end" path): every data
+ * pointer is a HOST pointer (pinned memory recommended).  The call copies the inputs to the device
+ * buffers in `dev` (caller-allocated device scratch, sf_e2e_device_bytes() bytes, 256-byte
+ * aligned), runs sf_chain_fwd + sf_chain_bwd and copies o, dq, dk, dv, dg, the final state and
+ * dS_init back, all on `stream`, then synchronises the stream.  Section 3.1, Eq. 4-7.
+ */
+size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg);
+
+sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg,
+                                  const void* q, const void* k, const void* v, const float* g,
+                                  const float* S_init, const void* dO, const float* dS_final,
+                                  void* o, float* S_final, void* dq, void* dk, void* dv, float* dg,
+                                  float* dS_init, void* dev, size_t dev_bytes, sf_stream_t stream);
+
+/*
+ * Device-side status word of the most recent kernels launched by this library on the current
+ * device (host function, synchronises nothing: it reads a mapped host word).  0 means no bounded
+ * wait has run out since sf_device_status_clear().  Kernels never spin without a limit; when a
+ * limit is hit they record a code here, stop waiting and return normally, leaving their outputs
+ * undefined.  No counterpart in the paper.
+ */
+int32_t sf_device_status(void);
+void sf_device_status_clear(void);
+
+/* Number of kernels this library has launched in this process (host counter). No paper counterpart. */
+int64_t sf_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STATEFLOW_H */

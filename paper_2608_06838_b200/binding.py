@@ -1,0 +1,214 @@
+"""Thin ctypes binding of libstateflow.so: argument marshalling only.
+
+Every function has the name and meaning of the C entry point in include/stateflow.h and takes
+torch CUDA tensors for the device pointers.  PyTorch provides device memory and streams; all
+arithmetic runs in the library's kernels.  There is no fallback: if the library is missing or a
+call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstateflow.so")
+_lib = None
+
+SF_BF16, SF_F32 = 0, 1
+STATUS = {0: "SF_OK", 1: "SF_ERR_INVALID_ARG", 2: "SF_ERR_UNSUPPORTED", 3: "SF_ERR_WORKSPACE", 4: "SF_ERR_CUDA",
+          5: "SF_ERR_TIMEOUT"}
+
+
+class SfError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s (%s)" % (where, STATUS.get(code, code), status_string(code)))
+
+
+class SegDesc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32),
+                ("seg_len", ctypes.c_int32), ("chunk", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("chunks_per_block", ctypes.c_int32),
+                ("tok_stride_qk", ctypes.c_int64), ("tok_stride_v", ctypes.c_int64), ("tok_stride_g", ctypes.c_int64),
+                ("batch_stride_qk", ctypes.c_int64), ("batch_stride_v", ctypes.c_int64), ("batch_stride_g", ctypes.c_int64)]
+
+
+def load() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built (there is no CPU path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libstateflow.so is missing: run `python -m paper_2608_06838_b200.build` "
+                               "(or __graft_entry__.build()); this package has no CPU fallback")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+        dp = ctypes.POINTER(SegDesc)
+        ip = ctypes.POINTER(ctypes.c_int32)
+        lib.sf_status_string.restype = ctypes.c_char_p
+        lib.sf_status_string.argtypes = [ctypes.c_int]
+        lib.sf_num_blocks.restype = i32
+        lib.sf_num_blocks.argtypes = [dp]
+        lib.sf_workspace_bytes.restype = sz
+        lib.sf_workspace_bytes.argtypes = [dp, ctypes.c_int]
+        lib.sf_segment_fwd.restype = ctypes.c_int
+        lib.sf_segment_fwd.argtypes = [dp] + [vp] * 7 + [vp, sz, vp]
+        lib.sf_segment_bwd.restype = ctypes.c_int
+        lib.sf_segment_bwd.argtypes = [dp] + [vp] * 12 + [vp, vp, sz, vp]
+        lib.sf_state_scan.restype = ctypes.c_int
+        lib.sf_state_scan.argtypes = [dp, i32, i32] + [vp] * 5 + [vp]
+        lib.sf_chain_workspace_bytes.restype = sz
+        lib.sf_chain_workspace_bytes.argtypes = [dp, ip, i32, ctypes.c_int]
+        lib.sf_chain_fwd.restype = ctypes.c_int
+        lib.sf_chain_fwd.argtypes = [dp, ip, i32] + [vp] * 7 + [vp, sz, i32, vp]
+        lib.sf_chain_bwd.restype = ctypes.c_int
+        lib.sf_chain_bwd.argtypes = [dp, ip, i32] + [vp] * 12 + [vp, vp, sz, i32, vp]
+        lib.sf_e2e_device_bytes.restype = sz
+        lib.sf_e2e_device_bytes.argtypes = [dp, ip, i32]
+        lib.sf_chain_fwd_bwd_host.restype = ctypes.c_int
+        lib.sf_chain_fwd_bwd_host.argtypes = [dp, ip, i32] + [vp] * 14 + [vp, sz, vp]
+        lib.sf_device_status.restype = i32
+        lib.sf_device_status_clear.restype = None
+        lib.sf_launch_count.restype = ctypes.c_int64
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load().sf_status_string(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise SfError(code, where)
+
+
+def make_desc(q: torch.Tensor, v: torch.Tensor, g: torch.Tensor, chunk: int, chunks_per_block: int = 0,
+              seg_len: Optional[int] = None) -> SegDesc:
+    """Descriptor for q [B,T,H,d_k], v [B,T,H,d_v], g [B,T,H] (views along T are fine)."""
+    B, T, H, dk = q.shape
+    dv = v.shape[-1]
+    if q.stride(3) != 1 or v.stride(3) != 1 or q.stride(2) != dk or v.stride(2) != dv or g.stride(2) != 1:
+        raise ValueError("heads and features must be densely packed inside a token")
+    dt = {torch.bfloat16: SF_BF16, torch.float32: SF_F32}[q.dtype]
+    return SegDesc(B, H, dk, dv, T if seg_len is None else seg_len, chunk, dt, chunks_per_block,
+                   q.stride(1), v.stride(1), g.stride(1), q.stride(0), v.stride(0), g.stride(0))
+
+
+def sf_num_blocks(desc: SegDesc) -> int:
+    return int(load().sf_num_blocks(ctypes.byref(desc)))
+
+
+def sf_workspace_bytes(desc: SegDesc, backward: int) -> int:
+    return int(load().sf_workspace_bytes(ctypes.byref(desc), backward))
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+def sf_segment_fwd(desc: SegDesc, q, k, v, g, S_in, o, S_out, workspace: torch.Tensor, stream=None):
+    _check(load().sf_segment_fwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(S_in), _ptr(o), _ptr(S_out),
+                                 _ptr(workspace), workspace.numel(), _stream(stream)), "sf_segment_fwd")
+
+
+def sf_segment_bwd(desc: SegDesc, q, k, v, g, S_in, dO, dS_out, dq, dk, dv, dg, dS_in, fwd_saved, workspace, stream=None):
+    _check(load().sf_segment_bwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(S_in), _ptr(dO), _ptr(dS_out),
+                                 _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dg), _ptr(dS_in), _ptr(fwd_saved), _ptr(workspace),
+                                 workspace.numel(), _stream(stream)), "sf_segment_bwd")
+
+
+def sf_state_scan(desc: SegDesc, chunks_per_block: int, reverse: bool, log_decay, U, S_boundary_in, states, S_boundary_out,
+                  stream=None):
+    _check(load().sf_state_scan(ctypes.byref(desc), chunks_per_block, int(reverse), _ptr(log_decay), _ptr(U),
+                                _ptr(S_boundary_in), _ptr(states), _ptr(S_boundary_out), _stream(stream)), "sf_state_scan")
+
+
+def _seg_array(seg_lens: Sequence[int]):
+    return (ctypes.c_int32 * len(seg_lens))(*[int(s) for s in seg_lens])
+
+
+def sf_chain_workspace_bytes(desc: SegDesc, seg_lens: Sequence[int], backward: int) -> int:
+    return int(load().sf_chain_workspace_bytes(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens), backward))
+
+
+def sf_chain_fwd(desc: SegDesc, seg_lens, q, k, v, g, S_init, o, S_bounds, workspace, overlap=True, stream=None):
+    _check(load().sf_chain_fwd(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens), _ptr(q), _ptr(k), _ptr(v), _ptr(g),
+                               _ptr(S_init), _ptr(o), _ptr(S_bounds), _ptr(workspace), workspace.numel(), int(overlap),
+                               _stream(stream)), "sf_chain_fwd")
+
+
+def sf_chain_bwd(desc: SegDesc, seg_lens, q, k, v, g, S_bounds, dO, dS_final, dq, dk, dv, dg, dS_init, fwd_workspace,
+                 workspace, overlap=True, stream=None):
+    _check(load().sf_chain_bwd(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens), _ptr(q), _ptr(k), _ptr(v), _ptr(g),
+                               _ptr(S_bounds), _ptr(dO), _ptr(dS_final), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dg),
+                               _ptr(dS_init), _ptr(fwd_workspace), _ptr(workspace), workspace.numel(), int(overlap),
+                               _stream(stream)), "sf_chain_bwd")
+
+
+def sf_e2e_device_bytes(desc: SegDesc, seg_lens) -> int:
+    return int(load().sf_e2e_device_bytes(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens)))
+
+
+def sf_chain_fwd_bwd_host(desc: SegDesc, seg_lens, q, k, v, g, S_init, dO, dS_final, o, S_final, dq, dk, dv, dg, dS_init,
+                          dev: torch.Tensor, stream=None):
+    """All data tensors are HOST tensors (pinned recommended); dev is device scratch."""
+    _check(load().sf_chain_fwd_bwd_host(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens), _ptr(q), _ptr(k), _ptr(v),
+                                        _ptr(g), _ptr(S_init), _ptr(dO), _ptr(dS_final), _ptr(o), _ptr(S_final), _ptr(dq),
+                                        _ptr(dk), _ptr(dv), _ptr(dg), _ptr(dS_init), _ptr(dev), dev.numel(),
+                                        _stream(stream)), "sf_chain_fwd_bwd_host")
+
+
+def sf_device_status() -> int:
+    return int(load().sf_device_status())
+
+
+def sf_device_status_clear() -> None:
+    load().sf_device_status_clear()
+
+
+def sf_launch_count() -> int:
+    return int(load().sf_launch_count())
+
+
+# ---- conveniences built only from the calls above (allocation + one call each) --------------------
+
+class ChainRun:
+    """Device buffers for one chained forward+backward over a whole sequence."""
+
+    def __init__(self, q, k, v, g, dO, seg_lens: List[int], chunk: int, chunks_per_block: int = 0, save_states: bool = True):
+        self.seg_lens = [int(s) for s in seg_lens]
+        self.desc = make_desc(q, v, g, chunk, chunks_per_block, seg_len=self.seg_lens[0])
+        dev = q.device
+        B, T, H, dk = q.shape
+        dv = v.shape[-1]
+        self.q, self.k, self.v, self.g, self.dO = q, k, v, g, dO
+        self.o = torch.empty_like(v)
+        self.dq, self.dk, self.dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+        self.dg = torch.empty_like(g)
+        self.S_bounds = torch.empty(len(self.seg_lens) + 1, B, H, dk, dv, dtype=torch.float32, device=dev)
+        self.dS_init = torch.empty(B, H, dk, dv, dtype=torch.float32, device=dev)
+        self.save_states = save_states
+        self.ws_f = _workspace(sf_chain_workspace_bytes(self.desc, self.seg_lens, 0), dev)
+        state_bytes = (B * H * dk * dv * 4 + 255) // 256 * 256
+        self.ws_b = _workspace(sf_chain_workspace_bytes(self.desc, self.seg_lens, 1 if save_states else 2) + 2 * state_bytes, dev)
+
+    def forward(self, S_init=None, overlap=True, stream=None):
+        sf_chain_fwd(self.desc, self.seg_lens, self.q, self.k, self.v, self.g, S_init, self.o, self.S_bounds, self.ws_f,
+                     overlap, stream)
+
+    def backward(self, dS_final=None, overlap=True, stream=None):
+        sf_chain_bwd(self.desc, self.seg_lens, self.q, self.k, self.v, self.g, self.S_bounds, self.dO, dS_final, self.dq,
+                     self.dk, self.dv, self.dg, self.dS_init, self.ws_f if self.save_states else None, self.ws_b, overlap,
+                     stream)

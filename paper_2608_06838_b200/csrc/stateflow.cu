@@ -1,0 +1,644 @@
+// Host side of the C ABI declared in include/stateflow.h: validation, workspace layout, kernel
+// dispatch, the segment-chaining driver and the host-memory end-to-end wrapper.
+#include "../../include/stateflow.h"
+
+#include <atomic>
+#include <mutex>
+
+#include "sf_common.cuh"
+#include "sf_scan.cuh"
+#include "sf_simt.cuh"
+#include "sf_tc.cuh"
+
+namespace {
+
+using sf::SegParams;
+
+std::atomic<long long> g_launches{0};
+
+constexpr int kDefaultChunksPerBlock = 16;
+constexpr size_t kAlign = 256;
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+enum class Path { Invalid, Unsupported, Simt, Tc };
+
+Path classify(const sf_seg_desc_t* d) {
+    if (!d) return Path::Invalid;
+    if (d->B <= 0 || d->H <= 0 || d->d_k <= 0 || d->d_v <= 0 || d->chunk <= 0 || d->seg_len <= 0) return Path::Invalid;
+    if (d->seg_len % d->chunk != 0) return Path::Invalid;
+    if (d->chunks_per_block < 0 || d->chunks_per_block > sf::simt::MAXR) return Path::Invalid;
+    if (d->dtype != SF_BF16 && d->dtype != SF_F32) return Path::Invalid;
+    if (d->tok_stride_qk < (long long)d->H * d->d_k || d->tok_stride_v < (long long)d->H * d->d_v || d->tok_stride_g < d->H)
+        return Path::Invalid;
+    if (d->B > 1 && (d->batch_stride_qk <= 0 || d->batch_stride_v <= 0 || d->batch_stride_g <= 0)) return Path::Invalid;
+    if ((long long)d->B * d->H > 65535LL * 65535LL) return Path::Invalid;
+    if (d->H > 65535 || d->B > 65535) return Path::Invalid;
+    const bool c_ok = d->chunk == 16 || d->chunk == 32 || d->chunk == 64;
+    auto d_ok = [](int x) { return x == 32 || x == 64 || x == 128; };
+    if (!c_ok || !d_ok(d->d_k) || !d_ok(d->d_v)) return Path::Unsupported;
+    if (d->dtype == SF_BF16) {
+        if (d->tok_stride_qk % 8 || d->tok_stride_v % 8 || d->batch_stride_qk % 8 || d->batch_stride_v % 8) return Path::Invalid;
+        if (d->d_k == 128 && d->d_v == 128) return d->chunk == 64 ? Path::Tc : Path::Unsupported;
+        if (d->d_k == 128 || d->d_v == 128) return Path::Unsupported;
+        return d->d_k == d->d_v || (d->d_k == 32 && d->d_v == 64) ? Path::Simt : Path::Unsupported;
+    }
+    if (d->tok_stride_qk % 4 || d->tok_stride_v % 4 || d->batch_stride_qk % 4 || d->batch_stride_v % 4) return Path::Invalid;
+    return d->d_k == d->d_v || (d->d_k == 32 && d->d_v == 64) ? Path::Simt : Path::Unsupported;
+}
+
+SegParams make_params(const sf_seg_desc_t* d, int cpb_override = 0) {
+    SegParams p;
+    p.B = d->B; p.H = d->H; p.L = d->seg_len; p.C = d->chunk;
+    p.NC = d->seg_len / d->chunk;
+    int r = cpb_override > 0 ? cpb_override : d->chunks_per_block;
+    p.R = r > 0 ? r : kDefaultChunksPerBlock;
+    p.NB = (p.NC + p.R - 1) / p.R;
+    p.tqk = d->tok_stride_qk; p.tv = d->tok_stride_v; p.tg = d->tok_stride_g;
+    p.bqk = d->batch_stride_qk; p.bv = d->batch_stride_v; p.bg = d->batch_stride_g;
+    return p;
+}
+
+// ---- workspace layout -------------------------------------------------------------------------
+// forward           : [beta B*H*NB f32][UH B*H*NB*dk*dv f32]       UH: block aggregates, scanned in place
+//                                                                   into block-entering states
+// backward (saved)  : [GU B*H*NB*dk*dv][xq B*H*L][xk B*H*L][dc B*H*NC]
+// backward (replay) : backward (saved) ++ forward ++ [Sfin B*H*dk*dv]
+struct FwdWs { float* beta; float* UH; size_t bytes; };
+struct BwdWs { float* GU; float* xq; float* xk; float* dc; size_t bytes; };
+
+FwdWs fwd_ws(const sf_seg_desc_t* d, const SegParams& p, void* base) {
+    FwdWs w;
+    char* c = static_cast<char*>(base);
+    size_t off = 0;
+    const size_t bh = (size_t)p.B * p.H;
+    w.beta = reinterpret_cast<float*>(c + off); off += align_up(bh * p.NB * sizeof(float));
+    w.UH = reinterpret_cast<float*>(c + off);   off += align_up(bh * p.NB * (size_t)d->d_k * d->d_v * sizeof(float));
+    w.bytes = off;
+    return w;
+}
+
+BwdWs bwd_ws(const sf_seg_desc_t* d, const SegParams& p, void* base) {
+    BwdWs w;
+    char* c = static_cast<char*>(base);
+    size_t off = 0;
+    const size_t bh = (size_t)p.B * p.H;
+    w.GU = reinterpret_cast<float*>(c + off); off += align_up(bh * p.NB * (size_t)d->d_k * d->d_v * sizeof(float));
+    w.xq = reinterpret_cast<float*>(c + off); off += align_up(bh * p.L * sizeof(float));
+    w.xk = reinterpret_cast<float*>(c + off); off += align_up(bh * p.L * sizeof(float));
+    w.dc = reinterpret_cast<float*>(c + off); off += align_up(bh * p.NC * sizeof(float));
+    w.bytes = off;
+    return w;
+}
+
+size_t state_bytes(const sf_seg_desc_t* d) { return align_up((size_t)d->B * d->H * d->d_k * d->d_v * sizeof(float)); }
+
+inline sf_status_t check_launch() {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? SF_OK : SF_ERR_CUDA;
+}
+
+#define SF_TRY(expr) do { sf_status_t st__ = (expr); if (st__ != SF_OK) return st__; } while (0)
+
+// ---- SIMT dispatch ------------------------------------------------------------------------------
+template <typename K>
+sf_status_t set_smem(K kernel, size_t bytes) {
+    if (bytes > 48 * 1024) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+            cudaGetLastError();
+            return SF_ERR_CUDA;
+        }
+    }
+    return SF_OK;
+}
+
+enum class Role { Aggregate, FwdOut, BwdDq, BwdDkDv };
+
+struct RoleArgs {
+    const void *q, *k, *v, *dO;
+    const float* g;
+    int mode;                 // Aggregate: 0 forward (k,v), 1 backward (q,dO)
+    float *U, *beta;          // Aggregate outputs
+    const float* states;      // FwdOut/BwdDq: Hs ; BwdDkDv: Gs
+    void *o, *dq, *dk, *dv;
+    float *xq, *xk, *dc;
+};
+
+template <typename T, int DK, int DV>
+sf_status_t launch_simt(Role role, const SegParams& p, const RoleArgs& a, cudaStream_t st) {
+    using namespace sf::simt;
+    dim3 grid(p.NB, p.H, p.B), block(NT);
+    switch (role) {
+        case Role::Aggregate: {
+            auto kern = block_aggregate_kernel<T, DK, DV>;
+            constexpr size_t sm = smem_aggregate<DK, DV>();
+            SF_TRY(set_smem(kern, sm));
+            const T* X = static_cast<const T*>(a.mode == 0 ? a.k : a.q);
+            const T* Y = static_cast<const T*>(a.mode == 0 ? a.v : a.dO);
+            kern<<<grid, block, sm, st>>>(p, X, Y, a.g, a.mode, a.U, a.beta);
+            break;
+        }
+        case Role::FwdOut: {
+            auto kern = fwd_out_kernel<T, DK, DV>;
+            constexpr size_t sm = smem_fwd_out<DK, DV>();
+            SF_TRY(set_smem(kern, sm));
+            kern<<<grid, block, sm, st>>>(p, static_cast<const T*>(a.q), static_cast<const T*>(a.k),
+                                          static_cast<const T*>(a.v), a.g, a.states, static_cast<T*>(a.o));
+            break;
+        }
+        case Role::BwdDq: {
+            auto kern = bwd_dq_kernel<T, DK, DV>;
+            constexpr size_t sm = smem_bwd_dq<DK, DV>();
+            SF_TRY(set_smem(kern, sm));
+            kern<<<grid, block, sm, st>>>(p, static_cast<const T*>(a.q), static_cast<const T*>(a.k),
+                                          static_cast<const T*>(a.v), a.g, static_cast<const T*>(a.dO), a.states,
+                                          static_cast<T*>(a.dq), a.xq);
+            break;
+        }
+        case Role::BwdDkDv: {
+            auto kern = bwd_dkdv_kernel<T, DK, DV>;
+            constexpr size_t sm = smem_bwd_dkdv<DK, DV>();
+            SF_TRY(set_smem(kern, sm));
+            kern<<<grid, block, sm, st>>>(p, static_cast<const T*>(a.q), static_cast<const T*>(a.k),
+                                          static_cast<const T*>(a.v), a.g, static_cast<const T*>(a.dO), a.states,
+                                          static_cast<T*>(a.dk), static_cast<T*>(a.dv), a.xk, a.dc);
+            break;
+        }
+    }
+    return check_launch();
+}
+
+template <typename T>
+sf_status_t launch_simt_d(Role role, const sf_seg_desc_t* d, const SegParams& p, const RoleArgs& a, cudaStream_t st) {
+    if (d->d_k == 32 && d->d_v == 32) return launch_simt<T, 32, 32>(role, p, a, st);
+    if (d->d_k == 64 && d->d_v == 64) return launch_simt<T, 64, 64>(role, p, a, st);
+    if (d->d_k == 32 && d->d_v == 64) return launch_simt<T, 32, 64>(role, p, a, st);
+    if constexpr (sizeof(T) == 4) {
+        if (d->d_k == 128 && d->d_v == 128) return launch_simt<T, 128, 128>(role, p, a, st);
+    }
+    return SF_ERR_UNSUPPORTED;
+}
+
+sf_status_t launch_role(Path path, Role role, const sf_seg_desc_t* d, const SegParams& p, const RoleArgs& a, cudaStream_t st) {
+    if (path == Path::Tc) {
+        long long n = 0;
+        sf_status_t s = sf::tc::launch(static_cast<int>(role), d, p, a.q, a.k, a.v, a.dO, a.g, a.mode, a.U, a.beta, a.states,
+                                       a.o, a.dq, a.dk, a.dv, a.xq, a.xk, a.dc, st, &n);
+        g_launches.fetch_add(n, std::memory_order_relaxed);
+        return s;
+    }
+    if (d->dtype == SF_F32) return launch_simt_d<float>(role, d, p, a, st);
+    return launch_simt_d<__nv_bfloat16>(role, d, p, a, st);
+}
+
+sf_status_t launch_scan(const sf_seg_desc_t* d, const SegParams& p, int reverse, const float* ld, const float* U,
+                        const float* init, float* states, float* fin, cudaStream_t st) {
+    const int m = d->d_k * d->d_v;
+    dim3 grid((m / 4 + sf::SCAN_NT - 1) / sf::SCAN_NT, p.B * p.H);
+    sf::state_scan_kernel<<<grid, sf::SCAN_NT, 0, st>>>(p.NB, m, reverse, ld, U, init, states, fin);
+    return check_launch();
+}
+
+// ---- one segment -------------------------------------------------------------------------------
+struct FwdPtrs { const void *q, *k, *v; const float* g; const float* S_in; void* o; float* S_out; };
+
+// Stage split used by the chaining driver: `pre` needs no boundary state, `post` does.
+sf_status_t fwd_pre(Path path, const sf_seg_desc_t* d, const SegParams& p, const FwdPtrs& x, const FwdWs& w, cudaStream_t st) {
+    RoleArgs a{};
+    a.k = x.k; a.v = x.v; a.g = x.g; a.mode = 0; a.U = w.UH; a.beta = w.beta;
+    return launch_role(path, Role::Aggregate, d, p, a, st);
+}
+sf_status_t fwd_scan(const sf_seg_desc_t* d, const SegParams& p, const FwdPtrs& x, const FwdWs& w, cudaStream_t st) {
+    return launch_scan(d, p, 0, w.beta, w.UH, x.S_in, w.UH, x.S_out, st);
+}
+sf_status_t fwd_out(Path path, const sf_seg_desc_t* d, const SegParams& p, const FwdPtrs& x, const FwdWs& w, cudaStream_t st) {
+    RoleArgs a{};
+    a.q = x.q; a.k = x.k; a.v = x.v; a.g = x.g; a.states = w.UH; a.o = x.o;
+    return launch_role(path, Role::FwdOut, d, p, a, st);
+}
+
+struct BwdPtrs {
+    const void *q, *k, *v; const float* g; const float* S_in; const void* dO; const float* dS_out;
+    void *dq, *dk, *dv; float* dg; float* dS_in;
+};
+
+sf_status_t bwd_pre(Path path, const sf_seg_desc_t* d, const SegParams& p, const BwdPtrs& x, const BwdWs& w, float* beta_out,
+                    cudaStream_t st) {
+    RoleArgs a{};
+    a.q = x.q; a.dO = x.dO; a.g = x.g; a.mode = 1; a.U = w.GU; a.beta = beta_out;
+    return launch_role(path, Role::Aggregate, d, p, a, st);
+}
+sf_status_t bwd_scan(const sf_seg_desc_t* d, const SegParams& p, const BwdPtrs& x, const BwdWs& w, const float* beta, cudaStream_t st) {
+    return launch_scan(d, p, 1, beta, w.GU, x.dS_out, w.GU, x.dS_in, st);
+}
+sf_status_t bwd_dq(Path path, const sf_seg_desc_t* d, const SegParams& p, const BwdPtrs& x, const BwdWs& w, const float* Hs, cudaStream_t st) {
+    RoleArgs a{};
+    a.q = x.q; a.k = x.k; a.v = x.v; a.dO = x.dO; a.g = x.g; a.states = Hs; a.dq = x.dq; a.xq = w.xq;
+    return launch_role(path, Role::BwdDq, d, p, a, st);
+}
+sf_status_t bwd_dkdv(Path path, const sf_seg_desc_t* d, const SegParams& p, const BwdPtrs& x, const BwdWs& w, cudaStream_t st) {
+    RoleArgs a{};
+    a.q = x.q; a.k = x.k; a.v = x.v; a.dO = x.dO; a.g = x.g; a.states = w.GU; a.dk = x.dk; a.dv = x.dv; a.xk = w.xk; a.dc = w.dc;
+    return launch_role(path, Role::BwdDkDv, d, p, a, st);
+}
+sf_status_t bwd_dg(const sf_seg_desc_t* d, const SegParams& p, const BwdPtrs& x, const BwdWs& w, const float* Hs, cudaStream_t st) {
+    dim3 grid(p.NB, p.H, p.B);
+    sf::dg_epilogue_kernel<<<grid, sf::DG_NT, 0, st>>>(p, d->d_k * d->d_v, w.xq, w.xk, w.dc, Hs, w.GU, x.dS_in, x.dg);
+    return check_launch();
+}
+
+sf_status_t validate_fwd(const sf_seg_desc_t* d, const FwdPtrs& x, const void* ws, size_t ws_bytes, Path* path) {
+    *path = classify(d);
+    if (*path == Path::Invalid) return SF_ERR_INVALID_ARG;
+    if (*path == Path::Unsupported) return SF_ERR_UNSUPPORTED;
+    if (!x.q || !x.k || !x.v || !x.g || !x.o || !x.S_out) return SF_ERR_INVALID_ARG;
+    if (x.S_in == x.S_out) return SF_ERR_INVALID_ARG;
+    const void* ptrs[] = {x.q, x.k, x.v, x.g, x.S_in, x.o, x.S_out};
+    for (const void* ptr : ptrs) if (ptr && !aligned16(ptr)) return SF_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < sf_workspace_bytes(d, 0)) return SF_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) % kAlign) return SF_ERR_INVALID_ARG;
+    return SF_OK;
+}
+
+sf_status_t validate_bwd(const sf_seg_desc_t* d, const BwdPtrs& x, const void* saved, const void* ws, size_t ws_bytes, Path* path) {
+    *path = classify(d);
+    if (*path == Path::Invalid) return SF_ERR_INVALID_ARG;
+    if (*path == Path::Unsupported) return SF_ERR_UNSUPPORTED;
+    if (!x.q || !x.k || !x.v || !x.g || !x.dO || !x.dq || !x.dk || !x.dv || !x.dg || !x.dS_in) return SF_ERR_INVALID_ARG;
+    if (x.dS_out == x.dS_in) return SF_ERR_INVALID_ARG;
+    const void* ptrs[] = {x.q, x.k, x.v, x.g, x.S_in, x.dO, x.dS_out, x.dq, x.dk, x.dv, x.dg, x.dS_in, saved};
+    for (const void* ptr : ptrs) if (ptr && !aligned16(ptr)) return SF_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < sf_workspace_bytes(d, saved ? 1 : 2)) return SF_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) % kAlign) return SF_ERR_INVALID_ARG;
+    if (saved && saved == ws) return SF_ERR_INVALID_ARG;
+    if (saved && reinterpret_cast<uintptr_t>(saved) % kAlign) return SF_ERR_INVALID_ARG;
+    return SF_OK;
+}
+
+// Side streams and events of the chaining driver (host objects only; created once per process).
+struct ChainRes {
+    cudaStream_t side[2] = {nullptr, nullptr};
+    cudaEvent_t ev[64] = {};
+    bool ok = false;
+    int device = -1;
+};
+std::mutex g_chain_mu;
+ChainRes g_chain;
+
+sf_status_t chain_resources(ChainRes** out) {
+    std::lock_guard<std::mutex> lk(g_chain_mu);
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SF_ERR_CUDA;
+    if (!g_chain.ok || g_chain.device != dev) {
+        for (auto& s : g_chain.side)
+            if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SF_ERR_CUDA;
+        for (auto& e : g_chain.ev)
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return SF_ERR_CUDA;
+        g_chain.ok = true;
+        g_chain.device = dev;
+    }
+    *out = &g_chain;
+    return SF_OK;
+}
+
+#define SF_CUDA(expr) do { if ((expr) != cudaSuccess) { cudaGetLastError(); return SF_ERR_CUDA; } } while (0)
+
+struct SeqPtr {
+    // byte pointer arithmetic over a [B,T,H,d] tensor along T
+    static const void* at(const void* base, long long tok, long long stride, size_t esz) {
+        return base ? static_cast<const char*>(base) + tok * stride * (long long)esz : nullptr;
+    }
+    static void* at(void* base, long long tok, long long stride, size_t esz) {
+        return base ? static_cast<char*>(base) + tok * stride * (long long)esz : nullptr;
+    }
+};
+
+sf_status_t validate_chain(const sf_seg_desc_t* d, const int32_t* seg_lens, int32_t n_seg, long long* T_out) {
+    if (!d || !seg_lens || n_seg <= 0 || n_seg > 1 << 20) return SF_ERR_INVALID_ARG;
+    long long T = 0;
+    for (int i = 0; i < n_seg; ++i) {
+        if (seg_lens[i] <= 0 || d->chunk <= 0 || seg_lens[i] % d->chunk) return SF_ERR_INVALID_ARG;
+        T += seg_lens[i];
+    }
+    sf_seg_desc_t t = *d;
+    t.seg_len = seg_lens[0];
+    Path p = classify(&t);
+    if (p == Path::Invalid) return SF_ERR_INVALID_ARG;
+    if (p == Path::Unsupported) return SF_ERR_UNSUPPORTED;
+    if (T_out) *T_out = T;
+    return SF_OK;
+}
+
+}  // namespace
+
+// ================================================================================================
+extern "C" {
+
+const char* sf_status_string(sf_status_t s) {
+    switch (s) {
+        case SF_OK: return "ok";
+        case SF_ERR_INVALID_ARG: return "invalid argument";
+        case SF_ERR_UNSUPPORTED: return "unsupported (dtype, d_k, d_v, chunk) combination";
+        case SF_ERR_WORKSPACE: return "workspace missing or too small";
+        case SF_ERR_CUDA: return "CUDA call or kernel launch failed";
+        case SF_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+int32_t sf_num_blocks(const sf_seg_desc_t* desc) {
+    Path p = classify(desc);
+    if (p == Path::Invalid || p == Path::Unsupported) return 0;
+    return make_params(desc).NB;
+}
+
+size_t sf_workspace_bytes(const sf_seg_desc_t* desc, int backward) {
+    Path path = classify(desc);
+    if (path == Path::Invalid || path == Path::Unsupported) return 0;
+    const SegParams p = make_params(desc);
+    const size_t f = fwd_ws(desc, p, nullptr).bytes;
+    if (backward == 0) return f;
+    const size_t b = bwd_ws(desc, p, nullptr).bytes;
+    if (backward == 1) return b;
+    return b + f + state_bytes(desc);
+}
+
+sf_status_t sf_segment_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                           const float* S_in, void* o, float* S_out, void* workspace, size_t workspace_bytes,
+                           sf_stream_t stream) {
+    FwdPtrs x{q, k, v, g, S_in, o, S_out};
+    Path path;
+    SF_TRY(validate_fwd(desc, x, workspace, workspace_bytes, &path));
+    const SegParams p = make_params(desc);
+    const FwdWs w = fwd_ws(desc, p, workspace);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    SF_TRY(fwd_pre(path, desc, p, x, w, st));
+    SF_TRY(fwd_scan(desc, p, x, w, st));
+    SF_TRY(fwd_out(path, desc, p, x, w, st));
+    return SF_OK;
+}
+
+sf_status_t sf_segment_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                           const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk, void* dv, float* dg,
+                           float* dS_in, const void* fwd_saved, void* workspace, size_t workspace_bytes, sf_stream_t stream) {
+    BwdPtrs x{q, k, v, g, S_in, dO, dS_out, dq, dk, dv, dg, dS_in};
+    Path path;
+    SF_TRY(validate_bwd(desc, x, fwd_saved, workspace, workspace_bytes, &path));
+    const SegParams p = make_params(desc);
+    const BwdWs w = bwd_ws(desc, p, workspace);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    FwdWs fw;
+    if (fwd_saved) {
+        fw = fwd_ws(desc, p, const_cast<void*>(fwd_saved));
+    } else {
+        // SR: replay the block-entering states from S_in
+        char* base = static_cast<char*>(workspace) + w.bytes;
+        fw = fwd_ws(desc, p, base);
+        float* sfin = reinterpret_cast<float*>(base + fw.bytes);
+        FwdPtrs fx{q, k, v, g, S_in, nullptr, sfin};
+        SF_TRY(fwd_pre(path, desc, p, fx, fw, st));
+        SF_TRY(fwd_scan(desc, p, fx, fw, st));
+    }
+    SF_TRY(bwd_pre(path, desc, p, x, w, nullptr, st));
+    SF_TRY(bwd_scan(desc, p, x, w, fw.beta, st));
+    SF_TRY(bwd_dq(path, desc, p, x, w, fw.UH, st));
+    SF_TRY(bwd_dkdv(path, desc, p, x, w, st));
+    SF_TRY(bwd_dg(desc, p, x, w, fw.UH, st));
+    return SF_OK;
+}
+
+sf_status_t sf_state_scan(const sf_seg_desc_t* desc, int32_t chunks_per_block, int32_t reverse, const float* log_decay,
+                          const float* U, const float* S_boundary_in, float* states, float* S_boundary_out,
+                          sf_stream_t stream) {
+    Path path = classify(desc);
+    if (path == Path::Invalid) return SF_ERR_INVALID_ARG;
+    if (path == Path::Unsupported) return SF_ERR_UNSUPPORTED;
+    if (chunks_per_block < 0 || chunks_per_block > sf::simt::MAXR) return SF_ERR_INVALID_ARG;
+    if (!log_decay || !U || !states || !S_boundary_out || S_boundary_in == S_boundary_out) return SF_ERR_INVALID_ARG;
+    if (!aligned16(U) || !aligned16(states) || !aligned16(S_boundary_out) || (S_boundary_in && !aligned16(S_boundary_in)))
+        return SF_ERR_INVALID_ARG;
+    const SegParams p = make_params(desc, chunks_per_block);
+    return launch_scan(desc, p, reverse != 0, log_decay, U, S_boundary_in, states, S_boundary_out,
+                       reinterpret_cast<cudaStream_t>(stream));
+}
+
+size_t sf_chain_workspace_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, int backward) {
+    if (validate_chain(desc, seg_lens, n_seg, nullptr) != SF_OK) return 0;
+    size_t total = 0, mx = 0;
+    for (int i = 0; i < n_seg; ++i) {
+        sf_seg_desc_t t = *desc;
+        t.seg_len = seg_lens[i];
+        const size_t b = sf_workspace_bytes(&t, backward);
+        total += b;
+        mx = b > mx ? b : mx;
+    }
+    // forward keeps every segment's block states for the backward; the backward ping-pongs two
+    // per-segment workspaces so that neighbouring segments can overlap
+    return backward == 0 ? total : 2 * mx;
+}
+
+sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q, const void* k,
+                         const void* v, const float* g, const float* S_init, void* o, float* S_bounds, void* workspace,
+                         size_t workspace_bytes, int32_t overlap, sf_stream_t stream) {
+    long long T = 0;
+    SF_TRY(validate_chain(desc, seg_lens, n_seg, &T));
+    if (!q || !k || !v || !g || !o || !S_bounds) return SF_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < sf_chain_workspace_bytes(desc, seg_lens, n_seg, 0)) return SF_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return SF_ERR_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, g, S_init, o, S_bounds};
+    for (const void* ptr : ptrs) if (ptr && !aligned16(ptr)) return SF_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t esz = desc->dtype == SF_BF16 ? 2 : 4;
+    const size_t sN = (size_t)desc->B * desc->H * desc->d_k * desc->d_v;
+
+    // S_bounds[0] = S_init (or zero)
+    if (S_init) SF_CUDA(cudaMemcpyAsync(S_bounds, S_init, sN * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    else        SF_CUDA(cudaMemsetAsync(S_bounds, 0, sN * sizeof(float), st));
+
+    ChainRes* res = nullptr;
+    if (overlap) SF_TRY(chain_resources(&res));
+    // overlap schedule (the forward wavefront of Section 3.4, Eq. 17, across segments):
+    //   side stream : Pre(0) Pre(1) Pre(2) ...            (block aggregates need no boundary state)
+    //   main stream : [wait Pre(i)] ST(i) Out(i)          (ST(i) also overlaps Out(i-1)'s tail)
+    if (overlap) {
+        SF_CUDA(cudaEventRecord(res->ev[0], st));
+        SF_CUDA(cudaStreamWaitEvent(res->side[0], res->ev[0], 0));
+    }
+    size_t ws_off = 0;
+    long long tok = 0;
+    for (int i = 0; i < n_seg; ++i) {
+        sf_seg_desc_t t = *desc;
+        t.seg_len = seg_lens[i];
+        const Path path = classify(&t);
+        const SegParams p = make_params(&t);
+        const FwdWs w = fwd_ws(&t, p, static_cast<char*>(workspace) + ws_off);
+        ws_off += w.bytes;
+        FwdPtrs x{SeqPtr::at(q, tok, t.tok_stride_qk, esz), SeqPtr::at(k, tok, t.tok_stride_qk, esz),
+                  SeqPtr::at(v, tok, t.tok_stride_v, esz),
+                  static_cast<const float*>(SeqPtr::at(g, tok, t.tok_stride_g, sizeof(float))),
+                  S_bounds + (size_t)i * sN, SeqPtr::at(o, tok, t.tok_stride_v, esz), S_bounds + (size_t)(i + 1) * sN};
+        if (overlap) {
+            cudaEvent_t e = res->ev[1 + (i % 32)];
+            SF_TRY(fwd_pre(path, &t, p, x, w, res->side[0]));
+            SF_CUDA(cudaEventRecord(e, res->side[0]));
+            SF_CUDA(cudaStreamWaitEvent(st, e, 0));
+        } else {
+            SF_TRY(fwd_pre(path, &t, p, x, w, st));
+        }
+        SF_TRY(fwd_scan(&t, p, x, w, st));
+        SF_TRY(fwd_out(path, &t, p, x, w, st));
+        tok += seg_lens[i];
+    }
+    return SF_OK;
+}
+
+sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q, const void* k,
+                         const void* v, const float* g, const float* S_bounds, const void* dO, const float* dS_final,
+                         void* dq, void* dk, void* dv, float* dg, float* dS_init, const void* fwd_workspace, void* workspace,
+                         size_t workspace_bytes, int32_t overlap, sf_stream_t stream) {
+    long long T = 0;
+    SF_TRY(validate_chain(desc, seg_lens, n_seg, &T));
+    if (!q || !k || !v || !g || !S_bounds || !dO || !dq || !dk || !dv || !dg || !dS_init) return SF_ERR_INVALID_ARG;
+    const int mode = fwd_workspace ? 1 : 2;
+    const size_t need = sf_chain_workspace_bytes(desc, seg_lens, n_seg, mode);
+    const size_t sB = state_bytes(desc);
+    if (!workspace || workspace_bytes < need + 2 * sB) return SF_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return SF_ERR_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, g, S_bounds, dO, dS_final, dq, dk, dv, dg, dS_init, fwd_workspace};
+    for (const void* ptr : ptrs) if (ptr && !aligned16(ptr)) return SF_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t esz = desc->dtype == SF_BF16 ? 2 : 4;
+    const size_t sN = (size_t)desc->B * desc->H * desc->d_k * desc->d_v;
+    (void)overlap;
+
+    // layout: [seg ws A][seg ws B][dS ping][dS pong]
+    char* base = static_cast<char*>(workspace);
+    const size_t half = need / 2;
+    float* dS_buf[2] = {reinterpret_cast<float*>(base + need), reinterpret_cast<float*>(base + need + sB)};
+
+    // offsets of every segment's saved forward workspace
+    size_t fwd_off_end = 0;
+    for (int i = 0; i < n_seg; ++i) {
+        sf_seg_desc_t t = *desc;
+        t.seg_len = seg_lens[i];
+        fwd_off_end += sf_workspace_bytes(&t, 0);
+    }
+    long long tok = T;
+    const float* dS_next = dS_final;
+    for (int i = n_seg - 1; i >= 0; --i) {
+        sf_seg_desc_t t = *desc;
+        t.seg_len = seg_lens[i];
+        tok -= seg_lens[i];
+        fwd_off_end -= sf_workspace_bytes(&t, 0);
+        const Path path = classify(&t);
+        const SegParams p = make_params(&t);
+        char* wsi = base + (size_t)(i & 1) * half;
+        const BwdWs w = bwd_ws(&t, p, wsi);
+        float* dS_here = (i == 0) ? dS_init : dS_buf[i & 1];
+        BwdPtrs x{SeqPtr::at(q, tok, t.tok_stride_qk, esz), SeqPtr::at(k, tok, t.tok_stride_qk, esz),
+                  SeqPtr::at(v, tok, t.tok_stride_v, esz),
+                  static_cast<const float*>(SeqPtr::at(g, tok, t.tok_stride_g, sizeof(float))),
+                  S_bounds + (size_t)i * sN, SeqPtr::at(dO, tok, t.tok_stride_v, esz), dS_next,
+                  SeqPtr::at(dq, tok, t.tok_stride_qk, esz), SeqPtr::at(dk, tok, t.tok_stride_qk, esz),
+                  SeqPtr::at(dv, tok, t.tok_stride_v, esz),
+                  static_cast<float*>(SeqPtr::at(dg, tok, t.tok_stride_g, sizeof(float))), dS_here};
+        FwdWs fw;
+        if (fwd_workspace) {
+            fw = fwd_ws(&t, p, const_cast<char*>(static_cast<const char*>(fwd_workspace)) + fwd_off_end);
+        } else {
+            char* fbase = wsi + w.bytes;
+            fw = fwd_ws(&t, p, fbase);
+            float* sfin = reinterpret_cast<float*>(fbase + fw.bytes);
+            FwdPtrs fx{x.q, x.k, x.v, x.g, x.S_in, nullptr, sfin};
+            SF_TRY(fwd_pre(path, &t, p, fx, fw, st));
+            SF_TRY(fwd_scan(&t, p, fx, fw, st));
+        }
+        SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, st));
+        SF_TRY(bwd_scan(&t, p, x, w, fw.beta, st));
+        SF_TRY(bwd_dq(path, &t, p, x, w, fw.UH, st));
+        SF_TRY(bwd_dkdv(path, &t, p, x, w, st));
+        SF_TRY(bwd_dg(&t, p, x, w, fw.UH, st));
+        dS_next = dS_here;
+    }
+    return SF_OK;
+}
+
+size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg) {
+    long long T = 0;
+    if (validate_chain(desc, seg_lens, n_seg, &T) != SF_OK) return 0;
+    const size_t esz = desc->dtype == SF_BF16 ? 2 : 4;
+    const size_t nqk = align_up((size_t)desc->B * T * desc->H * desc->d_k * esz);
+    const size_t nv = align_up((size_t)desc->B * T * desc->H * desc->d_v * esz);
+    const size_t ng = align_up((size_t)desc->B * T * desc->H * sizeof(float));
+    const size_t sB = state_bytes(desc);
+    return 4 * nqk + 4 * nv + 2 * ng + (size_t)(n_seg + 1) * sB + 3 * sB +
+           sf_chain_workspace_bytes(desc, seg_lens, n_seg, 0) + sf_chain_workspace_bytes(desc, seg_lens, n_seg, 1) + 2 * sB;
+}
+
+sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q,
+                                  const void* k, const void* v, const float* g, const float* S_init, const void* dO,
+                                  const float* dS_final, void* o, float* S_final, void* dq, void* dk, void* dv, float* dg,
+                                  float* dS_init, void* dev, size_t dev_bytes, sf_stream_t stream) {
+    long long T = 0;
+    SF_TRY(validate_chain(desc, seg_lens, n_seg, &T));
+    if (!q || !k || !v || !g || !dO || !o || !dq || !dk || !dv || !dg || !dS_init) return SF_ERR_INVALID_ARG;
+    if (!dev || dev_bytes < sf_e2e_device_bytes(desc, seg_lens, n_seg)) return SF_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(dev) % kAlign) return SF_ERR_INVALID_ARG;
+    // the wrapper works on a densely packed device copy
+    sf_seg_desc_t d = *desc;
+    if (d.tok_stride_qk != (long long)d.H * d.d_k || d.tok_stride_v != (long long)d.H * d.d_v || d.tok_stride_g != d.H)
+        return SF_ERR_INVALID_ARG;
+    if (d.B > 1 && (d.batch_stride_qk != T * d.tok_stride_qk || d.batch_stride_v != T * d.tok_stride_v ||
+                    d.batch_stride_g != T * d.tok_stride_g))
+        return SF_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t esz = d.dtype == SF_BF16 ? 2 : 4;
+    const size_t bqk = (size_t)d.B * T * d.H * d.d_k * esz, bv = (size_t)d.B * T * d.H * d.d_v * esz;
+    const size_t bg = (size_t)d.B * T * d.H * sizeof(float);
+    const size_t nqk = align_up(bqk), nv = align_up(bv), ng = align_up(bg), sB = state_bytes(&d);
+    const size_t sbytes = (size_t)d.B * d.H * d.d_k * d.d_v * sizeof(float);
+    char* c = static_cast<char*>(dev);
+    auto take = [&](size_t n) { char* r = c; c += n; return r; };
+    char *dq_ = take(nqk), *dk_ = take(nqk), *q_ = take(nqk), *k_ = take(nqk);
+    char *v_ = take(nv), *dO_ = take(nv), *o_ = take(nv), *dv_ = take(nv);
+    char *g_ = take(ng), *dg_ = take(ng);
+    float* bounds = reinterpret_cast<float*>(take((size_t)(n_seg + 1) * sB));
+    float* sinit = reinterpret_cast<float*>(take(sB));
+    float* dsfin = reinterpret_cast<float*>(take(sB));
+    float* dsinit = reinterpret_cast<float*>(take(sB));
+    const size_t wf = sf_chain_workspace_bytes(&d, seg_lens, n_seg, 0), wb = sf_chain_workspace_bytes(&d, seg_lens, n_seg, 1);
+    char* wsf = take(wf);
+    char* wsb = take(wb + 2 * sB);
+
+    SF_CUDA(cudaMemcpyAsync(q_, q, bqk, cudaMemcpyHostToDevice, st));
+    SF_CUDA(cudaMemcpyAsync(k_, k, bqk, cudaMemcpyHostToDevice, st));
+    SF_CUDA(cudaMemcpyAsync(v_, v, bv, cudaMemcpyHostToDevice, st));
+    SF_CUDA(cudaMemcpyAsync(g_, g, bg, cudaMemcpyHostToDevice, st));
+    SF_CUDA(cudaMemcpyAsync(dO_, dO, bv, cudaMemcpyHostToDevice, st));
+    if (S_init) SF_CUDA(cudaMemcpyAsync(sinit, S_init, sbytes, cudaMemcpyHostToDevice, st));
+    if (dS_final) SF_CUDA(cudaMemcpyAsync(dsfin, dS_final, sbytes, cudaMemcpyHostToDevice, st));
+    // sB is a multiple of 256 but the chain driver indexes bounds densely
+    float* bounds_dense = bounds;
+    SF_TRY(sf_chain_fwd(&d, seg_lens, n_seg, q_, k_, v_, reinterpret_cast<float*>(g_), S_init ? sinit : nullptr, o_,
+                        bounds_dense, wsf, wf, 1, stream));
+    SF_TRY(sf_chain_bwd(&d, seg_lens, n_seg, q_, k_, v_, reinterpret_cast<float*>(g_), bounds_dense, dO_,
+                        dS_final ? dsfin : nullptr, dq_, dk_, dv_, reinterpret_cast<float*>(dg_), dsinit, wsf, wsb,
+                        wb + 2 * sB, 1, stream));
+    SF_CUDA(cudaMemcpyAsync(o, o_, bv, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaMemcpyAsync(dq, dq_, bqk, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaMemcpyAsync(dk, dk_, bqk, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaMemcpyAsync(dv, dv_, bv, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaMemcpyAsync(dg, dg_, bg, cudaMemcpyDeviceToHost, st));
+    if (S_final)
+        SF_CUDA(cudaMemcpyAsync(S_final, bounds_dense + (size_t)n_seg * (sbytes / sizeof(float)), sbytes, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaMemcpyAsync(dS_init, dsinit, sbytes, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaStreamSynchronize(st));
+    return SF_OK;
+}
+
+int32_t sf_device_status(void) { return sf::tc::read_device_status(); }
+void sf_device_status_clear(void) { sf::tc::clear_device_status(); }
+int64_t sf_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"
