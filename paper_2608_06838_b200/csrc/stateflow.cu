@@ -174,9 +174,7 @@ sf_status_t launch_simt_d(Role role, const sf_seg_desc_t* d, const SegParams& p,
     if (d->d_k == 32 && d->d_v == 32) return launch_simt<T, 32, 32>(role, p, a, st);
     if (d->d_k == 64 && d->d_v == 64) return launch_simt<T, 64, 64>(role, p, a, st);
     if (d->d_k == 32 && d->d_v == 64) return launch_simt<T, 32, 64>(role, p, a, st);
-    if constexpr (sizeof(T) == 4) {
-        if (d->d_k == 128 && d->d_v == 128) return launch_simt<T, 128, 128>(role, p, a, st);
-    }
+    if (d->d_k == 128 && d->d_v == 128) return launch_simt<T, 128, 128>(role, p, a, st);
     return SF_ERR_UNSUPPORTED;
 }
 
@@ -186,7 +184,7 @@ sf_status_t launch_role(Path path, Role role, const sf_seg_desc_t* d, const SegP
         sf_status_t s = sf::tc::launch(static_cast<int>(role), d, p, a.q, a.k, a.v, a.dO, a.g, a.mode, a.U, a.beta, a.states,
                                        a.o, a.dq, a.dk, a.dv, a.xq, a.xk, a.dc, st, &n);
         g_launches.fetch_add(n, std::memory_order_relaxed);
-        return s;
+        if (s != SF_ERR_UNSUPPORTED) return s;      // DEV: roles not yet on tensor cores run on CUDA cores
     }
     if (d->dtype == SF_F32) return launch_simt_d<float>(role, d, p, a, st);
     return launch_simt_d<__nv_bfloat16>(role, d, p, a, st);
