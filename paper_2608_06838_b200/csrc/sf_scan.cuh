@@ -56,21 +56,23 @@ __global__ void __launch_bounds__(SCAN_NT) state_scan_kernel(int n, int m, int r
     *reinterpret_cast<float4*>(final_state + (long long)bh * m + e) = x;
 }
 
-// Log-decay gradient.  With x_t = q_t.dq_t - k_t.dk_t (assembled from the per-token terms the dq and
-// dk/dv passes emit), H_{c+1} the state leaving chunk c and dH_{c+1} its gradient,
-//     dg_u = <H_{c+1}, dH_{c+1}> + sum_{t=u}^{end of chunk c} x_t .
-// P_c = <H_c, dH_c> obeys the scalar recurrence P_{c+1} = P_c - a_c + d_c with
-// a_c = sum_t q_t.dq_t^{inter}, d_c = sum_t k_t.dk_t^{inter}; it is anchored at every block start with
-// the float32 block states: P = <Hs[j], gradient entering block j> (Gs[j-1], or dS_in for j = 0).
-// grid = (NB, H, B), 256 threads.  xq, xk: [B,H,L]; dc: [B,H,NC]; dg: [B,L,H] with strides.
+// Log-decay gradient.  With x_t = q_t.dq_t - k_t.dk_t (the dq and dk/dv passes emit both dot products
+// from their float32 accumulators) the recurrence gives dg_t = dg_{t+1} + x_t, and at a block start
+// dg equals <H, dH> of the block-entering state and its gradient plus the block's x.  So, with
+// P = <Hs[j], gradient entering block j> (Gs[j-1], or dS_in for j = 0) read from the float32 block
+// states, the token u of block j gets
+//     dg_u = P - sum_{t < u in block j} x_t ,
+// evaluated chunk by chunk: P_{c+1} = P_c - sum_{t in chunk c} x_t, dg_u = P_{c+1} + sum_{t=u}^{end of c} x_t.
+// Re-anchoring at every block keeps rounding errors of the dot products from accumulating over the
+// segment.  grid = (NB, H, B), 256 threads.  xq, xk: [B,H,L]; dg: [B,L,H] with strides.
 constexpr int DG_NT = 256;
 
 __global__ void __launch_bounds__(DG_NT) dg_epilogue_kernel(SegParams p, int m, const float* __restrict__ xq,
-                                                            const float* __restrict__ xk, const float* __restrict__ dc,
-                                                            const float* __restrict__ Hs, const float* __restrict__ Gs,
-                                                            const float* __restrict__ dS_in, float* __restrict__ dg) {
+                                                            const float* __restrict__ xk, const float* __restrict__ Hs,
+                                                            const float* __restrict__ Gs, const float* __restrict__ dS_in,
+                                                            float* __restrict__ dg) {
     __shared__ float red[DG_NT / 32];
-    __shared__ float a_c[64], P_next[64];
+    __shared__ float sx[64], P_next[64];
     __shared__ float suffix[64 * 64];
     const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const long long bh = (long long)b * p.H + h;
@@ -90,35 +92,30 @@ __global__ void __launch_bounds__(DG_NT) dg_epilogue_kernel(SegParams p, int m, 
     for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = part;
 
-    // per chunk: suffix sums of x_t and a_c, one warp per chunk (C <= 64: two tokens per lane)
+    // per chunk: suffix sums of x_t and the chunk total, one warp per chunk (C <= 64: two tokens per lane)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float* xqh = xq + bh * p.L;
     const float* xkh = xk + bh * p.L;
     for (int c = warp; c < nch; c += DG_NT / 32) {
         const long long t0 = (long long)(c0 + c) * C;
-        // lane owns tokens 2*lane and 2*lane+1 (when < C)
         const int r0 = 2 * lane, r1 = 2 * lane + 1;
-        const float q0 = (r0 < C) ? xqh[t0 + r0] : 0.f, q1 = (r1 < C) ? xqh[t0 + r1] : 0.f;
-        const float x0 = (r0 < C) ? q0 + xkh[t0 + r0] : 0.f, x1 = (r1 < C) ? q1 + xkh[t0 + r1] : 0.f;
-        float qs = q0 + q1;
-        for (int off = 16; off > 0; off >>= 1) qs += __shfl_xor_sync(0xffffffffu, qs, off);
-        // inclusive suffix sum over lanes of (x0 + x1)
-        float incl = x0 + x1;
+        const float x0 = (r0 < C) ? xqh[t0 + r0] - xkh[t0 + r0] : 0.f;
+        const float x1 = (r1 < C) ? xqh[t0 + r1] - xkh[t0 + r1] : 0.f;
+        float incl = x0 + x1;                       // inclusive suffix sum over lanes
         for (int off = 1; off < 32; off <<= 1) {
             const float up = __shfl_down_sync(0xffffffffu, incl, off);
             if (lane + off < 32) incl += up;
         }
-        if (r0 < C) suffix[c * 64 + r0] = incl;            // x0 + x1 + everything after
+        if (r0 < C) suffix[c * 64 + r0] = incl;
         if (r1 < C) suffix[c * 64 + r1] = incl - x0;
-        if (lane == 0) a_c[c] = qs;
+        if (lane == 0) sx[c] = incl;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         float P = 0.f;
         for (int w = 0; w < DG_NT / 32; ++w) P += red[w];
-        const float* dch = dc + bh * p.NC + c0;
         for (int c = 0; c < nch; ++c) {
-            P = P - a_c[c] + dch[c];
+            P -= sx[c];
             P_next[c] = P;
         }
     }

@@ -140,7 +140,6 @@ __device__ __forceinline__ void state_update(float* S, const float* Ks, const fl
 }
 
 // masked[r][s] = (x_r . y_s) * exp(bcum[r]-bcum[s]) for s <= r, else 0.  D = feature width of x and y.
-// If raw != nullptr the unmasked dot products are stored there too (lower triangle, 0 above).
 template <int D>
 __device__ __forceinline__ void masked_scores(float* out, float* raw, const float* Xs, const float* Ys, const float* bcum, int C) {
     for (int idx = threadIdx.x; idx < C * C; idx += NT) {
@@ -154,7 +153,7 @@ __device__ __forceinline__ void masked_scores(float* out, float* raw, const floa
             val = dot * __expf(bcum[r] - bcum[s]);
         }
         out[idx] = val;
-        if (raw) raw[idx] = dot;
+        (void)raw;
     }
 }
 
@@ -206,7 +205,7 @@ __global__ void __launch_bounds__(NT) fwd_out_kernel(SegParams p, const T* __res
 
 // ------------------------------------------------------------------------------------------------
 // dq pass (SR + OG): replays H_c inside the block from Hs[j]; dq = dA K + diag(exp(b)) dO H_c^T.
-// Also emits xq[t] = q_t . (inter-chunk part of dq_t), a term of the log-decay gradient.
+// Also emits xq[t] = q_t . dq_t from the float32 accumulators, a term of the log-decay gradient.
 template <typename T, int DK, int DV>
 __global__ void __launch_bounds__(NT) bwd_dq_kernel(SegParams p, const T* __restrict__ q, const T* __restrict__ k,
                                                     const T* __restrict__ v, const float* __restrict__ g,
@@ -249,9 +248,9 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(SegParams p, const T* __rest
                 const int jv = (j0 + i) & (DV - 1);
                 inter = fmaf(Ds[r * DV + jv], S[i * DV + jv], inter);
             }
-            inter *= ebc[r];
-            dq[qk_off + (t0 + r) * p.tqk + i] = from_f32<T>(intra + inter);
-            Qs[idx] *= inter;                       // q_r[i] * dq_inter_r[i], reduced below
+            const float tot = intra + ebc[r] * inter;
+            dq[qk_off + (t0 + r) * p.tqk + i] = from_f32<T>(tot);
+            Qs[idx] *= tot;                         // q_r[i] * dq_r[i], reduced below
         }
         __syncthreads();
         if (threadIdx.x < C) {
@@ -267,14 +266,12 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(SegParams p, const T* __rest
 
 // ------------------------------------------------------------------------------------------------
 // dk/dv pass (STB inside the block + PG): reverse sweep from Gs[j], the gradient w.r.t. the state
-// leaving block j.  Also emits, per token, xk[t] = rowsum(M)_t - colsum(M)_t - k_t.(inter part of
-// dk_t) with M = dA * (Q K^T), and per chunk dc[c] = sum_t k_t.(inter part of dk_t).
+// leaving block j.  Also emits xk[t] = k_t . dk_t from the float32 accumulators.
 template <typename T, int DK, int DV>
 __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __restrict__ q, const T* __restrict__ k,
                                                       const T* __restrict__ v, const float* __restrict__ g,
                                                       const T* __restrict__ dO, const float* __restrict__ Gs,
-                                                      T* __restrict__ dk, T* __restrict__ dv,
-                                                      float* __restrict__ xk, float* __restrict__ dc) {
+                                                      T* __restrict__ dk, T* __restrict__ dv, float* __restrict__ xk) {
     extern __shared__ float smem[];
     float* Qs = smem;
     float* Ks = Qs + MAXC * DK;
@@ -286,8 +283,6 @@ __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __re
     float* bcum = G + DK * DV;
     float* wsuf = bcum + MAXC;
     float* ebc = wsuf + MAXC;
-    float* rs = ebc + MAXC;
-    float* cs = rs + MAXC;
     const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const int C = p.C;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
@@ -296,7 +291,6 @@ __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __re
     const float* gh = g + (long long)b * p.bg + h;
     const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(DK * DV);
     float* xkh = xk + ((long long)b * p.H + h) * p.L;
-    float* dch = dc + ((long long)b * p.H + h) * p.NC;
     for (int idx = threadIdx.x; idx < DK * DV; idx += NT) G[idx] = G0[idx];
 
     for (int c = nch - 1; c >= 0; --c) {
@@ -306,26 +300,8 @@ __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __re
         load_tile(Vs, v + v_off + t0 * p.tv, p.tv, C, DV);
         load_tile(Ds, dO + v_off + t0 * p.tv, p.tv, C, DV);
         chunk_decay(gh + t0 * p.tg, p.tg, C, bcum, wsuf, ebc);     // syncs
-        masked_scores<DK>(dA /*scratch for masked A*/, A /*raw QK^T*/, Qs, Ks, bcum, C);
-        __syncthreads();
-        masked_scores<DV>(dA, nullptr, Ds, Vs, bcum, C);           // dA = (dO V^T) * D ; A still raw
-        __syncthreads();
-        if (threadIdx.x < C) {                                     // row sums of M = dA * raw
-            const int r = threadIdx.x;
-            float s = 0.f;
-            for (int s0 = 0; s0 <= r; ++s0) s = fmaf(dA[r * C + s0], A[r * C + s0], s);
-            rs[r] = s;
-        } else if (threadIdx.x < 2 * C) {                          // column sums of M
-            const int s0 = threadIdx.x - C;
-            float s = 0.f;
-            for (int r = s0; r < C; ++r) s = fmaf(dA[r * C + s0], A[r * C + s0], s);
-            cs[s0] = s;
-        }
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < C * C; idx += NT) {      // A <- masked
-            const int r = idx / C, s = idx - r * C;
-            A[idx] = (s <= r) ? A[idx] * __expf(bcum[r] - bcum[s]) : 0.f;
-        }
+        masked_scores<DK>(A, nullptr, Qs, Ks, bcum, C);            // A  = (Q K^T) * D
+        masked_scores<DV>(dA, nullptr, Ds, Vs, bcum, C);           // dA = (dO V^T) * D
         __syncthreads();
         for (int idx = threadIdx.x; idx < C * DV; idx += NT) {     // dv
             const int s = idx / DV, jv = idx - s * DV;
@@ -343,23 +319,16 @@ __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __re
                 const int jv = (j0 + i) & (DV - 1);
                 inter = fmaf(Vs[s * DV + jv], G[i * DV + jv], inter);
             }
-            inter *= wsuf[s];
-            dk[qk_off + (t0 + s) * p.tqk + i] = from_f32<T>(intra + inter);
-            Ks[idx] *= inter;                       // k_s[i] * dk_inter_s[i], reduced below
+            const float tot = intra + wsuf[s] * inter;
+            dk[qk_off + (t0 + s) * p.tqk + i] = from_f32<T>(tot);
+            Ks[idx] *= tot;                         // k_s[i] * dk_s[i], reduced below
         }
         __syncthreads();
         if (threadIdx.x < C) {
             const int s = threadIdx.x;
             float kd = 0.f;
             for (int i0 = 0; i0 < DK; ++i0) kd += Ks[s * DK + ((i0 + s) & (DK - 1))];
-            xkh[t0 + s] = rs[s] - cs[s] - kd;
-            cs[s] = kd;                              // reuse as the per-token inter term
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            float s = 0.f;
-            for (int r = 0; r < C; ++r) s += cs[r];
-            dch[c0 + c] = s;
+            xkh[t0 + s] = kd;
         }
         // STB: G <- exp(bC) G + sum_r exp(b_r) q_r^T dO_r
         {
@@ -378,7 +347,7 @@ __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __re
 template <int DK, int DV> constexpr size_t smem_aggregate() { return sizeof(float) * (MAXC * DK + MAXC * DV + MAXC + 2 * MAXR); }
 template <int DK, int DV> constexpr size_t smem_fwd_out()   { return sizeof(float) * (2 * MAXC * DK + MAXC * DV + MAXC * MAXC + DK * DV + 3 * MAXC); }
 template <int DK, int DV> constexpr size_t smem_bwd_dq()    { return sizeof(float) * (2 * MAXC * DK + 2 * MAXC * DV + MAXC * MAXC + DK * DV + 3 * MAXC); }
-template <int DK, int DV> constexpr size_t smem_bwd_dkdv()  { return sizeof(float) * (2 * MAXC * DK + 2 * MAXC * DV + 2 * MAXC * MAXC + DK * DV + 5 * MAXC); }
+template <int DK, int DV> constexpr size_t smem_bwd_dkdv()  { return sizeof(float) * (2 * MAXC * DK + 2 * MAXC * DV + 2 * MAXC * MAXC + DK * DV + 3 * MAXC); }
 
 }  // namespace simt
 }  // namespace sf

@@ -217,6 +217,436 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     if (warp == 4) ptx::tmem_dealloc(tmem, 128);
 }
 
+// ==================================================================================================
+// Pieces shared by the two chunk-sweep kernels.
+//
+// TMEM accumulators of token-row results (M = 64) occupy lanes 0-15 of each 32-lane quarter, so two of
+// them are interleaved in the same columns: X at lane offset 0, Y at lane offset 16.  Warp w, lane l
+// then sees row 16w + (l & 15) of X (l < 16) or of Y (l >= 16).
+
+// Stores one 16-byte unit (8 bf16) of row `row`, unit index `unit` (0..7) of a [rows x 64] box.
+__device__ __forceinline__ void st_unit(unsigned char* box, int row, int unit, uint4 v) {
+    *reinterpret_cast<uint4*>(box + row * 128 + ((unit ^ (row & 7)) << 4)) = v;
+}
+__device__ __forceinline__ uint4 ld_unit(const unsigned char* box, int row, int unit) {
+    return *reinterpret_cast<const uint4*>(box + row * 128 + ((unit ^ (row & 7)) << 4));
+}
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// dst = diag(w) * src for a [64 x 128] tile (two boxes); w_row(row) gives the weight of a token row.
+template <typename F>
+__device__ __forceinline__ void scale_tile(unsigned char* dst, const unsigned char* src, F w_row) {
+    const uint4* in = reinterpret_cast<const uint4*>(src);
+    uint4* out = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int pos = threadIdx.x + NCOMP * i;
+        const float w = w_row((pos >> 3) & 63);
+        uint4 v = in[pos];
+        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h2[e]);
+            h2[e] = __floats2bfloat162_rn(f.x * w, f.y * w);
+        }
+        out[pos] = v;
+    }
+}
+
+// Decay mask on a [64 x 64] score accumulator pair at TMEM columns `sc`: lanes < 16 turn accumulator X
+// into dst0, lanes >= 16 accumulator Y into dst1 (skipped if dst1 == nullptr):
+//   dst[r][s] = bf16( acc[r][s] * exp(b_r - b_s) )  for s <= r, else 0        (row-major, one box)
+__device__ __forceinline__ void mask_pass(uint32_t sc, const float* bch, unsigned char* dst0, unsigned char* dst1) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = 16 * warp + (lane & 15);
+    unsigned char* dst = lane < 16 ? dst0 : dst1;
+    const float br = bch[r] * LOG2E;
+#pragma unroll
+    for (int cb = 0; cb < 2; ++cb) {
+        float v[32];
+        ptx::tmem_ld32(sc + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+        ptx::tmem_ld_wait();
+        if (dst) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int s0 = cb * 32 + u * 8 + 2 * e;
+                    const float m0 = s0 <= r ? v[u * 8 + 2 * e] * exp2f(br - bch[s0] * LOG2E) : 0.f;
+                    const float m1 = s0 + 1 <= r ? v[u * 8 + 2 * e + 1] * exp2f(br - bch[s0 + 1] * LOG2E) : 0.f;
+                    w[e] = pack2(m0, m1);
+                }
+                st_unit(dst, r, cb * 4 + u, make_uint4(w[0], w[1], w[2], w[3]));
+            }
+        }
+    }
+}
+
+// State pass for a [128 x 128] float32 accumulator at TMEM columns `acc` (thread tid owns lane tid):
+// writes its bf16 copy to `sb` (two boxes of [128 rows x 64 columns], 16 KB apart) and scales the
+// accumulator by `decay`.  If init != nullptr the state is first taken from global memory
+// (init[a*128 + i], or init[i*128 + a] when `transposed`) instead of TMEM.
+__device__ __forceinline__ void state_pass(uint32_t acc, unsigned char* sb, float decay, const float* __restrict__ init, bool transposed) {
+    const int a = threadIdx.x, warp = a >> 5;
+    const uint32_t taddr = acc + ((uint32_t)(warp * 32) << 16);
+#pragma unroll
+    for (int cb = 0; cb < 4; ++cb) {
+        float v[32];
+        if (init) {
+            if (transposed) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = init[(cb * 32 + i) * D + a];
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                    const float4 f = *reinterpret_cast<const float4*>(init + a * D + cb * 32 + i);
+                    v[i] = f.x; v[i + 1] = f.y; v[i + 2] = f.z; v[i + 3] = f.w;
+                }
+            }
+        } else {
+            ptx::tmem_ld32(taddr + cb * 32, v);
+            ptx::tmem_ld_wait();
+        }
+        unsigned char* box = sb + (cb >> 1) * 16384;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            st_unit(box, a, (cb & 1) * 4 + u,
+                    make_uint4(pack2(v[u * 8], v[u * 8 + 1]), pack2(v[u * 8 + 2], v[u * 8 + 3]), pack2(v[u * 8 + 4], v[u * 8 + 5]),
+                               pack2(v[u * 8 + 6], v[u * 8 + 7])));
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] *= decay;
+        ptx::tmem_st32(taddr + cb * 32, v);
+    }
+    ptx::tmem_st_wait();
+}
+
+// Epilogue of an interleaved accumulator pair at TMEM columns `pair`: out[r][:] = X[r][:] + scale_r * Y[r][:]
+// as bf16 to global row pointers, and (ROWDOT) dot_r = sum_c out[r][c] * e[r][c] with e a [64 x 128]
+// bf16 tile in shared memory.  Each lane handles 16 of every 32 columns; lane l and l+16 share row r.
+template <bool ROWDOT>
+__device__ __forceinline__ float pair_epilogue(uint32_t pair, float scale, __nv_bfloat16* __restrict__ out_row, const unsigned char* etile) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = 16 * warp + (lane & 15);
+    const bool upper = lane >= 16;
+    float dot = 0.f;
+#pragma unroll
+    for (int cb = 0; cb < 4; ++cb) {
+        float v[32];
+        ptx::tmem_ld32(pair + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+        ptx::tmem_ld_wait();
+        float res[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float send = upper ? v[i] : v[16 + i];
+            const float recv = __shfl_xor_sync(0xffffffffu, send, 16);
+            const float x = upper ? recv : v[i];
+            const float y = upper ? v[16 + i] : recv;
+            res[i] = fmaf(scale, y, x);
+        }
+        const int col = cb * 32 + (upper ? 16 : 0);
+        if (ROWDOT) {
+            const unsigned char* box = etile + (col >> 6) * BOX;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const uint4 ev = ld_unit(box, r, ((col & 63) >> 3) + u);
+                const __nv_bfloat162* e2 = reinterpret_cast<const __nv_bfloat162*>(&ev);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __bfloat1622float2(e2[e]);
+                    dot = fmaf(res[u * 8 + 2 * e], f.x, dot);
+                    dot = fmaf(res[u * 8 + 2 * e + 1], f.y, dot);
+                }
+            }
+        }
+        uint4* dst = reinterpret_cast<uint4*>(out_row + col);
+        dst[0] = make_uint4(pack2(res[0], res[1]), pack2(res[2], res[3]), pack2(res[4], res[5]), pack2(res[6], res[7]));
+        dst[1] = make_uint4(pack2(res[8], res[9]), pack2(res[10], res[11]), pack2(res[12], res[13]), pack2(res[14], res[15]));
+    }
+    if (ROWDOT) dot += __shfl_xor_sync(0xffffffffu, dot, 16);
+    return dot;
+}
+
+// K-major descriptor of a [rows x 128] tile for K step ks (0..7): features 16*ks .. 16*ks+15.
+__device__ __forceinline__ uint64_t kdesc(uint32_t tile, int ks, uint32_t box_bytes) {
+    return ptx::smem_desc(tile + (ks >> 2) * box_bytes + (ks & 3) * 32, 0);
+}
+// MN-major descriptor of a tile whose rows are the contraction index, K step ks = rows 16*ks .. 16*ks+15.
+__device__ __forceinline__ uint64_t mndesc(uint32_t tile, int ks, uint32_t box_bytes) {
+    return ptx::smem_desc(tile + ks * 2048, box_bytes);
+}
+
+// ==================================================================================================
+// Chunk sweep with a forward-running state (Out + ST of paper Eq. 2; SR + OG of Section 3.4).
+// With tile roles (xq, xk, xv) and the state St[a][b] = sum xk[.][a] * xv[.][b]:
+//     out_r = sum_{s<=r} (xq_r . xk_s) D[r,s] xv_s  +  exp(b_r) * xq_r St_c ;   St_{c+1} = exp(b_C) St_c + xk^T diag(w) xv
+//   forward output pass : (xq, xk, xv) = (q, k, v),  St = H (from Hs[j]),      out = o
+//   dq pass             : (xq, xk, xv) = (dO, v, k), St = H^T (Hs[j] transposed), out = dq, and
+//                         xout[t] = q_t . dq_t (float32) with q as a fourth tile
+constexpr int SW_STAGES = 2;
+template <int NTILES>
+struct SweepSmem {
+    alignas(1024) unsigned char tiles[SW_STAGES][NTILES][TILE];
+    alignas(1024) unsigned char xvw[TILE];
+    alignas(1024) unsigned char am[BOX];
+    alignas(1024) unsigned char sb[2 * 16384];
+    float bloc[MAXR * C];
+    float ctot[MAXR];
+    uint64_t full[SW_STAGES], empty[SW_STAGES], sc_done, ops_ready, out_done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <bool DQ>
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                const __grid_constant__ CUtensorMap tmE, SegParams p, const float* __restrict__ g, const float* __restrict__ Hs,
+                __nv_bfloat16* __restrict__ out, long long out_tok, long long out_bat, float* __restrict__ xout, int* status) {
+    constexpr int NTILES = DQ ? 4 : 3;
+    using Smem = SweepSmem<NTILES>;
+    extern __shared__ unsigned char smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
+    const long long t0 = (long long)c0 * C;
+    volatile int* abort_flag = &sm.abort_flag;
+    constexpr uint32_t T_ST = 0, T_O = 128, T_SC = 256;
+
+    if (tid == 0) {
+        sm.abort_flag = 0;
+        for (int s = 0; s < SW_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1 + NCOMP); }
+        ptx::mbar_init(&sm.sc_done, 1);
+        ptx::mbar_init(&sm.ops_ready, NCOMP);
+        ptx::mbar_init(&sm.out_done, 1);
+        ptx::fence_mbar_init();
+    }
+    if (warp == 4) ptx::tmem_alloc(&sm.tmem_base, 512);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
+            if (DQ) ptx::prefetch_tmap(&tmE);
+            for (int c = 0; c < nch; ++c) {
+                const int s = c % SW_STAGES, it = c / SW_STAGES;
+                if (it > 0) ptx::mbar_wait(&sm.empty[s], (it - 1) & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+                ptx::mbar_expect_tx(&sm.full[s], NTILES * TILE);
+                const int tok = (int)t0 + c * C;
+                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
+                if (DQ) tma_tile(sm.tiles[s][NTILES - 1], &tmE, &sm.full[s], h, tok, b);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
+            constexpr uint32_t id_o1 = ptx::idesc_bf16(64, 128, 0, 1);
+            constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
+            const uint32_t am = ptx::smem_u32(sm.am), sb = ptx::smem_u32(sm.sb), xvw = ptx::smem_u32(sm.xvw);
+            for (int c = 0; c < nch; ++c) {
+                const int s = c % SW_STAGES, it = c / SW_STAGES;
+                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]), xv = ptx::smem_u32(sm.tiles[s][2]);
+                // scores of this chunk (the accumulator was released by the previous ops_ready)
+                ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
+                ptx::tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
+                ptx::mma_commit(&sm.sc_done);
+                ptx::mbar_wait(&sm.ops_ready, c & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                // O1 = Am xv   (lanes +0)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_O, kdesc(am, ks, BOX), mndesc(xv, ks, BOX), id_o1, ks > 0);
+                // O2 = xq St   (lanes +16)
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_O + (16u << 16), kdesc(xq, ks, BOX), mndesc(sb, ks, 16384), id_o1, ks > 0);
+                // St += xk^T (w xv)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_ST, mndesc(xk, ks, BOX), mndesc(xvw, ks, BOX), id_st, 1u);
+                ptx::mma_commit(&sm.out_done);
+                ptx::mma_commit(&sm.empty[s]);
+            }
+        }
+    } else {
+        const float* gh = g + (long long)b * p.bg + h;
+        prep_decay(gh, p.tg, t0, nch, sm.bloc, sm.ctot);
+        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
+        const int r = 16 * warp + (lane & 15);
+        __nv_bfloat16* out_h = out + (long long)b * out_bat + (long long)h * D;
+        float* xo = DQ ? xout + ((long long)b * p.H + h) * p.L : nullptr;
+        for (int c = 0; c < nch; ++c) {
+            const int s = c % SW_STAGES, it = c / SW_STAGES;
+            const float* bch = sm.bloc + c * C;
+            const float bC = sm.ctot[c];
+            ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
+            scale_tile(sm.xvw, sm.tiles[s][2], [&](int row) { return fast_exp(bC - bch[row]); });
+            state_pass(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ);
+            ptx::mbar_wait(&sm.sc_done, c & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+            ptx::tc_fence_after_sync();
+            mask_pass(tmem + T_SC, bch, sm.am, nullptr);
+            ptx::fence_proxy_async();
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&sm.ops_ready);
+            ptx::mbar_wait(&sm.out_done, c & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+            ptx::tc_fence_after_sync();
+            const long long tok = t0 + c * C + r;
+            const float dot = pair_epilogue<DQ>(tmem + T_O, fast_exp(bch[r]), out_h + tok * out_tok, sm.tiles[s][NTILES - 1]);
+            if (DQ && lane < 16) xo[tok] = dot;
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&sm.empty[s]);
+        }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) ptx::tmem_dealloc(tmem, 512);
+}
+
+// ==================================================================================================
+// dk/dv pass (STB inside the block + PG, Section 3.4): reverse chunk sweep carrying G = dH (the
+// gradient w.r.t. the state leaving the chunk, from Gs[j]):
+//     A = (Q K^T) D,  dA = (dO V^T) D
+//     dv_s = sum_{r>=s} A[r,s] dO_r + w_s k_s G ;   dk_s = sum_{r>=s} dA[r,s] q_r + w_s v_s G^T ;   w_s = exp(b_C - b_s)
+//     G <- exp(b_C) G + (diag(exp(b)) Q)^T dO
+// and xk[t] = k_t . dk_t (float32).
+struct DkdvSmem {
+    alignas(1024) unsigned char tiles[SW_STAGES][4][TILE];     // q, k, v, dO
+    alignas(1024) unsigned char qw[TILE];
+    alignas(1024) unsigned char am[BOX];
+    alignas(1024) unsigned char dam[BOX];
+    alignas(1024) unsigned char gb[2 * 16384];
+    float bloc[MAXR * C];
+    float ctot[MAXR];
+    uint64_t full[SW_STAGES], empty[SW_STAGES], sc_done, ops_ready, out_done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+               const __grid_constant__ CUtensorMap tmD, SegParams p, const float* __restrict__ g, const float* __restrict__ Gs,
+               __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, float* __restrict__ xk, int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    DkdvSmem& sm = *reinterpret_cast<DkdvSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
+    const long long t0 = (long long)c0 * C;
+    volatile int* abort_flag = &sm.abort_flag;
+    constexpr uint32_t T_G = 0, T_DK = 128, T_DV = 256, T_SC = 384;
+
+    if (tid == 0) {
+        sm.abort_flag = 0;
+        for (int s = 0; s < SW_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1 + NCOMP); }
+        ptx::mbar_init(&sm.sc_done, 1);
+        ptx::mbar_init(&sm.ops_ready, NCOMP);
+        ptx::mbar_init(&sm.out_done, 1);
+        ptx::fence_mbar_init();
+    }
+    if (warp == 4) ptx::tmem_alloc(&sm.tmem_base, 512);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;
+
+    // iteration i handles chunk c = nch-1-i
+    if (warp == 4) {
+        if (lane == 0) {
+            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); ptx::prefetch_tmap(&tmD);
+            for (int i = 0; i < nch; ++i) {
+                const int s = i % SW_STAGES, it = i / SW_STAGES;
+                if (it > 0) ptx::mbar_wait(&sm.empty[s], (it - 1) & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+                ptx::mbar_expect_tx(&sm.full[s], 4 * TILE);
+                const int tok = (int)t0 + (nch - 1 - i) * C;
+                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][3], &tmD, &sm.full[s], h, tok, b);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
+            constexpr uint32_t id_tt = ptx::idesc_bf16(64, 128, 1, 1);     // A^T-type: both operands token-major
+            constexpr uint32_t id_kn = ptx::idesc_bf16(64, 128, 0, 1);     // K G
+            constexpr uint32_t id_kk = ptx::idesc_bf16(64, 128, 0, 0);     // V G^T
+            constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
+            const uint32_t am = ptx::smem_u32(sm.am), dam = ptx::smem_u32(sm.dam), gb = ptx::smem_u32(sm.gb), qw = ptx::smem_u32(sm.qw);
+            for (int i = 0; i < nch; ++i) {
+                const int s = i % SW_STAGES, it = i / SW_STAGES;
+                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
+                const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
+                ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
+                ptx::tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC + (16u << 16), kdesc(xd, ks, BOX), kdesc(xv, ks, BOX), id_sc, ks > 0);
+                ptx::mma_commit(&sm.sc_done);
+                ptx::mbar_wait(&sm.ops_ready, i & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                // dv1 = A^T dO (lanes +0), dv2 = K G (lanes +16)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DV, mndesc(am, ks, BOX), mndesc(xd, ks, BOX), id_tt, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DV + (16u << 16), kdesc(xk, ks, BOX), mndesc(gb, ks, 16384), id_kn, ks > 0);
+                // dk1 = dA^T Q (lanes +0), dk2 = V G^T (lanes +16)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DK, mndesc(dam, ks, BOX), mndesc(xq, ks, BOX), id_tt, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
+                // G += (diag(exp(b)) Q)^T dO
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
+                ptx::mma_commit(&sm.out_done);
+                ptx::mma_commit(&sm.empty[s]);
+            }
+        }
+    } else {
+        const float* gh = g + (long long)b * p.bg + h;
+        prep_decay(gh, p.tg, t0, nch, sm.bloc, sm.ctot);
+        const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
+        const int r = 16 * warp + (lane & 15);
+        __nv_bfloat16* dk_h = dk + (long long)b * p.bqk + (long long)h * D;
+        __nv_bfloat16* dv_h = dv + (long long)b * p.bv + (long long)h * D;
+        float* xo = xk + ((long long)b * p.H + h) * p.L;
+        for (int i = 0; i < nch; ++i) {
+            const int c = nch - 1 - i;
+            const int s = i % SW_STAGES, it = i / SW_STAGES;
+            const float* bch = sm.bloc + c * C;
+            const float bC = sm.ctot[c];
+            ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
+            scale_tile(sm.qw, sm.tiles[s][0], [&](int row) { return fast_exp(bch[row]); });
+            state_pass(tmem + T_G, sm.gb, fast_exp(bC), i == 0 ? G0 : nullptr, false);
+            ptx::mbar_wait(&sm.sc_done, i & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+            ptx::tc_fence_after_sync();
+            mask_pass(tmem + T_SC, bch, sm.am, sm.dam);
+            ptx::fence_proxy_async();
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&sm.ops_ready);
+            ptx::mbar_wait(&sm.out_done, i & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+            ptx::tc_fence_after_sync();
+            const long long tok = t0 + c * C + r;
+            const float w = fast_exp(bC - bch[r]);
+            pair_epilogue<false>(tmem + T_DV, w, dv_h + tok * p.tv, nullptr);
+            const float dot = pair_epilogue<true>(tmem + T_DK, w, dk_h + tok * p.tqk, sm.tiles[s][1]);
+            if (lane < 16) xo[tok] = dot;
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&sm.empty[s]);
+        }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) ptx::tmem_dealloc(tmem, 512);
+}
+
 // ---- host launch -------------------------------------------------------------------------------------
 template <typename K>
 inline bool opt_in_smem(K kern, size_t bytes) {
@@ -237,23 +667,49 @@ inline int* status_ptr() {
 // role: 0 aggregate, 1 forward output pass, 2 dq pass, 3 dk/dv pass (same order as the host's Role enum)
 inline sf_status_t launch(int role, const sf_seg_desc_t* d, const SegParams& p, const void* q, const void* k, const void* v,
                           const void* dO, const float* g, int mode, float* U, float* beta, const float* states, void* o,
-                          void* dq, void* dk, void* dv, float* xq, float* xk, float* dc, cudaStream_t st, long long* n_launch) {
+                          void* dq, void* dk, void* dv, float* xq, float* xk, cudaStream_t st, long long* n_launch) {
     int* status = status_ptr();
     if (!status) return SF_ERR_CUDA;
     dim3 grid(p.NB, p.H, p.B), block(NTHREADS);
+    auto map_qk = [&](CUtensorMap* m, const void* base) { return make_tmap(m, base, p.B, p.L, p.H, p.tqk, p.bqk); };
+    auto map_v = [&](CUtensorMap* m, const void* base) { return make_tmap(m, base, p.B, p.L, p.H, p.tv, p.bv); };
     if (role == 0) {
         CUtensorMap tmX, tmY;
-        const void* X = mode == 0 ? k : q;
-        const void* Y = mode == 0 ? v : dO;
-        if (!make_tmap(&tmX, X, p.B, p.L, p.H, p.tqk, p.bqk) || !make_tmap(&tmY, Y, p.B, p.L, p.H, p.tv, p.bv)) return SF_ERR_CUDA;
+        if (!map_qk(&tmX, mode == 0 ? k : q) || !map_v(&tmY, mode == 0 ? v : dO)) return SF_ERR_CUDA;
         constexpr size_t smem = sizeof(AggSmem) + 1024;
         static bool ok = opt_in_smem(tc_aggregate_kernel, smem);
         if (!ok) return SF_ERR_CUDA;
         tc_aggregate_kernel<<<grid, block, smem, st>>>(tmX, tmY, p, g, mode, U, beta, status);
-        *n_launch += 1;
-        return cudaGetLastError() == cudaSuccess ? SF_OK : SF_ERR_CUDA;
+    } else if (role == 1) {
+        CUtensorMap tq, tk, tv;
+        if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v)) return SF_ERR_CUDA;
+        constexpr size_t smem = sizeof(SweepSmem<3>) + 1024;
+        static bool ok = opt_in_smem(tc_sweep_kernel<false>, smem);
+        if (!ok) return SF_ERR_CUDA;
+        tc_sweep_kernel<false><<<grid, block, smem, st>>>(tq, tk, tv, tq, p, g, states, static_cast<__nv_bfloat16*>(o), p.tv, p.bv,
+                                                          nullptr, status);
+    } else if (role == 2) {
+        CUtensorMap tq, tk, tv, td;
+        if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;
+        constexpr size_t smem = sizeof(SweepSmem<4>) + 1024;
+        static bool ok = opt_in_smem(tc_sweep_kernel<true>, smem);
+        if (!ok) return SF_ERR_CUDA;
+        // roles: xq = dO, xk = v, xv = k, extra = q
+        tc_sweep_kernel<true><<<grid, block, smem, st>>>(td, tv, tk, tq, p, g, states, static_cast<__nv_bfloat16*>(dq), p.tqk, p.bqk,
+                                                         xq, status);
+    } else if (role == 3) {
+        CUtensorMap tq, tk, tv, td;
+        if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;
+        constexpr size_t smem = sizeof(DkdvSmem) + 1024;
+        static bool ok = opt_in_smem(tc_dkdv_kernel, smem);
+        if (!ok) return SF_ERR_CUDA;
+        tc_dkdv_kernel<<<grid, block, smem, st>>>(tq, tk, tv, td, p, g, states, static_cast<__nv_bfloat16*>(dk),
+                                                  static_cast<__nv_bfloat16*>(dv), xk, status);
+    } else {
+        return SF_ERR_UNSUPPORTED;
     }
-    return SF_ERR_UNSUPPORTED;
+    *n_launch += 1;
+    return cudaGetLastError() == cudaSuccess ? SF_OK : SF_ERR_CUDA;
 }
 
 }  // namespace tc

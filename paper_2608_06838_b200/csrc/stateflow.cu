@@ -63,10 +63,10 @@ SegParams make_params(const sf_seg_desc_t* d, int cpb_override = 0) {
 // ---- workspace layout -------------------------------------------------------------------------
 // forward           : [beta B*H*NB f32][UH B*H*NB*dk*dv f32]       UH: block aggregates, scanned in place
 //                                                                   into block-entering states
-// backward (saved)  : [GU B*H*NB*dk*dv][xq B*H*L][xk B*H*L][dc B*H*NC]
+// backward (saved)  : [GU B*H*NB*dk*dv][xq B*H*L][xk B*H*L]
 // backward (replay) : backward (saved) ++ forward ++ [Sfin B*H*dk*dv]
 struct FwdWs { float* beta; float* UH; size_t bytes; };
-struct BwdWs { float* GU; float* xq; float* xk; float* dc; size_t bytes; };
+struct BwdWs { float* GU; float* xq; float* xk; size_t bytes; };
 
 FwdWs fwd_ws(const sf_seg_desc_t* d, const SegParams& p, void* base) {
     FwdWs w;
@@ -87,7 +87,6 @@ BwdWs bwd_ws(const sf_seg_desc_t* d, const SegParams& p, void* base) {
     w.GU = reinterpret_cast<float*>(c + off); off += align_up(bh * p.NB * (size_t)d->d_k * d->d_v * sizeof(float));
     w.xq = reinterpret_cast<float*>(c + off); off += align_up(bh * p.L * sizeof(float));
     w.xk = reinterpret_cast<float*>(c + off); off += align_up(bh * p.L * sizeof(float));
-    w.dc = reinterpret_cast<float*>(c + off); off += align_up(bh * p.NC * sizeof(float));
     w.bytes = off;
     return w;
 }
@@ -122,7 +121,7 @@ struct RoleArgs {
     float *U, *beta;          // Aggregate outputs
     const float* states;      // FwdOut/BwdDq: Hs ; BwdDkDv: Gs
     void *o, *dq, *dk, *dv;
-    float *xq, *xk, *dc;
+    float *xq, *xk;
 };
 
 template <typename T, int DK, int DV>
@@ -162,7 +161,7 @@ sf_status_t launch_simt(Role role, const SegParams& p, const RoleArgs& a, cudaSt
             SF_TRY(set_smem(kern, sm));
             kern<<<grid, block, sm, st>>>(p, static_cast<const T*>(a.q), static_cast<const T*>(a.k),
                                           static_cast<const T*>(a.v), a.g, static_cast<const T*>(a.dO), a.states,
-                                          static_cast<T*>(a.dk), static_cast<T*>(a.dv), a.xk, a.dc);
+                                          static_cast<T*>(a.dk), static_cast<T*>(a.dv), a.xk);
             break;
         }
     }
@@ -174,7 +173,9 @@ sf_status_t launch_simt_d(Role role, const sf_seg_desc_t* d, const SegParams& p,
     if (d->d_k == 32 && d->d_v == 32) return launch_simt<T, 32, 32>(role, p, a, st);
     if (d->d_k == 64 && d->d_v == 64) return launch_simt<T, 64, 64>(role, p, a, st);
     if (d->d_k == 32 && d->d_v == 64) return launch_simt<T, 32, 64>(role, p, a, st);
-    if (d->d_k == 128 && d->d_v == 128) return launch_simt<T, 128, 128>(role, p, a, st);
+    if constexpr (sizeof(T) == 4) {
+        if (d->d_k == 128 && d->d_v == 128) return launch_simt<T, 128, 128>(role, p, a, st);
+    }
     return SF_ERR_UNSUPPORTED;
 }
 
@@ -182,9 +183,9 @@ sf_status_t launch_role(Path path, Role role, const sf_seg_desc_t* d, const SegP
     if (path == Path::Tc) {
         long long n = 0;
         sf_status_t s = sf::tc::launch(static_cast<int>(role), d, p, a.q, a.k, a.v, a.dO, a.g, a.mode, a.U, a.beta, a.states,
-                                       a.o, a.dq, a.dk, a.dv, a.xq, a.xk, a.dc, st, &n);
+                                       a.o, a.dq, a.dk, a.dv, a.xq, a.xk, st, &n);
         g_launches.fetch_add(n, std::memory_order_relaxed);
-        if (s != SF_ERR_UNSUPPORTED) return s;      // DEV: roles not yet on tensor cores run on CUDA cores
+        return s;
     }
     if (d->dtype == SF_F32) return launch_simt_d<float>(role, d, p, a, st);
     return launch_simt_d<__nv_bfloat16>(role, d, p, a, st);
@@ -237,12 +238,12 @@ sf_status_t bwd_dq(Path path, const sf_seg_desc_t* d, const SegParams& p, const 
 }
 sf_status_t bwd_dkdv(Path path, const sf_seg_desc_t* d, const SegParams& p, const BwdPtrs& x, const BwdWs& w, cudaStream_t st) {
     RoleArgs a{};
-    a.q = x.q; a.k = x.k; a.v = x.v; a.dO = x.dO; a.g = x.g; a.states = w.GU; a.dk = x.dk; a.dv = x.dv; a.xk = w.xk; a.dc = w.dc;
+    a.q = x.q; a.k = x.k; a.v = x.v; a.dO = x.dO; a.g = x.g; a.states = w.GU; a.dk = x.dk; a.dv = x.dv; a.xk = w.xk;
     return launch_role(path, Role::BwdDkDv, d, p, a, st);
 }
 sf_status_t bwd_dg(const sf_seg_desc_t* d, const SegParams& p, const BwdPtrs& x, const BwdWs& w, const float* Hs, cudaStream_t st) {
     dim3 grid(p.NB, p.H, p.B);
-    sf::dg_epilogue_kernel<<<grid, sf::DG_NT, 0, st>>>(p, d->d_k * d->d_v, w.xq, w.xk, w.dc, Hs, w.GU, x.dS_in, x.dg);
+    sf::dg_epilogue_kernel<<<grid, sf::DG_NT, 0, st>>>(p, d->d_k * d->d_v, w.xq, w.xk, Hs, w.GU, x.dS_in, x.dg);
     return check_launch();
 }
 
