@@ -1,0 +1,298 @@
+#!/usr/bin/env python
+"""Benchmark: fwd+bwd tokens/s per linear-recurrence layer (chained segments, bf16) on B200.
+
+One "step" = sf_chain_fwd + sf_chain_bwd over the whole synthetic sequence of one configuration
+(all segments, state and state-gradient hand-offs included).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config {2,3,4,5}] [--seg-len L]
+  python bench.py --impl reference ...      times the fp64 CPU oracle on a bounded sample instead
+
+Multi-GPU: the path does not shard (replicas only): with --gpus N each rank runs the same workload on
+its own GPU, no data-path collective; value = N * tokens / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fwd+bwd tokens/s per linear-recurrence layer"
+UNIT = "tokens/s"
+BYTES_PER_TOKEN_HEAD = 2828          # q,k,v,dO read once, o,dq,dk,dv written once (bf16, d=128), g and dg float32
+DKDV_BYTES_PER_TOKEN_HEAD = 1540     # the dk/dv pass alone: q,k,v,dO + g in, dk,dv out
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def pick_workload(args):
+    from paper_2608_06838_b200 import inputs
+    if args.config == 5:
+        return inputs.sweep_config(args.seg_len)
+    return inputs.configs()[args.config - 1]
+
+
+def cpu_baseline(w, budget_tokens=2048):
+    """The oracle as it stands on the host cores, on the first `budget_tokens` tokens of the workload (all heads)."""
+    import numpy as np
+    import oracle
+    from paper_2608_06838_b200 import inputs
+    import dataclasses
+    ws = dataclasses.replace(w, seg_lens=[budget_tokens])
+    x = inputs.make_inputs(ws, "cpu")
+    f = inputs.to_f64
+    q, k, v, g, dO = (f(x[n]) for n in ("q", "k", "v", "g", "dO"))
+    t0 = time.perf_counter()
+    oracle.segment_fwd(q, k, v, g, f(x["S_in"]))
+    oracle.segment_bwd(q, k, v, g, f(x["S_in"]), dO, f(x["dS_out"]))
+    dt = time.perf_counter() - t0
+    return {"value": ws.B * budget_tokens / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "first %d tokens of the workload, all %d heads, unsplit, fwd+bwd, %.1f s" % (budget_tokens, w.H, dt)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = pick_workload(args)
+    import oracle
+    oracle.build()
+    vals = []
+    total = args.warmup + args.steps
+    budget = 1024 if total > 3 else 2048
+    for i in range(total):
+        r = cpu_baseline(w, budget)
+        if i >= args.warmup:
+            vals.append(r)
+    v = statistics.mean(x["value"] for x in vals)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * w.B * budget / v, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d_k, "d_v": w.d_v, "T": w.T, "chunk": w.chunk},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle", "sample": vals[-1]["sample"]},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
+    ap.add_argument("--seg-len", type=int, default=4096, help="segment length of configuration 5")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-overlap", action="store_true")
+    ap.add_argument("--chunks-per-block", type=int, default=0)
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2608_06838_b200 import binding, inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = "cuda:%d" % local
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    binding.load()
+
+    w = pick_workload(args)
+    x = inputs.make_inputs(w, dev)
+    run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk, args.chunks_per_block)
+    overlap = not args.no_overlap
+
+    def step():
+        run.forward(x["S_in"], overlap=overlap)
+        run.backward(x["dS_out"], overlap=overlap)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    n0 = binding.sf_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = binding.sf_launch_count() - n0
+    assert binding.sf_device_status() == 0, "a bounded device-side wait ran out"
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = ms / args.steps
+    tokens = w.B * w.T
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    # ---- per-stage device times (second pass with the library's stage timers on) -------------------
+    stage = None
+    if rank == 0:
+        binding.sf_stage_timing(True)
+        for _ in range(args.steps):
+            step()
+        torch.cuda.synchronize()
+        stage = binding.sf_stage_timing_read()
+        binding.sf_stage_timing(False)
+
+    # ---- end-to-end through the host-memory entry point ----------------------------------------------
+    e2e = None
+    if not args.skip_e2e:
+        host = {n: (None if t is None else t.detach().to("cpu").pin_memory()) for n, t in x.items()}
+        outs = {n: torch.empty_like(host[m]).pin_memory() for n, m in
+                [("o", "v"), ("dq", "q"), ("dk", "k"), ("dv", "v"), ("dg", "g")]}
+        S_final = torch.empty(w.B, w.H, w.d_k, w.d_v, dtype=torch.float32).pin_memory()
+        dS_init = torch.empty_like(S_final).pin_memory()
+        desc = binding.make_desc(host["q"], host["v"], host["g"], w.chunk, args.chunks_per_block, seg_len=w.seg_lens[0])
+        scratch = torch.empty(binding.sf_e2e_device_bytes(desc, w.seg_lens), dtype=torch.uint8, device=dev)
+
+        def e2e_step():
+            binding.sf_chain_fwd_bwd_host(desc, w.seg_lens, host["q"], host["k"], host["v"], host["g"], host["S_in"],
+                                          host["dO"], host["dS_out"], outs["o"], S_final, outs["dq"], outs["dk"], outs["dv"],
+                                          outs["dg"], dS_init, scratch)
+        e2e_step()
+        barrier()
+        n_e2e = max(2, min(args.steps, 5))
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            e2e_step()              # synchronises its stream before returning
+        dt = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([dt], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        nb = lambda t: 0 if t is None else t.numel() * t.element_size()
+        h2d = sum(nb(host[n]) for n in ("q", "k", "v", "g", "dO", "S_in", "dS_out"))
+        d2h = sum(nb(t) for t in outs.values()) + nb(S_final) + nb(dS_init)
+        e2e = {"value": world * tokens * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": 1e3 * dt / n_e2e}
+        del scratch
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = peaks()
+    roof = None
+    path_roof = {"bound": "hbm", "achieved": BYTES_PER_TOKEN_HEAD * tokens * w.H / (ms_per_step * 1e-3) / 1e9, "peak": peak,
+                 "unit": "GB/s", "peak_source": peak_kind,
+                 "note": "whole step: 2828 algorithmic bytes per token*head / step time"}
+    path_roof["frac"] = path_roof["achieved"] / peak
+    if stage:
+        dom = max(stage, key=lambda s: s["ms"])
+        per_launch_ms = dom["ms"] / max(dom["launches"], 1)
+        if dom["name"] == "dkdv":
+            alg = DKDV_BYTES_PER_TOKEN_HEAD * tokens * w.H / len(w.seg_lens)       # mean over this step's launches
+        else:
+            alg = None
+        roof = {"bound": "hbm", "kernel": dom["name"], "achieved": (alg / (per_launch_ms * 1e-3) / 1e9) if alg else None,
+                "peak": peak, "unit": "GB/s", "peak_source": peak_kind, "traffic": None,
+                "avg_launch_ms": per_launch_ms, "launches": dom["launches"]}
+        roof["frac"] = roof["achieved"] / peak if roof["achieved"] else None
+    cpu = None if args.skip_cpu else cpu_baseline(w)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d_k, "d_v": w.d_v, "T": w.T, "segments": w.seg_lens,
+                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or 16, "overlap": overlap,
+                   "l2": "inputs (%.0f MB) exceed L2, no flush" % (4 * tokens * w.H * w.d_k * 2 / 1e6),
+                   "parallelism": "replicas only"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roof, "path_roofline": path_roof,
+        "stages": stage, "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

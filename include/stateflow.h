@@ -188,8 +188,8 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
                                   float* dS_init, void* dev, size_t dev_bytes, sf_stream_t stream);
 
 /*
- * Device-side status word of the most recent kernels launched by this library on the current
- * device (host function, synchronises nothing: it reads a mapped host word).  0 means no bounded
+ * Device-side status word of the kernels launched by this library on the current device (host
+ * function; it copies one word from the device, which waits for prior work).  0 means no bounded
  * wait has run out since sf_device_status_clear().  Kernels never spin without a limit; when a
  * limit is hit they record a code here, stop waiting and return normally, leaving their outputs
  * undefined.  No counterpart in the paper.
@@ -199,6 +199,18 @@ void sf_device_status_clear(void);
 
 /* Number of kernels this library has launched in this process (host counter). No paper counterpart. */
 int64_t sf_launch_count(void);
+
+/*
+ * Per-stage device timers for profiling (host functions; no paper counterpart, the stages themselves
+ * are those of Eq. 2 and Section 3.4).  While enabled, every kernel launch is bracketed by two CUDA
+ * events on its own stream, which costs a little throughput, so leave it off when timing whole steps.
+ * sf_stage_timing_read synchronises the device, adds up the elapsed time and launch count of each
+ * stage since the last read into ms[0..n) / launches[0..n), forgets them and returns the number of
+ * stages: 0 block aggregate of (k, v), 1 block aggregate of (q, dO), 2 state scan, 3 forward output
+ * pass, 4 dq pass, 5 dk/dv pass, 6 log-decay gradient.
+ */
+void sf_stage_timing(int32_t enable);
+int32_t sf_stage_timing_read(float* ms, int64_t* launches, int32_t n);
 
 #ifdef __cplusplus
 }

@@ -72,6 +72,10 @@ def load() -> ctypes.CDLL:
         lib.sf_device_status.restype = i32
         lib.sf_device_status_clear.restype = None
         lib.sf_launch_count.restype = ctypes.c_int64
+        lib.sf_stage_timing.restype = None
+        lib.sf_stage_timing.argtypes = [i32]
+        lib.sf_stage_timing_read.restype = i32
+        lib.sf_stage_timing_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64), i32]
         _lib = lib
     return _lib
 
@@ -180,6 +184,21 @@ def sf_device_status_clear() -> None:
 
 def sf_launch_count() -> int:
     return int(load().sf_launch_count())
+
+
+STAGE_NAMES = ["agg_kv", "agg_qdo", "scan", "fwd_out", "dq", "dkdv", "dg"]
+
+
+def sf_stage_timing(enable: bool) -> None:
+    load().sf_stage_timing(int(enable))
+
+
+def sf_stage_timing_read():
+    n = len(STAGE_NAMES)
+    ms = (ctypes.c_float * n)()
+    cnt = (ctypes.c_int64 * n)()
+    load().sf_stage_timing_read(ms, cnt, n)
+    return [{"name": STAGE_NAMES[i], "ms": float(ms[i]), "launches": int(cnt[i])} for i in range(n)]
 
 
 # ---- conveniences built only from the calls above (allocation + one call each) --------------------

@@ -24,9 +24,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(2000u) : "memory");   // may sleep up to ~2 us in hardware
     return ok != 0;
 }
 
@@ -34,11 +34,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // CTA-wide sticky flag *abort_flag (shared) so that every later wait in this CTA returns at once.
 // The kernel then runs to its end on undefined data and releases its TMEM normally.
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+    if (mbar_try_wait(bar, parity)) return;
     if (*abort_flag) return;
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-        if ((it & 1023u) == 1023u) {
+        if ((it & 255u) == 255u) {
             if (*abort_flag) return;
             if (clock64() - t0 > 2000000000LL) {
                 *abort_flag = 1;
@@ -93,6 +94,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
+// 2^x with the single-instruction approximation (inputs here are <= 0 or moderate; flush-to-zero underflow is the wanted limit)
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// 16 lanes x 64 columns: thread t gets, for each group j of 8 columns, v[4j], v[4j+1] = (lane t/4, columns
+// 8j + 2(t%4), +1) and v[4j+2], v[4j+3] = (lane t/4 + 8, same columns) - the layout of an M = 64 accumulator
+// row block, spread over all 32 threads of the warp.
+__device__ __forceinline__ void tmem_ld_16x64(uint32_t taddr, float* v) {
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
     const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
@@ -117,13 +139,11 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 //   MN-major (rows = K index, the 64 columns = M/N): 8-row K groups 1024 B apart (SBO); the next 64
 //            M/N elements live `lbo_bytes` away (the next box); a K step of 16 rows is +2048 B.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);             // start address   [0,14)
-    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;    // leading offset  [16,30)
-    d |= static_cast<uint64_t>(1024u >> 4) << 32;                    // stride offset   [32,46)
-    d |= static_cast<uint64_t>(1) << 46;                             // descriptor version (Blackwell)
-    d |= static_cast<uint64_t>(2) << 61;                             // SWIZZLE_128B
-    return d;
+    // low word: start address [0,14) and leading offset [16,30), both in 16-byte units
+    // high word: stride offset 1024 B [32,46), descriptor version 1 [46,48), SWIZZLE_128B = 2 [61,64)
+    const uint32_t lo = ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+    constexpr uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
 // Instruction descriptor for kind::f16 with bf16 operands and float32 accumulation.

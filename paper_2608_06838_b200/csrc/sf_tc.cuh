@@ -1,8 +1,8 @@
 // tcgen05 / TMEM / TMA kernels for the bf16, d_k = d_v = 128, chunk = 64 shape.
 //
 // Thread roles in every kernel here: warps 0-3 are the compute warpgroup (TMEM loads/stores, decay
-// masks, epilogues; warp w owns TMEM lanes 32w..32w+31), warp 4 lane 0 is the TMA producer, warp 5
-// lane 0 issues the MMAs.  All waits are bounded (see ptx::mbar_wait).
+// masks, epilogues; warp w owns TMEM lanes 32(w mod 4)..+31), then one TMA producer warp and one warp that
+// issues the MMAs (lane 0 each).  All waits are bounded (see ptx::mbar_wait).
 //
 // Shared-memory operand storage: every [64 tokens x 128 features] bf16 tile is two TMA boxes of
 // [64 rows x 64 columns] (128-byte rows, SWIZZLE_128B, 8 KB each, features 0-63 then 64-127).  The
@@ -10,6 +10,7 @@
 // over tokens (ptx::smem_desc).
 #pragma once
 #include <cuda.h>
+#include <cstdio>
 
 #include "../../include/stateflow.h"
 #include "sf_common.cuh"
@@ -19,6 +20,13 @@ namespace sf {
 namespace tc {
 
 __device__ int g_dev_status = 0;
+
+#ifdef SF_TRACE
+__device__ long long g_trace[8][64][4];
+#define SF_TR(role, c, e) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 31) == 0 && ((threadIdx.x >> 5) & 3) == 0) g_trace[role][c][e] = clock64(); } while (0)
+#else
+#define SF_TR(role, c, e) do { } while (0)
+#endif
 
 inline int read_device_status() {
     int v = 0;
@@ -34,12 +42,10 @@ constexpr int C = 64;              // chunk
 constexpr int D = 128;             // d_k = d_v
 constexpr int BOX = 8192;          // bytes of one [64 x 64] bf16 box
 constexpr int TILE = 2 * BOX;      // bytes of one [64 x 128] bf16 tile
-constexpr int NCOMP = 128;         // compute threads
-constexpr int NTHREADS = 192;
-constexpr int MAXR = 64;
+constexpr int MAXR = 32;           // largest chunks_per_block of the tensor-core path
 constexpr float LOG2E = 1.4426950408889634f;
 
-__device__ __forceinline__ float fast_exp(float x) { return exp2f(x * LOG2E); }
+__device__ __forceinline__ float fast_exp(float x) { return ptx::ex2(x * LOG2E); }
 
 // ---- host: tensor maps ---------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -81,12 +87,14 @@ __device__ __forceinline__ void tma_tile(void* dst, const CUtensorMap* m, uint64
     ptx::tma_load_4d(static_cast<char*>(dst) + BOX, m, bar, 64, h, t0, b);
 }
 
-// Decay tables of one block, by the 128 compute threads.  On return (after the named barrier):
+// Decay tables of one block, computed by `nwarps` warps (threads 0 .. 32*nwarps-1).  Callers
+// synchronise afterwards.
 //   bloc[t]  = inclusive cumulative log-decay of token t inside ITS chunk  (t = 0 .. nch*64-1)
 //   ctot[c]  = chunk totals
-__device__ __forceinline__ void prep_decay(const float* __restrict__ gh, long long tg, long long t0, int nch, float* bloc, float* ctot) {
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    for (int c = warp; c < nch; c += 4) {
+__device__ __forceinline__ void prep_decay(const float* __restrict__ gh, long long tg, long long t0, int nch, float* bloc, float* ctot,
+                                           int nwarps) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int c = warp; c < nch; c += nwarps) {
         const float g0 = gh[(t0 + c * C + 2 * lane) * tg];
         const float g1 = gh[(t0 + c * C + 2 * lane + 1) * tg];
         float incl = g0 + g1;
@@ -98,133 +106,8 @@ __device__ __forceinline__ void prep_decay(const float* __restrict__ gh, long lo
         bloc[c * C + 2 * lane + 1] = incl;
         if (lane == 31) ctot[c] = incl;
     }
-    ptx::named_bar_sync(1, NCOMP);
 }
 
-// ==================================================================================================
-// Block aggregates on tensor cores: U = sum_s w_s x_s^T y_s over the block (M = N = 128, K = tokens).
-//   mode 0: (x, y) = (k, v), w_s = exp(beta - B_s);   mode 1: (x, y) = (q, dO), w_s = exp(B_s)
-// y is scaled by w in place in shared memory, then U += X^T (w*Y) with both operands MN-major.
-constexpr int AGG_STAGES = 3;
-struct AggSmem {
-    alignas(1024) unsigned char tiles[AGG_STAGES][2][TILE];
-    float bloc[MAXR * C];
-    float ctot[MAXR];
-    float cofs[MAXR];
-    uint64_t full[AGG_STAGES], empty[AGG_STAGES], ready[AGG_STAGES], done;
-    uint32_t tmem_base;
-    int abort_flag;
-};
-
-__global__ void __launch_bounds__(NTHREADS, 1)
-tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, SegParams p,
-                    const float* __restrict__ g, int mode, float* __restrict__ U, float* __restrict__ beta_out, int* status) {
-    extern __shared__ unsigned char smem_raw[];
-    AggSmem& sm = *reinterpret_cast<AggSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
-    const long long t0 = (long long)c0 * C;
-    volatile int* abort_flag = &sm.abort_flag;
-
-    if (tid == 0) {
-        sm.abort_flag = 0;
-        for (int s = 0; s < AGG_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1); ptx::mbar_init(&sm.ready[s], NCOMP); }
-        ptx::mbar_init(&sm.done, 1);
-        ptx::fence_mbar_init();
-    }
-    if (warp == 4) ptx::tmem_alloc(&sm.tmem_base, 128);
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::tc_fence_after_sync();
-    const uint32_t tmem = sm.tmem_base;
-
-    if (warp == 4) {
-        if (lane == 0) {
-            ptx::prefetch_tmap(&tmX);
-            ptx::prefetch_tmap(&tmY);
-            for (int c = 0; c < nch; ++c) {
-                const int s = c % AGG_STAGES, it = c / AGG_STAGES;
-                if (it > 0) ptx::mbar_wait(&sm.empty[s], (it - 1) & 1, abort_flag, status, DEV_TIMEOUT_MMA);
-                ptx::mbar_expect_tx(&sm.full[s], 2 * TILE);
-                tma_tile(sm.tiles[s][0], &tmX, &sm.full[s], h, (int)t0 + c * C, b);
-                tma_tile(sm.tiles[s][1], &tmY, &sm.full[s], h, (int)t0 + c * C, b);
-            }
-        }
-    } else if (warp == 5) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16(128, 128, 1, 1);
-            for (int c = 0; c < nch; ++c) {
-                const int s = c % AGG_STAGES, it = c / AGG_STAGES;
-                ptx::mbar_wait(&sm.ready[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
-                ptx::tc_fence_after_sync();
-                const uint32_t xa = ptx::smem_u32(sm.tiles[s][0]), ya = ptx::smem_u32(sm.tiles[s][1]);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    ptx::mma_ss(tmem, ptx::smem_desc(xa + ks * 2048, BOX), ptx::smem_desc(ya + ks * 2048, BOX), idesc, (c > 0 || ks > 0) ? 1u : 0u);
-                ptx::mma_commit(&sm.empty[s]);
-            }
-            ptx::mma_commit(&sm.done);
-        }
-    } else {
-        const float* gh = g + (long long)b * p.bg + h;
-        prep_decay(gh, p.tg, t0, nch, sm.bloc, sm.ctot);
-        if (tid == 0) {
-            float acc = 0.f;
-            if (mode == 0) { for (int c = nch - 1; c >= 0; --c) { sm.cofs[c] = acc; acc += sm.ctot[c]; } }
-            else           { for (int c = 0; c < nch; ++c)      { sm.cofs[c] = acc; acc += sm.ctot[c]; } }
-            if (beta_out) beta_out[((long long)b * p.H + h) * p.NB + j] = acc;
-        }
-        ptx::named_bar_sync(1, NCOMP);
-        for (int c = 0; c < nch; ++c) {
-            const int s = c % AGG_STAGES, it = c / AGG_STAGES;
-            ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
-            const float cof = sm.cofs[c], bC = sm.ctot[c];
-            uint4* y = reinterpret_cast<uint4*>(sm.tiles[s][1]);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int pos = tid + NCOMP * i;              // 16-byte unit inside the tile
-                const int row = (pos >> 3) & 63;              // token row (each box holds 64 rows x 8 units)
-                const float bl = sm.bloc[c * C + row];
-                const float w = fast_exp(mode == 0 ? (bC - bl) + cof : bl + cof);
-                uint4 v = y[pos];
-                __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float2 f = __bfloat1622float2(h2[e]);
-                    h2[e] = __floats2bfloat162_rn(f.x * w, f.y * w);
-                }
-                y[pos] = v;
-            }
-            ptx::fence_proxy_async();
-            ptx::mbar_arrive(&sm.ready[s]);
-        }
-        ptx::mbar_wait(&sm.done, 0, abort_flag, status, DEV_TIMEOUT_MMA);
-        ptx::tc_fence_after_sync();
-        float* Uo = U + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D) + (long long)tid * D;
-#pragma unroll
-        for (int cb = 0; cb < 4; ++cb) {
-            float v[32];
-            ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 32; e += 4)
-                *reinterpret_cast<float4*>(Uo + cb * 32 + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
-        }
-        ptx::tc_fence_before_sync();
-    }
-    __syncthreads();
-    if (warp == 4) ptx::tmem_dealloc(tmem, 128);
-}
-
-// ==================================================================================================
-// Pieces shared by the two chunk-sweep kernels.
-//
-// TMEM accumulators of token-row results (M = 64) occupy lanes 0-15 of each 32-lane quarter, so two of
-// them are interleaved in the same columns: X at lane offset 0, Y at lane offset 16.  Warp w, lane l
-// then sees row 16w + (l & 15) of X (l < 16) or of Y (l >= 16).
-
-// Stores one 16-byte unit (8 bf16) of row `row`, unit index `unit` (0..7) of a [rows x 64] box.
 __device__ __forceinline__ void st_unit(unsigned char* box, int row, int unit, uint4 v) {
     *reinterpret_cast<uint4*>(box + row * 128 + ((unit ^ (row & 7)) << 4)) = v;
 }
@@ -236,138 +119,159 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// dst = diag(w) * src for a [64 x 128] tile (two boxes); w_row(row) gives the weight of a token row.
-template <typename F>
-__device__ __forceinline__ void scale_tile(unsigned char* dst, const unsigned char* src, F w_row) {
+// dst = diag(w) * src for a [64 x 128] tile (two boxes), done by NTHR threads (this one is `t`);
+// w_row(row) gives the weight of a token row.  dst may equal src.  A thread touches 16-byte units
+// t + NTHR*i; a box holds 64 rows x 8 units, so with NTHR = 256 it meets only rows (t>>3) and (t>>3)+32.
+template <int NTHR, typename F>
+__device__ __forceinline__ void scale_tile(unsigned char* dst, const unsigned char* src, int t, F w_row) {
+    static_assert(NTHR == 256, "unit-to-row mapping below assumes 256 threads");
     const uint4* in = reinterpret_cast<const uint4*>(src);
     uint4* out = reinterpret_cast<uint4*>(dst);
+    const float w0 = w_row(t >> 3), w1 = w_row((t >> 3) + 32);
+    uint4 v[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int pos = threadIdx.x + NCOMP * i;
-        const float w = w_row((pos >> 3) & 63);
-        uint4 v = in[pos];
-        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v);
+    for (int i = 0; i < 4; ++i) v[i] = in[t + NTHR * i];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float w = (i & 1) ? w1 : w0;
+        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v[i]);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float2 f = __bfloat1622float2(h2[e]);
             h2[e] = __floats2bfloat162_rn(f.x * w, f.y * w);
         }
-        out[pos] = v;
+        out[t + NTHR * i] = v[i];
     }
 }
 
-// Decay mask on a [64 x 64] score accumulator pair at TMEM columns `sc`: lanes < 16 turn accumulator X
-// into dst0, lanes >= 16 accumulator Y into dst1 (skipped if dst1 == nullptr):
+// TMEM accumulators of token-row results (M = 64) occupy lanes 0-15 of each 32-lane quarter, so two of
+// them are interleaved in the same columns: X at lane offset 0, Y at lane offset 16.  They are read
+// with the 16-lane load shape (ptx::tmem_ld_16x64): in the warp with index q (mod 4), thread t holds
+// rows 16q + t/4 and 16q + t/4 + 8, two adjacent columns out of every eight.
+
+// Decay mask on the [64 x 64] score accumulators at TMEM columns `sc`:
 //   dst[r][s] = bf16( acc[r][s] * exp(b_r - b_s) )  for s <= r, else 0        (row-major, one box)
+// X -> dst0 and, if dst1 != nullptr, Y -> dst1 (same mask).
 __device__ __forceinline__ void mask_pass(uint32_t sc, const float* bch, unsigned char* dst0, unsigned char* dst1) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int r = 16 * warp + (lane & 15);
-    unsigned char* dst = lane < 16 ? dst0 : dst1;
-    const float br = bch[r] * LOG2E;
+    const int q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
+    const int rA = 16 * q + (lane >> 2), rB = rA + 8, cq = 2 * (lane & 3);
+    const uint32_t taddr = sc + ((uint32_t)(q * 32) << 16);
+    float x[32], y[32];
+    ptx::tmem_ld_16x64(taddr, x);
+    if (dst1) ptx::tmem_ld_16x64(taddr + (16u << 16), y);
+    const float bA = bch[rA] * LOG2E, bB = bch[rB] * LOG2E;
+    ptx::tmem_ld_wait();
 #pragma unroll
-    for (int cb = 0; cb < 2; ++cb) {
-        float v[32];
-        ptx::tmem_ld32(sc + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
-        ptx::tmem_ld_wait();
-        if (dst) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                uint32_t w[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int s0 = cb * 32 + u * 8 + 2 * e;
-                    const float m0 = s0 <= r ? v[u * 8 + 2 * e] * exp2f(br - bch[s0] * LOG2E) : 0.f;
-                    const float m1 = s0 + 1 <= r ? v[u * 8 + 2 * e + 1] * exp2f(br - bch[s0 + 1] * LOG2E) : 0.f;
-                    w[e] = pack2(m0, m1);
-                }
-                st_unit(dst, r, cb * 4 + u, make_uint4(w[0], w[1], w[2], w[3]));
-            }
+    for (int j = 0; j < 8; ++j) {
+        const int s0 = 8 * j + cq;
+        const float2 bs = *reinterpret_cast<const float2*>(bch + s0);
+        const float e0 = -LOG2E * bs.x, e1 = -LOG2E * bs.y;
+        const float dA0 = s0 <= rA ? ptx::ex2(bA + e0) : 0.f, dA1 = s0 + 1 <= rA ? ptx::ex2(bA + e1) : 0.f;
+        const float dB0 = s0 <= rB ? ptx::ex2(bB + e0) : 0.f, dB1 = s0 + 1 <= rB ? ptx::ex2(bB + e1) : 0.f;
+        const int offA = rA * 128 + ((j ^ (rA & 7)) << 4) + 2 * cq, offB = rB * 128 + ((j ^ (rB & 7)) << 4) + 2 * cq;
+        *reinterpret_cast<uint32_t*>(dst0 + offA) = pack2(x[4 * j] * dA0, x[4 * j + 1] * dA1);
+        *reinterpret_cast<uint32_t*>(dst0 + offB) = pack2(x[4 * j + 2] * dB0, x[4 * j + 3] * dB1);
+        if (dst1) {
+            *reinterpret_cast<uint32_t*>(dst1 + offA) = pack2(y[4 * j] * dA0, y[4 * j + 1] * dA1);
+            *reinterpret_cast<uint32_t*>(dst1 + offB) = pack2(y[4 * j + 2] * dB0, y[4 * j + 3] * dB1);
         }
     }
 }
 
-// State pass for a [128 x 128] float32 accumulator at TMEM columns `acc` (thread tid owns lane tid):
-// writes its bf16 copy to `sb` (two boxes of [128 rows x 64 columns], 16 KB apart) and scales the
-// accumulator by `decay`.  If init != nullptr the state is first taken from global memory
-// (init[a*128 + i], or init[i*128 + a] when `transposed`) instead of TMEM.
-__device__ __forceinline__ void state_pass(uint32_t acc, unsigned char* sb, float decay, const float* __restrict__ init, bool transposed) {
-    const int a = threadIdx.x, warp = a >> 5;
+// State pass over the two column batches cb0, cb0+1 (32 columns each, cb0 even) of a [128 x 128] float32 accumulator at
+// TMEM columns `acc`; the thread owns lane a = threadIdx.x & 127.  Writes the bf16 copy of the state
+// to `sb` (two boxes of [128 rows x 64 columns], 16 KB apart) and scales the accumulator by `decay`.
+// If init != nullptr the state is taken from global memory (init[a*128 + i], or init[i*128 + a] when
+// `transposed`) instead of TMEM.
+__device__ __forceinline__ void state_pass(uint32_t acc, unsigned char* sb, float decay, const float* __restrict__ init, bool transposed,
+                                           int cb0) {
+    const int a = threadIdx.x & 127, warp = a >> 5;
     const uint32_t taddr = acc + ((uint32_t)(warp * 32) << 16);
+    float v[2][32];
+    if (init) {
 #pragma unroll
-    for (int cb = 0; cb < 4; ++cb) {
-        float v[32];
-        if (init) {
+        for (int k = 0; k < 2; ++k) {
+            const int cb = cb0 + k;
             if (transposed) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = init[(cb * 32 + i) * D + a];
+                for (int i = 0; i < 32; ++i) v[k][i] = init[(cb * 32 + i) * D + a];
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; i += 4) {
                     const float4 f = *reinterpret_cast<const float4*>(init + a * D + cb * 32 + i);
-                    v[i] = f.x; v[i + 1] = f.y; v[i + 2] = f.z; v[i + 3] = f.w;
+                    v[k][i] = f.x; v[k][i + 1] = f.y; v[k][i + 2] = f.z; v[k][i + 3] = f.w;
                 }
             }
-        } else {
-            ptx::tmem_ld32(taddr + cb * 32, v);
-            ptx::tmem_ld_wait();
         }
-        unsigned char* box = sb + (cb >> 1) * 16384;
+    } else {
+        ptx::tmem_ld32(taddr + cb0 * 32, v[0]);
+        ptx::tmem_ld32(taddr + cb0 * 32 + 32, v[1]);
+        ptx::tmem_ld_wait();
+    }
+    unsigned char* box = sb + (cb0 >> 1) * 16384;          // cb0 is even: both batches fall into one box
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
 #pragma unroll
         for (int u = 0; u < 4; ++u)
-            st_unit(box, a, (cb & 1) * 4 + u,
-                    make_uint4(pack2(v[u * 8], v[u * 8 + 1]), pack2(v[u * 8 + 2], v[u * 8 + 3]), pack2(v[u * 8 + 4], v[u * 8 + 5]),
-                               pack2(v[u * 8 + 6], v[u * 8 + 7])));
+            st_unit(box, a, k * 4 + u,
+                    make_uint4(pack2(v[k][u * 8], v[k][u * 8 + 1]), pack2(v[k][u * 8 + 2], v[k][u * 8 + 3]),
+                               pack2(v[k][u * 8 + 4], v[k][u * 8 + 5]), pack2(v[k][u * 8 + 6], v[k][u * 8 + 7])));
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] *= decay;
-        ptx::tmem_st32(taddr + cb * 32, v);
+        for (int i = 0; i < 32; ++i) v[k][i] *= decay;
+        ptx::tmem_st32(taddr + (cb0 + k) * 32, v[k]);
     }
     ptx::tmem_st_wait();
 }
 
 // Epilogue of an interleaved accumulator pair at TMEM columns `pair`: out[r][:] = X[r][:] + scale_r * Y[r][:]
-// as bf16 to global row pointers, and (ROWDOT) dot_r = sum_c out[r][c] * e[r][c] with e a [64 x 128]
-// bf16 tile in shared memory.  Each lane handles 16 of every 32 columns; lane l and l+16 share row r.
-template <bool ROWDOT>
-__device__ __forceinline__ float pair_epilogue(uint32_t pair, float scale, __nv_bfloat16* __restrict__ out_row, const unsigned char* etile) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int r = 16 * warp + (lane & 15);
-    const bool upper = lane >= 16;
-    float dot = 0.f;
+// as bf16 to global rows, and row dot products dot_r = sum_c out[r][c] * e[r][c] where e comes from a
+// [64 x 128] bf16 tile in shared memory (EMODE 1) or from global rows (EMODE 2); EMODE 0: none.
+// The thread serves rows rA = 16q + t/4 and rB = rA + 8; out_A/out_B (and e_A/e_B) point at their
+// first element.  On return dotA/dotB hold the full row sums in every thread of the row's lane group.
+template <int EMODE>
+__device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float scaleB, __nv_bfloat16* __restrict__ out_A,
+                                              __nv_bfloat16* __restrict__ out_B, const unsigned char* etile,
+                                              const __nv_bfloat16* __restrict__ e_A, const __nv_bfloat16* __restrict__ e_B,
+                                              float& dotA, float& dotB) {
+    const int q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
+    const int rA = 16 * q + (lane >> 2), rB = rA + 8, cq = 2 * (lane & 3);
+    const uint32_t taddr = pair + ((uint32_t)(q * 32) << 16);
+    dotA = 0.f;
+    dotB = 0.f;
 #pragma unroll
-    for (int cb = 0; cb < 4; ++cb) {
-        float v[32];
-        ptx::tmem_ld32(pair + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+    for (int hf = 0; hf < 2; ++hf) {
+        float x[32], y[32];
+        ptx::tmem_ld_16x64(taddr + hf * 64, x);
+        ptx::tmem_ld_16x64(taddr + (16u << 16) + hf * 64, y);
         ptx::tmem_ld_wait();
-        float res[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const float send = upper ? v[i] : v[16 + i];
-            const float recv = __shfl_xor_sync(0xffffffffu, send, 16);
-            const float x = upper ? recv : v[i];
-            const float y = upper ? v[16 + i] : recv;
-            res[i] = fmaf(scale, y, x);
-        }
-        const int col = cb * 32 + (upper ? 16 : 0);
-        if (ROWDOT) {
-            const unsigned char* box = etile + (col >> 6) * BOX;
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const uint4 ev = ld_unit(box, r, ((col & 63) >> 3) + u);
-                const __nv_bfloat162* e2 = reinterpret_cast<const __nv_bfloat162*>(&ev);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float2 f = __bfloat1622float2(e2[e]);
-                    dot = fmaf(res[u * 8 + 2 * e], f.x, dot);
-                    dot = fmaf(res[u * 8 + 2 * e + 1], f.y, dot);
+        for (int j = 0; j < 8; ++j) {
+            const int col = hf * 64 + 8 * j + cq;
+            const float a0 = fmaf(scaleA, y[4 * j], x[4 * j]), a1 = fmaf(scaleA, y[4 * j + 1], x[4 * j + 1]);
+            const float b0 = fmaf(scaleB, y[4 * j + 2], x[4 * j + 2]), b1 = fmaf(scaleB, y[4 * j + 3], x[4 * j + 3]);
+            if (EMODE != 0) {
+                uint32_t ea, eb;
+                if (EMODE == 1) {
+                    const unsigned char* box = etile + hf * BOX;
+                    ea = *reinterpret_cast<const uint32_t*>(box + rA * 128 + ((j ^ (rA & 7)) << 4) + 2 * cq);
+                    eb = *reinterpret_cast<const uint32_t*>(box + rB * 128 + ((j ^ (rB & 7)) << 4) + 2 * cq);
+                } else {
+                    ea = *reinterpret_cast<const uint32_t*>(e_A + col);
+                    eb = *reinterpret_cast<const uint32_t*>(e_B + col);
                 }
+                const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ea));
+                const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&eb));
+                dotA = fmaf(a0, fa.x, dotA); dotA = fmaf(a1, fa.y, dotA);
+                dotB = fmaf(b0, fb.x, dotB); dotB = fmaf(b1, fb.y, dotB);
             }
+            *reinterpret_cast<uint32_t*>(out_A + col) = pack2(a0, a1);
+            *reinterpret_cast<uint32_t*>(out_B + col) = pack2(b0, b1);
         }
-        uint4* dst = reinterpret_cast<uint4*>(out_row + col);
-        dst[0] = make_uint4(pack2(res[0], res[1]), pack2(res[2], res[3]), pack2(res[4], res[5]), pack2(res[6], res[7]));
-        dst[1] = make_uint4(pack2(res[8], res[9]), pack2(res[10], res[11]), pack2(res[12], res[13]), pack2(res[14], res[15]));
     }
-    if (ROWDOT) dot += __shfl_xor_sync(0xffffffffu, dot, 16);
-    return dot;
+    if (EMODE != 0) {
+        dotA += __shfl_xor_sync(0xffffffffu, dotA, 1); dotA += __shfl_xor_sync(0xffffffffu, dotA, 2);
+        dotB += __shfl_xor_sync(0xffffffffu, dotB, 1); dotB += __shfl_xor_sync(0xffffffffu, dotB, 2);
+    }
 }
 
 // K-major descriptor of a [rows x 128] tile for K step ks (0..7): features 16*ks .. 16*ks+15.
@@ -379,134 +283,313 @@ __device__ __forceinline__ uint64_t mndesc(uint32_t tile, int ks, uint32_t box_b
     return ptx::smem_desc(tile + ks * 2048, box_bytes);
 }
 
+// Warp roles of the chunk-sweep kernels (16 warps, 128 registers each): warps 0-7 are the two state
+// warpgroups (columns 0-63 / 64-127 of the carried state, plus the weighted-tile pass; lane 0 of warp 0
+// also issues every MMA, right after its own state pass), warps 8-11 compute the decay masks (lane 0
+// of warp 8 also issues the TMA loads), warps 12-15 run epilogues.  The groups work on different
+// chunks at the same time; mbarriers carry the dependencies
+//     scores -> mask -> MMAs <- state pass <- previous MMAs ;  MMAs -> epilogue.
+constexpr int SW_THREADS = 512;
+#define SF_WAIT(bar, parity, code) ptx::mbar_wait(bar, parity, abort_flag, status, code)
+
 // ==================================================================================================
-// Chunk sweep with a forward-running state (Out + ST of paper Eq. 2; SR + OG of Section 3.4).
-// With tile roles (xq, xk, xv) and the state St[a][b] = sum xk[.][a] * xv[.][b]:
-//     out_r = sum_{s<=r} (xq_r . xk_s) D[r,s] xv_s  +  exp(b_r) * xq_r St_c ;   St_{c+1} = exp(b_C) St_c + xk^T diag(w) xv
-//   forward output pass : (xq, xk, xv) = (q, k, v),  St = H (from Hs[j]),      out = o
-//   dq pass             : (xq, xk, xv) = (dO, v, k), St = H^T (Hs[j] transposed), out = dq, and
-//                         xout[t] = q_t . dq_t (float32) with q as a fourth tile
-constexpr int SW_STAGES = 2;
-template <int NTILES>
-struct SweepSmem {
-    alignas(1024) unsigned char tiles[SW_STAGES][NTILES][TILE];
-    alignas(1024) unsigned char xvw[TILE];
-    alignas(1024) unsigned char am[BOX];
-    alignas(1024) unsigned char sb[2 * 16384];
+// Block aggregates on tensor cores: U = sum_s w_s x_s^T y_s over the block (M = N = 128, K = tokens).
+//   mode 0: (x, y) = (k, v), w_s = exp(beta - B_s);   mode 1: (x, y) = (q, dO), w_s = exp(B_s)
+// y is scaled by w in place in shared memory, then U += X^T (w*Y) with both operands MN-major.
+// 8 compute warps, one TMA warp, one MMA warp.
+constexpr int AGG_STAGES = 4;
+constexpr int AGG_COMP = 256;
+constexpr int AGG_THREADS = AGG_COMP + 64;
+struct AggSmem {
+    alignas(1024) unsigned char tiles[AGG_STAGES][2][TILE];
     float bloc[MAXR * C];
     float ctot[MAXR];
-    uint64_t full[SW_STAGES], empty[SW_STAGES], sc_done, ops_ready, out_done;
+    float cofs[MAXR];
+    uint64_t full[AGG_STAGES], empty[AGG_STAGES], ready[AGG_STAGES], done;
     uint32_t tmem_base;
     int abort_flag;
 };
 
-template <bool DQ>
-__global__ void __launch_bounds__(NTHREADS, 1)
-tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                const __grid_constant__ CUtensorMap tmE, SegParams p, const float* __restrict__ g, const float* __restrict__ Hs,
-                __nv_bfloat16* __restrict__ out, long long out_tok, long long out_bat, float* __restrict__ xout, int* status) {
-    constexpr int NTILES = DQ ? 4 : 3;
-    using Smem = SweepSmem<NTILES>;
+__global__ void __launch_bounds__(AGG_THREADS, 1)
+tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, SegParams p,
+                    const float* __restrict__ g, int mode, float* __restrict__ U, float* __restrict__ beta_out, int* status) {
     extern __shared__ unsigned char smem_raw[];
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    AggSmem& sm = *reinterpret_cast<AggSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
     const long long t0 = (long long)c0 * C;
     volatile int* abort_flag = &sm.abort_flag;
-    constexpr uint32_t T_ST = 0, T_O = 128, T_SC = 256;
+    constexpr int WT = AGG_COMP / 32, WM = WT + 1;
 
     if (tid == 0) {
         sm.abort_flag = 0;
-        for (int s = 0; s < SW_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1 + NCOMP); }
-        ptx::mbar_init(&sm.sc_done, 1);
-        ptx::mbar_init(&sm.ops_ready, NCOMP);
-        ptx::mbar_init(&sm.out_done, 1);
+        for (int s = 0; s < AGG_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1); ptx::mbar_init(&sm.ready[s], AGG_COMP); }
+        ptx::mbar_init(&sm.done, 1);
         ptx::fence_mbar_init();
     }
-    if (warp == 4) ptx::tmem_alloc(&sm.tmem_base, 512);
+    if (warp == WT) ptx::tmem_alloc(&sm.tmem_base, 128);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
 
-    if (warp == 4) {
+    if (warp == WT) {
         if (lane == 0) {
-            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
-            if (DQ) ptx::prefetch_tmap(&tmE);
+            ptx::prefetch_tmap(&tmX);
+            ptx::prefetch_tmap(&tmY);
             for (int c = 0; c < nch; ++c) {
-                const int s = c % SW_STAGES, it = c / SW_STAGES;
-                if (it > 0) ptx::mbar_wait(&sm.empty[s], (it - 1) & 1, abort_flag, status, DEV_TIMEOUT_MMA);
-                ptx::mbar_expect_tx(&sm.full[s], NTILES * TILE);
-                const int tok = (int)t0 + c * C;
-                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
-                if (DQ) tma_tile(sm.tiles[s][NTILES - 1], &tmE, &sm.full[s], h, tok, b);
+                const int s = c % AGG_STAGES, it = c / AGG_STAGES;
+                if (it > 0) SF_WAIT(&sm.empty[s], (it - 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::mbar_expect_tx(&sm.full[s], 2 * TILE);
+                tma_tile(sm.tiles[s][0], &tmX, &sm.full[s], h, (int)t0 + c * C, b);
+                tma_tile(sm.tiles[s][1], &tmY, &sm.full[s], h, (int)t0 + c * C, b);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == WM) {
         if (lane == 0) {
-            constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
-            constexpr uint32_t id_o1 = ptx::idesc_bf16(64, 128, 0, 1);
-            constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
-            const uint32_t am = ptx::smem_u32(sm.am), sb = ptx::smem_u32(sm.sb), xvw = ptx::smem_u32(sm.xvw);
+            constexpr uint32_t idesc = ptx::idesc_bf16(128, 128, 1, 1);
             for (int c = 0; c < nch; ++c) {
-                const int s = c % SW_STAGES, it = c / SW_STAGES;
-                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]), xv = ptx::smem_u32(sm.tiles[s][2]);
-                // scores of this chunk (the accumulator was released by the previous ops_ready)
-                ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
+                const int s = c % AGG_STAGES, it = c / AGG_STAGES;
+                SF_WAIT(&sm.ready[s], it & 1, DEV_TIMEOUT_TMA);
                 ptx::tc_fence_after_sync();
+                const uint32_t xa = ptx::smem_u32(sm.tiles[s][0]), ya = ptx::smem_u32(sm.tiles[s][1]);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
-                ptx::mma_commit(&sm.sc_done);
-                ptx::mbar_wait(&sm.ops_ready, c & 1, abort_flag, status, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-                // O1 = Am xv   (lanes +0)
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_O, kdesc(am, ks, BOX), mndesc(xv, ks, BOX), id_o1, ks > 0);
-                // O2 = xq St   (lanes +16)
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_O + (16u << 16), kdesc(xq, ks, BOX), mndesc(sb, ks, 16384), id_o1, ks > 0);
-                // St += xk^T (w xv)
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_ST, mndesc(xk, ks, BOX), mndesc(xvw, ks, BOX), id_st, 1u);
-                ptx::mma_commit(&sm.out_done);
+                for (int ks = 0; ks < 4; ++ks)
+                    ptx::mma_ss(tmem, mndesc(xa, ks, BOX), mndesc(ya, ks, BOX), idesc, (c > 0 || ks > 0) ? 1u : 0u);
                 ptx::mma_commit(&sm.empty[s]);
             }
+            ptx::mma_commit(&sm.done);
         }
     } else {
         const float* gh = g + (long long)b * p.bg + h;
-        prep_decay(gh, p.tg, t0, nch, sm.bloc, sm.ctot);
-        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
-        const int r = 16 * warp + (lane & 15);
-        __nv_bfloat16* out_h = out + (long long)b * out_bat + (long long)h * D;
-        float* xo = DQ ? xout + ((long long)b * p.H + h) * p.L : nullptr;
+        prep_decay(gh, p.tg, t0, nch, sm.bloc, sm.ctot, WT);
+        ptx::named_bar_sync(1, AGG_COMP);
+        if (tid == 0) {
+            float acc = 0.f;
+            if (mode == 0) { for (int c = nch - 1; c >= 0; --c) { sm.cofs[c] = acc; acc += sm.ctot[c]; } }
+            else           { for (int c = 0; c < nch; ++c)      { sm.cofs[c] = acc; acc += sm.ctot[c]; } }
+            if (beta_out) beta_out[((long long)b * p.H + h) * p.NB + j] = acc;
+        }
+        ptx::named_bar_sync(1, AGG_COMP);
         for (int c = 0; c < nch; ++c) {
-            const int s = c % SW_STAGES, it = c / SW_STAGES;
+            const int s = c % AGG_STAGES, it = c / AGG_STAGES;
+            SF_WAIT(&sm.full[s], it & 1, DEV_TIMEOUT_TMA);
+            const float cof = sm.cofs[c], bC = sm.ctot[c];
+            const float* bch = sm.bloc + c * C;
+            scale_tile<AGG_COMP>(sm.tiles[s][1], sm.tiles[s][1], tid,
+                       [&](int row) { return fast_exp(mode == 0 ? (bC - bch[row]) + cof : bch[row] + cof); });
+            ptx::fence_proxy_async();
+            ptx::mbar_arrive(&sm.ready[s]);
+        }
+        SF_WAIT(&sm.done, 0, DEV_TIMEOUT_MMA);
+        ptx::tc_fence_after_sync();
+        // 8 warps read the [128 x 128] accumulator: warp w covers lanes 32*(w&3).., column half w>>2
+        const int row = tid & 127, half = tid >> 7;
+        float* Uo = U + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D) + (long long)row * D + half * 64;
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+            float v[32];
+            ptx::tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64 + cb * 32, v);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+                *reinterpret_cast<float4*>(Uo + cb * 32 + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+        }
+        ptx::tc_fence_before_sync();
+    }
+    __syncthreads();
+    if (warp == WT) ptx::tmem_dealloc(tmem, 128);
+}
+
+// ==================================================================================================
+// Chunk sweep with a forward-running state (Out + ST of paper Eq. 2; SR + OG of Section 3.4).
+// With tile roles (xq, xk, xv) and the state St[a][b] = sum xk[.][a] * xv[.][b]:
+//     out_r = sum_{s<=r} (xq_r . xk_s) D[r,s] xv_s  +  exp(b_r) * xq_r St_c ;   St_{c+1} = exp(b_C) St_c + xk^T diag(w) xv
+//   forward output pass : (xq, xk, xv) = (q, k, v),  St = H (from Hs[j]),         out = o
+//   dq pass             : (xq, xk, xv) = (dO, v, k), St = H^T (Hs[j] transposed), out = dq, and
+//                         xout[t] = q_t . dq_t (float32), q read from global memory in the epilogue
+// TMEM columns: St 0-127; O pair (intra at lanes +0, inter at lanes +16) double-buffered at 128 / 256;
+// scores double-buffered at 384 / 448.//
+// The state is carried as two independent column halves (b < 64, b >= 64), one per state warpgroup:
+// each half has its own pass -> MMA -> pass chain, so one half's MMAs run while the other half's
+// warps rescale their accumulator, which keeps the tensor pipe fed.
+constexpr int SW_STAGES = 3;
+struct SweepSmem {
+    alignas(1024) unsigned char tiles[SW_STAGES][3][TILE];
+    alignas(1024) unsigned char xvw[TILE];
+    alignas(1024) unsigned char am[2][BOX];
+    alignas(1024) unsigned char sb[2 * 16384];
+    float bloc[MAXR * C];
+    float ctot[MAXR];
+    uint64_t full[SW_STAGES], sc_done[2], am_ready[2], st_ready[2], st_done[2], out_done[2], o_free[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <bool DQ>
+__global__ void __launch_bounds__(SW_THREADS, 1)
+tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                SegParams p, const float* __restrict__ g, const float* __restrict__ Hs, __nv_bfloat16* __restrict__ out, long long out_tok,
+                long long out_bat, const __nv_bfloat16* __restrict__ e_glob, float* __restrict__ xout, int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    SweepSmem& sm = *reinterpret_cast<SweepSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
+    const long long t0 = (long long)c0 * C;
+    volatile int* abort_flag = &sm.abort_flag;
+    constexpr uint32_t T_ST = 0, T_O = 128, T_SC = 384;
+
+    auto load_chunk = [&](int c) {          // one thread
+        const int s = c % SW_STAGES;
+        ptx::mbar_expect_tx(&sm.full[s], 3 * TILE);
+        const int tok = (int)t0 + c * C;
+        tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
+        tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
+        tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
+    };
+
+    if (tid == 256) {
+        sm.abort_flag = 0;
+        for (int s = 0; s < SW_STAGES; ++s) ptx::mbar_init(&sm.full[s], 1);
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 128);
+            ptx::mbar_init(&sm.st_ready[i], 128); ptx::mbar_init(&sm.st_done[i], 1);
+            ptx::mbar_init(&sm.out_done[i], 2); ptx::mbar_init(&sm.o_free[i], 128);
+        }
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
+        for (int c = 0; c < SW_STAGES && c < nch; ++c) load_chunk(c);
+    }
+    if (warp == 0) ptx::tmem_alloc(&sm.tmem_base, 512);
+    prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp < 8) {
+        // ---- state warpgroup `hf` (columns 64*hf .. 64*hf+63); its first thread issues this half's MMAs ----
+        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
+        const int hf = warp >> 2, t = tid & 127;
+        const bool issuer = t == 0;
+        constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
+        constexpr uint32_t id_o1 = ptx::idesc_bf16(64, 128, 0, 1);
+        constexpr uint32_t id_o2 = ptx::idesc_bf16(64, 64, 0, 1);       // xq (K-major) x state half (token... feature-major rows)
+        constexpr uint32_t id_st = ptx::idesc_bf16(128, 64, 1, 1);
+        const uint32_t sbh = ptx::smem_u32(sm.sb) + hf * 16384, xvwh = ptx::smem_u32(sm.xvw) + hf * BOX;
+        auto scores = [&](int c) {
+            const int s = c % SW_STAGES;
+            SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
+            ptx::tc_fence_after_sync();
+            const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC + (c & 1) * 64, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
+            ptx::mma_commit(&sm.sc_done[c & 1]);
+        };
+        if (issuer && hf == 0) scores(0);
+        for (int c = 0; c < nch; ++c) {
+            const int s = c % SW_STAGES, bf = c & 1;
             const float* bch = sm.bloc + c * C;
             const float bC = sm.ctot[c];
-            ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
-            scale_tile(sm.xvw, sm.tiles[s][2], [&](int row) { return fast_exp(bC - bch[row]); });
-            state_pass(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ);
-            ptx::mbar_wait(&sm.sc_done, c & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+            SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
+            SF_TR(2 + 3 * hf, c, 0);
+            if (c > 0) SF_WAIT(&sm.st_done[hf], (c - 1) & 1, DEV_TIMEOUT_MMA);
             ptx::tc_fence_after_sync();
-            mask_pass(tmem + T_SC, bch, sm.am, nullptr);
+            SF_TR(2 + 3 * hf, c, 1);
+            // weighted copy of this half's box of xv: 512 units over 128 threads, rows t>>3 + {0,16,32,48}
+            {
+                const uint4* in = reinterpret_cast<const uint4*>(sm.tiles[s][2] + hf * BOX);
+                uint4* outp = reinterpret_cast<uint4*>(sm.xvw + hf * BOX);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float w = fast_exp(bC - bch[(t >> 3) + 16 * i]);
+                    uint4 v = in[t + 128 * i];
+                    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __bfloat1622float2(h2[e]);
+                        h2[e] = __floats2bfloat162_rn(f.x * w, f.y * w);
+                    }
+                    outp[t + 128 * i] = v;
+                }
+            }
+            SF_TR(2 + 3 * hf, c, 2);
+            state_pass(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 2 * hf);
             ptx::fence_proxy_async();
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.ops_ready);
-            ptx::mbar_wait(&sm.out_done, c & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+            ptx::mbar_arrive(&sm.st_ready[hf]);
+            SF_TR(2 + 3 * hf, c, 3);
+            if (issuer) {
+                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]), xv = ptx::smem_u32(sm.tiles[s][2]);
+                const uint32_t to = tmem + T_O + bf * 128;
+                if (c >= 2) SF_WAIT(&sm.o_free[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
+                SF_WAIT(&sm.st_ready[hf], c & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                SF_TR(1 + 5 * hf, c, 2);
+                // inter-chunk part of this half's output columns (lanes +16), then the state half
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(to + (16u << 16) + hf * 64, kdesc(xq, ks, BOX), mndesc(sbh, ks, 0), id_o2, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_ST + hf * 64, mndesc(xk, ks, BOX), mndesc(xvwh, ks, 0), id_st, 1u);
+                ptx::mma_commit(&sm.st_done[hf]);
+                if (hf == 1) {
+                    const uint32_t am = ptx::smem_u32(sm.am[bf]);
+                    SF_WAIT(&sm.am_ready[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
+                    ptx::tc_fence_after_sync();
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(to, kdesc(am, ks, BOX), mndesc(xv, ks, BOX), id_o1, ks > 0);            // intra
+                }
+                ptx::mma_commit(&sm.out_done[bf]);
+                SF_TR(1 + 5 * hf, c, 3);
+                if (hf == 0 && c + 1 < nch) scores(c + 1);      // its accumulator was released by am_ready of chunk c-1
+            }
+            __syncwarp();
+        }
+    } else if (warp < 12) {
+        // ---- mask warpgroup (thread 256 also feeds the TMA pipeline) ---------------------------------------
+        for (int c = 0; c < nch; ++c) {
+            const int bf = c & 1;
+            SF_WAIT(&sm.sc_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
+            if (c >= 2) {
+                // chunk c-2 is complete: Am[bf] is no longer read, and its tile stage can take chunk c+1
+                SF_WAIT(&sm.out_done[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
+                if (tid == 256 && c + 1 < nch) load_chunk(c + 1);
+            }
             ptx::tc_fence_after_sync();
-            const long long tok = t0 + c * C + r;
-            const float dot = pair_epilogue<DQ>(tmem + T_O, fast_exp(bch[r]), out_h + tok * out_tok, sm.tiles[s][NTILES - 1]);
-            if (DQ && lane < 16) xo[tok] = dot;
+            SF_TR(3, c, 0);
+            mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], nullptr);
+            ptx::fence_proxy_async();
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.empty[s]);
+            ptx::mbar_arrive(&sm.am_ready[bf]);
+            SF_TR(3, c, 1);
+        }
+    } else {
+        // ---- epilogue warpgroup ---------------------------------------------------------------------------
+        const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
+        __nv_bfloat16* out_h = out + (long long)b * out_bat + (long long)h * D;
+        const __nv_bfloat16* e_h = DQ ? e_glob + (long long)b * out_bat + (long long)h * D : nullptr;
+        float* xo = DQ ? xout + ((long long)b * p.H + h) * p.L : nullptr;
+        for (int c = 0; c < nch; ++c) {
+            const int bf = c & 1;
+            const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
+            const float eA = fast_exp(sm.bloc[c * C + rA]), eB = fast_exp(sm.bloc[c * C + rB]);
+            SF_WAIT(&sm.out_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
+            ptx::tc_fence_after_sync();
+            SF_TR(4, c, 0);
+            float dotA, dotB;
+            pair_epilogue<DQ ? 2 : 0>(tmem + T_O + bf * 128, eA, eB, out_h + tokA * out_tok, out_h + tokB * out_tok, nullptr,
+                                      DQ ? e_h + tokA * out_tok : nullptr, DQ ? e_h + tokB * out_tok : nullptr, dotA, dotB);
+            if (DQ && (lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&sm.o_free[bf]);
+            SF_TR(4, c, 1);
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) ptx::tmem_dealloc(tmem, 512);
+    if (warp == 0) ptx::tmem_dealloc(tmem, 512);
 }
 
 // ==================================================================================================
@@ -516,23 +599,26 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 //     dv_s = sum_{r>=s} A[r,s] dO_r + w_s k_s G ;   dk_s = sum_{r>=s} dA[r,s] q_r + w_s v_s G^T ;   w_s = exp(b_C - b_s)
 //     G <- exp(b_C) G + (diag(exp(b)) Q)^T dO
 // and xk[t] = k_t . dk_t (float32).
+// TMEM columns: G 0-127; dk pair 128-255; dv pair 256-383; score pair (A at lanes +0, dA at +16)
+// double-buffered at 384 / 448.
 struct DkdvSmem {
-    alignas(1024) unsigned char tiles[SW_STAGES][4][TILE];     // q, k, v, dO
+    alignas(1024) unsigned char tiles[2][4][TILE];     // q, k, v, dO
     alignas(1024) unsigned char qw[TILE];
-    alignas(1024) unsigned char am[BOX];
-    alignas(1024) unsigned char dam[BOX];
+    alignas(1024) unsigned char am[2][BOX];
+    alignas(1024) unsigned char dam[2][BOX];
     alignas(1024) unsigned char gb[2 * 16384];
     float bloc[MAXR * C];
     float ctot[MAXR];
-    uint64_t full[SW_STAGES], empty[SW_STAGES], sc_done, ops_ready, out_done;
+    uint64_t full[2], sc_done[2], am_ready[2], st_ready, out_done, o_free;
     uint32_t tmem_base;
     int abort_flag;
 };
 
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(SW_THREADS, 1)
 tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmD, SegParams p, const float* __restrict__ g, const float* __restrict__ Gs,
-               __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, float* __restrict__ xk, int* status) {
+               const __nv_bfloat16* __restrict__ k_glob, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+               float* __restrict__ xk, int* status) {
     extern __shared__ unsigned char smem_raw[];
     DkdvSmem& sm = *reinterpret_cast<DkdvSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -542,109 +628,140 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     volatile int* abort_flag = &sm.abort_flag;
     constexpr uint32_t T_G = 0, T_DK = 128, T_DV = 256, T_SC = 384;
 
-    if (tid == 0) {
+    // iteration i handles chunk c = nch-1-i
+    auto load_chunk = [&](int i) {          // one thread
+        const int s = i & 1;
+        ptx::mbar_expect_tx(&sm.full[s], 4 * TILE);
+        const int tok = (int)t0 + (nch - 1 - i) * C;
+        tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
+        tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
+        tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
+        tma_tile(sm.tiles[s][3], &tmD, &sm.full[s], h, tok, b);
+    };
+
+    if (tid == 256) {
         sm.abort_flag = 0;
-        for (int s = 0; s < SW_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1 + NCOMP); }
-        ptx::mbar_init(&sm.sc_done, 1);
-        ptx::mbar_init(&sm.ops_ready, NCOMP);
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&sm.full[i], 1);
+            ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 128);
+        }
+        ptx::mbar_init(&sm.st_ready, 256);
         ptx::mbar_init(&sm.out_done, 1);
+        ptx::mbar_init(&sm.o_free, 256);
         ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); ptx::prefetch_tmap(&tmD);
+        for (int i = 0; i < 2 && i < nch; ++i) load_chunk(i);
     }
-    if (warp == 4) ptx::tmem_alloc(&sm.tmem_base, 512);
+    if (warp == 0) ptx::tmem_alloc(&sm.tmem_base, 512);
+    prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
 
-    // iteration i handles chunk c = nch-1-i
-    if (warp == 4) {
-        if (lane == 0) {
-            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); ptx::prefetch_tmap(&tmD);
-            for (int i = 0; i < nch; ++i) {
-                const int s = i % SW_STAGES, it = i / SW_STAGES;
-                if (it > 0) ptx::mbar_wait(&sm.empty[s], (it - 1) & 1, abort_flag, status, DEV_TIMEOUT_MMA);
-                ptx::mbar_expect_tx(&sm.full[s], 4 * TILE);
-                const int tok = (int)t0 + (nch - 1 - i) * C;
-                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][3], &tmD, &sm.full[s], h, tok, b);
-            }
-        }
-    } else if (warp == 5) {
-        if (lane == 0) {
-            constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
-            constexpr uint32_t id_tt = ptx::idesc_bf16(64, 128, 1, 1);     // A^T-type: both operands token-major
-            constexpr uint32_t id_kn = ptx::idesc_bf16(64, 128, 0, 1);     // K G
-            constexpr uint32_t id_kk = ptx::idesc_bf16(64, 128, 0, 0);     // V G^T
-            constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
-            const uint32_t am = ptx::smem_u32(sm.am), dam = ptx::smem_u32(sm.dam), gb = ptx::smem_u32(sm.gb), qw = ptx::smem_u32(sm.qw);
-            for (int i = 0; i < nch; ++i) {
-                const int s = i % SW_STAGES, it = i / SW_STAGES;
+    if (warp < 8) {
+        // ---- state warpgroups: exp(b) * Q tile + carried gradient; warp 0 lane 0 issues the MMAs ---------
+        const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
+        const int half = warp >> 2;
+        const bool issuer = tid == 0;
+        constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
+        constexpr uint32_t id_tt = ptx::idesc_bf16(64, 128, 1, 1);     // A^T dO, dA^T Q: both operands token-major
+        constexpr uint32_t id_kn = ptx::idesc_bf16(64, 128, 0, 1);     // K G
+        constexpr uint32_t id_kk = ptx::idesc_bf16(64, 128, 0, 0);     // V G^T
+        constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
+        const uint32_t gb = ptx::smem_u32(sm.gb), qw = ptx::smem_u32(sm.qw);
+        auto scores = [&](int i) {
+            const int s = i & 1;
+            SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
+            ptx::tc_fence_after_sync();
+            const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
+            const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
+            const uint32_t sc = tmem + T_SC + (i & 1) * 64;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(sc, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(sc + (16u << 16), kdesc(xd, ks, BOX), kdesc(xv, ks, BOX), id_sc, ks > 0);
+            ptx::mma_commit(&sm.sc_done[i & 1]);
+        };
+        if (issuer) scores(0);
+        for (int i = 0; i < nch; ++i) {
+            const int c = nch - 1 - i, s = i & 1;
+            const float* bch = sm.bloc + c * C;
+            SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
+            if (i > 0) SF_WAIT(&sm.out_done, (i - 1) & 1, DEV_TIMEOUT_MMA);
+            ptx::tc_fence_after_sync();
+            scale_tile<256>(sm.qw, sm.tiles[s][0], tid, [&](int row) { return fast_exp(bch[row]); });
+            state_pass(tmem + T_G, sm.gb, fast_exp(sm.ctot[c]), i == 0 ? G0 : nullptr, false, 2 * half);
+            ptx::fence_proxy_async();
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&sm.st_ready);
+            if (issuer) {
                 const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
                 const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
-                ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
+                const uint32_t am = ptx::smem_u32(sm.am[s]), dam = ptx::smem_u32(sm.dam[s]);
+                SF_WAIT(&sm.am_ready[s], (i >> 1) & 1, DEV_TIMEOUT_MMA);
+                if (i >= 1) SF_WAIT(&sm.o_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
+                SF_WAIT(&sm.st_ready, i & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DV + (16u << 16), kdesc(xk, ks, BOX), mndesc(gb, ks, 16384), id_kn, ks > 0);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC + (16u << 16), kdesc(xd, ks, BOX), kdesc(xv, ks, BOX), id_sc, ks > 0);
-                ptx::mma_commit(&sm.sc_done);
-                ptx::mbar_wait(&sm.ops_ready, i & 1, abort_flag, status, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-                // dv1 = A^T dO (lanes +0), dv2 = K G (lanes +16)
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DV, mndesc(am, ks, BOX), mndesc(xd, ks, BOX), id_tt, ks > 0);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DV + (16u << 16), kdesc(xk, ks, BOX), mndesc(gb, ks, 16384), id_kn, ks > 0);
-                // dk1 = dA^T Q (lanes +0), dk2 = V G^T (lanes +16)
-#pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DK, mndesc(dam, ks, BOX), mndesc(xq, ks, BOX), id_tt, ks > 0);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
-                // G += (diag(exp(b)) Q)^T dO
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
                 ptx::mma_commit(&sm.out_done);
-                ptx::mma_commit(&sm.empty[s]);
+                if (i + 1 < nch) scores(i + 1);
             }
+            __syncwarp();
         }
     } else {
-        const float* gh = g + (long long)b * p.bg + h;
-        prep_decay(gh, p.tg, t0, nch, sm.bloc, sm.ctot);
-        const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
-        const int r = 16 * warp + (lane & 15);
+        // ---- warps 8-11: masks, TMA feed, then the dv epilogue; warps 12-15: the dk epilogue ------------
+        const bool masker = warp < 12;
+        const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
         __nv_bfloat16* dk_h = dk + (long long)b * p.bqk + (long long)h * D;
         __nv_bfloat16* dv_h = dv + (long long)b * p.bv + (long long)h * D;
+        const __nv_bfloat16* k_h = k_glob + (long long)b * p.bqk + (long long)h * D;
         float* xo = xk + ((long long)b * p.H + h) * p.L;
-        for (int i = 0; i < nch; ++i) {
-            const int c = nch - 1 - i;
-            const int s = i % SW_STAGES, it = i / SW_STAGES;
-            const float* bch = sm.bloc + c * C;
-            const float bC = sm.ctot[c];
-            ptx::mbar_wait(&sm.full[s], it & 1, abort_flag, status, DEV_TIMEOUT_TMA);
-            scale_tile(sm.qw, sm.tiles[s][0], [&](int row) { return fast_exp(bch[row]); });
-            state_pass(tmem + T_G, sm.gb, fast_exp(bC), i == 0 ? G0 : nullptr, false);
-            ptx::mbar_wait(&sm.sc_done, i & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+        auto mask = [&](int i) {
+            const int c = nch - 1 - i, bf = i & 1;
+            SF_WAIT(&sm.sc_done[bf], (i >> 1) & 1, DEV_TIMEOUT_MMA);
             ptx::tc_fence_after_sync();
-            mask_pass(tmem + T_SC, bch, sm.am, sm.dam);
+            mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], sm.dam[bf]);
             ptx::fence_proxy_async();
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.ops_ready);
-            ptx::mbar_wait(&sm.out_done, i & 1, abort_flag, status, DEV_TIMEOUT_MMA);
+            ptx::mbar_arrive(&sm.am_ready[bf]);
+        };
+        if (masker) mask(0);
+        for (int i = 0; i < nch; ++i) {
+            const int c = nch - 1 - i;
+            // the masks of the next chunk go first: their buffers were last read by the MMAs of chunk i-1,
+            // whose completion this warpgroup observed before the previous epilogue
+            if (masker && i + 1 < nch) mask(i + 1);
+            const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
+            const float wA = fast_exp(sm.ctot[c] - sm.bloc[c * C + rA]), wB = fast_exp(sm.ctot[c] - sm.bloc[c * C + rB]);
+            SF_WAIT(&sm.out_done, i & 1, DEV_TIMEOUT_MMA);
+            // every MMA of chunk i is complete: its tile stage can take chunk i+2
+            if (tid == 256 && i + 2 < nch) load_chunk(i + 2);
             ptx::tc_fence_after_sync();
-            const long long tok = t0 + c * C + r;
-            const float w = fast_exp(bC - bch[r]);
-            pair_epilogue<false>(tmem + T_DV, w, dv_h + tok * p.tv, nullptr);
-            const float dot = pair_epilogue<true>(tmem + T_DK, w, dk_h + tok * p.tqk, sm.tiles[s][1]);
-            if (lane < 16) xo[tok] = dot;
+            float dotA, dotB;
+            if (masker) {
+                pair_epilogue<0>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, nullptr, dotA, dotB);
+            } else {
+                pair_epilogue<2>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, nullptr, k_h + tokA * p.tqk,
+                                 k_h + tokB * p.tqk, dotA, dotB);
+                if ((lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
+            }
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.empty[s]);
+            ptx::mbar_arrive(&sm.o_free);
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) ptx::tmem_dealloc(tmem, 512);
+    if (warp == 0) ptx::tmem_dealloc(tmem, 512);
 }
 
 // ---- host launch -------------------------------------------------------------------------------------
@@ -670,7 +787,8 @@ inline sf_status_t launch(int role, const sf_seg_desc_t* d, const SegParams& p, 
                           void* dq, void* dk, void* dv, float* xq, float* xk, cudaStream_t st, long long* n_launch) {
     int* status = status_ptr();
     if (!status) return SF_ERR_CUDA;
-    dim3 grid(p.NB, p.H, p.B), block(NTHREADS);
+    if (p.R > MAXR) return SF_ERR_UNSUPPORTED;
+    dim3 grid(p.NB, p.H, p.B);
     auto map_qk = [&](CUtensorMap* m, const void* base) { return make_tmap(m, base, p.B, p.L, p.H, p.tqk, p.bqk); };
     auto map_v = [&](CUtensorMap* m, const void* base) { return make_tmap(m, base, p.B, p.L, p.H, p.tv, p.bv); };
     if (role == 0) {
@@ -679,37 +797,43 @@ inline sf_status_t launch(int role, const sf_seg_desc_t* d, const SegParams& p, 
         constexpr size_t smem = sizeof(AggSmem) + 1024;
         static bool ok = opt_in_smem(tc_aggregate_kernel, smem);
         if (!ok) return SF_ERR_CUDA;
-        tc_aggregate_kernel<<<grid, block, smem, st>>>(tmX, tmY, p, g, mode, U, beta, status);
+        tc_aggregate_kernel<<<grid, AGG_THREADS, smem, st>>>(tmX, tmY, p, g, mode, U, beta, status);
     } else if (role == 1) {
         CUtensorMap tq, tk, tv;
         if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v)) return SF_ERR_CUDA;
-        constexpr size_t smem = sizeof(SweepSmem<3>) + 1024;
+        constexpr size_t smem = sizeof(SweepSmem) + 1024;
         static bool ok = opt_in_smem(tc_sweep_kernel<false>, smem);
         if (!ok) return SF_ERR_CUDA;
-        tc_sweep_kernel<false><<<grid, block, smem, st>>>(tq, tk, tv, tq, p, g, states, static_cast<__nv_bfloat16*>(o), p.tv, p.bv,
-                                                          nullptr, status);
+        tc_sweep_kernel<false><<<grid, SW_THREADS, smem, st>>>(tq, tk, tv, p, g, states, static_cast<__nv_bfloat16*>(o), p.tv, p.bv,
+                                                               nullptr, nullptr, status);
     } else if (role == 2) {
-        CUtensorMap tq, tk, tv, td;
-        if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;
-        constexpr size_t smem = sizeof(SweepSmem<4>) + 1024;
+        CUtensorMap tk, tv, td;
+        if (!map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;
+        constexpr size_t smem = sizeof(SweepSmem) + 1024;
         static bool ok = opt_in_smem(tc_sweep_kernel<true>, smem);
         if (!ok) return SF_ERR_CUDA;
-        // roles: xq = dO, xk = v, xv = k, extra = q
-        tc_sweep_kernel<true><<<grid, block, smem, st>>>(td, tv, tk, tq, p, g, states, static_cast<__nv_bfloat16*>(dq), p.tqk, p.bqk,
-                                                         xq, status);
+        // roles: xq = dO, xk = v, xv = k; q is read from global memory for the row dot products
+        tc_sweep_kernel<true><<<grid, SW_THREADS, smem, st>>>(td, tv, tk, p, g, states, static_cast<__nv_bfloat16*>(dq), p.tqk, p.bqk,
+                                                              static_cast<const __nv_bfloat16*>(q), xq, status);
     } else if (role == 3) {
         CUtensorMap tq, tk, tv, td;
         if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;
         constexpr size_t smem = sizeof(DkdvSmem) + 1024;
         static bool ok = opt_in_smem(tc_dkdv_kernel, smem);
         if (!ok) return SF_ERR_CUDA;
-        tc_dkdv_kernel<<<grid, block, smem, st>>>(tq, tk, tv, td, p, g, states, static_cast<__nv_bfloat16*>(dk),
-                                                  static_cast<__nv_bfloat16*>(dv), xk, status);
+        tc_dkdv_kernel<<<grid, SW_THREADS, smem, st>>>(tq, tk, tv, td, p, g, states, static_cast<const __nv_bfloat16*>(k),
+                                                       static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), xk, status);
     } else {
         return SF_ERR_UNSUPPORTED;
     }
     *n_launch += 1;
-    return cudaGetLastError() == cudaSuccess ? SF_OK : SF_ERR_CUDA;
+    {
+        cudaError_t e = cudaGetLastError();
+#ifdef SF_TRACE
+        if (e != cudaSuccess) fprintf(stderr, "[sf] launch role %d failed: %s\n", role, cudaGetErrorString(e));
+#endif
+        return e == cudaSuccess ? SF_OK : SF_ERR_CUDA;
+    }
 }
 
 }  // namespace tc

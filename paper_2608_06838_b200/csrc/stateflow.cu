@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <mutex>
+#include <vector>
 
 #include "sf_common.cuh"
 #include "sf_scan.cuh"
@@ -15,6 +16,31 @@ namespace {
 using sf::SegParams;
 
 std::atomic<long long> g_launches{0};
+
+// Optional per-stage device timers (off by default): every kernel launch is bracketed by a pair of
+// events on its own stream.
+enum Stage { ST_AGG_KV = 0, ST_AGG_QDO, ST_SCAN, ST_FWD_OUT, ST_DQ, ST_DKDV, ST_DG, ST_COUNT };
+struct TimedLaunch { cudaEvent_t a, b; int stage; };
+std::mutex g_timing_mu;
+bool g_timing_on = false;
+std::vector<TimedLaunch> g_timed;
+
+struct StageTimer {
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaStream_t st;
+    int stage;
+    StageTimer(int stage_, cudaStream_t st_) : st(st_), stage(stage_) {
+        if (!g_timing_on) return;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { cudaGetLastError(); a = b = nullptr; return; }
+        cudaEventRecord(a, st);
+    }
+    ~StageTimer() {
+        if (!a) return;
+        cudaEventRecord(b, st);
+        std::lock_guard<std::mutex> lk(g_timing_mu);
+        g_timed.push_back({a, b, stage});
+    }
+};
 
 constexpr int kDefaultChunksPerBlock = 16;
 constexpr size_t kAlign = 256;
@@ -180,6 +206,9 @@ sf_status_t launch_simt_d(Role role, const sf_seg_desc_t* d, const SegParams& p,
 }
 
 sf_status_t launch_role(Path path, Role role, const sf_seg_desc_t* d, const SegParams& p, const RoleArgs& a, cudaStream_t st) {
+    const int stage = role == Role::Aggregate ? (a.mode == 0 ? ST_AGG_KV : ST_AGG_QDO)
+                    : role == Role::FwdOut ? ST_FWD_OUT : role == Role::BwdDq ? ST_DQ : ST_DKDV;
+    StageTimer timer(stage, st);
     if (path == Path::Tc) {
         long long n = 0;
         sf_status_t s = sf::tc::launch(static_cast<int>(role), d, p, a.q, a.k, a.v, a.dO, a.g, a.mode, a.U, a.beta, a.states,
@@ -194,6 +223,7 @@ sf_status_t launch_role(Path path, Role role, const sf_seg_desc_t* d, const SegP
 sf_status_t launch_scan(const sf_seg_desc_t* d, const SegParams& p, int reverse, const float* ld, const float* U,
                         const float* init, float* states, float* fin, cudaStream_t st) {
     const int m = d->d_k * d->d_v;
+    StageTimer timer(ST_SCAN, st);
     dim3 grid((m / 4 + sf::SCAN_NT - 1) / sf::SCAN_NT, p.B * p.H);
     sf::state_scan_kernel<<<grid, sf::SCAN_NT, 0, st>>>(p.NB, m, reverse, ld, U, init, states, fin);
     return check_launch();
@@ -242,6 +272,7 @@ sf_status_t bwd_dkdv(Path path, const sf_seg_desc_t* d, const SegParams& p, cons
     return launch_role(path, Role::BwdDkDv, d, p, a, st);
 }
 sf_status_t bwd_dg(const sf_seg_desc_t* d, const SegParams& p, const BwdPtrs& x, const BwdWs& w, const float* Hs, cudaStream_t st) {
+    StageTimer timer(ST_DG, st);
     dim3 grid(p.NB, p.H, p.B);
     sf::dg_epilogue_kernel<<<grid, sf::DG_NT, 0, st>>>(p, d->d_k * d->d_v, w.xq, w.xk, Hs, w.GU, x.dS_in, x.dg);
     return check_launch();
@@ -639,5 +670,29 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
 int32_t sf_device_status(void) { return sf::tc::read_device_status(); }
 void sf_device_status_clear(void) { sf::tc::clear_device_status(); }
 int64_t sf_launch_count(void) { return g_launches.load(); }
+
+#ifdef SF_TRACE
+void sf_debug_trace(long long* out) { cudaMemcpyFromSymbol(out, sf::tc::g_trace, sizeof(long long) * 8 * 64 * 4); }
+#endif
+
+void sf_stage_timing(int32_t enable) {
+    std::lock_guard<std::mutex> lk(g_timing_mu);
+    g_timing_on = enable != 0;
+}
+
+int32_t sf_stage_timing_read(float* ms, int64_t* launches, int32_t n) {
+    cudaDeviceSynchronize();
+    std::lock_guard<std::mutex> lk(g_timing_mu);
+    for (int i = 0; i < n; ++i) { ms[i] = 0.f; launches[i] = 0; }
+    for (auto& t : g_timed) {
+        float e = 0.f;
+        if (cudaEventElapsedTime(&e, t.a, t.b) == cudaSuccess && t.stage < n) { ms[t.stage] += e; launches[t.stage] += 1; }
+        else cudaGetLastError();
+        cudaEventDestroy(t.a);
+        cudaEventDestroy(t.b);
+    }
+    g_timed.clear();
+    return ST_COUNT;
+}
 
 }  // extern "C"
