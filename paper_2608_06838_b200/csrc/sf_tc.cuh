@@ -156,71 +156,98 @@ __device__ __forceinline__ void mask_pass(uint32_t sc, const float* bch, unsigne
     const int q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
     const int rA = 16 * q + (lane >> 2), rB = rA + 8, cq = 2 * (lane & 3);
     const uint32_t taddr = sc + ((uint32_t)(q * 32) << 16);
-    float x[32], y[32];
-    ptx::tmem_ld_16x64(taddr, x);
-    if (dst1) ptx::tmem_ld_16x64(taddr + (16u << 16), y);
     const float bA = bch[rA] * LOG2E, bB = bch[rB] * LOG2E;
-    ptx::tmem_ld_wait();
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int s0 = 8 * j + cq;
-        const float2 bs = *reinterpret_cast<const float2*>(bch + s0);
-        const float e0 = -LOG2E * bs.x, e1 = -LOG2E * bs.y;
-        const float dA0 = s0 <= rA ? ptx::ex2(bA + e0) : 0.f, dA1 = s0 + 1 <= rA ? ptx::ex2(bA + e1) : 0.f;
-        const float dB0 = s0 <= rB ? ptx::ex2(bB + e0) : 0.f, dB1 = s0 + 1 <= rB ? ptx::ex2(bB + e1) : 0.f;
-        const int offA = rA * 128 + ((j ^ (rA & 7)) << 4) + 2 * cq, offB = rB * 128 + ((j ^ (rB & 7)) << 4) + 2 * cq;
-        *reinterpret_cast<uint32_t*>(dst0 + offA) = pack2(x[4 * j] * dA0, x[4 * j + 1] * dA1);
-        *reinterpret_cast<uint32_t*>(dst0 + offB) = pack2(x[4 * j + 2] * dB0, x[4 * j + 3] * dB1);
-        if (dst1) {
-            *reinterpret_cast<uint32_t*>(dst1 + offA) = pack2(y[4 * j] * dA0, y[4 * j + 1] * dA1);
-            *reinterpret_cast<uint32_t*>(dst1 + offB) = pack2(y[4 * j + 2] * dB0, y[4 * j + 3] * dB1);
+    for (int hf = 0; hf < 2; ++hf) {
+        float x[16], y[16];
+        ptx::tmem_ld_16x32(taddr + hf * 32, x);
+        if (dst1) ptx::tmem_ld_16x32(taddr + (16u << 16) + hf * 32, y);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const int j = hf * 4 + jj, s0 = 8 * j + cq;
+            const float2 bs = *reinterpret_cast<const float2*>(bch + s0);
+            const float e0 = -LOG2E * bs.x, e1 = -LOG2E * bs.y;
+            const float dA0 = s0 <= rA ? ptx::ex2(bA + e0) : 0.f, dA1 = s0 + 1 <= rA ? ptx::ex2(bA + e1) : 0.f;
+            const float dB0 = s0 <= rB ? ptx::ex2(bB + e0) : 0.f, dB1 = s0 + 1 <= rB ? ptx::ex2(bB + e1) : 0.f;
+            const int offA = rA * 128 + ((j ^ (rA & 7)) << 4) + 2 * cq, offB = rB * 128 + ((j ^ (rB & 7)) << 4) + 2 * cq;
+            *reinterpret_cast<uint32_t*>(dst0 + offA) = pack2(x[4 * jj] * dA0, x[4 * jj + 1] * dA1);
+            *reinterpret_cast<uint32_t*>(dst0 + offB) = pack2(x[4 * jj + 2] * dB0, x[4 * jj + 3] * dB1);
+            if (dst1) {
+                *reinterpret_cast<uint32_t*>(dst1 + offA) = pack2(y[4 * jj] * dA0, y[4 * jj + 1] * dA1);
+                *reinterpret_cast<uint32_t*>(dst1 + offB) = pack2(y[4 * jj + 2] * dB0, y[4 * jj + 3] * dB1);
+            }
         }
     }
 }
 
-// State pass over the two column batches cb0, cb0+1 (32 columns each, cb0 even) of a [128 x 128] float32 accumulator at
-// TMEM columns `acc`; the thread owns lane a = threadIdx.x & 127.  Writes the bf16 copy of the state
-// to `sb` (two boxes of [128 rows x 64 columns], 16 KB apart) and scales the accumulator by `decay`.
-// If init != nullptr the state is taken from global memory (init[a*128 + i], or init[i*128 + a] when
-// `transposed`) instead of TMEM.
+// State pass over NU consecutive 16-column units starting at unit u0 of a [128 x 128] float32
+// accumulator at TMEM columns `acc`; the thread owns lane a = threadIdx.x & 127.  Writes the bf16 copy
+// of the state to `sb` (two boxes of [128 rows x 64 columns], 16 KB apart) and scales the accumulator
+// by `decay`.  If init != nullptr the state is taken from global memory (init[a*128 + i], or
+// init[i*128 + a] when `transposed`) instead of TMEM.
+template <int NU>
 __device__ __forceinline__ void state_pass(uint32_t acc, unsigned char* sb, float decay, const float* __restrict__ init, bool transposed,
-                                           int cb0) {
+                                           int u0) {
     const int a = threadIdx.x & 127, warp = a >> 5;
     const uint32_t taddr = acc + ((uint32_t)(warp * 32) << 16);
-    float v[2][32];
+    float v[NU][16];
     if (init) {
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            const int cb = cb0 + k;
+        for (int k = 0; k < NU; ++k) {
+            const int col = (u0 + k) * 16;
             if (transposed) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[k][i] = init[(cb * 32 + i) * D + a];
+                for (int i = 0; i < 16; ++i) v[k][i] = init[(col + i) * D + a];
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    const float4 f = *reinterpret_cast<const float4*>(init + a * D + cb * 32 + i);
+                for (int i = 0; i < 16; i += 4) {
+                    const float4 f = *reinterpret_cast<const float4*>(init + a * D + col + i);
                     v[k][i] = f.x; v[k][i + 1] = f.y; v[k][i + 2] = f.z; v[k][i + 3] = f.w;
                 }
             }
         }
     } else {
-        ptx::tmem_ld32(taddr + cb0 * 32, v[0]);
-        ptx::tmem_ld32(taddr + cb0 * 32 + 32, v[1]);
+#pragma unroll
+        for (int k = 0; k < NU; ++k) ptx::tmem_ld16(taddr + (u0 + k) * 16, v[k]);
         ptx::tmem_ld_wait();
     }
-    unsigned char* box = sb + (cb0 >> 1) * 16384;          // cb0 is even: both batches fall into one box
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
+    for (int k = 0; k < NU; ++k) {
+        const int u = u0 + k;
+        unsigned char* box = sb + (u >> 2) * 16384;
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-            st_unit(box, a, k * 4 + u,
-                    make_uint4(pack2(v[k][u * 8], v[k][u * 8 + 1]), pack2(v[k][u * 8 + 2], v[k][u * 8 + 3]),
-                               pack2(v[k][u * 8 + 4], v[k][u * 8 + 5]), pack2(v[k][u * 8 + 6], v[k][u * 8 + 7])));
+        for (int e = 0; e < 2; ++e)
+            st_unit(box, a, (u & 3) * 2 + e,
+                    make_uint4(pack2(v[k][e * 8], v[k][e * 8 + 1]), pack2(v[k][e * 8 + 2], v[k][e * 8 + 3]),
+                               pack2(v[k][e * 8 + 4], v[k][e * 8 + 5]), pack2(v[k][e * 8 + 6], v[k][e * 8 + 7])));
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[k][i] *= decay;
-        ptx::tmem_st32(taddr + (cb0 + k) * 32, v[k]);
+        for (int i = 0; i < 16; ++i) v[k][i] *= decay;
+        ptx::tmem_st16(taddr + u * 16, v[k]);
     }
     ptx::tmem_st_wait();
+}
+
+// Weighted copy of one [64 x 64] box: dst = diag(w) src, by the 128 threads of a warpgroup (t = 0..127);
+// a thread meets rows (t>>3) + {0, 16, 32, 48}.
+template <typename F>
+__device__ __forceinline__ void scale_box(unsigned char* dst, const unsigned char* src, int t, F w_row) {
+    const uint4* in = reinterpret_cast<const uint4*>(src);
+    uint4* out = reinterpret_cast<uint4*>(dst);
+    uint4 v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = in[t + 128 * i];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float w = w_row((t >> 3) + 16 * i);
+        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v[i]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h2[e]);
+            h2[e] = __floats2bfloat162_rn(f.x * w, f.y * w);
+        }
+        out[t + 128 * i] = v[i];
+    }
 }
 
 // Epilogue of an interleaved accumulator pair at TMEM columns `pair`: out[r][:] = X[r][:] + scale_r * Y[r][:]
@@ -239,16 +266,18 @@ __device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float
     dotA = 0.f;
     dotB = 0.f;
 #pragma unroll
-    for (int hf = 0; hf < 2; ++hf) {
-        float x[32], y[32];
-        ptx::tmem_ld_16x64(taddr + hf * 64, x);
-        ptx::tmem_ld_16x64(taddr + (16u << 16) + hf * 64, y);
+    for (int qt = 0; qt < 4; ++qt) {
+        const int hf = qt >> 1;
+        float x[16], y[16];
+        ptx::tmem_ld_16x32(taddr + qt * 32, x);
+        ptx::tmem_ld_16x32(taddr + (16u << 16) + qt * 32, y);
         ptx::tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int jj = 0; jj < 4; ++jj) {
+            const int j = (qt & 1) * 4 + jj;
             const int col = hf * 64 + 8 * j + cq;
-            const float a0 = fmaf(scaleA, y[4 * j], x[4 * j]), a1 = fmaf(scaleA, y[4 * j + 1], x[4 * j + 1]);
-            const float b0 = fmaf(scaleB, y[4 * j + 2], x[4 * j + 2]), b1 = fmaf(scaleB, y[4 * j + 3], x[4 * j + 3]);
+            const float a0 = fmaf(scaleA, y[4 * jj], x[4 * jj]), a1 = fmaf(scaleA, y[4 * jj + 1], x[4 * jj + 1]);
+            const float b0 = fmaf(scaleB, y[4 * jj + 2], x[4 * jj + 2]), b1 = fmaf(scaleB, y[4 * jj + 3], x[4 * jj + 3]);
             if (EMODE != 0) {
                 uint32_t ea, eb;
                 if (EMODE == 1) {
@@ -283,13 +312,15 @@ __device__ __forceinline__ uint64_t mndesc(uint32_t tile, int ks, uint32_t box_b
     return ptx::smem_desc(tile + ks * 2048, box_bytes);
 }
 
-// Warp roles of the chunk-sweep kernels (16 warps, 128 registers each): warps 0-7 are the two state
-// warpgroups (columns 0-63 / 64-127 of the carried state, plus the weighted-tile pass; lane 0 of warp 0
-// also issues every MMA, right after its own state pass), warps 8-11 compute the decay masks (lane 0
-// of warp 8 also issues the TMA loads), warps 12-15 run epilogues.  The groups work on different
-// chunks at the same time; mbarriers carry the dependencies
-//     scores -> mask -> MMAs <- state pass <- previous MMAs ;  MMAs -> epilogue.
-constexpr int SW_THREADS = 512;
+// Warp roles of the chunk-sweep kernels (20 warps): four compute warpgroups, warp 16 issues the MMAs,
+// warp 17 the TMA loads (lane 0 each), warps 18-19 only fill the fifth warpgroup.  The carried state
+// sits on the critical path (MMA -> rescale -> MMA), so several warpgroups share its rescaling (16-column
+// units) as soon as the previous chunk's state MMAs retire and only then turn to their other jobs:
+//   WG0, WG1: state units, then the weighted tile halves      WG2: state units (forward-state sweeps), decay mask of
+//   the NEXT chunk, dv epilogue (dk/dv pass)                  WG3: epilogues
+// mbarriers carry the dependencies  scores -> mask -> MMAs <- state pass <- previous state MMAs;  MMAs -> epilogue.
+constexpr int SW_THREADS = 640;
+constexpr int W_MMA = 16, W_TMA = 17;
 #define SF_WAIT(bar, parity, code) ptx::mbar_wait(bar, parity, abort_flag, status, code)
 
 // ==================================================================================================
@@ -410,10 +441,7 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 //   dq pass             : (xq, xk, xv) = (dO, v, k), St = H^T (Hs[j] transposed), out = dq, and
 //                         xout[t] = q_t . dq_t (float32), q read from global memory in the epilogue
 // TMEM columns: St 0-127; O pair (intra at lanes +0, inter at lanes +16) double-buffered at 128 / 256;
-// scores double-buffered at 384 / 448.//
-// The state is carried as two independent column halves (b < 64, b >= 64), one per state warpgroup:
-// each half has its own pass -> MMA -> pass chain, so one half's MMAs run while the other half's
-// warps rescale their accumulator, which keeps the tensor pipe fed.
+// scores double-buffered at 384 / 448.
 constexpr int SW_STAGES = 3;
 struct SweepSmem {
     alignas(1024) unsigned char tiles[SW_STAGES][3][TILE];
@@ -422,7 +450,7 @@ struct SweepSmem {
     alignas(1024) unsigned char sb[2 * 16384];
     float bloc[MAXR * C];
     float ctot[MAXR];
-    uint64_t full[SW_STAGES], sc_done[2], am_ready[2], st_ready[2], st_done[2], out_done[2], o_free[2];
+    uint64_t full[SW_STAGES], sc_done[2], am_ready[2], st_ready, w_ready, st_done, out_done[2], o_free[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -441,122 +469,95 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     volatile int* abort_flag = &sm.abort_flag;
     constexpr uint32_t T_ST = 0, T_O = 128, T_SC = 384;
 
-    auto load_chunk = [&](int c) {          // one thread
-        const int s = c % SW_STAGES;
-        ptx::mbar_expect_tx(&sm.full[s], 3 * TILE);
-        const int tok = (int)t0 + c * C;
-        tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
-        tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
-        tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
-    };
-
-    if (tid == 256) {
+    if (tid == 0) {
         sm.abort_flag = 0;
         for (int s = 0; s < SW_STAGES; ++s) ptx::mbar_init(&sm.full[s], 1);
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 128);
-            ptx::mbar_init(&sm.st_ready[i], 128); ptx::mbar_init(&sm.st_done[i], 1);
-            ptx::mbar_init(&sm.out_done[i], 2); ptx::mbar_init(&sm.o_free[i], 128);
+            ptx::mbar_init(&sm.out_done[i], 1); ptx::mbar_init(&sm.o_free[i], 128);
         }
+        ptx::mbar_init(&sm.st_ready, 384);
+        ptx::mbar_init(&sm.w_ready, 256);
+        ptx::mbar_init(&sm.st_done, 1);
         ptx::fence_mbar_init();
-        ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
-        for (int c = 0; c < SW_STAGES && c < nch; ++c) load_chunk(c);
     }
-    if (warp == 0) ptx::tmem_alloc(&sm.tmem_base, 512);
-    prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
+    if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
+    if (warp < 16) prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
 
-    if (warp < 8) {
-        // ---- state warpgroup `hf` (columns 64*hf .. 64*hf+63); its first thread issues this half's MMAs ----
-        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
-        const int hf = warp >> 2, t = tid & 127;
-        const bool issuer = t == 0;
-        constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
-        constexpr uint32_t id_o1 = ptx::idesc_bf16(64, 128, 0, 1);
-        constexpr uint32_t id_o2 = ptx::idesc_bf16(64, 64, 0, 1);       // xq (K-major) x state half (token... feature-major rows)
-        constexpr uint32_t id_st = ptx::idesc_bf16(128, 64, 1, 1);
-        const uint32_t sbh = ptx::smem_u32(sm.sb) + hf * 16384, xvwh = ptx::smem_u32(sm.xvw) + hf * BOX;
-        auto scores = [&](int c) {
-            const int s = c % SW_STAGES;
-            SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
-            ptx::tc_fence_after_sync();
-            const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC + (c & 1) * 64, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
-            ptx::mma_commit(&sm.sc_done[c & 1]);
-        };
-        if (issuer && hf == 0) scores(0);
-        for (int c = 0; c < nch; ++c) {
-            const int s = c % SW_STAGES, bf = c & 1;
-            const float* bch = sm.bloc + c * C;
-            const float bC = sm.ctot[c];
-            SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
-            SF_TR(2 + 3 * hf, c, 0);
-            if (c > 0) SF_WAIT(&sm.st_done[hf], (c - 1) & 1, DEV_TIMEOUT_MMA);
-            ptx::tc_fence_after_sync();
-            SF_TR(2 + 3 * hf, c, 1);
-            // weighted copy of this half's box of xv: 512 units over 128 threads, rows t>>3 + {0,16,32,48}
-            {
-                const uint4* in = reinterpret_cast<const uint4*>(sm.tiles[s][2] + hf * BOX);
-                uint4* outp = reinterpret_cast<uint4*>(sm.xvw + hf * BOX);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float w = fast_exp(bC - bch[(t >> 3) + 16 * i]);
-                    uint4 v = in[t + 128 * i];
-                    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&v);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 f = __bfloat1622float2(h2[e]);
-                        h2[e] = __floats2bfloat162_rn(f.x * w, f.y * w);
-                    }
-                    outp[t + 128 * i] = v;
-                }
+    if (warp == W_TMA) {
+        if (lane == 0) {
+            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
+            for (int c = 0; c < nch; ++c) {
+                const int s = c % SW_STAGES;
+                // the stage was last used by chunk c-3, complete once all its MMAs retired
+                if (c >= SW_STAGES) SF_WAIT(&sm.out_done[(c - SW_STAGES) & 1], ((c - SW_STAGES) >> 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::mbar_expect_tx(&sm.full[s], 3 * TILE);
+                const int tok = (int)t0 + c * C;
+                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
             }
-            SF_TR(2 + 3 * hf, c, 2);
-            state_pass(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 2 * hf);
-            ptx::fence_proxy_async();
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.st_ready[hf]);
-            SF_TR(2 + 3 * hf, c, 3);
-            if (issuer) {
+        }
+    } else if (warp == W_MMA) {
+        if (lane == 0) {
+            constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
+            constexpr uint32_t id_o1 = ptx::idesc_bf16(64, 128, 0, 1);
+            constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
+            const uint32_t sb = ptx::smem_u32(sm.sb), xvw = ptx::smem_u32(sm.xvw);
+            auto scores = [&](int c) {
+                const int s = c % SW_STAGES;
+                SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
+                ptx::tc_fence_after_sync();
+                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC + (c & 1) * 64, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
+                ptx::mma_commit(&sm.sc_done[c & 1]);
+            };
+            scores(0);
+            if (nch > 1) scores(1);
+            for (int c = 0; c < nch; ++c) {
+                const int s = c % SW_STAGES, bf = c & 1;
                 const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]), xv = ptx::smem_u32(sm.tiles[s][2]);
+                const uint32_t am = ptx::smem_u32(sm.am[bf]);
                 const uint32_t to = tmem + T_O + bf * 128;
                 if (c >= 2) SF_WAIT(&sm.o_free[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
-                SF_WAIT(&sm.st_ready[hf], c & 1, DEV_TIMEOUT_MMA);
+                SF_WAIT(&sm.st_ready, c & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                SF_TR(1 + 5 * hf, c, 2);
-                // inter-chunk part of this half's output columns (lanes +16), then the state half
+                SF_TR(1, c, 0);
+                // the state-dependent MMAs first: inter-chunk output (lanes +16), then the state update
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(to + (16u << 16) + hf * 64, kdesc(xq, ks, BOX), mndesc(sbh, ks, 0), id_o2, ks > 0);
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(to + (16u << 16), kdesc(xq, ks, BOX), mndesc(sb, ks, 16384), id_o1, ks > 0);
+                SF_WAIT(&sm.w_ready, c & 1, DEV_TIMEOUT_MMA);        // the weighted tile is written while the MMAs above run
+                ptx::tc_fence_after_sync();
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_ST + hf * 64, mndesc(xk, ks, BOX), mndesc(xvwh, ks, 0), id_st, 1u);
-                ptx::mma_commit(&sm.st_done[hf]);
-                if (hf == 1) {
-                    const uint32_t am = ptx::smem_u32(sm.am[bf]);
-                    SF_WAIT(&sm.am_ready[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
-                    ptx::tc_fence_after_sync();
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_ST, mndesc(xk, ks, BOX), mndesc(xvw, ks, BOX), id_st, 1u);
+                ptx::mma_commit(&sm.st_done);
+                SF_TR(1, c, 1);
+                SF_WAIT(&sm.am_ready[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(to, kdesc(am, ks, BOX), mndesc(xv, ks, BOX), id_o1, ks > 0);            // intra
-                }
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(to, kdesc(am, ks, BOX), mndesc(xv, ks, BOX), id_o1, ks > 0);                // intra
                 ptx::mma_commit(&sm.out_done[bf]);
-                SF_TR(1 + 5 * hf, c, 3);
-                if (hf == 0 && c + 1 < nch) scores(c + 1);      // its accumulator was released by am_ready of chunk c-1
+                SF_TR(1, c, 2);
+                if (c + 2 < nch) scores(c + 2);          // into the score buffer the mask of chunk c has released
+                SF_TR(1, c, 3);
             }
-            __syncwarp();
         }
-    } else if (warp < 12) {
-        // ---- mask warpgroup (thread 256 also feeds the TMA pipeline) ---------------------------------------
-        for (int c = 0; c < nch; ++c) {
+    } else if (warp < 16) {
+        const int wg = warp >> 2, t = tid & 127;
+        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
+        const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
+        __nv_bfloat16* out_h = out + (long long)b * out_bat + (long long)h * D;
+        const __nv_bfloat16* e_h = DQ ? e_glob + (long long)b * out_bat + (long long)h * D : nullptr;
+        float* xo = DQ ? xout + ((long long)b * p.H + h) * p.L : nullptr;
+        auto mask = [&](int c) {
             const int bf = c & 1;
             SF_WAIT(&sm.sc_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
-            if (c >= 2) {
-                // chunk c-2 is complete: Am[bf] is no longer read, and its tile stage can take chunk c+1
-                SF_WAIT(&sm.out_done[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
-                if (tid == 256 && c + 1 < nch) load_chunk(c + 1);
-            }
+            if (c >= 2) SF_WAIT(&sm.out_done[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);      // Am[bf] no longer read
             ptx::tc_fence_after_sync();
             SF_TR(3, c, 0);
             mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], nullptr);
@@ -564,14 +565,8 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(&sm.am_ready[bf]);
             SF_TR(3, c, 1);
-        }
-    } else {
-        // ---- epilogue warpgroup ---------------------------------------------------------------------------
-        const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
-        __nv_bfloat16* out_h = out + (long long)b * out_bat + (long long)h * D;
-        const __nv_bfloat16* e_h = DQ ? e_glob + (long long)b * out_bat + (long long)h * D : nullptr;
-        float* xo = DQ ? xout + ((long long)b * p.H + h) * p.L : nullptr;
-        for (int c = 0; c < nch; ++c) {
+        };
+        auto epilogue = [&](int c) {
             const int bf = c & 1;
             const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
             const float eA = fast_exp(sm.bloc[c * C + rA]), eB = fast_exp(sm.bloc[c * C + rB]);
@@ -585,11 +580,40 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(&sm.o_free[bf]);
             SF_TR(4, c, 1);
+        };
+        if (wg == 3) {
+            for (int c = 0; c < nch; ++c) epilogue(c);
+        } else {
+            if (wg == 2) mask(0);
+            for (int c = 0; c < nch; ++c) {
+                const int s = c % SW_STAGES;
+                const float* bch = sm.bloc + c * C;
+                const float bC = sm.ctot[c];
+                if (wg < 2) SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
+                SF_TR(2, c, 0);
+                if (c > 0) SF_WAIT(&sm.st_done, (c - 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                SF_TR(2, c, 1);
+                // 16-column units: WG0 0-2, WG1 3-5, WG2 6-7
+                if (wg < 2) state_pass<3>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 3 * wg);
+                else        state_pass<2>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 6);
+                ptx::fence_proxy_async();
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive(&sm.st_ready);
+                SF_TR(2, c, 2);
+                if (wg < 2) {
+                    scale_box(sm.xvw + wg * BOX, sm.tiles[s][2] + wg * BOX, t, [&](int row) { return fast_exp(bC - bch[row]); });
+                    ptx::fence_proxy_async();
+                    ptx::mbar_arrive(&sm.w_ready);
+                }
+                SF_TR(2, c, 3);
+                if (wg == 2 && c + 1 < nch) mask(c + 1);
+            }
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) ptx::tmem_dealloc(tmem, 512);
+    if (warp == W_MMA) ptx::tmem_dealloc(tmem, 512);
 }
 
 // ==================================================================================================
@@ -609,7 +633,7 @@ struct DkdvSmem {
     alignas(1024) unsigned char gb[2 * 16384];
     float bloc[MAXR * C];
     float ctot[MAXR];
-    uint64_t full[2], sc_done[2], am_ready[2], st_ready, out_done, o_free;
+    uint64_t full[2], sc_done[2], am_ready[2], st_ready, w_ready, st_done, out_done, o_free;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -628,99 +652,94 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     volatile int* abort_flag = &sm.abort_flag;
     constexpr uint32_t T_G = 0, T_DK = 128, T_DV = 256, T_SC = 384;
 
-    // iteration i handles chunk c = nch-1-i
-    auto load_chunk = [&](int i) {          // one thread
-        const int s = i & 1;
-        ptx::mbar_expect_tx(&sm.full[s], 4 * TILE);
-        const int tok = (int)t0 + (nch - 1 - i) * C;
-        tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
-        tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
-        tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
-        tma_tile(sm.tiles[s][3], &tmD, &sm.full[s], h, tok, b);
-    };
-
-    if (tid == 256) {
+    if (tid == 0) {
         sm.abort_flag = 0;
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&sm.full[i], 1);
             ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 128);
         }
         ptx::mbar_init(&sm.st_ready, 256);
+        ptx::mbar_init(&sm.w_ready, 256);
+        ptx::mbar_init(&sm.st_done, 1);
         ptx::mbar_init(&sm.out_done, 1);
         ptx::mbar_init(&sm.o_free, 256);
         ptx::fence_mbar_init();
-        ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); ptx::prefetch_tmap(&tmD);
-        for (int i = 0; i < 2 && i < nch; ++i) load_chunk(i);
     }
-    if (warp == 0) ptx::tmem_alloc(&sm.tmem_base, 512);
-    prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
+    if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
+    if (warp < 16) prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
 
-    if (warp < 8) {
-        // ---- state warpgroups: exp(b) * Q tile + carried gradient; warp 0 lane 0 issues the MMAs ---------
-        const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
-        const int half = warp >> 2;
-        const bool issuer = tid == 0;
-        constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
-        constexpr uint32_t id_tt = ptx::idesc_bf16(64, 128, 1, 1);     // A^T dO, dA^T Q: both operands token-major
-        constexpr uint32_t id_kn = ptx::idesc_bf16(64, 128, 0, 1);     // K G
-        constexpr uint32_t id_kk = ptx::idesc_bf16(64, 128, 0, 0);     // V G^T
-        constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
-        const uint32_t gb = ptx::smem_u32(sm.gb), qw = ptx::smem_u32(sm.qw);
-        auto scores = [&](int i) {
-            const int s = i & 1;
-            SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
-            ptx::tc_fence_after_sync();
-            const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
-            const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
-            const uint32_t sc = tmem + T_SC + (i & 1) * 64;
+    // iteration i handles chunk c = nch-1-i
+    if (warp == W_TMA) {
+        if (lane == 0) {
+            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); ptx::prefetch_tmap(&tmD);
+            for (int i = 0; i < nch; ++i) {
+                const int s = i & 1;
+                if (i >= 2) SF_WAIT(&sm.out_done, (i - 2) & 1, DEV_TIMEOUT_MMA);       // every MMA of chunk i-2 has retired
+                ptx::mbar_expect_tx(&sm.full[s], 4 * TILE);
+                const int tok = (int)t0 + (nch - 1 - i) * C;
+                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][3], &tmD, &sm.full[s], h, tok, b);
+            }
+        }
+    } else if (warp == W_MMA) {
+        if (lane == 0) {
+            constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
+            constexpr uint32_t id_tt = ptx::idesc_bf16(64, 128, 1, 1);     // A^T dO, dA^T Q: both operands token-major
+            constexpr uint32_t id_kn = ptx::idesc_bf16(64, 128, 0, 1);     // K G
+            constexpr uint32_t id_kk = ptx::idesc_bf16(64, 128, 0, 0);     // V G^T
+            constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
+            const uint32_t gb = ptx::smem_u32(sm.gb), qw = ptx::smem_u32(sm.qw);
+            auto scores = [&](int i) {
+                const int s = i & 1;
+                SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
+                ptx::tc_fence_after_sync();
+                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
+                const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
+                const uint32_t sc = tmem + T_SC + (i & 1) * 64;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(sc, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(sc, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(sc + (16u << 16), kdesc(xd, ks, BOX), kdesc(xv, ks, BOX), id_sc, ks > 0);
-            ptx::mma_commit(&sm.sc_done[i & 1]);
-        };
-        if (issuer) scores(0);
-        for (int i = 0; i < nch; ++i) {
-            const int c = nch - 1 - i, s = i & 1;
-            const float* bch = sm.bloc + c * C;
-            SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
-            if (i > 0) SF_WAIT(&sm.out_done, (i - 1) & 1, DEV_TIMEOUT_MMA);
-            ptx::tc_fence_after_sync();
-            scale_tile<256>(sm.qw, sm.tiles[s][0], tid, [&](int row) { return fast_exp(bch[row]); });
-            state_pass(tmem + T_G, sm.gb, fast_exp(sm.ctot[c]), i == 0 ? G0 : nullptr, false, 2 * half);
-            ptx::fence_proxy_async();
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.st_ready);
-            if (issuer) {
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(sc + (16u << 16), kdesc(xd, ks, BOX), kdesc(xv, ks, BOX), id_sc, ks > 0);
+                ptx::mma_commit(&sm.sc_done[i & 1]);
+            };
+            scores(0);
+            for (int i = 0; i < nch; ++i) {
+                const int s = i & 1;
                 const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
                 const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
                 const uint32_t am = ptx::smem_u32(sm.am[s]), dam = ptx::smem_u32(sm.dam[s]);
-                SF_WAIT(&sm.am_ready[s], (i >> 1) & 1, DEV_TIMEOUT_MMA);
-                if (i >= 1) SF_WAIT(&sm.o_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
                 SF_WAIT(&sm.st_ready, i & 1, DEV_TIMEOUT_MMA);
+                if (i >= 1) SF_WAIT(&sm.o_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
+                // the MMAs that read the bf16 copy of G, then (its weighted tile is written meanwhile) the update of G
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DV + (16u << 16), kdesc(xk, ks, BOX), mndesc(gb, ks, 16384), id_kn, ks > 0);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
+                SF_WAIT(&sm.w_ready, i & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
+                ptx::mma_commit(&sm.st_done);
+                if (i + 1 < nch) scores(i + 1);      // two stages: the next chunk's tiles are already resident
+                SF_WAIT(&sm.am_ready[s], (i >> 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DV, mndesc(am, ks, BOX), mndesc(xd, ks, BOX), id_tt, ks > 0);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DK, mndesc(dam, ks, BOX), mndesc(xq, ks, BOX), id_tt, ks > 0);
                 ptx::mma_commit(&sm.out_done);
-                if (i + 1 < nch) scores(i + 1);
             }
-            __syncwarp();
         }
-    } else {
-        // ---- warps 8-11: masks, TMA feed, then the dv epilogue; warps 12-15: the dk epilogue ------------
-        const bool masker = warp < 12;
+    } else if (warp < 16) {
+        const int wg = warp >> 2, t = tid & 127;
+        const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
         const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
         __nv_bfloat16* dk_h = dk + (long long)b * p.bqk + (long long)h * D;
         __nv_bfloat16* dv_h = dv + (long long)b * p.bv + (long long)h * D;
@@ -729,26 +748,21 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         auto mask = [&](int i) {
             const int c = nch - 1 - i, bf = i & 1;
             SF_WAIT(&sm.sc_done[bf], (i >> 1) & 1, DEV_TIMEOUT_MMA);
+            if (i >= 2) SF_WAIT(&sm.out_done, (i - 2) & 1, DEV_TIMEOUT_MMA);            // am/dam[bf] no longer read
             ptx::tc_fence_after_sync();
             mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], sm.dam[bf]);
             ptx::fence_proxy_async();
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(&sm.am_ready[bf]);
         };
-        if (masker) mask(0);
-        for (int i = 0; i < nch; ++i) {
+        auto epilogue = [&](int i) {
             const int c = nch - 1 - i;
-            // the masks of the next chunk go first: their buffers were last read by the MMAs of chunk i-1,
-            // whose completion this warpgroup observed before the previous epilogue
-            if (masker && i + 1 < nch) mask(i + 1);
             const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
             const float wA = fast_exp(sm.ctot[c] - sm.bloc[c * C + rA]), wB = fast_exp(sm.ctot[c] - sm.bloc[c * C + rB]);
             SF_WAIT(&sm.out_done, i & 1, DEV_TIMEOUT_MMA);
-            // every MMA of chunk i is complete: its tile stage can take chunk i+2
-            if (tid == 256 && i + 2 < nch) load_chunk(i + 2);
             ptx::tc_fence_after_sync();
             float dotA, dotB;
-            if (masker) {
+            if (wg == 2) {
                 pair_epilogue<0>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, nullptr, dotA, dotB);
             } else {
                 pair_epilogue<2>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, nullptr, k_h + tokA * p.tqk,
@@ -757,11 +771,35 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(&sm.o_free);
+        };
+        if (wg >= 2) {
+            if (wg == 2) mask(0);
+            for (int i = 0; i < nch; ++i) {
+                if (wg == 2 && i + 1 < nch) mask(i + 1);
+                epilogue(i);
+            }
+        } else {
+            for (int i = 0; i < nch; ++i) {
+                const int c = nch - 1 - i, s = i & 1;
+                const float* bch = sm.bloc + c * C;
+                SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
+                // qw and the bf16 copy of G are rewritten below; both were last read by MMAs that precede the
+                // state update of the previous chunk in issue order, so its completion covers them
+                if (i > 0) SF_WAIT(&sm.st_done, (i - 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                state_pass<4>(tmem + T_G, sm.gb, fast_exp(sm.ctot[c]), i == 0 ? G0 : nullptr, false, 4 * wg);
+                ptx::fence_proxy_async();
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive(&sm.st_ready);
+                scale_box(sm.qw + wg * BOX, sm.tiles[s][0] + wg * BOX, t, [&](int row) { return fast_exp(bch[row]); });
+                ptx::fence_proxy_async();
+                ptx::mbar_arrive(&sm.w_ready);
+            }
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) ptx::tmem_dealloc(tmem, 512);
+    if (warp == W_MMA) ptx::tmem_dealloc(tmem, 512);
 }
 
 // ---- host launch -------------------------------------------------------------------------------------
