@@ -346,7 +346,7 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                     const float* __restrict__ g, int mode, float* __restrict__ U, float* __restrict__ beta_out, int* status) {
     extern __shared__ unsigned char smem_raw[];
     AggSmem& sm = *reinterpret_cast<AggSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
     const long long t0 = (long long)c0 * C;
@@ -462,7 +462,7 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 long long out_bat, const __nv_bfloat16* __restrict__ e_glob, float* __restrict__ xout, int* status) {
     extern __shared__ unsigned char smem_raw[];
     SweepSmem& sm = *reinterpret_cast<SweepSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
     const long long t0 = (long long)c0 * C;
@@ -645,7 +645,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                float* __restrict__ xk, int* status) {
     extern __shared__ unsigned char smem_raw[];
     DkdvSmem& sm = *reinterpret_cast<DkdvSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int j = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
     const long long t0 = (long long)c0 * C;
@@ -826,7 +826,7 @@ inline sf_status_t launch(int role, const sf_seg_desc_t* d, const SegParams& p, 
     int* status = status_ptr();
     if (!status) return SF_ERR_CUDA;
     if (p.R > MAXR) return SF_ERR_UNSUPPORTED;
-    dim3 grid(p.NB, p.H, p.B);
+    dim3 grid(p.H, p.NB, p.B);
     auto map_qk = [&](CUtensorMap* m, const void* base) { return make_tmap(m, base, p.B, p.L, p.H, p.tqk, p.bqk); };
     auto map_v = [&](CUtensorMap* m, const void* base) { return make_tmap(m, base, p.B, p.L, p.H, p.tv, p.bv); };
     if (role == 0) {
