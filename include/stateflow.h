@@ -122,6 +122,35 @@ sf_status_t sf_segment_bwd(const sf_seg_desc_t* desc, const void* q, const void*
                            sf_stream_t stream);
 
 /*
+ * sf_segment_fwd for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for the library's users, not for the method.)
+ *
+ * Some callers have no way to hand over a workspace: code running inside a CUDA-graph capture or
+ * under a memory pool that forbids new allocations, plug-ins that receive only their input and
+ * output pointers from a host framework, and real-time loops that must not touch the allocator.
+ * For them the block aggregates and block-entering states live in a scratch array that is part of
+ * the library image itself (SF_STATIC_SCRATCH_BYTES bytes, held by every GPU that loads the library
+ * until the process exits).  The call allocates nothing: no cudaMalloc, no cudaFree, no allocating
+ * library routine.  Inputs and outputs are still the caller's, exactly as for sf_segment_fwd.
+ *
+ *  - Limit: sf_workspace_bytes(desc, 0) must not exceed SF_STATIC_SCRATCH_BYTES, i.e. roughly
+ *    B * H * sf_num_blocks(desc) <= 255 for d_k = d_v = 128; larger shapes get SF_ERR_WORKSPACE and
+ *    nothing is launched.
+ *  - The first call on each device looks up the device address of the scratch array (once per
+ *    device, with that device current).  Make that first call before any stream capture begins.
+ *  - All calls share the one array and it keeps whatever the previous call left in it.  The forward
+ *    pass overwrites every scratch element it later reads, so nothing has to be cleared; but two
+ *    calls whose kernels overlap on the GPU (different streams, no ordering between them) race on
+ *    it.  Order such calls yourself.
+ *  - The scratch content cannot be passed to sf_segment_bwd as fwd_saved once another call has run;
+ *    use fwd_saved == NULL (state replay) for the backward of such a segment.
+ */
+#define SF_STATIC_SCRATCH_BYTES (16u << 20)
+sf_status_t sf_segment_fwd_static(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v,
+                                  const float* g, const float* S_in, void* o, float* S_out,
+                                  sf_stream_t stream);
+
+/*
  * The ST stage alone (paper Eq. 2, second line; Eq. 5 / Eq. 7 across boundaries): the first-order
  * linear recurrence over the n = sf_num_blocks(desc) blocks of a segment, element-wise over
  * B*H*d_k*d_v lanes.  B, H, d_k, d_v, seg_len, chunk come from desc; chunks_per_block overrides

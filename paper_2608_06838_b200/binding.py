@@ -55,6 +55,8 @@ def load() -> ctypes.CDLL:
         lib.sf_workspace_bytes.argtypes = [dp, ctypes.c_int]
         lib.sf_segment_fwd.restype = ctypes.c_int
         lib.sf_segment_fwd.argtypes = [dp] + [vp] * 7 + [vp, sz, vp]
+        lib.sf_segment_fwd_static.restype = ctypes.c_int
+        lib.sf_segment_fwd_static.argtypes = [dp] + [vp] * 7 + [vp]
         lib.sf_segment_bwd.restype = ctypes.c_int
         lib.sf_segment_bwd.argtypes = [dp] + [vp] * 12 + [vp, vp, sz, vp]
         lib.sf_state_scan.restype = ctypes.c_int
@@ -125,6 +127,18 @@ def _workspace(nbytes: int, device) -> torch.Tensor:
 def sf_segment_fwd(desc: SegDesc, q, k, v, g, S_in, o, S_out, workspace: torch.Tensor, stream=None):
     _check(load().sf_segment_fwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(S_in), _ptr(o), _ptr(S_out),
                                  _ptr(workspace), workspace.numel(), _stream(stream)), "sf_segment_fwd")
+
+
+SF_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def sf_segment_fwd_static(desc: SegDesc, q, k, v, g, S_in, o, S_out, stream=None):
+    """sf_segment_fwd without a workspace argument: for callers that cannot allocate device memory
+    (graph capture, no-allocation memory pools, plug-ins that only get input/output pointers).  The
+    scratch is a fixed array inside the library; shapes needing more than SF_STATIC_SCRATCH_BYTES
+    raise SF_ERR_WORKSPACE.  Calls share the array, so calls that overlap on the GPU race."""
+    _check(load().sf_segment_fwd_static(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(S_in), _ptr(o), _ptr(S_out),
+                                        _stream(stream)), "sf_segment_fwd_static")
 
 
 def sf_segment_bwd(desc: SegDesc, q, k, v, g, S_in, dO, dS_out, dq, dk, dv, dg, dS_in, fwd_saved, workspace, stream=None):

@@ -362,6 +362,10 @@ sf_status_t validate_chain(const sf_seg_desc_t* d, const int32_t* seg_lens, int3
 
 }  // namespace
 
+// Scratch of sf_segment_fwd_static: part of the library image, one copy per GPU that loads it.  In host
+// code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[SF_STATIC_SCRATCH_BYTES];
+
 // ================================================================================================
 extern "C" {
 
@@ -436,6 +440,31 @@ sf_status_t sf_segment_bwd(const sf_seg_desc_t* desc, const void* q, const void*
     SF_TRY(bwd_dkdv(path, desc, p, x, w, st));
     SF_TRY(bwd_dg(desc, p, x, w, fw.UH, st));
     return SF_OK;
+}
+
+sf_status_t sf_segment_fwd_static(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                  const float* S_in, void* o, float* S_out, sf_stream_t stream) {
+    const Path path = classify(desc);
+    if (path == Path::Invalid) return SF_ERR_INVALID_ARG;
+    if (path == Path::Unsupported) return SF_ERR_UNSUPPORTED;
+    if (sf_workspace_bytes(desc, 0) > SF_STATIC_SCRATCH_BYTES) return SF_ERR_WORKSPACE;
+    // device address of the scratch array, looked up once per device with that device current
+    constexpr int kMaxDevices = 64;
+    static void* scratch_of_device[kMaxDevices] = {};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return SF_ERR_CUDA; }
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        if (!scratch_of_device[dev]) {
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return SF_ERR_CUDA; }
+            scratch_of_device[dev] = ptr;
+        }
+        scratch = scratch_of_device[dev];
+    }
+    return sf_segment_fwd(desc, q, k, v, g, S_in, o, S_out, scratch, SF_STATIC_SCRATCH_BYTES, stream);
 }
 
 sf_status_t sf_state_scan(const sf_seg_desc_t* desc, int32_t chunks_per_block, int32_t reverse, const float* log_decay,
