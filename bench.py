@@ -88,6 +88,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(x: float, dist, device) -> float:
+    """Max of a per-rank scalar (the timing rule for replicas: the slowest rank sets the step time)."""
+    if dist is None:
+        return float(x)
+    import torch
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job tokens/s of `world` independent replicas that each process tokens_per_rank per step."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def pick_workload(args):
     from paper_2608_06838_b200 import inputs
     if args.config == 5:
@@ -203,14 +218,11 @@ def main():
     ms = e0.elapsed_time(e1)
     launches = binding.sf_launch_count() - n0
     assert binding.sf_device_status() == 0, "a bounded device-side wait ran out"
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, dev)
     clocks = sampler.stop() if rank == 0 else None
     ms_per_step = ms / args.steps
     tokens = w.B * w.T
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = replica_throughput(tokens, world, ms_per_step)
 
     # ---- per-stage device times (second pass with the library's stage timers on) -------------------
     stage = None
@@ -244,10 +256,7 @@ def main():
         for _ in range(n_e2e):
             e2e_step()              # synchronises its stream before returning
         dt = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([dt], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(dt, dist, dev)
         nb = lambda t: 0 if t is None else t.numel() * t.element_size()
         h2d = sum(nb(host[n]) for n in ("q", "k", "v", "g", "dO", "S_in", "dS_out"))
         d2h = sum(nb(t) for t in outs.values()) + nb(S_final) + nb(dS_init)

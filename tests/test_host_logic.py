@@ -1,0 +1,149 @@
+"""CPU-only checks: exported symbols, argument validation before any launch, workspace arithmetic,
+the golden regression pin of the oracle, and the multi-rank (replica) bookkeeping on gloo."""
+import ctypes
+import os
+import re
+import sys
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+from paper_2608_06838_b200 import binding, build  # noqa: E402
+from paper_2608_06838_b200.binding import SegDesc  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "stateflow.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sf_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_functions()
+    assert {"sf_segment_fwd", "sf_segment_bwd", "sf_state_scan", "sf_chain_fwd", "sf_chain_bwd"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def desc(**kw):
+    d = dict(B=1, H=2, d_k=128, d_v=128, seg_len=1024, chunk=64, dtype=binding.SF_BF16, chunks_per_block=0)
+    d.update(kw)
+    H, dk, dv = d["H"], d["d_k"], d["d_v"]
+    return SegDesc(d["B"], H, dk, dv, d["seg_len"], d["chunk"], d["dtype"], d["chunks_per_block"],
+                   H * dk, H * dv, H, 0, 0, 0)
+
+
+P = ctypes.c_void_p(0x10000)        # never dereferenced: every call below must fail validation first
+
+
+def fwd(lib, d, q=P, k=P, v=P, g=P, S_in=None, o=P, S_out=ctypes.c_void_p(0x20000), ws=ctypes.c_void_p(0x30000), nbytes=1 << 40):
+    return lib.sf_segment_fwd(ctypes.byref(d), q, k, v, g, S_in, o, S_out, ws, nbytes, None)
+
+
+def test_forward_validation_happens_before_any_launch(lib):
+    assert fwd(lib, desc(), q=None) == 1
+    assert fwd(lib, desc(), S_out=None) == 1
+    assert fwd(lib, desc(seg_len=1000)) == 1                       # not a multiple of the chunk
+    assert fwd(lib, desc(B=0)) == 1
+    assert fwd(lib, desc(d_k=96, d_v=96)) == 2                      # unsupported head width
+    assert fwd(lib, desc(chunk=32)) == 2                            # bf16 d=128 needs chunk 64
+    assert fwd(lib, desc(chunks_per_block=65)) == 1
+    assert fwd(lib, desc(), q=ctypes.c_void_p(0x10004)) == 1        # misaligned
+    assert fwd(lib, desc(), S_in=ctypes.c_void_p(0x20000)) == 1     # S_in aliases S_out
+    assert fwd(lib, desc(), nbytes=16) == 3
+    assert fwd(lib, desc(), ws=None) == 3
+    assert fwd(lib, desc(), ws=ctypes.c_void_p(0x30010)) == 1       # workspace not 256-byte aligned
+
+
+def test_backward_and_scan_validation(lib):
+    d = desc()
+    args = [P] * 4 + [None, P, None] + [P] * 4 + [ctypes.c_void_p(0x40000)]
+    assert lib.sf_segment_bwd(ctypes.byref(d), *args, None, ctypes.c_void_p(0x30000), 16, None) == 3
+    bad = list(args)
+    bad[5] = None                                                   # dO missing
+    assert lib.sf_segment_bwd(ctypes.byref(d), *bad, None, ctypes.c_void_p(0x30000), 1 << 40, None) == 1
+    alias = list(args)
+    alias[6] = ctypes.c_void_p(0x40000)                             # dS_out aliases dS_in
+    assert lib.sf_segment_bwd(ctypes.byref(d), *alias, None, ctypes.c_void_p(0x30000), 1 << 40, None) == 1
+    assert lib.sf_state_scan(ctypes.byref(d), 0, 0, None, P, None, P, P, None) == 1
+    assert lib.sf_state_scan(ctypes.byref(d), 0, 0, P, P, P, P, P, None) == 1       # in aliases out
+    assert lib.sf_segment_fwd_static(ctypes.byref(desc(H=64, seg_len=4096)), P, P, P, P, None, P, P, None) == 3
+
+
+def test_workspace_arithmetic(lib):
+    d = desc(H=32, seg_len=8192)
+    assert binding.sf_num_blocks(d) == 8
+    state = 128 * 128 * 4
+    f = binding.sf_workspace_bytes(d, 0)
+    assert f == 32 * 8 * state + 1024                               # block states + 32*8 block totals (256-byte padded)
+    b1 = binding.sf_workspace_bytes(d, 1)
+    assert b1 == 32 * 8 * state + 2 * 32 * 8192 * 4
+    assert binding.sf_workspace_bytes(d, 2) == b1 + f + 32 * state
+    assert binding.sf_num_blocks(desc(seg_len=17 * 64, chunks_per_block=4)) == 5
+    assert binding.sf_workspace_bytes(desc(seg_len=1000), 0) == 0
+    segs = [12288, 10240, 8192]
+    tot = sum(binding.sf_workspace_bytes(desc(H=32, seg_len=s), 0) for s in segs)
+    assert binding.sf_chain_workspace_bytes(d, segs, 0) == tot
+    assert binding.sf_chain_workspace_bytes(d, segs, 1) == 2 * binding.sf_workspace_bytes(desc(H=32, seg_len=12288), 1)
+    assert binding.sf_chain_workspace_bytes(d, [100], 0) == 0
+
+
+def test_status_strings(lib):
+    assert binding.status_string(0) == "ok"
+    assert "workspace" in binding.status_string(3)
+    assert binding.sf_launch_count() == 0                            # nothing above launched a kernel
+
+
+def test_oracle_reproduces_the_golden_case():
+    import oracle
+    vals = {}
+    with open(os.path.join(ROOT, "tests", "golden", "tiny_case.txt")) as f:
+        lines = [ln for ln in f.read().splitlines() if not ln.startswith("#")]
+    for head, data in zip(lines[0::2], lines[1::2]):
+        name, *shape = head.split()
+        vals[name] = np.array([float(t) for t in data.split()]).reshape([int(s) for s in shape])
+    o, S_out = oracle.segment_fwd(vals["q"], vals["k"], vals["v"], vals["g"], vals["S_in"])
+    grads = oracle.segment_bwd(vals["q"], vals["k"], vals["v"], vals["g"], vals["S_in"], vals["dO"], vals["dS_out"])
+    for name, a in zip(["o", "S_out", "dq", "dk", "dv", "dg", "dS_in"], (o, S_out) + tuple(grads)):
+        np.testing.assert_allclose(a, vals[name], rtol=1e-13, atol=1e-13, err_msg=name)
+    # the first output row can be checked by hand: o_0 = q_0 (e^{g_0} S_in + k_0^T v_0)
+    S1 = np.exp(vals["g"][0, 0, 0]) * vals["S_in"][0, 0] + np.outer(vals["k"][0, 0, 0], vals["v"][0, 0, 0])
+    np.testing.assert_allclose(vals["o"][0, 0, 0], vals["q"][0, 0, 0] @ S1, atol=1e-12)
+
+
+def _replica_rank(rank, world, port, out):
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
+    ms = bench.max_over_ranks(10.0 + 5.0 * rank, dist, "cpu")          # rank 1 is the slow one
+    dist.barrier()
+    if rank == 0:
+        out.put((ms, bench.replica_throughput(1000, world, ms)))
+    dist.destroy_process_group()
+
+
+def test_replica_timing_takes_the_slowest_rank_on_gloo():
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_replica_rank, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    ms, value = out.get(timeout=120)
+    for p in procs:
+        p.join(60)
+        assert p.exitcode == 0
+    assert ms == 15.0
+    assert abs(value - 2 * 1000 / 15e-3) < 1e-6
