@@ -105,6 +105,8 @@ def replica_throughput(tokens_per_rank: int, world: int, ms_per_step: float) -> 
 
 def pick_workload(args):
     from paper_2608_06838_b200 import inputs
+    if getattr(args, "small", False):
+        return inputs.Workload("small-8k", 1, 32, 128, 128, [8192], 64, s_in_sigma=0.02, ds_out_sigma=0.02)
     if args.config == 5:
         return inputs.sweep_config(args.seg_len)
     return inputs.configs()[args.config - 1]
@@ -163,10 +165,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-overlap", action="store_true")
     ap.add_argument("--chunks-per-block", type=int, default=0)
+    ap.add_argument("--small", action="store_true",
+                    help="profiling case: one 8192-token segment, H=32 (tensors still exceed L2); implies no e2e / cpu legs")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.small:
+        args.skip_e2e = args.skip_cpu = True
     if args.impl == "reference":
         run_reference(args)
         return
@@ -292,7 +298,7 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d_k, "d_v": w.d_v, "T": w.T, "segments": w.seg_lens,
-                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or 16, "overlap": overlap,
+                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or "auto", "overlap": overlap,
                    "l2": "inputs (%.0f MB) exceed L2, no flush" % (4 * tokens * w.H * w.d_k * 2 / 1e6),
                    "parallelism": "replicas only"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roof, "path_roofline": path_roof,

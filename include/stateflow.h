@@ -65,7 +65,8 @@ typedef enum { SF_BF16 = 0, SF_F32 = 1 } sf_dtype_t;
  *             d_k, d_v in {32, 64}, chunk in {16, 32, 64}               (CUDA-core kernels)
  * seg_len must be a positive multiple of chunk (the paper rounds boundaries to multiples of 128,
  * Section 3.2).  chunks_per_block sets how many chunks form one block, the only granularity
- * whose states are written to the workspace; 0 picks the default (16).  Heads are independent.
+ * whose states are written to the workspace (at most 32 on the tensor-core path); 0 lets the library
+ * pick the length in [4, 32] that fills the device's SMs best for this shape.  Heads are independent.
  */
 typedef struct {
     int32_t B, H, d_k, d_v;
@@ -78,7 +79,8 @@ typedef struct {
 
 const char* sf_status_string(sf_status_t s);
 
-/* Number of blocks of the segment: ceil((seg_len / chunk) / chunks_per_block).  0 on an invalid descriptor. */
+/* Number of blocks of the segment: ceil((seg_len / chunk) / chunks_per_block), with the library's own choice
+   of chunks_per_block when the descriptor leaves it 0.  0 on an invalid descriptor. */
 int32_t sf_num_blocks(const sf_seg_desc_t* desc);
 
 /*

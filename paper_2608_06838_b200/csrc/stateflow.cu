@@ -74,12 +74,40 @@ Path classify(const sf_seg_desc_t* d) {
     return d->d_k == d->d_v || (d->d_k == 32 && d->d_v == 64) ? Path::Simt : Path::Unsupported;
 }
 
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+        else { cudaGetLastError(); n = 148; }
+    }
+    return n;
+}
+
+// Block length when the caller leaves it open: one CTA per (batch, head, block) and one CTA per SM, so a
+// kernel takes waves * (chunks per block + a fixed per-CTA cost of about three chunk times).  Pick the
+// length in [4, 32] that minimises this; ties go to the longer block (fewer block states in HBM).
+int auto_chunks_per_block(int NC, long long bh) {
+    const int sms = sm_count();
+    int best = kDefaultChunksPerBlock;
+    long long best_cost = -1;
+    for (int r = 4; r <= 32; ++r) {
+        const int reff = r < NC ? r : NC;
+        const long long nb = (NC + reff - 1) / reff;
+        const long long waves = (nb * bh + sms - 1) / sms;
+        const long long cost = waves * (reff + 3);
+        if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = reff; }
+        if (r >= NC) break;
+    }
+    return best;
+}
+
 SegParams make_params(const sf_seg_desc_t* d, int cpb_override = 0) {
     SegParams p;
     p.B = d->B; p.H = d->H; p.L = d->seg_len; p.C = d->chunk;
     p.NC = d->seg_len / d->chunk;
     int r = cpb_override > 0 ? cpb_override : d->chunks_per_block;
-    p.R = r > 0 ? r : kDefaultChunksPerBlock;
+    p.R = r > 0 ? r : auto_chunks_per_block(p.NC, (long long)d->B * d->H);
     p.NB = (p.NC + p.R - 1) / p.R;
     p.tqk = d->tok_stride_qk; p.tv = d->tok_stride_v; p.tg = d->tok_stride_g;
     p.bqk = d->batch_stride_qk; p.bv = d->batch_stride_v; p.bg = d->batch_stride_g;

@@ -76,11 +76,11 @@ def test_backward_and_scan_validation(lib):
     assert lib.sf_segment_bwd(ctypes.byref(d), *alias, None, ctypes.c_void_p(0x30000), 1 << 40, None) == 1
     assert lib.sf_state_scan(ctypes.byref(d), 0, 0, None, P, None, P, P, None) == 1
     assert lib.sf_state_scan(ctypes.byref(d), 0, 0, P, P, P, P, P, None) == 1       # in aliases out
-    assert lib.sf_segment_fwd_static(ctypes.byref(desc(H=64, seg_len=4096)), P, P, P, P, None, P, P, None) == 3
+    assert lib.sf_segment_fwd_static(ctypes.byref(desc(H=64, seg_len=4096, chunks_per_block=16)), P, P, P, P, None, P, P, None) == 3
 
 
 def test_workspace_arithmetic(lib):
-    d = desc(H=32, seg_len=8192)
+    d = desc(H=32, seg_len=8192, chunks_per_block=16)
     assert binding.sf_num_blocks(d) == 8
     state = 128 * 128 * 4
     f = binding.sf_workspace_bytes(d, 0)
@@ -91,9 +91,14 @@ def test_workspace_arithmetic(lib):
     assert binding.sf_num_blocks(desc(seg_len=17 * 64, chunks_per_block=4)) == 5
     assert binding.sf_workspace_bytes(desc(seg_len=1000), 0) == 0
     segs = [12288, 10240, 8192]
-    tot = sum(binding.sf_workspace_bytes(desc(H=32, seg_len=s), 0) for s in segs)
+    tot = sum(binding.sf_workspace_bytes(desc(H=32, seg_len=s, chunks_per_block=16), 0) for s in segs)
     assert binding.sf_chain_workspace_bytes(d, segs, 0) == tot
-    assert binding.sf_chain_workspace_bytes(d, segs, 1) == 2 * binding.sf_workspace_bytes(desc(H=32, seg_len=12288), 1)
+    assert binding.sf_chain_workspace_bytes(d, segs, 1) == 2 * binding.sf_workspace_bytes(desc(H=32, seg_len=12288, chunks_per_block=16), 1)
+    # left open, the block length is chosen per shape (148 SMs assumed without a device): one wave where possible
+    auto = desc(H=32, seg_len=8192)
+    assert binding.sf_num_blocks(auto) == 4                          # 32 chunks per block: 128 CTAs, one wave
+    assert binding.sf_num_blocks(desc(H=16, seg_len=4096)) == 8      # 8 chunks per block: 128 CTAs
+    assert 1 <= binding.sf_num_blocks(desc(H=1, seg_len=64)) <= 1
     assert binding.sf_chain_workspace_bytes(d, [100], 0) == 0
 
 

@@ -51,7 +51,7 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(dtype, d, chunk, tol
 def test_shapes_beyond_the_static_scratch_are_rejected():
     w = Workload("na-big", 1, 64, 128, 128, [64 * 64], 64, seed=23)      # 64 heads x 4 blocks x 64 KB = 16 MiB + totals
     x = inputs.make_inputs(w, DEV)
-    desc = binding.make_desc(x["q"], x["v"], x["g"], w.chunk)
+    desc = binding.make_desc(x["q"], x["v"], x["g"], w.chunk, chunks_per_block=16)
     assert binding.sf_workspace_bytes(desc, 0) > binding.SF_STATIC_SCRATCH_BYTES
     o = torch.empty_like(x["v"])
     S = torch.empty(1, 64, 128, 128, dtype=torch.float32, device=DEV)
