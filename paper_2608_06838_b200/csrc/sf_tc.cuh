@@ -355,7 +355,7 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 
     if (tid == 0) {
         sm.abort_flag = 0;
-        for (int s = 0; s < AGG_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1); ptx::mbar_init(&sm.ready[s], AGG_COMP); }
+        for (int s = 0; s < AGG_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1); ptx::mbar_init(&sm.ready[s], AGG_COMP / 32); }
         ptx::mbar_init(&sm.done, 1);
         ptx::fence_mbar_init();
     }
@@ -411,7 +411,7 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             scale_tile<AGG_COMP>(sm.tiles[s][1], sm.tiles[s][1], tid,
                        [&](int row) { return fast_exp(mode == 0 ? (bC - bch[row]) + cof : bch[row] + cof); });
             ptx::fence_proxy_async();
-            ptx::mbar_arrive(&sm.ready[s]);
+            ptx::mbar_arrive_warp(&sm.ready[s]);
         }
         SF_WAIT(&sm.done, 0, DEV_TIMEOUT_MMA);
         ptx::tc_fence_after_sync();
@@ -473,11 +473,11 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         sm.abort_flag = 0;
         for (int s = 0; s < SW_STAGES; ++s) ptx::mbar_init(&sm.full[s], 1);
         for (int i = 0; i < 2; ++i) {
-            ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 128);
-            ptx::mbar_init(&sm.out_done[i], 1); ptx::mbar_init(&sm.o_free[i], 128);
+            ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 4);
+            ptx::mbar_init(&sm.out_done[i], 1); ptx::mbar_init(&sm.o_free[i], 4);
         }
-        ptx::mbar_init(&sm.st_ready, 384);
-        ptx::mbar_init(&sm.w_ready, 256);
+        ptx::mbar_init(&sm.st_ready, 12);
+        ptx::mbar_init(&sm.w_ready, 8);
         ptx::mbar_init(&sm.st_done, 1);
         ptx::fence_mbar_init();
     }
@@ -525,14 +525,17 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const uint32_t am = ptx::smem_u32(sm.am[bf]);
                 const uint32_t to = tmem + T_O + bf * 128;
                 if (c >= 2) SF_WAIT(&sm.o_free[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
+                SF_TR(7, c, 0);
                 SF_WAIT(&sm.st_ready, c & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
                 SF_TR(1, c, 0);
                 // the state-dependent MMAs first: inter-chunk output (lanes +16), then the state update
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(to + (16u << 16), kdesc(xq, ks, BOX), mndesc(sb, ks, 16384), id_o1, ks > 0);
+                SF_TR(7, c, 1);
                 SF_WAIT(&sm.w_ready, c & 1, DEV_TIMEOUT_MMA);        // the weighted tile is written while the MMAs above run
                 ptx::tc_fence_after_sync();
+                SF_TR(7, c, 2);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_ST, mndesc(xk, ks, BOX), mndesc(xvw, ks, BOX), id_st, 1u);
                 ptx::mma_commit(&sm.st_done);
@@ -563,7 +566,7 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], nullptr);
             ptx::fence_proxy_async();
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.am_ready[bf]);
+            ptx::mbar_arrive_warp(&sm.am_ready[bf]);
             SF_TR(3, c, 1);
         };
         auto epilogue = [&](int c) {
@@ -578,7 +581,7 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                                       DQ ? e_h + tokA * out_tok : nullptr, DQ ? e_h + tokB * out_tok : nullptr, dotA, dotB);
             if (DQ && (lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.o_free[bf]);
+            ptx::mbar_arrive_warp(&sm.o_free[bf]);
             SF_TR(4, c, 1);
         };
         if (wg == 3) {
@@ -590,23 +593,26 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const float* bch = sm.bloc + c * C;
                 const float bC = sm.ctot[c];
                 if (wg < 2) SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
-                SF_TR(2, c, 0);
+                SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 0);
                 if (c > 0) SF_WAIT(&sm.st_done, (c - 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                SF_TR(2, c, 1);
+                SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 1);
                 // 16-column units: WG0 0-2, WG1 3-5, WG2 6-7
                 if (wg < 2) state_pass<3>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 3 * wg);
                 else        state_pass<2>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 6);
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before_sync();
-                ptx::mbar_arrive(&sm.st_ready);
-                SF_TR(2, c, 2);
+                ptx::mbar_arrive_warp(&sm.st_ready);
+                SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 2);
                 if (wg < 2) {
                     scale_box(sm.xvw + wg * BOX, sm.tiles[s][2] + wg * BOX, t, [&](int row) { return fast_exp(bC - bch[row]); });
+                    if (wg == 0) SF_TR(0, c, 1);
                     ptx::fence_proxy_async();
-                    ptx::mbar_arrive(&sm.w_ready);
+                    if (wg == 0) SF_TR(0, c, 2);
+                    ptx::mbar_arrive_warp(&sm.w_ready);
+                    if (wg == 0) SF_TR(0, c, 3);
                 }
-                SF_TR(2, c, 3);
+                SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 3);
                 if (wg == 2 && c + 1 < nch) mask(c + 1);
             }
         }
@@ -656,13 +662,13 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         sm.abort_flag = 0;
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&sm.full[i], 1);
-            ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 128);
+            ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 4);
         }
-        ptx::mbar_init(&sm.st_ready, 256);
-        ptx::mbar_init(&sm.w_ready, 256);
+        ptx::mbar_init(&sm.st_ready, 8);
+        ptx::mbar_init(&sm.w_ready, 8);
         ptx::mbar_init(&sm.st_done, 1);
         ptx::mbar_init(&sm.out_done, 1);
-        ptx::mbar_init(&sm.o_free, 256);
+        ptx::mbar_init(&sm.o_free, 8);
         ptx::fence_mbar_init();
     }
     if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
@@ -753,7 +759,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], sm.dam[bf]);
             ptx::fence_proxy_async();
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.am_ready[bf]);
+            ptx::mbar_arrive_warp(&sm.am_ready[bf]);
         };
         auto epilogue = [&](int i) {
             const int c = nch - 1 - i;
@@ -770,7 +776,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if ((lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
             }
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&sm.o_free);
+            ptx::mbar_arrive_warp(&sm.o_free);
         };
         if (wg >= 2) {
             if (wg == 2) mask(0);
@@ -790,10 +796,10 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 state_pass<4>(tmem + T_G, sm.gb, fast_exp(sm.ctot[c]), i == 0 ? G0 : nullptr, false, 4 * wg);
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before_sync();
-                ptx::mbar_arrive(&sm.st_ready);
+                ptx::mbar_arrive_warp(&sm.st_ready);
                 scale_box(sm.qw + wg * BOX, sm.tiles[s][0] + wg * BOX, t, [&](int row) { return fast_exp(bch[row]); });
                 ptx::fence_proxy_async();
-                ptx::mbar_arrive(&sm.w_ready);
+                ptx::mbar_arrive_warp(&sm.w_ready);
             }
         }
     }
