@@ -639,11 +639,14 @@ struct DkdvSmem {
     alignas(1024) unsigned char gb[2 * 16384];
     float bloc[MAXR * C];
     float ctot[MAXR];
-    uint64_t full[2], sc_done[2], am_ready[2], st_ready, w_ready, st_done, out_done, o_free;
+    uint64_t full[2], sc_done[2], am_ready[2], st_ready, w_ready, st_done[2], dv_done, dk_done, dv_free, dk_free;
     uint32_t tmem_base;
     int abort_flag;
 };
 
+// The dk and dv accumulator pairs are single-buffered (TMEM is full), so each has its own completion and
+// release barrier: the dv epilogue runs while the dk MMAs execute, the dk epilogue while the state update and
+// the next chunk's scores execute, and the next chunk's dv MMAs start as soon as the dv pair is free.
 __global__ void __launch_bounds__(SW_THREADS, 1)
 tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmD, SegParams p, const float* __restrict__ g, const float* __restrict__ Gs,
@@ -663,12 +666,14 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&sm.full[i], 1);
             ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 4);
+            ptx::mbar_init(&sm.st_done[i], 1);
         }
         ptx::mbar_init(&sm.st_ready, 8);
         ptx::mbar_init(&sm.w_ready, 8);
-        ptx::mbar_init(&sm.st_done, 1);
-        ptx::mbar_init(&sm.out_done, 1);
-        ptx::mbar_init(&sm.o_free, 8);
+        ptx::mbar_init(&sm.dv_done, 1);
+        ptx::mbar_init(&sm.dk_done, 1);
+        ptx::mbar_init(&sm.dv_free, 4);
+        ptx::mbar_init(&sm.dk_free, 4);
         ptx::fence_mbar_init();
     }
     if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
@@ -684,7 +689,8 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); ptx::prefetch_tmap(&tmD);
             for (int i = 0; i < nch; ++i) {
                 const int s = i & 1;
-                if (i >= 2) SF_WAIT(&sm.out_done, (i - 2) & 1, DEV_TIMEOUT_MMA);       // every MMA of chunk i-2 has retired
+                // the stage was last used by chunk i-2; st_done is committed after all of that chunk's MMAs
+                if (i >= 2) SF_WAIT(&sm.st_done[s], ((i - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::mbar_expect_tx(&sm.full[s], 4 * TILE);
                 const int tok = (int)t0 + (nch - 1 - i) * C;
                 tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
@@ -721,26 +727,31 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
                 const uint32_t am = ptx::smem_u32(sm.am[s]), dam = ptx::smem_u32(sm.dam[s]);
                 SF_WAIT(&sm.st_ready, i & 1, DEV_TIMEOUT_MMA);
-                if (i >= 1) SF_WAIT(&sm.o_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
+                if (i >= 1) SF_WAIT(&sm.dv_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                // the MMAs that read the bf16 copy of G, then (its weighted tile is written meanwhile) the update of G
+                // dv = A^T dO (lanes +0) + K G (lanes +16)
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DV + (16u << 16), kdesc(xk, ks, BOX), mndesc(gb, ks, 16384), id_kn, ks > 0);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
-                SF_WAIT(&sm.w_ready, i & 1, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
-                ptx::mma_commit(&sm.st_done);
-                if (i + 1 < nch) scores(i + 1);      // two stages: the next chunk's tiles are already resident
                 SF_WAIT(&sm.am_ready[s], (i >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DV, mndesc(am, ks, BOX), mndesc(xd, ks, BOX), id_tt, ks > 0);
+                ptx::mma_commit(&sm.dv_done);
+                // dk = dA^T Q (lanes +0) + V G^T (lanes +16)
+                if (i >= 1) SF_WAIT(&sm.dk_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DK, mndesc(dam, ks, BOX), mndesc(xq, ks, BOX), id_tt, ks > 0);
-                ptx::mma_commit(&sm.out_done);
+                ptx::mma_commit(&sm.dk_done);
+                // G += (diag(exp(b)) Q)^T dO; its completion (and that of everything above) frees G, gb, qw and the tiles
+                SF_WAIT(&sm.w_ready, i & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
+                ptx::mma_commit(&sm.st_done[s]);
+                if (i + 1 < nch) scores(i + 1);      // two stages: the next chunk's tiles are already resident
             }
         }
     } else if (warp < 16) {
@@ -754,44 +765,45 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         auto mask = [&](int i) {
             const int c = nch - 1 - i, bf = i & 1;
             SF_WAIT(&sm.sc_done[bf], (i >> 1) & 1, DEV_TIMEOUT_MMA);
-            if (i >= 2) SF_WAIT(&sm.out_done, (i - 2) & 1, DEV_TIMEOUT_MMA);            // am/dam[bf] no longer read
+            if (i >= 2) SF_WAIT(&sm.st_done[bf], ((i - 2) >> 1) & 1, DEV_TIMEOUT_MMA);     // am/dam[bf] no longer read
             ptx::tc_fence_after_sync();
             mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], sm.dam[bf]);
             ptx::fence_proxy_async();
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive_warp(&sm.am_ready[bf]);
         };
-        auto epilogue = [&](int i) {
-            const int c = nch - 1 - i;
-            const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
-            const float wA = fast_exp(sm.ctot[c] - sm.bloc[c * C + rA]), wB = fast_exp(sm.ctot[c] - sm.bloc[c * C + rB]);
-            SF_WAIT(&sm.out_done, i & 1, DEV_TIMEOUT_MMA);
-            ptx::tc_fence_after_sync();
-            float dotA, dotB;
-            if (wg == 2) {
-                pair_epilogue<0>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, nullptr, dotA, dotB);
-            } else {
-                pair_epilogue<2>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, nullptr, k_h + tokA * p.tqk,
-                                 k_h + tokB * p.tqk, dotA, dotB);
-                if ((lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
-            }
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive_warp(&sm.o_free);
-        };
         if (wg >= 2) {
             if (wg == 2) mask(0);
             for (int i = 0; i < nch; ++i) {
-                if (wg == 2 && i + 1 < nch) mask(i + 1);
-                epilogue(i);
+                const int c = nch - 1 - i;
+                const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
+                const float wA = fast_exp(sm.ctot[c] - sm.bloc[c * C + rA]), wB = fast_exp(sm.ctot[c] - sm.bloc[c * C + rB]);
+                float dotA, dotB;
+                if (wg == 2) {
+                    SF_WAIT(&sm.dv_done, i & 1, DEV_TIMEOUT_MMA);
+                    ptx::tc_fence_after_sync();
+                    pair_epilogue<0>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, nullptr, dotA, dotB);
+                    ptx::tc_fence_before_sync();
+                    ptx::mbar_arrive_warp(&sm.dv_free);
+                    if (i + 1 < nch) mask(i + 1);
+                } else {
+                    SF_WAIT(&sm.dk_done, i & 1, DEV_TIMEOUT_MMA);
+                    ptx::tc_fence_after_sync();
+                    pair_epilogue<2>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, nullptr, k_h + tokA * p.tqk,
+                                     k_h + tokB * p.tqk, dotA, dotB);
+                    if ((lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
+                    ptx::tc_fence_before_sync();
+                    ptx::mbar_arrive_warp(&sm.dk_free);
+                }
             }
         } else {
             for (int i = 0; i < nch; ++i) {
                 const int c = nch - 1 - i, s = i & 1;
                 const float* bch = sm.bloc + c * C;
                 SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
-                // qw and the bf16 copy of G are rewritten below; both were last read by MMAs that precede the
-                // state update of the previous chunk in issue order, so its completion covers them
-                if (i > 0) SF_WAIT(&sm.st_done, (i - 1) & 1, DEV_TIMEOUT_MMA);
+                // G, its bf16 copy and qw are rewritten below; the state update of the previous chunk is committed
+                // after every MMA that read them
+                if (i > 0) SF_WAIT(&sm.st_done[(i - 1) & 1], ((i - 1) >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
                 state_pass<4>(tmem + T_G, sm.gb, fast_exp(sm.ctot[c]), i == 0 ? G0 : nullptr, false, 4 * wg);
                 ptx::fence_proxy_async();
