@@ -183,9 +183,12 @@ sf_status_t sf_state_scan(const sf_seg_desc_t* desc, int32_t chunks_per_block, i
  *   dS_final : nullable = zero;   dS_init : required, receives dS_0^in
  *   fwd_workspace : the workspace sf_chain_fwd filled, or NULL to replay block states
  *   workspace: sf_chain_workspace_bytes(..., fwd_workspace ? 1 : 2) bytes
- * overlap != 0 lets the driver run state-independent stages of neighbouring segments on internal
- * side streams concurrently with the state scans (the split-and-overlap idea of Section 3.4,
- * Eq. 17-18); the result is bit-identical to overlap == 0.  The side streams are joined back
+ * overlap != 0 lets the driver run state-independent stages on internal side streams concurrently
+ * with the state scans (the split-and-overlap idea of Section 3.4, Eq. 17-18): forward, the block
+ * aggregates of the next segment run under the scan and sweep of the current one; backward (with
+ * fwd_workspace given), all aggregates run ahead, the reverse scans chain on `stream`, and each
+ * segment's dq sweep and dk/dv sweep run on two further streams as soon as its own scan is done.
+ * The result is bit-identical to overlap == 0.  The side streams are joined back
  * into `stream` before the call returns, so later work on `stream` sees all outputs.
  */
 size_t sf_chain_workspace_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg,

@@ -234,8 +234,7 @@ class ChainRun:
         self.dS_init = torch.empty(B, H, dk, dv, dtype=torch.float32, device=dev)
         self.save_states = save_states
         self.ws_f = _workspace(sf_chain_workspace_bytes(self.desc, self.seg_lens, 0), dev)
-        state_bytes = (B * H * dk * dv * 4 + 255) // 256 * 256
-        self.ws_b = _workspace(sf_chain_workspace_bytes(self.desc, self.seg_lens, 1 if save_states else 2) + 2 * state_bytes, dev)
+        self.ws_b = _workspace(sf_chain_workspace_bytes(self.desc, self.seg_lens, 1 if save_states else 2), dev)
 
     def forward(self, S_init=None, overlap=True, stream=None):
         sf_chain_fwd(self.desc, self.seg_lens, self.q, self.k, self.v, self.g, S_init, self.o, self.S_bounds, self.ws_f,

@@ -336,8 +336,9 @@ sf_status_t validate_bwd(const sf_seg_desc_t* d, const BwdPtrs& x, const void* s
 
 // Side streams and events of the chaining driver (host objects only; created once per process).
 struct ChainRes {
-    cudaStream_t side[2] = {nullptr, nullptr};
+    cudaStream_t side[3] = {nullptr, nullptr, nullptr};
     cudaEvent_t ev[64] = {};
+    std::vector<cudaEvent_t> pool;          // extra events of the backward driver, grown on demand
     bool ok = false;
     int device = -1;
 };
@@ -357,6 +358,16 @@ sf_status_t chain_resources(ChainRes** out) {
         g_chain.device = dev;
     }
     *out = &g_chain;
+    return SF_OK;
+}
+
+sf_status_t chain_events(ChainRes* res, size_t n) {
+    std::lock_guard<std::mutex> lk(g_chain_mu);
+    while (res->pool.size() < n) {
+        cudaEvent_t e;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return SF_ERR_CUDA; }
+        res->pool.push_back(e);
+    }
     return SF_OK;
 }
 
@@ -520,9 +531,10 @@ size_t sf_chain_workspace_bytes(const sf_seg_desc_t* desc, const int32_t* seg_le
         total += b;
         mx = b > mx ? b : mx;
     }
-    // forward keeps every segment's block states for the backward; the backward ping-pongs two
-    // per-segment workspaces so that neighbouring segments can overlap
-    return backward == 0 ? total : 2 * mx;
+    // forward keeps every segment's block states for the backward; the backward gives every segment its own
+    // workspace and boundary-gradient buffer so that the stages of different segments can run concurrently
+    (void)mx;
+    return backward == 0 ? total : total + (size_t)n_seg * state_bytes(desc);
 }
 
 sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q, const void* k,
@@ -590,49 +602,89 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     const int mode = fwd_workspace ? 1 : 2;
     const size_t need = sf_chain_workspace_bytes(desc, seg_lens, n_seg, mode);
     const size_t sB = state_bytes(desc);
-    if (!workspace || workspace_bytes < need + 2 * sB) return SF_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < need) return SF_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return SF_ERR_INVALID_ARG;
     const void* ptrs[] = {q, k, v, g, S_bounds, dO, dS_final, dq, dk, dv, dg, dS_init, fwd_workspace};
     for (const void* ptr : ptrs) if (ptr && !aligned16(ptr)) return SF_ERR_INVALID_ARG;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const size_t esz = desc->dtype == SF_BF16 ? 2 : 4;
     const size_t sN = (size_t)desc->B * desc->H * desc->d_k * desc->d_v;
-    (void)overlap;
 
-    // layout: [seg ws A][seg ws B][dS ping][dS pong]
+    // layout: [dS buffers: one state per segment][segment workspaces in order]
     char* base = static_cast<char*>(workspace);
-    const size_t half = need / 2;
-    float* dS_buf[2] = {reinterpret_cast<float*>(base + need), reinterpret_cast<float*>(base + need + sB)};
+    char* seg_base = base + (size_t)n_seg * sB;
 
-    // offsets of every segment's saved forward workspace
-    size_t fwd_off_end = 0;
-    for (int i = 0; i < n_seg; ++i) {
-        sf_seg_desc_t t = *desc;
-        t.seg_len = seg_lens[i];
-        fwd_off_end += sf_workspace_bytes(&t, 0);
+    // overlap schedule (Section 3.4, Eq. 18, across segments): only the reverse scans carry the boundary
+    // gradient from segment to segment.  The backward aggregates need no boundary gradient (side stream 0,
+    // ahead of everything), the scans chain on the main stream, and the two sweeps of a segment need only
+    // its own scan: dq sweeps queue on side stream 1, dk/dv sweeps and the dg epilogue on side stream 2.
+    const bool ov = overlap != 0 && fwd_workspace != nullptr;
+    ChainRes* res = nullptr;
+    cudaStream_t s_pre = st, s_dq = st, s_kv = st;
+    if (ov) {
+        SF_TRY(chain_resources(&res));
+        SF_TRY(chain_events(res, 3 * (size_t)n_seg + 4));
+        s_pre = res->side[0]; s_dq = res->side[1]; s_kv = res->side[2];
+        cudaEvent_t e0 = res->pool[3 * (size_t)n_seg];
+        SF_CUDA(cudaEventRecord(e0, st));
+        SF_CUDA(cudaStreamWaitEvent(s_pre, e0, 0));
+        SF_CUDA(cudaStreamWaitEvent(s_dq, e0, 0));
+        SF_CUDA(cudaStreamWaitEvent(s_kv, e0, 0));
     }
-    long long tok = T;
+
+    // per-segment offsets
+    std::vector<size_t> fwd_off(n_seg), bwd_off(n_seg);
+    std::vector<long long> tok0(n_seg);
+    {
+        size_t fo = 0, bo = 0;
+        long long t = 0;
+        for (int i = 0; i < n_seg; ++i) {
+            sf_seg_desc_t d1 = *desc;
+            d1.seg_len = seg_lens[i];
+            fwd_off[i] = fo; bwd_off[i] = bo; tok0[i] = t;
+            fo += sf_workspace_bytes(&d1, 0);
+            bo += sf_workspace_bytes(&d1, mode);
+            t += seg_lens[i];
+        }
+    }
+    auto seg_ptrs = [&](int i, const sf_seg_desc_t& t, const float* dS_next, float* dS_here) {
+        const long long tok = tok0[i];
+        return BwdPtrs{SeqPtr::at(q, tok, t.tok_stride_qk, esz), SeqPtr::at(k, tok, t.tok_stride_qk, esz),
+                       SeqPtr::at(v, tok, t.tok_stride_v, esz),
+                       static_cast<const float*>(SeqPtr::at(g, tok, t.tok_stride_g, sizeof(float))),
+                       S_bounds + (size_t)i * sN, SeqPtr::at(dO, tok, t.tok_stride_v, esz), dS_next,
+                       SeqPtr::at(dq, tok, t.tok_stride_qk, esz), SeqPtr::at(dk, tok, t.tok_stride_qk, esz),
+                       SeqPtr::at(dv, tok, t.tok_stride_v, esz),
+                       static_cast<float*>(SeqPtr::at(dg, tok, t.tok_stride_g, sizeof(float))), dS_here};
+    };
+    auto dS_buf = [&](int i) { return i == 0 ? dS_init : reinterpret_cast<float*>(base + (size_t)i * sB); };
+
+    if (ov) {
+        // all backward aggregates first, in the order the scans will need them
+        for (int i = n_seg - 1; i >= 0; --i) {
+            sf_seg_desc_t t = *desc;
+            t.seg_len = seg_lens[i];
+            const Path path = classify(&t);
+            const SegParams p = make_params(&t);
+            const BwdWs w = bwd_ws(&t, p, seg_base + bwd_off[i]);
+            BwdPtrs x = seg_ptrs(i, t, nullptr, nullptr);
+            SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, s_pre));
+            SF_CUDA(cudaEventRecord(res->pool[3 * (size_t)i], s_pre));
+        }
+    }
     const float* dS_next = dS_final;
     for (int i = n_seg - 1; i >= 0; --i) {
         sf_seg_desc_t t = *desc;
         t.seg_len = seg_lens[i];
-        tok -= seg_lens[i];
-        fwd_off_end -= sf_workspace_bytes(&t, 0);
         const Path path = classify(&t);
         const SegParams p = make_params(&t);
-        char* wsi = base + (size_t)(i & 1) * half;
+        char* wsi = seg_base + bwd_off[i];
         const BwdWs w = bwd_ws(&t, p, wsi);
-        float* dS_here = (i == 0) ? dS_init : dS_buf[i & 1];
-        BwdPtrs x{SeqPtr::at(q, tok, t.tok_stride_qk, esz), SeqPtr::at(k, tok, t.tok_stride_qk, esz),
-                  SeqPtr::at(v, tok, t.tok_stride_v, esz),
-                  static_cast<const float*>(SeqPtr::at(g, tok, t.tok_stride_g, sizeof(float))),
-                  S_bounds + (size_t)i * sN, SeqPtr::at(dO, tok, t.tok_stride_v, esz), dS_next,
-                  SeqPtr::at(dq, tok, t.tok_stride_qk, esz), SeqPtr::at(dk, tok, t.tok_stride_qk, esz),
-                  SeqPtr::at(dv, tok, t.tok_stride_v, esz),
-                  static_cast<float*>(SeqPtr::at(dg, tok, t.tok_stride_g, sizeof(float))), dS_here};
+        float* dS_here = dS_buf(i);
+        BwdPtrs x = seg_ptrs(i, t, dS_next, dS_here);
         FwdWs fw;
         if (fwd_workspace) {
-            fw = fwd_ws(&t, p, const_cast<char*>(static_cast<const char*>(fwd_workspace)) + fwd_off_end);
+            fw = fwd_ws(&t, p, const_cast<char*>(static_cast<const char*>(fwd_workspace)) + fwd_off[i]);
         } else {
             char* fbase = wsi + w.bytes;
             fw = fwd_ws(&t, p, fbase);
@@ -641,12 +693,36 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
             SF_TRY(fwd_pre(path, &t, p, fx, fw, st));
             SF_TRY(fwd_scan(&t, p, fx, fw, st));
         }
-        SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, st));
+        if (ov) {
+            SF_CUDA(cudaStreamWaitEvent(st, res->pool[3 * (size_t)i], 0));
+        } else {
+            SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, st));
+        }
         SF_TRY(bwd_scan(&t, p, x, w, fw.beta, st));
-        SF_TRY(bwd_dq(path, &t, p, x, w, fw.UH, st));
-        SF_TRY(bwd_dkdv(path, &t, p, x, w, st));
-        SF_TRY(bwd_dg(&t, p, x, w, fw.UH, st));
+        if (ov) {
+            cudaEvent_t e_scan = res->pool[3 * (size_t)i + 1], e_dq = res->pool[3 * (size_t)i + 2];
+            SF_CUDA(cudaEventRecord(e_scan, st));
+            SF_CUDA(cudaStreamWaitEvent(s_dq, e_scan, 0));
+            SF_CUDA(cudaStreamWaitEvent(s_kv, e_scan, 0));
+            SF_TRY(bwd_dq(path, &t, p, x, w, fw.UH, s_dq));
+            SF_CUDA(cudaEventRecord(e_dq, s_dq));
+            SF_TRY(bwd_dkdv(path, &t, p, x, w, s_kv));
+            SF_CUDA(cudaStreamWaitEvent(s_kv, e_dq, 0));
+            SF_TRY(bwd_dg(&t, p, x, w, fw.UH, s_kv));
+        } else {
+            SF_TRY(bwd_dq(path, &t, p, x, w, fw.UH, st));
+            SF_TRY(bwd_dkdv(path, &t, p, x, w, st));
+            SF_TRY(bwd_dg(&t, p, x, w, fw.UH, st));
+        }
         dS_next = dS_here;
+    }
+    if (ov) {
+        // join the side streams back into the caller's stream
+        cudaEvent_t e1 = res->pool[3 * (size_t)n_seg + 1], e2 = res->pool[3 * (size_t)n_seg + 2];
+        SF_CUDA(cudaEventRecord(e1, s_dq));
+        SF_CUDA(cudaEventRecord(e2, s_kv));
+        SF_CUDA(cudaStreamWaitEvent(st, e1, 0));
+        SF_CUDA(cudaStreamWaitEvent(st, e2, 0));
     }
     return SF_OK;
 }
@@ -660,7 +736,7 @@ size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, i
     const size_t ng = align_up((size_t)desc->B * T * desc->H * sizeof(float));
     const size_t sB = state_bytes(desc);
     return 4 * nqk + 4 * nv + 2 * ng + (size_t)(n_seg + 1) * sB + 3 * sB +
-           sf_chain_workspace_bytes(desc, seg_lens, n_seg, 0) + sf_chain_workspace_bytes(desc, seg_lens, n_seg, 1) + 2 * sB;
+           sf_chain_workspace_bytes(desc, seg_lens, n_seg, 0) + sf_chain_workspace_bytes(desc, seg_lens, n_seg, 1);
 }
 
 sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q,
@@ -696,7 +772,7 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
     float* dsinit = reinterpret_cast<float*>(take(sB));
     const size_t wf = sf_chain_workspace_bytes(&d, seg_lens, n_seg, 0), wb = sf_chain_workspace_bytes(&d, seg_lens, n_seg, 1);
     char* wsf = take(wf);
-    char* wsb = take(wb + 2 * sB);
+    char* wsb = take(wb);
 
     SF_CUDA(cudaMemcpyAsync(q_, q, bqk, cudaMemcpyHostToDevice, st));
     SF_CUDA(cudaMemcpyAsync(k_, k, bqk, cudaMemcpyHostToDevice, st));
@@ -711,7 +787,7 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
                         bounds_dense, wsf, wf, 1, stream));
     SF_TRY(sf_chain_bwd(&d, seg_lens, n_seg, q_, k_, v_, reinterpret_cast<float*>(g_), bounds_dense, dO_,
                         dS_final ? dsfin : nullptr, dq_, dk_, dv_, reinterpret_cast<float*>(dg_), dsinit, wsf, wsb,
-                        wb + 2 * sB, 1, stream));
+                        wb, 1, stream));
     SF_CUDA(cudaMemcpyAsync(o, o_, bv, cudaMemcpyDeviceToHost, st));
     SF_CUDA(cudaMemcpyAsync(dq, dq_, bqk, cudaMemcpyDeviceToHost, st));
     SF_CUDA(cudaMemcpyAsync(dk, dk_, bqk, cudaMemcpyDeviceToHost, st));
