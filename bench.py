@@ -28,6 +28,10 @@ METRIC = "fwd+bwd tokens/s per linear-recurrence layer"
 UNIT = "tokens/s"
 BYTES_PER_TOKEN_HEAD = 2828          # q,k,v,dO read once, o,dq,dk,dv written once (bf16, d=128), g and dg float32
 DKDV_BYTES_PER_TOKEN_HEAD = 1540     # the dk/dv pass alone: q,k,v,dO + g in, dk,dv out
+# DRAM bytes per token*head of the dk/dv pass from the ncu capture of the small case
+# (profiles/ncu_full_small_case_8k_h32_all_kernels.txt: 278.19 MB read + 105.72 MB written for 262144 token*heads),
+# scaled to a bench launch by the token*heads it processes (traffic grows in proportion)
+DKDV_NCU_TRAFFIC_PER_TOKEN_HEAD = (278.186e6 + 105.722e6) / 262144
 
 
 def peaks():
@@ -231,11 +235,14 @@ def main():
     value = replica_throughput(tokens, world, ms_per_step)
 
     # ---- per-stage device times (second pass with the library's stage timers on) -------------------
+    # (overlap off here: with the side streams on, a kernel's bracketed time would include waiting for SMs
+    # that kernels of other streams hold; the whole-step number above keeps the overlap)
     stage = None
     if rank == 0:
         binding.sf_stage_timing(True)
         for _ in range(args.steps):
-            step()
+            run.forward(x["S_in"], overlap=False)
+            run.backward(x["dS_out"], overlap=False)
         torch.cuda.synchronize()
         stage = binding.sf_stage_timing_read()
         binding.sf_stage_timing(False)
@@ -288,8 +295,9 @@ def main():
             alg = DKDV_BYTES_PER_TOKEN_HEAD * tokens * w.H / len(w.seg_lens)       # mean over this step's launches
         else:
             alg = None
+        traffic = DKDV_NCU_TRAFFIC_PER_TOKEN_HEAD * tokens * w.H / len(w.seg_lens) if dom["name"] == "dkdv" else None
         roof = {"bound": "hbm", "kernel": dom["name"], "achieved": (alg / (per_launch_ms * 1e-3) / 1e9) if alg else None,
-                "peak": peak, "unit": "GB/s", "peak_source": peak_kind, "traffic": None,
+                "peak": peak, "unit": "GB/s", "peak_source": peak_kind, "traffic": traffic,
                 "avg_launch_ms": per_launch_ms, "launches": dom["launches"]}
         roof["frac"] = roof["achieved"] / peak if roof["achieved"] else None
     cpu = None if args.skip_cpu else cpu_baseline(w)
