@@ -191,39 +191,49 @@ __device__ __forceinline__ void state_pass(uint32_t acc, unsigned char* sb, floa
                                            int u0) {
     const int a = threadIdx.x & 127, warp = a >> 5;
     const uint32_t taddr = acc + ((uint32_t)(warp * 32) << 16);
-    float v[NU][16];
-    if (init) {
+    // two units (32 registers) at a time keeps the register footprint small enough for the 96-register budget
 #pragma unroll
-        for (int k = 0; k < NU; ++k) {
-            const int col = (u0 + k) * 16;
-            if (transposed) {
+    for (int k0 = 0; k0 < NU; k0 += 2) {
+        const int nk = (NU - k0) < 2 ? (NU - k0) : 2;
+        float v[2][16];
+        if (init) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[k][i] = init[(col + i) * D + a];
-            } else {
+            for (int k = 0; k < 2; ++k) {
+                if (k < nk) {
+                    const int col = (u0 + k0 + k) * 16;
+                    if (transposed) {
 #pragma unroll
-                for (int i = 0; i < 16; i += 4) {
-                    const float4 f = *reinterpret_cast<const float4*>(init + a * D + col + i);
-                    v[k][i] = f.x; v[k][i + 1] = f.y; v[k][i + 2] = f.z; v[k][i + 3] = f.w;
+                        for (int i = 0; i < 16; ++i) v[k][i] = init[(col + i) * D + a];
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4) {
+                            const float4 f = *reinterpret_cast<const float4*>(init + a * D + col + i);
+                            v[k][i] = f.x; v[k][i + 1] = f.y; v[k][i + 2] = f.z; v[k][i + 3] = f.w;
+                        }
+                    }
                 }
             }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 2; ++k)
+                if (k < nk) ptx::tmem_ld16(taddr + (u0 + k0 + k) * 16, v[k]);
+            ptx::tmem_ld_wait();
         }
-    } else {
 #pragma unroll
-        for (int k = 0; k < NU; ++k) ptx::tmem_ld16(taddr + (u0 + k) * 16, v[k]);
-        ptx::tmem_ld_wait();
-    }
+        for (int k = 0; k < 2; ++k) {
+            if (k < nk) {
+                const int u = u0 + k0 + k;
+                unsigned char* box = sb + (u >> 2) * 16384;
 #pragma unroll
-    for (int k = 0; k < NU; ++k) {
-        const int u = u0 + k;
-        unsigned char* box = sb + (u >> 2) * 16384;
+                for (int e = 0; e < 2; ++e)
+                    st_unit(box, a, (u & 3) * 2 + e,
+                            make_uint4(pack2(v[k][e * 8], v[k][e * 8 + 1]), pack2(v[k][e * 8 + 2], v[k][e * 8 + 3]),
+                                       pack2(v[k][e * 8 + 4], v[k][e * 8 + 5]), pack2(v[k][e * 8 + 6], v[k][e * 8 + 7])));
 #pragma unroll
-        for (int e = 0; e < 2; ++e)
-            st_unit(box, a, (u & 3) * 2 + e,
-                    make_uint4(pack2(v[k][e * 8], v[k][e * 8 + 1]), pack2(v[k][e * 8 + 2], v[k][e * 8 + 3]),
-                               pack2(v[k][e * 8 + 4], v[k][e * 8 + 5]), pack2(v[k][e * 8 + 6], v[k][e * 8 + 7])));
-#pragma unroll
-        for (int i = 0; i < 16; ++i) v[k][i] *= decay;
-        ptx::tmem_st16(taddr + u * 16, v[k]);
+                for (int i = 0; i < 16; ++i) v[k][i] *= decay;
+                ptx::tmem_st16(taddr + u * 16, v[k]);
+            }
+        }
     }
     ptx::tmem_st_wait();
 }
@@ -255,6 +265,34 @@ __device__ __forceinline__ void scale_box(unsigned char* dst, const unsigned cha
 // [64 x 128] bf16 tile in shared memory (EMODE 1) or from global rows (EMODE 2); EMODE 0: none.
 // The thread serves rows rA = 16q + t/4 and rB = rA + 8; out_A/out_B (and e_A/e_B) point at their
 // first element.  On return dotA/dotB hold the full row sums in every thread of the row's lane group.
+// All-to-all among the 4 lanes that share an accumulator row: lane q holds w[j] = bf16 pair of columns
+// 8j + 2q, 8j + 2q + 1 (j = 0..7 of a 64-column half) and ends up with column groups j = q and j = 4 + q
+// complete: out[0..3] = columns 8q .. 8q+7, out[4..7] = columns 32 + 8q .. 32 + 8q + 7.  The four lanes then
+// write 64 contiguous bytes per store instruction.
+// 4 x 4 transpose across the four lanes of a row group by two butterfly exchanges (lane ^ 1, then lane ^ 2):
+// lane q gives up w[i] and ends with the w[q] of lanes 0..3, in lane order.  4 shuffles + 12 selects.
+__device__ __forceinline__ uint4 lanes4_transpose(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
+    const bool p0 = (threadIdx.x & 1) != 0, p1 = (threadIdx.x & 2) != 0;
+    uint32_t s0 = p0 ? w0 : w1, s1 = p0 ? w2 : w3;
+    uint32_t r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
+    const uint32_t a0 = p0 ? r0 : w0, a1 = p0 ? w1 : r0, a2 = p0 ? r1 : w2, a3 = p0 ? w3 : r1;
+    s0 = p1 ? a0 : a2; s1 = p1 ? a1 : a3;
+    r0 = __shfl_xor_sync(0xffffffffu, s0, 2); r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
+    return make_uint4(p1 ? r0 : a0, p1 ? r1 : a1, p1 ? a2 : r0, p1 ? a3 : r1);
+}
+// All-to-all among the 4 lanes that share an accumulator row: lane q holds w[j] = bf16 pair of columns
+// 8j + 2q, 8j + 2q + 1 (j = 0..7 of a 64-column half) and ends up with column groups j = q and j = 4 + q
+// complete: lo = columns 8q .. 8q+7, hi = columns 32 + 8q .. 32 + 8q + 7.  The four lanes then write 64
+// contiguous bytes per store instruction.  The mapping is its own inverse.
+struct Row8 { uint4 lo, hi; };
+__device__ __forceinline__ Row8 row_transpose4(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, uint32_t w4, uint32_t w5,
+                                               uint32_t w6, uint32_t w7) {
+    Row8 r;
+    r.lo = lanes4_transpose(w0, w1, w2, w3);
+    r.hi = lanes4_transpose(w4, w5, w6, w7);
+    return r;
+}
+
 template <int EMODE>
 __device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float scaleB, __nv_bfloat16* __restrict__ out_A,
                                               __nv_bfloat16* __restrict__ out_B, const unsigned char* etile,
@@ -266,35 +304,60 @@ __device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float
     dotA = 0.f;
     dotB = 0.f;
 #pragma unroll
-    for (int qt = 0; qt < 4; ++qt) {
-        const int hf = qt >> 1;
-        float x[16], y[16];
-        ptx::tmem_ld_16x32(taddr + qt * 32, x);
-        ptx::tmem_ld_16x32(taddr + (16u << 16) + qt * 32, y);
-        ptx::tmem_ld_wait();
+    for (int hf = 0; hf < 2; ++hf) {
+        uint32_t wa[8], wb[8];
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-            const int j = (qt & 1) * 4 + jj;
-            const int col = hf * 64 + 8 * j + cq;
-            const float a0 = fmaf(scaleA, y[4 * jj], x[4 * jj]), a1 = fmaf(scaleA, y[4 * jj + 1], x[4 * jj + 1]);
-            const float b0 = fmaf(scaleB, y[4 * jj + 2], x[4 * jj + 2]), b1 = fmaf(scaleB, y[4 * jj + 3], x[4 * jj + 3]);
-            if (EMODE != 0) {
-                uint32_t ea, eb;
-                if (EMODE == 1) {
-                    const unsigned char* box = etile + hf * BOX;
-                    ea = *reinterpret_cast<const uint32_t*>(box + rA * 128 + ((j ^ (rA & 7)) << 4) + 2 * cq);
-                    eb = *reinterpret_cast<const uint32_t*>(box + rB * 128 + ((j ^ (rB & 7)) << 4) + 2 * cq);
-                } else {
-                    ea = *reinterpret_cast<const uint32_t*>(e_A + col);
-                    eb = *reinterpret_cast<const uint32_t*>(e_B + col);
+        for (int qt = 0; qt < 2; ++qt) {
+            float x[16], y[16];
+            ptx::tmem_ld_16x32(taddr + hf * 64 + qt * 32, x);
+            ptx::tmem_ld_16x32(taddr + (16u << 16) + hf * 64 + qt * 32, y);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = qt * 4 + jj;
+                const float a0 = fmaf(scaleA, y[4 * jj], x[4 * jj]), a1 = fmaf(scaleA, y[4 * jj + 1], x[4 * jj + 1]);
+                const float b0 = fmaf(scaleB, y[4 * jj + 2], x[4 * jj + 2]), b1 = fmaf(scaleB, y[4 * jj + 3], x[4 * jj + 3]);
+                if (EMODE != 0) {
+                    uint32_t ea, eb;
+                    if (EMODE == 1) {
+                        const unsigned char* box = etile + hf * BOX;
+                        ea = *reinterpret_cast<const uint32_t*>(box + rA * 128 + ((j ^ (rA & 7)) << 4) + 2 * cq);
+                        eb = *reinterpret_cast<const uint32_t*>(box + rB * 128 + ((j ^ (rB & 7)) << 4) + 2 * cq);
+                    } else {
+                        const int col = hf * 64 + 8 * j + cq;
+                        ea = *reinterpret_cast<const uint32_t*>(e_A + col);
+                        eb = *reinterpret_cast<const uint32_t*>(e_B + col);
+                    }
+                    const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ea));
+                    const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&eb));
+                    dotA = fmaf(a0, fa.x, dotA); dotA = fmaf(a1, fa.y, dotA);
+                    dotB = fmaf(b0, fb.x, dotB); dotB = fmaf(b1, fb.y, dotB);
                 }
-                const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ea));
-                const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&eb));
-                dotA = fmaf(a0, fa.x, dotA); dotA = fmaf(a1, fa.y, dotA);
-                dotB = fmaf(b0, fb.x, dotB); dotB = fmaf(b1, fb.y, dotB);
+                if (EMODE == 2) {
+                    // with the dot products in the same loop the direct 4-byte stores measured faster than the
+                    // exchange below (register pressure), so this variant keeps them
+                    const int col = hf * 64 + 8 * j + cq;
+                    *reinterpret_cast<uint32_t*>(out_A + col) = pack2(a0, a1);
+                    *reinterpret_cast<uint32_t*>(out_B + col) = pack2(b0, b1);
+                } else {
+                    wa[j] = pack2(a0, a1);
+                    wb[j] = pack2(b0, b1);
+                }
             }
-            *reinterpret_cast<uint32_t*>(out_A + col) = pack2(a0, a1);
-            *reinterpret_cast<uint32_t*>(out_B + col) = pack2(b0, b1);
+        }
+        // 4-byte stores issue eight times as many store instructions: exchange within the row's four lanes
+        // so that they write 64 contiguous bytes per instruction
+        if (EMODE != 2) {
+            const Row8 o = row_transpose4(wa[0], wa[1], wa[2], wa[3], wa[4], wa[5], wa[6], wa[7]);
+            uint4* pa = reinterpret_cast<uint4*>(out_A + hf * 64 + 8 * (lane & 3));
+            pa[0] = o.lo;
+            pa[4] = o.hi;                                        // +32 columns = 4 x 16 bytes
+        }
+        if (EMODE != 2) {
+            const Row8 o = row_transpose4(wb[0], wb[1], wb[2], wb[3], wb[4], wb[5], wb[6], wb[7]);
+            uint4* pb = reinterpret_cast<uint4*>(out_B + hf * 64 + 8 * (lane & 3));
+            pb[0] = o.lo;
+            pb[4] = o.hi;
         }
     }
     if (EMODE != 0) {
@@ -530,20 +593,26 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 ptx::tc_fence_after_sync();
                 SF_TR(1, c, 0);
                 // the state-dependent MMAs first: inter-chunk output (lanes +16), then the state update
+                {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(to + (16u << 16), kdesc(xq, ks, BOX), mndesc(sb, ks, 16384), id_o1, ks > 0);
+                }
                 SF_TR(7, c, 1);
                 SF_WAIT(&sm.w_ready, c & 1, DEV_TIMEOUT_MMA);        // the weighted tile is written while the MMAs above run
                 ptx::tc_fence_after_sync();
                 SF_TR(7, c, 2);
+                {
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_ST, mndesc(xk, ks, BOX), mndesc(xvw, ks, BOX), id_st, 1u);
+                }
                 ptx::mma_commit(&sm.st_done);
                 SF_TR(1, c, 1);
                 SF_WAIT(&sm.am_ready[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
+                {
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(to, kdesc(am, ks, BOX), mndesc(xv, ks, BOX), id_o1, ks > 0);                // intra
+                }
                 ptx::mma_commit(&sm.out_done[bf]);
                 SF_TR(1, c, 2);
                 if (c + 2 < nch) scores(c + 2);          // into the score buffer the mask of chunk c has released
@@ -598,8 +667,10 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 ptx::tc_fence_after_sync();
                 SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 1);
                 // 16-column units: WG0 0-2, WG1 3-5, WG2 6-7
+                {
                 if (wg < 2) state_pass<3>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 3 * wg);
                 else        state_pass<2>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 6);
+                }
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive_warp(&sm.st_ready);
@@ -789,8 +860,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 } else {
                     SF_WAIT(&sm.dk_done, i & 1, DEV_TIMEOUT_MMA);
                     ptx::tc_fence_after_sync();
-                    pair_epilogue<2>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, nullptr, k_h + tokA * p.tqk,
-                                     k_h + tokB * p.tqk, dotA, dotB);
+                    pair_epilogue<2>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, nullptr, k_h + tokA * p.tqk, k_h + tokB * p.tqk, dotA, dotB);
                     if ((lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dk_free);
