@@ -260,17 +260,9 @@ __device__ __forceinline__ void scale_box(unsigned char* dst, const unsigned cha
     }
 }
 
-// Epilogue of an interleaved accumulator pair at TMEM columns `pair`: out[r][:] = X[r][:] + scale_r * Y[r][:]
-// as bf16 to global rows, and row dot products dot_r = sum_c out[r][c] * e[r][c] where e comes from a
-// [64 x 128] bf16 tile in shared memory (EMODE 1) or from global rows (EMODE 2); EMODE 0: none.
-// The thread serves rows rA = 16q + t/4 and rB = rA + 8; out_A/out_B (and e_A/e_B) point at their
-// first element.  On return dotA/dotB hold the full row sums in every thread of the row's lane group.
-// All-to-all among the 4 lanes that share an accumulator row: lane q holds w[j] = bf16 pair of columns
-// 8j + 2q, 8j + 2q + 1 (j = 0..7 of a 64-column half) and ends up with column groups j = q and j = 4 + q
-// complete: out[0..3] = columns 8q .. 8q+7, out[4..7] = columns 32 + 8q .. 32 + 8q + 7.  The four lanes then
-// write 64 contiguous bytes per store instruction.
 // 4 x 4 transpose across the four lanes of a row group by two butterfly exchanges (lane ^ 1, then lane ^ 2):
 // lane q gives up w[i] and ends with the w[q] of lanes 0..3, in lane order.  4 shuffles + 12 selects.
+// The mapping is its own inverse.
 __device__ __forceinline__ uint4 lanes4_transpose(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
     const bool p0 = (threadIdx.x & 1) != 0, p1 = (threadIdx.x & 2) != 0;
     uint32_t s0 = p0 ? w0 : w1, s1 = p0 ? w2 : w3;
@@ -280,87 +272,69 @@ __device__ __forceinline__ uint4 lanes4_transpose(uint32_t w0, uint32_t w1, uint
     r0 = __shfl_xor_sync(0xffffffffu, s0, 2); r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
     return make_uint4(p1 ? r0 : a0, p1 ? r1 : a1, p1 ? a2 : r0, p1 ? a3 : r1);
 }
-// All-to-all among the 4 lanes that share an accumulator row: lane q holds w[j] = bf16 pair of columns
-// 8j + 2q, 8j + 2q + 1 (j = 0..7 of a 64-column half) and ends up with column groups j = q and j = 4 + q
-// complete: lo = columns 8q .. 8q+7, hi = columns 32 + 8q .. 32 + 8q + 7.  The four lanes then write 64
-// contiguous bytes per store instruction.  The mapping is its own inverse.
-struct Row8 { uint4 lo, hi; };
-__device__ __forceinline__ Row8 row_transpose4(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, uint32_t w4, uint32_t w5,
-                                               uint32_t w6, uint32_t w7) {
-    Row8 r;
-    r.lo = lanes4_transpose(w0, w1, w2, w3);
-    r.hi = lanes4_transpose(w4, w5, w6, w7);
-    return r;
-}
 
-template <int EMODE>
+struct NoWait { __device__ __forceinline__ void operator()() const {} };
+
+// Epilogue of an interleaved accumulator pair at TMEM columns `pair`: out[r][:] = X[r][:] + scale_r * Y[r][:]
+// as bf16 to global rows and, with DOT, the row dot products dot_r = sum_c out[r][c] * e[r][c] (out in float32)
+// against global rows e.  The thread serves rows rA = 16q + t/4 and rB = rA + 8; out_A/out_B (and e_A/e_B)
+// point at their first element.  On return dotA/dotB hold the full row sums in every lane of the row's group.
+//
+// The accumulator layout gives lane q' = t%4 of a row the bf16 column pairs 8j + 2q' (j = 0..15): 4-byte
+// pieces 16 bytes apart.  Global memory is touched in 16-byte pieces instead (the four lanes of a row
+// cover 64 contiguous bytes per instruction: an eighth of the load/store instructions), and the butterfly
+// above converts between the two layouts in registers.  `ready` is called before the first TMEM read: the e
+// rows are fetched and rearranged before it, so the wait for the accumulator hides their latency.
+template <bool DOT, typename W = NoWait>
 __device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float scaleB, __nv_bfloat16* __restrict__ out_A,
-                                              __nv_bfloat16* __restrict__ out_B, const unsigned char* etile,
-                                              const __nv_bfloat16* __restrict__ e_A, const __nv_bfloat16* __restrict__ e_B,
-                                              float& dotA, float& dotB) {
+                                              __nv_bfloat16* __restrict__ out_B, const __nv_bfloat16* __restrict__ e_A,
+                                              const __nv_bfloat16* __restrict__ e_B, float& dotA, float& dotB, W ready = W()) {
     const int q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
-    const int rA = 16 * q + (lane >> 2), rB = rA + 8, cq = 2 * (lane & 3);
     const uint32_t taddr = pair + ((uint32_t)(q * 32) << 16);
+    const int c16 = 8 * (lane & 3);                      // first column of this lane's 16-byte pieces
     dotA = 0.f;
     dotB = 0.f;
+    uint32_t pa[DOT ? 16 : 1], pb[DOT ? 16 : 1];
+    if (DOT) {
+        uint4 va[4], vb[4];
 #pragma unroll
-    for (int hf = 0; hf < 2; ++hf) {
-        uint32_t wa[8], wb[8];
-#pragma unroll
-        for (int qt = 0; qt < 2; ++qt) {
-            float x[16], y[16];
-            ptx::tmem_ld_16x32(taddr + hf * 64 + qt * 32, x);
-            ptx::tmem_ld_16x32(taddr + (16u << 16) + hf * 64 + qt * 32, y);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-                const int j = qt * 4 + jj;
-                const float a0 = fmaf(scaleA, y[4 * jj], x[4 * jj]), a1 = fmaf(scaleA, y[4 * jj + 1], x[4 * jj + 1]);
-                const float b0 = fmaf(scaleB, y[4 * jj + 2], x[4 * jj + 2]), b1 = fmaf(scaleB, y[4 * jj + 3], x[4 * jj + 3]);
-                if (EMODE != 0) {
-                    uint32_t ea, eb;
-                    if (EMODE == 1) {
-                        const unsigned char* box = etile + hf * BOX;
-                        ea = *reinterpret_cast<const uint32_t*>(box + rA * 128 + ((j ^ (rA & 7)) << 4) + 2 * cq);
-                        eb = *reinterpret_cast<const uint32_t*>(box + rB * 128 + ((j ^ (rB & 7)) << 4) + 2 * cq);
-                    } else {
-                        const int col = hf * 64 + 8 * j + cq;
-                        ea = *reinterpret_cast<const uint32_t*>(e_A + col);
-                        eb = *reinterpret_cast<const uint32_t*>(e_B + col);
-                    }
-                    const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ea));
-                    const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&eb));
-                    dotA = fmaf(a0, fa.x, dotA); dotA = fmaf(a1, fa.y, dotA);
-                    dotB = fmaf(b0, fb.x, dotB); dotB = fmaf(b1, fb.y, dotB);
-                }
-                if (EMODE == 2) {
-                    // with the dot products in the same loop the direct 4-byte stores measured faster than the
-                    // exchange below (register pressure), so this variant keeps them
-                    const int col = hf * 64 + 8 * j + cq;
-                    *reinterpret_cast<uint32_t*>(out_A + col) = pack2(a0, a1);
-                    *reinterpret_cast<uint32_t*>(out_B + col) = pack2(b0, b1);
-                } else {
-                    wa[j] = pack2(a0, a1);
-                    wb[j] = pack2(b0, b1);
-                }
-            }
+        for (int i = 0; i < 4; ++i) {
+            va[i] = __ldg(reinterpret_cast<const uint4*>(e_A + 32 * i + c16));
+            vb[i] = __ldg(reinterpret_cast<const uint4*>(e_B + 32 * i + c16));
         }
-        // 4-byte stores issue eight times as many store instructions: exchange within the row's four lanes
-        // so that they write 64 contiguous bytes per instruction
-        if (EMODE != 2) {
-            const Row8 o = row_transpose4(wa[0], wa[1], wa[2], wa[3], wa[4], wa[5], wa[6], wa[7]);
-            uint4* pa = reinterpret_cast<uint4*>(out_A + hf * 64 + 8 * (lane & 3));
-            pa[0] = o.lo;
-            pa[4] = o.hi;                                        // +32 columns = 4 x 16 bytes
-        }
-        if (EMODE != 2) {
-            const Row8 o = row_transpose4(wb[0], wb[1], wb[2], wb[3], wb[4], wb[5], wb[6], wb[7]);
-            uint4* pb = reinterpret_cast<uint4*>(out_B + hf * 64 + 8 * (lane & 3));
-            pb[0] = o.lo;
-            pb[4] = o.hi;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint4 ta = lanes4_transpose(va[i].x, va[i].y, va[i].z, va[i].w);
+            const uint4 tb = lanes4_transpose(vb[i].x, vb[i].y, vb[i].z, vb[i].w);
+            pa[4 * i] = ta.x; pa[4 * i + 1] = ta.y; pa[4 * i + 2] = ta.z; pa[4 * i + 3] = ta.w;
+            pb[4 * i] = tb.x; pb[4 * i + 1] = tb.y; pb[4 * i + 2] = tb.z; pb[4 * i + 3] = tb.w;
         }
     }
-    if (EMODE != 0) {
+    ready();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {                        // 32 columns at a time: j = 4i .. 4i+3
+        float x[16], y[16];
+        ptx::tmem_ld_16x32(taddr + i * 32, x);
+        ptx::tmem_ld_16x32(taddr + (16u << 16) + i * 32, y);
+        ptx::tmem_ld_wait();
+        uint32_t wa[4], wb[4];
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const float a0 = fmaf(scaleA, y[4 * jj], x[4 * jj]), a1 = fmaf(scaleA, y[4 * jj + 1], x[4 * jj + 1]);
+            const float b0 = fmaf(scaleB, y[4 * jj + 2], x[4 * jj + 2]), b1 = fmaf(scaleB, y[4 * jj + 3], x[4 * jj + 3]);
+            if (DOT) {
+                const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pa[4 * i + jj]));
+                const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pb[4 * i + jj]));
+                dotA = fmaf(a0, fa.x, dotA); dotA = fmaf(a1, fa.y, dotA);
+                dotB = fmaf(b0, fb.x, dotB); dotB = fmaf(b1, fb.y, dotB);
+            }
+            wa[jj] = pack2(a0, a1);
+            wb[jj] = pack2(b0, b1);
+        }
+        *reinterpret_cast<uint4*>(out_A + 32 * i + c16) = lanes4_transpose(wa[0], wa[1], wa[2], wa[3]);
+        *reinterpret_cast<uint4*>(out_B + 32 * i + c16) = lanes4_transpose(wb[0], wb[1], wb[2], wb[3]);
+    }
+    if (DOT) {
         dotA += __shfl_xor_sync(0xffffffffu, dotA, 1); dotA += __shfl_xor_sync(0xffffffffu, dotA, 2);
         dotB += __shfl_xor_sync(0xffffffffu, dotB, 1); dotB += __shfl_xor_sync(0xffffffffu, dotB, 2);
     }
@@ -642,12 +616,14 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const int bf = c & 1;
             const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
             const float eA = fast_exp(sm.bloc[c * C + rA]), eB = fast_exp(sm.bloc[c * C + rB]);
-            SF_WAIT(&sm.out_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
-            ptx::tc_fence_after_sync();
-            SF_TR(4, c, 0);
+            auto ready = [&]() {
+                SF_WAIT(&sm.out_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                SF_TR(4, c, 0);
+            };
             float dotA, dotB;
-            pair_epilogue<DQ ? 2 : 0>(tmem + T_O + bf * 128, eA, eB, out_h + tokA * out_tok, out_h + tokB * out_tok, nullptr,
-                                      DQ ? e_h + tokA * out_tok : nullptr, DQ ? e_h + tokB * out_tok : nullptr, dotA, dotB);
+            pair_epilogue<DQ>(tmem + T_O + bf * 128, eA, eB, out_h + tokA * out_tok, out_h + tokB * out_tok,
+                              DQ ? e_h + tokA * out_tok : nullptr, DQ ? e_h + tokB * out_tok : nullptr, dotA, dotB, ready);
             if (DQ && (lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive_warp(&sm.o_free[bf]);
@@ -667,10 +643,8 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 ptx::tc_fence_after_sync();
                 SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 1);
                 // 16-column units: WG0 0-2, WG1 3-5, WG2 6-7
-                {
                 if (wg < 2) state_pass<3>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 3 * wg);
                 else        state_pass<2>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 6);
-                }
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive_warp(&sm.st_ready);
@@ -850,17 +824,19 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
                 const float wA = fast_exp(sm.ctot[c] - sm.bloc[c * C + rA]), wB = fast_exp(sm.ctot[c] - sm.bloc[c * C + rB]);
                 float dotA, dotB;
+                auto dk_ready = [&]() {
+                    SF_WAIT(&sm.dk_done, i & 1, DEV_TIMEOUT_MMA);
+                    ptx::tc_fence_after_sync();
+                };
                 if (wg == 2) {
                     SF_WAIT(&sm.dv_done, i & 1, DEV_TIMEOUT_MMA);
                     ptx::tc_fence_after_sync();
-                    pair_epilogue<0>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, nullptr, dotA, dotB);
+                    pair_epilogue<false>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, dotA, dotB);
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dv_free);
                     if (i + 1 < nch) mask(i + 1);
                 } else {
-                    SF_WAIT(&sm.dk_done, i & 1, DEV_TIMEOUT_MMA);
-                    ptx::tc_fence_after_sync();
-                    pair_epilogue<2>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, nullptr, k_h + tokA * p.tqk, k_h + tokB * p.tqk, dotA, dotB);
+                    pair_epilogue<true>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, k_h + tokA * p.tqk, k_h + tokB * p.tqk, dotA, dotB, dk_ready);
                     if ((lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dk_free);
