@@ -171,6 +171,9 @@ def main():
     ap.add_argument("--chunks-per-block", type=int, default=0)
     ap.add_argument("--small", action="store_true",
                     help="profiling case: one 8192-token segment, H=32 (tensors still exceed L2); implies no e2e / cpu legs")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="launch the chain from the host every step instead of replaying it as one CUDA graph "
+                         "(sf_chain_graph_*)")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     args = ap.parse_args()
@@ -200,9 +203,19 @@ def main():
     run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk, args.chunks_per_block)
     overlap = not args.no_overlap
 
+    # a graph cannot be recorded on the legacy default stream: that mode runs on a stream of its own
+    work_stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
+    if args.graph:
+        with torch.cuda.stream(work_stream):
+            run.capture(x["S_in"], x["dS_out"], overlap=overlap)
+        work_stream.synchronize()
+
     def step():
-        run.forward(x["S_in"], overlap=overlap)
-        run.backward(x["dS_out"], overlap=overlap)
+        if args.graph:
+            run.replay()
+        else:
+            run.forward(x["S_in"], overlap=overlap)
+            run.backward(x["dS_out"], overlap=overlap)
 
     def barrier():
         torch.cuda.synchronize()
@@ -210,8 +223,9 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step()
+    with torch.cuda.stream(work_stream):
+        for _ in range(args.warmup):
+            step()
     barrier()
     sampler = ClockSampler(local)
     if rank == 0:
@@ -220,10 +234,11 @@ def main():
     n0 = binding.sf_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
+    with torch.cuda.stream(work_stream):
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
     barrier()
     ms = e0.elapsed_time(e1)
     launches = binding.sf_launch_count() - n0
@@ -306,7 +321,7 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d_k, "d_v": w.d_v, "T": w.T, "segments": w.seg_lens,
-                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or "auto", "overlap": overlap,
+                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or "auto", "overlap": overlap, "graph": bool(args.graph),
                    "l2": "inputs (%.0f MB) exceed L2, no flush" % (4 * tokens * w.H * w.d_k * 2 / 1e6),
                    "parallelism": "replicas only"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roof, "path_roofline": path_roof,

@@ -207,6 +207,34 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
                          int32_t overlap, sf_stream_t stream);
 
 /*
+ * The same chain as one CUDA graph.  The paper's timings include inter-chunk state propagation and
+ * kernel-launch overhead (Section 4.4); with short segments the chain is a long list of small kernels
+ * and the host cannot launch them as fast as the device finishes them.  sf_chain_graph_create runs
+ * sf_chain_fwd (and, if dO is not NULL, sf_chain_bwd with the forward workspace) once on `stream` as
+ * it stands, then records the same calls, side streams included, into a graph; sf_chain_graph_launch
+ * replays it.  Arguments are those of sf_chain_fwd / sf_chain_bwd; every pointer is baked into the
+ * graph, so the buffers must stay alive, at the same addresses, until sf_chain_graph_destroy.
+ *   stream : a stream that can be captured (not the legacy default stream, SF_ERR_INVALID_ARG)
+ *   *out   : receives the handle (host object owned by the library); NULL on error
+ * Results are bit-identical to the direct calls.  Errors: those of the direct calls, SF_ERR_UNSUPPORTED
+ * while stage timing is enabled, SF_ERR_CUDA if capture or instantiation fails.
+ * sf_chain_graph_kernels: kernels (of this library) per replay.  The paper has no counterpart.
+ */
+typedef struct sf_chain_graph sf_chain_graph_t;
+
+sf_status_t sf_chain_graph_create(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg,
+                                  const void* q, const void* k, const void* v, const float* g,
+                                  const float* S_init, void* o, float* S_bounds,
+                                  void* fwd_workspace, size_t fwd_workspace_bytes,
+                                  const void* dO, const float* dS_final,
+                                  void* dq, void* dk, void* dv, float* dg, float* dS_init,
+                                  void* bwd_workspace, size_t bwd_workspace_bytes,
+                                  int32_t overlap, sf_stream_t stream, sf_chain_graph_t** out);
+sf_status_t sf_chain_graph_launch(sf_chain_graph_t* graph, sf_stream_t stream);
+int64_t sf_chain_graph_kernels(const sf_chain_graph_t* graph);
+void sf_chain_graph_destroy(sf_chain_graph_t* graph);
+
+/*
  * Host-memory convenience wrappers around the chain driver (the "end-to-end" path): every data
  * pointer is a HOST pointer (pinned memory recommended).  The call copies the inputs to the device
  * buffers in `dev` (caller-allocated device scratch, sf_e2e_device_bytes() bytes, 256-byte

@@ -71,6 +71,15 @@ def load() -> ctypes.CDLL:
         lib.sf_e2e_device_bytes.argtypes = [dp, ip, i32]
         lib.sf_chain_fwd_bwd_host.restype = ctypes.c_int
         lib.sf_chain_fwd_bwd_host.argtypes = [dp, ip, i32] + [vp] * 14 + [vp, sz, vp]
+        lib.sf_chain_graph_create.restype = ctypes.c_int
+        lib.sf_chain_graph_create.argtypes = [dp, ip, i32] + [vp] * 7 + [vp, sz] + [vp] * 7 + [vp, sz, i32, vp,
+                                                                                             ctypes.POINTER(vp)]
+        lib.sf_chain_graph_launch.restype = ctypes.c_int
+        lib.sf_chain_graph_launch.argtypes = [vp, vp]
+        lib.sf_chain_graph_kernels.restype = ctypes.c_int64
+        lib.sf_chain_graph_kernels.argtypes = [vp]
+        lib.sf_chain_graph_destroy.restype = None
+        lib.sf_chain_graph_destroy.argtypes = [vp]
         lib.sf_device_status.restype = i32
         lib.sf_device_status_clear.restype = None
         lib.sf_launch_count.restype = ctypes.c_int64
@@ -175,6 +184,31 @@ def sf_chain_bwd(desc: SegDesc, seg_lens, q, k, v, g, S_bounds, dO, dS_final, dq
                                _stream(stream)), "sf_chain_bwd")
 
 
+def sf_chain_graph_create(desc: SegDesc, seg_lens, q, k, v, g, S_init, o, S_bounds, fwd_workspace, dO, dS_final, dq, dk, dv,
+                          dg, dS_init, bwd_workspace, overlap=True, stream=None) -> ctypes.c_void_p:
+    """Returns the graph handle; `stream` (default: the current stream) must not be the legacy default stream."""
+    handle = ctypes.c_void_p()
+    _check(load().sf_chain_graph_create(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens), _ptr(q), _ptr(k), _ptr(v),
+                                        _ptr(g), _ptr(S_init), _ptr(o), _ptr(S_bounds), _ptr(fwd_workspace),
+                                        fwd_workspace.numel(), _ptr(dO), _ptr(dS_final), _ptr(dq), _ptr(dk), _ptr(dv),
+                                        _ptr(dg), _ptr(dS_init), _ptr(bwd_workspace),
+                                        0 if bwd_workspace is None else bwd_workspace.numel(), int(overlap),
+                                        _stream(stream), ctypes.byref(handle)), "sf_chain_graph_create")
+    return handle
+
+
+def sf_chain_graph_launch(handle, stream=None) -> None:
+    _check(load().sf_chain_graph_launch(handle, _stream(stream)), "sf_chain_graph_launch")
+
+
+def sf_chain_graph_kernels(handle) -> int:
+    return int(load().sf_chain_graph_kernels(handle))
+
+
+def sf_chain_graph_destroy(handle) -> None:
+    load().sf_chain_graph_destroy(handle)
+
+
 def sf_e2e_device_bytes(desc: SegDesc, seg_lens) -> int:
     return int(load().sf_e2e_device_bytes(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens)))
 
@@ -244,3 +278,28 @@ class ChainRun:
         sf_chain_bwd(self.desc, self.seg_lens, self.q, self.k, self.v, self.g, self.S_bounds, self.dO, dS_final, self.dq,
                      self.dk, self.dv, self.dg, self.dS_init, self.ws_f if self.save_states else None, self.ws_b, overlap,
                      stream)
+
+    def capture(self, S_init=None, dS_final=None, overlap=True, stream=None):
+        """Records forward + backward as one CUDA graph (needs saved states); S_init / dS_final must stay alive."""
+        if not self.save_states:
+            raise ValueError("graph capture needs the forward workspace")
+        self.release()
+        self._graph_keep = (S_init, dS_final)
+        self.graph = sf_chain_graph_create(self.desc, self.seg_lens, self.q, self.k, self.v, self.g, S_init, self.o,
+                                           self.S_bounds, self.ws_f, self.dO, dS_final, self.dq, self.dk, self.dv, self.dg,
+                                           self.dS_init, self.ws_b, overlap, stream)
+        return sf_chain_graph_kernels(self.graph)
+
+    def replay(self, stream=None):
+        sf_chain_graph_launch(self.graph, stream)
+
+    def release(self):
+        if getattr(self, "graph", None) is not None:
+            sf_chain_graph_destroy(self.graph)
+            self.graph = None
+
+    def __del__(self):
+        try:
+            self.release()
+        except Exception:
+            pass

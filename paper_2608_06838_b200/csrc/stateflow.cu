@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <mutex>
+#include <new>
 #include <vector>
 
 #include "sf_common.cuh"
@@ -335,8 +336,10 @@ sf_status_t validate_bwd(const sf_seg_desc_t* d, const BwdPtrs& x, const void* s
 }
 
 // Side streams and events of the chaining driver (host objects only; created once per process).
+// Sweeps of consecutive segments go to different streams: a short segment's sweep does not fill the device.
+constexpr int kSweepStreams = 4;
 struct ChainRes {
-    cudaStream_t side[3] = {nullptr, nullptr, nullptr};
+    cudaStream_t side[1 + 2 * kSweepStreams] = {};   // 0: aggregates; then two groups of sweep streams, used round-robin by segment
     cudaEvent_t ev[64] = {};
     std::vector<cudaEvent_t> pool;          // extra events of the backward driver, grown on demand
     bool ok = false;
@@ -558,11 +561,14 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     ChainRes* res = nullptr;
     if (overlap) SF_TRY(chain_resources(&res));
     // overlap schedule (the forward wavefront of Section 3.4, Eq. 17, across segments):
-    //   side stream : Pre(0) Pre(1) Pre(2) ...            (block aggregates need no boundary state)
-    //   main stream : [wait Pre(i)] ST(i) Out(i)          (ST(i) also overlaps Out(i-1)'s tail)
+    //   side stream 0   : Pre(0) Pre(1) Pre(2) ...        (block aggregates need no boundary state)
+    //   main stream     : [wait Pre(i)] ST(i)             (only the scans carry the state from segment to segment)
+    //   side streams 1..: [wait ST(i)] Out(i)             (round-robin, so that the sweeps of short neighbouring
+    //                                                      segments, which do not fill the device, run side by side)
     if (overlap) {
+        SF_TRY(chain_events(res, (size_t)n_seg + 2 + kSweepStreams));
         SF_CUDA(cudaEventRecord(res->ev[0], st));
-        SF_CUDA(cudaStreamWaitEvent(res->side[0], res->ev[0], 0));
+        for (int s = 0; s <= kSweepStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->side[s], res->ev[0], 0));
     }
     size_t ws_off = 0;
     long long tok = 0;
@@ -586,8 +592,23 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
             SF_TRY(fwd_pre(path, &t, p, x, w, st));
         }
         SF_TRY(fwd_scan(&t, p, x, w, st));
-        SF_TRY(fwd_out(path, &t, p, x, w, st));
+        if (overlap) {
+            cudaStream_t s_out = res->side[1 + (i % kSweepStreams)];
+            SF_CUDA(cudaEventRecord(res->pool[i], st));
+            SF_CUDA(cudaStreamWaitEvent(s_out, res->pool[i], 0));
+            SF_TRY(fwd_out(path, &t, p, x, w, s_out));
+        } else {
+            SF_TRY(fwd_out(path, &t, p, x, w, st));
+        }
         tok += seg_lens[i];
+    }
+    if (overlap) {
+        // join the sweep streams back into the caller's stream
+        for (int s = 1; s <= kSweepStreams; ++s) {
+            cudaEvent_t e = res->pool[(size_t)n_seg + s];
+            SF_CUDA(cudaEventRecord(e, res->side[s]));
+            SF_CUDA(cudaStreamWaitEvent(st, e, 0));
+        }
     }
     return SF_OK;
 }
@@ -617,19 +638,18 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     // overlap schedule (Section 3.4, Eq. 18, across segments): only the reverse scans carry the boundary
     // gradient from segment to segment.  The backward aggregates need no boundary gradient (side stream 0,
     // ahead of everything), the scans chain on the main stream, and the two sweeps of a segment need only
-    // its own scan: dq sweeps queue on side stream 1, dk/dv sweeps and the dg epilogue on side stream 2.
+    // its own scan: dq sweeps queue on one group of side streams, dk/dv sweeps and the dg epilogue on another
+    // (round-robin by segment, so that neighbouring short segments share the device).
     const bool ov = overlap != 0 && fwd_workspace != nullptr;
     ChainRes* res = nullptr;
-    cudaStream_t s_pre = st, s_dq = st, s_kv = st;
+    cudaStream_t s_pre = st;
     if (ov) {
         SF_TRY(chain_resources(&res));
-        SF_TRY(chain_events(res, 3 * (size_t)n_seg + 4));
-        s_pre = res->side[0]; s_dq = res->side[1]; s_kv = res->side[2];
+        SF_TRY(chain_events(res, 3 * (size_t)n_seg + 2 + 2 * kSweepStreams));
+        s_pre = res->side[0];
         cudaEvent_t e0 = res->pool[3 * (size_t)n_seg];
         SF_CUDA(cudaEventRecord(e0, st));
-        SF_CUDA(cudaStreamWaitEvent(s_pre, e0, 0));
-        SF_CUDA(cudaStreamWaitEvent(s_dq, e0, 0));
-        SF_CUDA(cudaStreamWaitEvent(s_kv, e0, 0));
+        for (int s = 0; s <= 2 * kSweepStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->side[s], e0, 0));
     }
 
     // per-segment offsets
@@ -701,6 +721,8 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
         SF_TRY(bwd_scan(&t, p, x, w, fw.beta, st));
         if (ov) {
             cudaEvent_t e_scan = res->pool[3 * (size_t)i + 1], e_dq = res->pool[3 * (size_t)i + 2];
+            // the sweeps of neighbouring segments alternate between two pairs of streams
+            cudaStream_t s_dq = res->side[1 + (i % kSweepStreams)], s_kv = res->side[1 + kSweepStreams + (i % kSweepStreams)];
             SF_CUDA(cudaEventRecord(e_scan, st));
             SF_CUDA(cudaStreamWaitEvent(s_dq, e_scan, 0));
             SF_CUDA(cudaStreamWaitEvent(s_kv, e_scan, 0));
@@ -718,13 +740,84 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     }
     if (ov) {
         // join the side streams back into the caller's stream
-        cudaEvent_t e1 = res->pool[3 * (size_t)n_seg + 1], e2 = res->pool[3 * (size_t)n_seg + 2];
-        SF_CUDA(cudaEventRecord(e1, s_dq));
-        SF_CUDA(cudaEventRecord(e2, s_kv));
-        SF_CUDA(cudaStreamWaitEvent(st, e1, 0));
-        SF_CUDA(cudaStreamWaitEvent(st, e2, 0));
+        for (int s = 1; s <= 2 * kSweepStreams; ++s) {
+            cudaEvent_t e = res->pool[3 * (size_t)n_seg + s];
+            SF_CUDA(cudaEventRecord(e, res->side[s]));
+            SF_CUDA(cudaStreamWaitEvent(st, e, 0));
+        }
     }
     return SF_OK;
+}
+
+struct sf_chain_graph {
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    long long kernels = 0;
+};
+
+sf_status_t sf_chain_graph_create(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q,
+                                  const void* k, const void* v, const float* g, const float* S_init, void* o,
+                                  float* S_bounds, void* fwd_workspace, size_t fwd_workspace_bytes, const void* dO,
+                                  const float* dS_final, void* dq, void* dk, void* dv, float* dg, float* dS_init,
+                                  void* bwd_workspace, size_t bwd_workspace_bytes, int32_t overlap, sf_stream_t stream,
+                                  sf_chain_graph_t** out) {
+    if (!out) return SF_ERR_INVALID_ARG;
+    *out = nullptr;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (st == nullptr || st == cudaStreamLegacy) return SF_ERR_INVALID_ARG;
+    {
+        std::lock_guard<std::mutex> lk(g_timing_mu);
+        if (g_timing_on) return SF_ERR_UNSUPPORTED;        // timing events do not belong in a graph
+    }
+    auto run = [&]() -> sf_status_t {
+        SF_TRY(sf_chain_fwd(desc, seg_lens, n_seg, q, k, v, g, S_init, o, S_bounds, fwd_workspace, fwd_workspace_bytes,
+                            overlap, stream));
+        if (dO)
+            SF_TRY(sf_chain_bwd(desc, seg_lens, n_seg, q, k, v, g, S_bounds, dO, dS_final, dq, dk, dv, dg, dS_init,
+                                fwd_workspace, bwd_workspace, bwd_workspace_bytes, overlap, stream));
+        return SF_OK;
+    };
+    // A plain pass first: it validates every argument and creates the per-process host objects (kernel attributes,
+    // side streams, events) outside the capture.
+    SF_TRY(run());
+    const long long before = g_launches.load();
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return SF_ERR_CUDA; }
+    const sf_status_t rs = run();
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+    if (rs != SF_OK || ce != cudaSuccess || !graph) {
+        cudaGetLastError();
+        if (graph) cudaGraphDestroy(graph);
+        return rs != SF_OK ? rs : SF_ERR_CUDA;
+    }
+    sf_chain_graph* h = new (std::nothrow) sf_chain_graph;
+    if (!h) { cudaGraphDestroy(graph); return SF_ERR_CUDA; }
+    h->graph = graph;
+    h->kernels = g_launches.load() - before;
+    if (cudaGraphInstantiate(&h->exec, graph, 0) != cudaSuccess) {
+        cudaGetLastError();
+        cudaGraphDestroy(graph);
+        delete h;
+        return SF_ERR_CUDA;
+    }
+    *out = h;
+    return SF_OK;
+}
+
+sf_status_t sf_chain_graph_launch(sf_chain_graph_t* graph, sf_stream_t stream) {
+    if (!graph || !graph->exec) return SF_ERR_INVALID_ARG;
+    if (cudaGraphLaunch(graph->exec, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return SF_ERR_CUDA; }
+    g_launches.fetch_add(graph->kernels, std::memory_order_relaxed);
+    return SF_OK;
+}
+
+int64_t sf_chain_graph_kernels(const sf_chain_graph_t* graph) { return graph ? graph->kernels : 0; }
+
+void sf_chain_graph_destroy(sf_chain_graph_t* graph) {
+    if (!graph) return;
+    if (graph->exec) cudaGraphExecDestroy(graph->exec);
+    if (graph->graph) cudaGraphDestroy(graph->graph);
+    delete graph;
 }
 
 size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg) {

@@ -1,0 +1,46 @@
+"""The chain recorded as one CUDA graph gives bit-identical results to the direct calls."""
+import pytest
+import torch
+
+from paper_2608_06838_b200 import binding, inputs
+from paper_2608_06838_b200.inputs import Workload
+
+from helpers import NAMES, compare, oracle_reference, run_chain, tolerance
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.mark.parametrize("overlap", [True, False])
+def test_graph_replay_matches_direct_calls(overlap):
+    w = Workload("graph", 1, 3, 128, 128, [1024, 512, 512, 256], 64, s_in_sigma=0.02, ds_out_sigma=0.02, seed=11)
+    x = inputs.make_inputs(w, DEV)
+    direct, _ = run_chain(w, x, overlap=overlap)
+    direct = {n: direct[n].clone() for n in NAMES}
+
+    run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        kernels = run.capture(x["S_in"], x["dS_out"], overlap=overlap)
+        assert kernels == 8 * len(w.seg_lens)        # forward: aggregate, scan, sweep; backward: aggregate, scan, dq, dk/dv, dg
+        for t in (run.o, run.dq, run.dk, run.dv, run.dg, run.dS_init, run.S_bounds):
+            t.zero_()
+        before = binding.sf_launch_count()
+        run.replay()
+        run.replay()
+        assert binding.sf_launch_count() - before == 2 * kernels
+    stream.synchronize()
+    assert binding.sf_device_status() == 0
+    got = dict(o=run.o, S_out=run.S_bounds[-1], dq=run.dq, dk=run.dk, dv=run.dv, dg=run.dg, dS_in=run.dS_init)
+    for n in NAMES:
+        assert torch.equal(got[n], direct[n]), n
+    compare(got, oracle_reference(x), tolerance(w), label="graph")
+    run.release()
+
+
+def test_graph_needs_a_capturable_stream():
+    w = Workload("graph-legacy", 1, 2, 128, 128, [256], 64, seed=12)
+    x = inputs.make_inputs(w, DEV)
+    run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk)
+    with pytest.raises(binding.SfError):
+        run.capture(None, None, stream=torch.cuda.default_stream())

@@ -153,3 +153,17 @@ def test_replica_timing_takes_the_slowest_rank_on_gloo():
         assert p.exitcode == 0
     assert ms == 15.0
     assert abs(value - 2 * 1000 / 15e-3) < 1e-6
+
+
+def test_graph_create_rejects_bad_arguments_before_any_cuda_call(lib):
+    d = desc()
+    segs = (ctypes.c_int32 * 1)(1024)
+    handle = ctypes.c_void_p(0x1)
+    args = [ctypes.byref(d), segs, 1] + [P] * 7 + [P, 1 << 40] + [P] * 7 + [P, 1 << 40, 1]
+    # no place for the handle; then the legacy default stream, which cannot be captured
+    assert lib.sf_chain_graph_create(*args, ctypes.c_void_p(0x40), None) == 1
+    assert lib.sf_chain_graph_create(*args, None, ctypes.byref(handle)) == 1
+    assert handle.value is None                      # cleared on error
+    assert lib.sf_chain_graph_launch(None, None) == 1
+    assert lib.sf_chain_graph_kernels(None) == 0
+    lib.sf_chain_graph_destroy(None)                 # a no-op
