@@ -684,14 +684,15 @@ struct DkdvSmem {
     alignas(1024) unsigned char gb[2 * 16384];
     float bloc[MAXR * C];
     float ctot[MAXR];
-    uint64_t full[2], sc_done[2], am_ready[2], st_ready, w_ready, st_done[2], dv_done, dk_done, dv_free, dk_free;
+    uint64_t full[2], sc_done[2], am_ready[2], st_ready, w_ready, st_done[2], it_done[2], dv_done, dk_done, dv_free, dk_free;
     uint32_t tmem_base;
     int abort_flag;
 };
 
 // The dk and dv accumulator pairs are single-buffered (TMEM is full), so each has its own completion and
-// release barrier: the dv epilogue runs while the dk MMAs execute, the dk epilogue while the state update and
-// the next chunk's scores execute, and the next chunk's dv MMAs start as soon as the dv pair is free.
+// release barrier.  Per iteration the MMAs that read or update the carried gradient G are issued first and
+// st_done is committed right behind them: the rescaling of G for the next chunk (the serial part of the sweep)
+// then overlaps the intra-chunk MMAs, the epilogues and the next chunk's scores.  it_done closes the iteration.
 __global__ void __launch_bounds__(SW_THREADS, 1)
 tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmD, SegParams p, const float* __restrict__ g, const float* __restrict__ Gs,
@@ -712,6 +713,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(&sm.full[i], 1);
             ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 4);
             ptx::mbar_init(&sm.st_done[i], 1);
+            ptx::mbar_init(&sm.it_done[i], 1);
         }
         ptx::mbar_init(&sm.st_ready, 8);
         ptx::mbar_init(&sm.w_ready, 8);
@@ -734,8 +736,8 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); ptx::prefetch_tmap(&tmD);
             for (int i = 0; i < nch; ++i) {
                 const int s = i & 1;
-                // the stage was last used by chunk i-2; st_done is committed after all of that chunk's MMAs
-                if (i >= 2) SF_WAIT(&sm.st_done[s], ((i - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
+                // the stage was last used by iteration i-2; it_done is committed after all of its MMAs
+                if (i >= 2) SF_WAIT(&sm.it_done[s], ((i - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::mbar_expect_tx(&sm.full[s], 4 * TILE);
                 const int tok = (int)t0 + (nch - 1 - i) * C;
                 tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
@@ -771,32 +773,44 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
                 const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
                 const uint32_t am = ptx::smem_u32(sm.am[s]), dam = ptx::smem_u32(sm.dam[s]);
+                SF_TR(1, i, 0);
                 SF_WAIT(&sm.st_ready, i & 1, DEV_TIMEOUT_MMA);
+                SF_TR(1, i, 1);
                 if (i >= 1) SF_WAIT(&sm.dv_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                // dv = A^T dO (lanes +0) + K G (lanes +16)
+                SF_TR(1, i, 2);
+                // Everything that touches the carried gradient goes first, so that its rescaling for the next chunk
+                // runs while the intra-chunk MMAs and the next scores execute:
+                //   dv (lanes +16) = K G,  dk (lanes +16) = V G^T,  G += (diag(exp(b)) Q)^T dO
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DV + (16u << 16), kdesc(xk, ks, BOX), mndesc(gb, ks, 16384), id_kn, ks > 0);
+                SF_TR(1, i, 3);
+                if (i >= 1) SF_WAIT(&sm.dk_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                SF_TR(7, i, 0);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
+                SF_WAIT(&sm.w_ready, i & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                SF_TR(7, i, 1);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
+                ptx::mma_commit(&sm.st_done[s]);                 // G, its bf16 copy and qw are free again
+                SF_TR(7, i, 2);
+                // intra-chunk parts: dv (lanes +0) = A^T dO, dk (lanes +0) = dA^T Q
                 SF_WAIT(&sm.am_ready[s], (i >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
+                SF_TR(7, i, 3);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DV, mndesc(am, ks, BOX), mndesc(xd, ks, BOX), id_tt, ks > 0);
                 ptx::mma_commit(&sm.dv_done);
-                // dk = dA^T Q (lanes +0) + V G^T (lanes +16)
-                if (i >= 1) SF_WAIT(&sm.dk_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DK, mndesc(dam, ks, BOX), mndesc(xq, ks, BOX), id_tt, ks > 0);
                 ptx::mma_commit(&sm.dk_done);
-                // G += (diag(exp(b)) Q)^T dO; its completion (and that of everything above) frees G, gb, qw and the tiles
-                SF_WAIT(&sm.w_ready, i & 1, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
-                ptx::mma_commit(&sm.st_done[s]);
+                ptx::mma_commit(&sm.it_done[s]);                 // tiles and masks of this iteration are free again
+                SF_TR(0, i, 0);
                 if (i + 1 < nch) scores(i + 1);      // two stages: the next chunk's tiles are already resident
+                SF_TR(0, i, 2);
             }
         }
     } else if (warp < 16) {
@@ -810,7 +824,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         auto mask = [&](int i) {
             const int c = nch - 1 - i, bf = i & 1;
             SF_WAIT(&sm.sc_done[bf], (i >> 1) & 1, DEV_TIMEOUT_MMA);
-            if (i >= 2) SF_WAIT(&sm.st_done[bf], ((i - 2) >> 1) & 1, DEV_TIMEOUT_MMA);     // am/dam[bf] no longer read
+            if (i >= 2) SF_WAIT(&sm.it_done[bf], ((i - 2) >> 1) & 1, DEV_TIMEOUT_MMA);     // am/dam[bf] no longer read
             ptx::tc_fence_after_sync();
             mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], sm.dam[bf]);
             ptx::fence_proxy_async();
@@ -825,21 +839,29 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const float wA = fast_exp(sm.ctot[c] - sm.bloc[c * C + rA]), wB = fast_exp(sm.ctot[c] - sm.bloc[c * C + rB]);
                 float dotA, dotB;
                 auto dk_ready = [&]() {
+                    SF_TR(4, i, 1);
                     SF_WAIT(&sm.dk_done, i & 1, DEV_TIMEOUT_MMA);
                     ptx::tc_fence_after_sync();
+                    SF_TR(4, i, 2);
                 };
                 if (wg == 2) {
+                    SF_TR(6, i, 0);
                     SF_WAIT(&sm.dv_done, i & 1, DEV_TIMEOUT_MMA);
                     ptx::tc_fence_after_sync();
+                    SF_TR(6, i, 1);
                     pair_epilogue<false>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, dotA, dotB);
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dv_free);
+                    SF_TR(6, i, 2);
                     if (i + 1 < nch) mask(i + 1);
+                    SF_TR(6, i, 3);
                 } else {
+                    SF_TR(4, i, 0);
                     pair_epilogue<true>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, k_h + tokA * p.tqk, k_h + tokB * p.tqk, dotA, dotB, dk_ready);
                     if ((lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dk_free);
+                    SF_TR(4, i, 3);
                 }
             }
         } else {
@@ -849,15 +871,19 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
                 // G, its bf16 copy and qw are rewritten below; the state update of the previous chunk is committed
                 // after every MMA that read them
+                SF_TR(wg == 0 ? 2 : 5, i, 0);
                 if (i > 0) SF_WAIT(&sm.st_done[(i - 1) & 1], ((i - 1) >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
+                SF_TR(wg == 0 ? 2 : 5, i, 1);
                 state_pass<4>(tmem + T_G, sm.gb, fast_exp(sm.ctot[c]), i == 0 ? G0 : nullptr, false, 4 * wg);
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive_warp(&sm.st_ready);
+                SF_TR(wg == 0 ? 2 : 5, i, 2);
                 scale_box(sm.qw + wg * BOX, sm.tiles[s][0] + wg * BOX, t, [&](int row) { return fast_exp(bch[row]); });
                 ptx::fence_proxy_async();
                 ptx::mbar_arrive_warp(&sm.w_ready);
+                SF_TR(wg == 0 ? 2 : 5, i, 3);
             }
         }
     }
