@@ -519,11 +519,11 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ptx::fence_mbar_init();
     }
     if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
-    if (warp < 16) prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
+    // the decay tables are built by the compute warps while the first tiles are already on their way
 
     if (warp == W_TMA) {
         if (lane == 0) {
@@ -594,6 +594,8 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
         }
     } else if (warp < 16) {
+        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
+        ptx::named_bar_sync(1, 512);
         const int wg = warp >> 2, t = tid & 127;
         const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
         const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
@@ -724,11 +726,11 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         ptx::fence_mbar_init();
     }
     if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
-    if (warp < 16) prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
+    // the decay tables are built by the compute warps while the first tiles are already on their way
 
     // iteration i handles chunk c = nch-1-i
     if (warp == W_TMA) {
@@ -814,6 +816,8 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
         }
     } else if (warp < 16) {
+        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
+        ptx::named_bar_sync(1, 512);
         const int wg = warp >> 2, t = tid & 127;
         const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
         const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
