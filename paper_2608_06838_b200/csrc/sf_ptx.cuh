@@ -197,6 +197,23 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// The same instruction from 32-bit pieces.  The issuing thread has no queue to hide behind: whatever it executes
+// between two tcgen05.mma instructions is idle time of the tensor pipe, so the descriptors of a K loop are formed
+// with one integer add each: the high word of every descriptor here is the same constant and a K step only moves
+// the 14-bit start-address field of the low word (shared memory is smaller than 2^18 bytes: no carry out of it).
+constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+template <int ACC>
+__device__ __forceinline__ void mma_lo(uint32_t d_tmem, uint32_t alo, uint32_t blo, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %4};\n\t"
+        "mov.b64 db, {%2, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, %5;\n\t}"
+        ::"r"(d_tmem), "r"(alo), "r"(blo), "r"(idesc), "r"(DESC_HI), "n"(ACC) : "memory");
+}
 // Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");

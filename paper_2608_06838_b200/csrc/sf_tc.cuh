@@ -349,6 +349,23 @@ __device__ __forceinline__ uint64_t mndesc(uint32_t tile, int ks, uint32_t box_b
     return ptx::smem_desc(tile + ks * 2048, box_bytes);
 }
 
+// One K loop of MMAs from precomputed low descriptor words.  Offset rules of a K step (16-byte units):
+//   DK8 / DK16: K-major operand whose two 64-feature boxes lie 8 KB / 16 KB apart (kdesc);  DMN: MN-major (mndesc).
+enum { DK8 = 0, DK16 = 1, DMN = 2 };
+template <int RULE>
+__host__ __device__ constexpr uint32_t dofs(int ks) {
+    return RULE == DMN ? 128u * ks : (RULE == DK8 ? 512u : 1024u) * (ks >> 2) + 2u * (ks & 3);
+}
+template <int NK, int RA, int RB, int ACC0, int KS = 0>
+__device__ __forceinline__ void mma_group(uint32_t d, uint32_t alo, uint32_t blo, uint32_t idesc) {
+    if constexpr (KS < NK) {
+        ptx::mma_lo<(ACC0 || KS > 0) ? 1 : 0>(d, alo + dofs<RA>(KS), blo + dofs<RB>(KS), idesc);
+        mma_group<NK, RA, RB, ACC0, KS + 1>(d, alo, blo, idesc);
+    }
+}
+__device__ __forceinline__ uint32_t klo(uint32_t tile) { return ptx::desc_lo(tile, 0); }
+__device__ __forceinline__ uint32_t mlo(uint32_t tile, uint32_t box_bytes) { return ptx::desc_lo(tile, box_bytes); }
+
 // Warp roles of the chunk-sweep kernels (20 warps): four compute warpgroups, warp 16 issues the MMAs,
 // warp 17 the TMA loads (lane 0 each), warps 18-19 only fill the fifth warpgroup.  The carried state
 // sits on the critical path (MMA -> rescale -> MMA), so several warpgroups share its rescaling (16-column
@@ -422,9 +439,8 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                 SF_WAIT(&sm.ready[s], it & 1, DEV_TIMEOUT_TMA);
                 ptx::tc_fence_after_sync();
                 const uint32_t xa = ptx::smem_u32(sm.tiles[s][0]), ya = ptx::smem_u32(sm.tiles[s][1]);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    ptx::mma_ss(tmem, mndesc(xa, ks, BOX), mndesc(ya, ks, BOX), idesc, (c > 0 || ks > 0) ? 1u : 0u);
+                if (c == 0) mma_group<4, DMN, DMN, 0>(tmem, mlo(xa, BOX), mlo(ya, BOX), idesc);
+                else        mma_group<4, DMN, DMN, 1>(tmem, mlo(xa, BOX), mlo(ya, BOX), idesc);
                 ptx::mma_commit(&sm.empty[s]);
             }
             ptx::mma_commit(&sm.done);
@@ -550,8 +566,7 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
                 ptx::tc_fence_after_sync();
                 const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_SC + (c & 1) * 64, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
+                mma_group<8, DK8, DK8, 0>(tmem + T_SC + (c & 1) * 64, klo(xq), klo(xk), id_sc);
                 ptx::mma_commit(&sm.sc_done[c & 1]);
             };
             scores(0);
@@ -567,26 +582,17 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 ptx::tc_fence_after_sync();
                 SF_TR(1, c, 0);
                 // the state-dependent MMAs first: inter-chunk output (lanes +16), then the state update
-                {
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(to + (16u << 16), kdesc(xq, ks, BOX), mndesc(sb, ks, 16384), id_o1, ks > 0);
-                }
+                mma_group<8, DK8, DMN, 0>(to + (16u << 16), klo(xq), mlo(sb, 16384), id_o1);
                 SF_TR(7, c, 1);
                 SF_WAIT(&sm.w_ready, c & 1, DEV_TIMEOUT_MMA);        // the weighted tile is written while the MMAs above run
                 ptx::tc_fence_after_sync();
                 SF_TR(7, c, 2);
-                {
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_ST, mndesc(xk, ks, BOX), mndesc(xvw, ks, BOX), id_st, 1u);
-                }
+                mma_group<4, DMN, DMN, 1>(tmem + T_ST, mlo(xk, BOX), mlo(xvw, BOX), id_st);
                 ptx::mma_commit(&sm.st_done);
                 SF_TR(1, c, 1);
                 SF_WAIT(&sm.am_ready[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                {
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(to, kdesc(am, ks, BOX), mndesc(xv, ks, BOX), id_o1, ks > 0);                // intra
-                }
+                mma_group<4, DK8, DMN, 0>(to, klo(am), mlo(xv, BOX), id_o1);                // intra
                 ptx::mma_commit(&sm.out_done[bf]);
                 SF_TR(1, c, 2);
                 if (c + 2 < nch) scores(c + 2);          // into the score buffer the mask of chunk c has released
@@ -763,10 +769,8 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
                 const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
                 const uint32_t sc = tmem + T_SC + (i & 1) * 64;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(sc, kdesc(xq, ks, BOX), kdesc(xk, ks, BOX), id_sc, ks > 0);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(sc + (16u << 16), kdesc(xd, ks, BOX), kdesc(xv, ks, BOX), id_sc, ks > 0);
+                mma_group<8, DK8, DK8, 0>(sc, klo(xq), klo(xk), id_sc);
+                mma_group<8, DK8, DK8, 0>(sc + (16u << 16), klo(xd), klo(xv), id_sc);
                 ptx::mma_commit(&sm.sc_done[i & 1]);
             };
             scores(0);
@@ -784,30 +788,25 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 // Everything that touches the carried gradient goes first, so that its rescaling for the next chunk
                 // runs while the intra-chunk MMAs and the next scores execute:
                 //   dv (lanes +16) = K G,  dk (lanes +16) = V G^T,  G += (diag(exp(b)) Q)^T dO
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DV + (16u << 16), kdesc(xk, ks, BOX), mndesc(gb, ks, 16384), id_kn, ks > 0);
+                mma_group<8, DK8, DMN, 0>(tmem + T_DV + (16u << 16), klo(xk), mlo(gb, 16384), id_kn);
                 SF_TR(1, i, 3);
                 if (i >= 1) SF_WAIT(&sm.dk_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
                 SF_TR(7, i, 0);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) ptx::mma_ss(tmem + T_DK + (16u << 16), kdesc(xv, ks, BOX), kdesc(gb, ks, 16384), id_kk, ks > 0);
+                mma_group<8, DK8, DK16, 0>(tmem + T_DK + (16u << 16), klo(xv), klo(gb), id_kk);
                 SF_WAIT(&sm.w_ready, i & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
                 SF_TR(7, i, 1);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_G, mndesc(qw, ks, BOX), mndesc(xd, ks, BOX), id_st, 1u);
+                mma_group<4, DMN, DMN, 1>(tmem + T_G, mlo(qw, BOX), mlo(xd, BOX), id_st);
                 ptx::mma_commit(&sm.st_done[s]);                 // G, its bf16 copy and qw are free again
                 SF_TR(7, i, 2);
                 // intra-chunk parts: dv (lanes +0) = A^T dO, dk (lanes +0) = dA^T Q
                 SF_WAIT(&sm.am_ready[s], (i >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
                 SF_TR(7, i, 3);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DV, mndesc(am, ks, BOX), mndesc(xd, ks, BOX), id_tt, ks > 0);
+                mma_group<4, DMN, DMN, 0>(tmem + T_DV, mlo(am, BOX), mlo(xd, BOX), id_tt);
                 ptx::mma_commit(&sm.dv_done);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ptx::mma_ss(tmem + T_DK, mndesc(dam, ks, BOX), mndesc(xq, ks, BOX), id_tt, ks > 0);
+                mma_group<4, DMN, DMN, 0>(tmem + T_DK, mlo(dam, BOX), mlo(xq, BOX), id_tt);
                 ptx::mma_commit(&sm.dk_done);
                 ptx::mma_commit(&sm.it_done[s]);                 // tiles and masks of this iteration are free again
                 SF_TR(0, i, 0);
