@@ -174,13 +174,8 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 //            elements is +32 B on the start address; K beyond 64 lives in the next box.
 //   MN-major (rows = K index, the 64 columns = M/N): 8-row K groups 1024 B apart (SBO); the next 64
 //            M/N elements live `lbo_bytes` away (the next box); a K step of 16 rows is +2048 B.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes) {
-    // low word: start address [0,14) and leading offset [16,30), both in 16-byte units
-    // high word: stride offset 1024 B [32,46), descriptor version 1 [46,48), SWIZZLE_128B = 2 [61,64)
-    const uint32_t lo = ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
-    constexpr uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-    return (static_cast<uint64_t>(hi) << 32) | lo;
-}
+// Descriptor fields: low word = start address [0,14) and leading offset [16,30), both in 16-byte units; high
+// word = stride offset 1024 B [32,46), descriptor version 1 [46,48), SWIZZLE_128B = 2 [61,64).
 
 // Instruction descriptor for kind::f16 with bf16 operands and float32 accumulation.
 __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn_major, int b_mn_major) {
@@ -189,17 +184,9 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn_major, 
            (static_cast<uint32_t>(M >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// The same instruction from 32-bit pieces.  The issuing thread has no queue to hide behind: whatever it executes
-// between two tcgen05.mma instructions is idle time of the tensor pipe, so the descriptors of a K loop are formed
-// with one integer add each: the high word of every descriptor here is the same constant and a K step only moves
+// D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread, descriptors passed as 32-bit pieces.
+// The issuing thread has no queue to hide behind: whatever it executes between two tcgen05.mma instructions
+// is idle time of the tensor pipe, so the descriptors of a K loop are formed with one integer add each: the high word of every descriptor here is the same constant and a K step only moves
 // the 14-bit start-address field of the low word (shared memory is smaller than 2^18 bytes: no carry out of it).
 constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {

@@ -7,7 +7,7 @@
 // Shared-memory operand storage: every [64 tokens x 128 features] bf16 tile is two TMA boxes of
 // [64 rows x 64 columns] (128-byte rows, SWIZZLE_128B, 8 KB each, features 0-63 then 64-127).  The
 // same storage is read K-major when the contraction runs over features and MN-major when it runs
-// over tokens (ptx::smem_desc).
+// over tokens (ptx::desc_lo).
 #pragma once
 #include <cuda.h>
 #include <cstdio>
@@ -340,17 +340,11 @@ __device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float
     }
 }
 
-// K-major descriptor of a [rows x 128] tile for K step ks (0..7): features 16*ks .. 16*ks+15.
-__device__ __forceinline__ uint64_t kdesc(uint32_t tile, int ks, uint32_t box_bytes) {
-    return ptx::smem_desc(tile + (ks >> 2) * box_bytes + (ks & 3) * 32, 0);
-}
-// MN-major descriptor of a tile whose rows are the contraction index, K step ks = rows 16*ks .. 16*ks+15.
-__device__ __forceinline__ uint64_t mndesc(uint32_t tile, int ks, uint32_t box_bytes) {
-    return ptx::smem_desc(tile + ks * 2048, box_bytes);
-}
-
 // One K loop of MMAs from precomputed low descriptor words.  Offset rules of a K step (16-byte units):
-//   DK8 / DK16: K-major operand whose two 64-feature boxes lie 8 KB / 16 KB apart (kdesc);  DMN: MN-major (mndesc).
+//   DK8 / DK16: K-major operand (a [rows x 128] tile, K step = features 16*ks .. 16*ks+15: +32 B inside a box, the
+//               second 64 features in the next box 8 KB / 16 KB away);
+//   DMN:        MN-major operand (rows are the contraction index: K step = rows 16*ks .. 16*ks+15 = +2048 B; the
+//               other 64 elements of M/N lie one box away, which is the descriptor's leading offset).
 enum { DK8 = 0, DK16 = 1, DMN = 2 };
 template <int RULE>
 __host__ __device__ constexpr uint32_t dofs(int ks) {
