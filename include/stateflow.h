@@ -235,6 +235,23 @@ int64_t sf_chain_graph_kernels(const sf_chain_graph_t* graph);
 void sf_chain_graph_destroy(sf_chain_graph_t* graph);
 
 /*
+ * Hybrid-aware sequence chunking (paper Section 3.2, Eq. 9-11): the segment lengths to hand to the chain
+ * driver.  Host code only; no CUDA call.  With boundaries 0 = c_0 < ... < c_N = T and s_i = c_{i+1} - c_i,
+ *     Cost_i = w_tok * s_i + w_soft * (c_i * s_i + s_i^2 / 2)                                       (Eq. 9)
+ * (w_tok = L_lin*C_lin + C_dense: token-wise work; w_soft = L_soft*C_soft: work per query-key pair of the
+ * softmax layers).  The FLOP-balanced boundaries c_i^hybrid make all Cost_i equal (Eq. 10); the candidate is
+ *     c_i(alpha) = (1 - alpha) * i*T/N + alpha * c_i^hybrid                                          (Eq. 11)
+ * rounded to the closest multiple of `multiple` (the paper uses 128; a tie goes up; c_N stays T).  After
+ * rounding, boundaries are pushed apart (forward, then backward) so that every segment keeps at least one
+ * multiple.  alpha = 0 or w_soft = 0 give equal lengths; alpha > 1 exaggerates the imbalance.
+ *   seg_lens : HOST array of N entries, written on success
+ * Errors (SF_ERR_INVALID_ARG): T < 1, N < 1, multiple < 1, negative or both-zero weights, non-finite alpha,
+ * seg_lens NULL, or T too short for N segments of one multiple each.
+ */
+sf_status_t sf_partition_hybrid(int64_t T, int32_t N, double w_tok, double w_soft, double alpha,
+                                int32_t multiple, int32_t* seg_lens);
+
+/*
  * Host-memory convenience wrappers around the chain driver (the "end-to-end" path): every data
  * pointer is a HOST pointer (pinned memory recommended).  The call copies the inputs to the device
  * buffers in `dev` (caller-allocated device scratch, sf_e2e_device_bytes() bytes, 256-byte

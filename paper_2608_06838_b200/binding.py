@@ -80,6 +80,8 @@ def load() -> ctypes.CDLL:
         lib.sf_chain_graph_kernels.argtypes = [vp]
         lib.sf_chain_graph_destroy.restype = None
         lib.sf_chain_graph_destroy.argtypes = [vp]
+        lib.sf_partition_hybrid.restype = ctypes.c_int
+        lib.sf_partition_hybrid.argtypes = [ctypes.c_int64, i32, ctypes.c_double, ctypes.c_double, ctypes.c_double, i32, ip]
         lib.sf_device_status.restype = i32
         lib.sf_device_status_clear.restype = None
         lib.sf_launch_count.restype = ctypes.c_int64
@@ -207,6 +209,14 @@ def sf_chain_graph_kernels(handle) -> int:
 
 def sf_chain_graph_destroy(handle) -> None:
     load().sf_chain_graph_destroy(handle)
+
+
+def sf_partition_hybrid(T: int, N: int, w_tok: float, w_soft: float, alpha: float, multiple: int = 128) -> List[int]:
+    """Segment lengths of the candidate partition (host only)."""
+    out = (ctypes.c_int32 * max(N, 1))()
+    _check(load().sf_partition_hybrid(int(T), int(N), float(w_tok), float(w_soft), float(alpha), int(multiple), out),
+           "sf_partition_hybrid")
+    return [int(v) for v in out[:N]]
 
 
 def sf_e2e_device_bytes(desc: SegDesc, seg_lens) -> int:

@@ -2,7 +2,10 @@
 // dispatch, the segment-chaining driver and the host-memory end-to-end wrapper.
 #include "../../include/stateflow.h"
 
+#include <algorithm>
 #include <atomic>
+#include <climits>
+#include <cmath>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -818,6 +821,34 @@ void sf_chain_graph_destroy(sf_chain_graph_t* graph) {
     if (graph->exec) cudaGraphExecDestroy(graph->exec);
     if (graph->graph) cudaGraphDestroy(graph->graph);
     delete graph;
+}
+
+sf_status_t sf_partition_hybrid(int64_t T, int32_t N, double w_tok, double w_soft, double alpha, int32_t multiple,
+                                int32_t* seg_lens) {
+    if (T < 1 || N < 1 || multiple < 1 || !seg_lens) return SF_ERR_INVALID_ARG;
+    if (!(w_tok >= 0.0) || !(w_soft >= 0.0) || (w_tok == 0.0 && w_soft == 0.0) || !std::isfinite(alpha) ||
+        !std::isfinite(w_tok) || !std::isfinite(w_soft))
+        return SF_ERR_INVALID_ARG;
+    if ((int64_t)N * multiple > T || T > INT32_MAX) return SF_ERR_INVALID_ARG;
+    // Equal Cost_i (Eq. 10) means the cost accumulated over the prefix [0, c), acc(c) = w_tok*c + w_soft*c^2/2
+    // (Cost_i = acc(c_{i+1}) - acc(c_i) by Eq. 9), grows by the same amount per segment: acc(c_i) = (i/N) acc(T).
+    // The positive root of that quadratic, in the form that stays exact as w_soft -> 0:
+    //     c_i = 2 K_i / (w_tok + sqrt(w_tok^2 + 2 w_soft K_i)),   K_i = (i/N) acc(T)
+    const double Td = (double)T, accT = w_tok * Td + 0.5 * w_soft * Td * Td;
+    std::vector<long long> r(N + 1);
+    r[0] = 0;
+    r[N] = T;
+    for (int i = 1; i < N; ++i) {
+        const double K = accT * ((double)i / (double)N);
+        const double hybrid = 2.0 * K / (w_tok + std::sqrt(w_tok * w_tok + 2.0 * w_soft * K));
+        const double c = (1.0 - alpha) * (Td * (double)i / (double)N) + alpha * hybrid;              // Eq. 11
+        r[i] = (long long)std::floor(c / (double)multiple + 0.5) * (long long)multiple;
+    }
+    for (int i = 1; i < N; ++i) r[i] = std::max(r[i], r[i - 1] + multiple);
+    for (int i = N - 1; i >= 1; --i) r[i] = std::min(r[i], r[i + 1] - multiple);
+    if (N > 1 && r[1] < multiple) return SF_ERR_INVALID_ARG;
+    for (int i = 0; i < N; ++i) seg_lens[i] = (int32_t)(r[i + 1] - r[i]);
+    return SF_OK;
 }
 
 size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg) {

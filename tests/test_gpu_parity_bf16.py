@@ -47,3 +47,11 @@ def test_mixed_heads_strong_and_zero_decay():
 def test_single_chunk_segments():
     w = Workload("bf16-128-1chunk", 1, 2, 128, 128, [64, 64, 128], 64, g_scale=0.05, s_in_sigma=0.1, ds_out_sigma=0.1, seed=6)
     check(w)
+
+
+def test_chain_on_a_hybrid_aware_partition():
+    # non-uniform, decreasing segment lengths as Section 3.2 (Eq. 9-11) produces them
+    lens = binding.sf_partition_hybrid(4096, 4, 1.0, 1e-3, 1.0)
+    assert sum(lens) == 4096 and lens == sorted(lens, reverse=True) and lens[0] > lens[-1]
+    w = Workload("bf16-128-hybrid", 1, 2, 128, 128, lens, 64, g_scale=0.05, s_in_sigma=0.02, ds_out_sigma=0.02, seed=9)
+    check(w)

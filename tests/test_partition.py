@@ -86,3 +86,76 @@ def test_rounding_keeps_every_segment_alive_or_rejects():
     assert P.round_boundaries([0.0, 1000.0, 1010.0, 1020.0, 1024.0], 1024, 128) == [0, 640, 768, 896, 1024]
     with pytest.raises(ValueError):
         P.round_boundaries([0.0, 100.0, 200.0, 300.0, 384.0], 384, 128)
+
+
+# ---- the library's host function against the oracle ---------------------------------------------------------------
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2608_06838_b200 import binding as b, build
+    build.build()
+    return b
+
+
+def _near_tie(T, N, wt, ws, alpha, multiple):
+    cand = P.candidate_boundaries(float(T), N, wt, ws, alpha)
+    return any(abs((c / multiple) % 1.0 - 0.5) < 1e-6 for c in cand[1:N])
+
+
+def test_library_matches_the_oracle_on_the_paper_grid(binding):
+    # N and alpha values the paper profiles (Section 3.2), model-like weights
+    for T in (32768, 65536, 131072, 262144):
+        for N in (2, 4, 6, 8, 16, 32):
+            for alpha in (0.0, 0.1, 0.2, 0.3, 0.4, 0.5, 0.6, 0.7, 0.8, 0.9, 1.0, 1.25):
+                for ws in (0.0, 3e-5, 4e-4):
+                    if _near_tie(T, N, 1.0, ws, alpha, 128):
+                        continue
+                    assert binding.sf_partition_hybrid(T, N, 1.0, ws, alpha, 128) == P.partition(T, N, 1.0, ws, alpha, 128), \
+                        (T, N, alpha, ws)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_library_matches_the_oracle_on_random_cases(binding, seed):
+    rng = random.Random(1000 + seed)
+    multiple = rng.choice([1, 64, 128, 256])
+    N = rng.randint(1, 32)
+    T = multiple * rng.randint(N, 40 * N) + (rng.randint(0, multiple - 1) if seed % 4 == 0 else 0)
+    wt = rng.choice([0.0, rng.uniform(0.1, 5.0)])
+    ws = rng.uniform(1e-6, 1e-2) if wt == 0.0 or seed % 3 else 0.0
+    alpha = rng.choice([0.0, 1.0, 1.25, rng.uniform(-0.5, 2.0)])
+    if _near_tie(T, N, wt, ws, alpha, multiple):
+        pytest.skip("rounding tie within 1e-6: both neighbours are correct")
+    try:
+        ref = P.partition(T, N, wt, ws, alpha, multiple)
+    except ValueError:
+        with pytest.raises(binding.SfError):
+            binding.sf_partition_hybrid(T, N, wt, ws, alpha, multiple)
+        return
+    got = binding.sf_partition_hybrid(T, N, wt, ws, alpha, multiple)
+    assert got == ref
+    assert sum(got) == T and min(got) >= multiple
+
+
+def test_library_rejects_bad_arguments(binding):
+    lib = binding.load()
+    out = (ctypes.c_int32 * 8)()
+    ok = dict(T=65536, N=8, w_tok=1.0, w_soft=1e-4, alpha=1.0, multiple=128)
+
+    def call(**kw):
+        a = dict(ok, **kw)
+        return lib.sf_partition_hybrid(a["T"], a["N"], a["w_tok"], a["w_soft"], a["alpha"], a["multiple"], kw.get("out", out))
+
+    assert call() == 0
+    for bad in (dict(T=0), dict(N=0), dict(multiple=0), dict(w_tok=-1.0), dict(w_soft=-1e-3), dict(w_tok=0.0, w_soft=0.0),
+                dict(alpha=float("nan")), dict(alpha=float("inf")), dict(w_tok=float("nan")), dict(T=512, N=8),
+                dict(out=None)):
+        assert call(**bad) == 1, bad
+
+
+def test_partition_feeds_the_chain_driver(binding):
+    # lengths are multiples of 128, hence of the chunk size: the chain driver accepts them as they are
+    lens = binding.sf_partition_hybrid(65536, 8, 1.0, 2e-4, 1.0)
+    from paper_2608_06838_b200.binding import SegDesc, SF_BF16
+    d = SegDesc(1, 32, 128, 128, lens[0], 64, SF_BF16, 0, 32 * 128, 32 * 128, 32, 0, 0, 0)
+    assert binding.sf_chain_workspace_bytes(d, lens, 0) > 0
+    assert lens == sorted(lens, reverse=True) and sum(lens) == 65536
