@@ -174,6 +174,9 @@ def main():
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="launch the chain from the host every step instead of replaying it as one CUDA graph "
                          "(sf_chain_graph_*)")
+    ap.add_argument("--no-autotune", dest="autotune", action="store_false",
+                    help="keep the library's model for the block length instead of timing the candidates first "
+                         "(sf_chain_autotune; only used when --chunks-per-block is 0)")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     args = ap.parse_args()
@@ -202,6 +205,13 @@ def main():
     x = inputs.make_inputs(w, dev)
     run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk, args.chunks_per_block)
     overlap = not args.no_overlap
+
+    # profile-guided block length (untimed preparation, like the graph capture below)
+    tuned = None
+    if args.autotune and args.chunks_per_block == 0:
+        cands = [0, 8, 11, 16, 22, 32]
+        best, cand_ms = run.autotune(x["S_in"], x["dS_out"], cands, reps=3, overlap=overlap)
+        tuned = {"candidates": cands, "ms": [round(v, 4) for v in cand_ms], "chosen": best}
 
     # a graph cannot be recorded on the legacy default stream: that mode runs on a stream of its own
     work_stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
@@ -270,7 +280,7 @@ def main():
                 [("o", "v"), ("dq", "q"), ("dk", "k"), ("dv", "v"), ("dg", "g")]}
         S_final = torch.empty(w.B, w.H, w.d_k, w.d_v, dtype=torch.float32).pin_memory()
         dS_init = torch.empty_like(S_final).pin_memory()
-        desc = binding.make_desc(host["q"], host["v"], host["g"], w.chunk, args.chunks_per_block, seg_len=w.seg_lens[0])
+        desc = binding.make_desc(host["q"], host["v"], host["g"], w.chunk, int(run.desc.chunks_per_block), seg_len=w.seg_lens[0])
         scratch = torch.empty(binding.sf_e2e_device_bytes(desc, w.seg_lens), dtype=torch.uint8, device=dev)
 
         def e2e_step():
@@ -322,7 +332,8 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d_k, "d_v": w.d_v, "T": w.T, "segments": w.seg_lens,
-                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or "auto", "overlap": overlap, "graph": bool(args.graph),
+                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or (tuned["chosen"] if tuned else "auto"),
+                   "autotune": tuned, "overlap": overlap, "graph": bool(args.graph),
                    "l2": "inputs (%.0f MB) exceed L2, no flush" % (4 * tokens * w.H * w.d_k * 2 / 1e6),
                    "parallelism": "replicas only"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roof, "path_roofline": path_roof,

@@ -235,6 +235,30 @@ int64_t sf_chain_graph_kernels(const sf_chain_graph_t* graph);
 void sf_chain_graph_destroy(sf_chain_graph_t* graph);
 
 /*
+ * Profile-guided choice of the block length (the paper tunes its kernels' tile sizes and overlap schedules
+ * "for each operator shape" by profiling, Section 3.4 end and Section 4.4; here the one tunable of that kind is
+ * chunks_per_block).  Runs the chain (sf_chain_fwd, and sf_chain_bwd with the forward workspace if dO is not
+ * NULL) once untimed and `reps` times timed (CUDA events on `stream`) for every candidate value and reports
+ * the fastest.  Arguments are those of sf_chain_graph_create, plus
+ *   candidates : HOST array of n_cand values for desc->chunks_per_block (0 = the library's own model)
+ *   best       : receives the fastest candidate (write it into desc->chunks_per_block for later calls)
+ *   ms         : nullable HOST array of n_cand mean times in milliseconds; -1 for a candidate that was skipped
+ *                because the given workspaces are too small for it (size them for the smallest nonzero
+ *                candidate, which has the most blocks) or that the descriptor rejects
+ * The outputs hold the result of the last run.  The call synchronises `stream`.  Errors: those of the chain
+ * calls for argument problems common to all candidates; SF_ERR_WORKSPACE if no candidate fits.
+ */
+sf_status_t sf_chain_autotune(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg,
+                              const void* q, const void* k, const void* v, const float* g,
+                              const float* S_init, void* o, float* S_bounds,
+                              void* fwd_workspace, size_t fwd_workspace_bytes,
+                              const void* dO, const float* dS_final,
+                              void* dq, void* dk, void* dv, float* dg, float* dS_init,
+                              void* bwd_workspace, size_t bwd_workspace_bytes,
+                              const int32_t* candidates, int32_t n_cand, int32_t reps, int32_t overlap,
+                              sf_stream_t stream, int32_t* best, float* ms);
+
+/*
  * Hybrid-aware sequence chunking (paper Section 3.2, Eq. 9-11): the segment lengths to hand to the chain
  * driver.  Host code only; no CUDA call.  With boundaries 0 = c_0 < ... < c_N = T and s_i = c_{i+1} - c_i,
  *     Cost_i = w_tok * s_i + w_soft * (c_i * s_i + s_i^2 / 2)                                       (Eq. 9)

@@ -80,6 +80,9 @@ def load() -> ctypes.CDLL:
         lib.sf_chain_graph_kernels.argtypes = [vp]
         lib.sf_chain_graph_destroy.restype = None
         lib.sf_chain_graph_destroy.argtypes = [vp]
+        lib.sf_chain_autotune.restype = ctypes.c_int
+        lib.sf_chain_autotune.argtypes = [dp, ip, i32] + [vp] * 7 + [vp, sz] + [vp] * 7 + [vp, sz, ip, i32, i32, i32, vp, ip,
+                                                                                         ctypes.POINTER(ctypes.c_float)]
         lib.sf_partition_hybrid.restype = ctypes.c_int
         lib.sf_partition_hybrid.argtypes = [ctypes.c_int64, i32, ctypes.c_double, ctypes.c_double, ctypes.c_double, i32, ip]
         lib.sf_device_status.restype = i32
@@ -211,6 +214,21 @@ def sf_chain_graph_destroy(handle) -> None:
     load().sf_chain_graph_destroy(handle)
 
 
+def sf_chain_autotune(desc: SegDesc, seg_lens, q, k, v, g, S_init, o, S_bounds, fwd_workspace, dO, dS_final, dq, dk, dv, dg,
+                      dS_init, bwd_workspace, candidates, reps=3, overlap=True, stream=None):
+    """Returns (best chunks_per_block, [mean ms per candidate, -1 = skipped])."""
+    cand = (ctypes.c_int32 * len(candidates))(*[int(c) for c in candidates])
+    ms = (ctypes.c_float * len(candidates))()
+    best = ctypes.c_int32(-1)
+    _check(load().sf_chain_autotune(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens), _ptr(q), _ptr(k), _ptr(v),
+                                    _ptr(g), _ptr(S_init), _ptr(o), _ptr(S_bounds), _ptr(fwd_workspace),
+                                    fwd_workspace.numel(), _ptr(dO), _ptr(dS_final), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dg),
+                                    _ptr(dS_init), _ptr(bwd_workspace),
+                                    0 if bwd_workspace is None else bwd_workspace.numel(), cand, len(candidates), int(reps),
+                                    int(overlap), _stream(stream), ctypes.byref(best), ms), "sf_chain_autotune")
+    return int(best.value), [float(x) for x in ms]
+
+
 def sf_partition_hybrid(T: int, N: int, w_tok: float, w_soft: float, alpha: float, multiple: int = 128) -> List[int]:
     """Segment lengths of the candidate partition (host only)."""
     out = (ctypes.c_int32 * max(N, 1))()
@@ -313,3 +331,24 @@ class ChainRun:
             self.release()
         except Exception:
             pass
+
+    def autotune(self, S_init=None, dS_final=None, candidates=(0, 8, 11, 16, 22, 32), reps=3, overlap=True, stream=None):
+        """Times the chain for every candidate block length, keeps the fastest in the descriptor and returns
+        (best, [ms per candidate]).  Workspaces are re-allocated for the candidate with the most blocks."""
+        if not self.save_states:
+            raise ValueError("tuning runs the backward from saved states")
+        self.release()
+        dev = self.q.device
+        need_f = need_b = 0
+        keep = self.desc.chunks_per_block
+        for c in candidates:
+            self.desc.chunks_per_block = int(c)
+            need_f = max(need_f, sf_chain_workspace_bytes(self.desc, self.seg_lens, 0))
+            need_b = max(need_b, sf_chain_workspace_bytes(self.desc, self.seg_lens, 1))
+        self.desc.chunks_per_block = keep
+        self.ws_f, self.ws_b = _workspace(need_f, dev), _workspace(need_b, dev)
+        best, ms = sf_chain_autotune(self.desc, self.seg_lens, self.q, self.k, self.v, self.g, S_init, self.o, self.S_bounds,
+                                     self.ws_f, self.dO, dS_final, self.dq, self.dk, self.dv, self.dg, self.dS_init,
+                                     self.ws_b, candidates, reps, overlap, stream)
+        self.desc.chunks_per_block = best
+        return best, ms

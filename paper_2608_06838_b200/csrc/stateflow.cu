@@ -823,6 +823,63 @@ void sf_chain_graph_destroy(sf_chain_graph_t* graph) {
     delete graph;
 }
 
+sf_status_t sf_chain_autotune(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q,
+                              const void* k, const void* v, const float* g, const float* S_init, void* o, float* S_bounds,
+                              void* fwd_workspace, size_t fwd_workspace_bytes, const void* dO, const float* dS_final,
+                              void* dq, void* dk, void* dv, float* dg, float* dS_init, void* bwd_workspace,
+                              size_t bwd_workspace_bytes, const int32_t* candidates, int32_t n_cand, int32_t reps,
+                              int32_t overlap, sf_stream_t stream, int32_t* best, float* ms) {
+    if (!desc || !candidates || n_cand < 1 || reps < 1 || !best) return SF_ERR_INVALID_ARG;
+    SF_TRY(validate_chain(desc, seg_lens, n_seg, nullptr));
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        cudaGetLastError();
+        if (e0) cudaEventDestroy(e0);
+        return SF_ERR_CUDA;
+    }
+    float best_ms = -1.f;
+    sf_status_t result = SF_ERR_WORKSPACE;
+    for (int c = 0; c < n_cand; ++c) {
+        if (ms) ms[c] = -1.f;
+        sf_seg_desc_t d = *desc;
+        d.chunks_per_block = candidates[c];
+        const size_t need_f = sf_chain_workspace_bytes(&d, seg_lens, n_seg, 0);
+        const size_t need_b = dO ? sf_chain_workspace_bytes(&d, seg_lens, n_seg, 1) : 0;
+        if (need_f == 0 || need_f > fwd_workspace_bytes || need_b > bwd_workspace_bytes) continue;
+        auto run = [&]() -> sf_status_t {
+            SF_TRY(sf_chain_fwd(&d, seg_lens, n_seg, q, k, v, g, S_init, o, S_bounds, fwd_workspace, fwd_workspace_bytes,
+                                overlap, stream));
+            if (dO)
+                SF_TRY(sf_chain_bwd(&d, seg_lens, n_seg, q, k, v, g, S_bounds, dO, dS_final, dq, dk, dv, dg, dS_init,
+                                    fwd_workspace, bwd_workspace, bwd_workspace_bytes, overlap, stream));
+            return SF_OK;
+        };
+        sf_status_t rs = run();                                   // untimed: first-use costs of this shape
+        if (rs == SF_ERR_UNSUPPORTED || rs == SF_ERR_INVALID_ARG) {  // this value is not available for this shape
+            if (result != SF_OK) result = rs;
+            continue;
+        }
+        bool ok = rs == SF_OK && cudaEventRecord(e0, st) == cudaSuccess;
+        for (int r = 0; ok && r < reps; ++r) ok = (rs = run()) == SF_OK;
+        float t = 0.f;
+        ok = ok && cudaEventRecord(e1, st) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess &&
+             cudaEventElapsedTime(&t, e0, e1) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            result = rs != SF_OK ? rs : SF_ERR_CUDA;
+            break;
+        }
+        t /= (float)reps;
+        if (ms) ms[c] = t;
+        if (best_ms < 0.f || t < best_ms) { best_ms = t; *best = candidates[c]; }
+        result = SF_OK;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return result;
+}
+
 sf_status_t sf_partition_hybrid(int64_t T, int32_t N, double w_tok, double w_soft, double alpha, int32_t multiple,
                                 int32_t* seg_lens) {
     if (T < 1 || N < 1 || multiple < 1 || !seg_lens) return SF_ERR_INVALID_ARG;

@@ -167,3 +167,18 @@ def test_graph_create_rejects_bad_arguments_before_any_cuda_call(lib):
     assert lib.sf_chain_graph_launch(None, None) == 1
     assert lib.sf_chain_graph_kernels(None) == 0
     lib.sf_chain_graph_destroy(None)                 # a no-op
+
+
+def test_autotune_rejects_bad_arguments_before_any_cuda_call(lib):
+    d = desc()
+    segs = (ctypes.c_int32 * 1)(1024)
+    cands = (ctypes.c_int32 * 2)(0, 16)
+    best = ctypes.c_int32(-7)
+    head = [ctypes.byref(d), segs, 1] + [P] * 7 + [P, 1 << 40] + [P] * 7 + [P, 1 << 40]
+    assert lib.sf_chain_autotune(*head, None, 2, 3, 1, None, ctypes.byref(best), None) == 1        # no candidates
+    assert lib.sf_chain_autotune(*head, cands, 0, 3, 1, None, ctypes.byref(best), None) == 1
+    assert lib.sf_chain_autotune(*head, cands, 2, 0, 1, None, ctypes.byref(best), None) == 1       # no repetitions
+    assert lib.sf_chain_autotune(*head, cands, 2, 3, 1, None, None, None) == 1                     # nowhere to report
+    bad = (ctypes.c_int32 * 1)(1000)                                                               # not a multiple of the chunk
+    assert lib.sf_chain_autotune(ctypes.byref(d), bad, 1, *head[3:], cands, 2, 3, 1, None, ctypes.byref(best), None) == 1
+    assert best.value == -7
