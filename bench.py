@@ -29,9 +29,9 @@ UNIT = "tokens/s"
 BYTES_PER_TOKEN_HEAD = 2828          # q,k,v,dO read once, o,dq,dk,dv written once (bf16, d=128), g and dg float32
 DKDV_BYTES_PER_TOKEN_HEAD = 1540     # the dk/dv pass alone: q,k,v,dO + g in, dk,dv out
 # DRAM bytes per token*head of the dk/dv pass from the ncu capture of the small case
-# (profiles/ncu_full_small_case_8k_h32_all_kernels.txt: 278.08 MB read + 108.57 MB written for 262144 token*heads),
+# (profiles/ncu_full_small_case_8k_h32_all_kernels.txt: 278.06 MB read + 107.46 MB written for 262144 token*heads),
 # scaled to a bench launch by the token*heads it processes (traffic grows in proportion)
-DKDV_NCU_TRAFFIC_PER_TOKEN_HEAD = (278.078e6 + 108.569e6) / 262144
+DKDV_NCU_TRAFFIC_PER_TOKEN_HEAD = (278.056e6 + 107.461e6) / 262144
 
 
 def peaks():
