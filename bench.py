@@ -209,7 +209,7 @@ def main():
     # profile-guided block length (untimed preparation, like the graph capture below)
     tuned = None
     if args.autotune and args.chunks_per_block == 0:
-        cands = [0, 8, 11, 16, 22, 32]
+        cands = [0, 8, 10, 11, 13, 16, 19, 22, 26, 29, 32]
         best, cand_ms = run.autotune(x["S_in"], x["dS_out"], cands, reps=3, overlap=overlap)
         tuned = {"candidates": cands, "ms": [round(v, 4) for v in cand_ms], "chosen": best}
 

@@ -332,7 +332,7 @@ class ChainRun:
         except Exception:
             pass
 
-    def autotune(self, S_init=None, dS_final=None, candidates=(0, 8, 11, 16, 22, 32), reps=3, overlap=True, stream=None):
+    def autotune(self, S_init=None, dS_final=None, candidates=(0, 8, 10, 11, 13, 16, 19, 22, 26, 29, 32), reps=3, overlap=True, stream=None):
         """Times the chain for every candidate block length, keeps the fastest in the descriptor and returns
         (best, [ms per candidate]).  Workspaces are re-allocated for the candidate with the most blocks."""
         if not self.save_states:
