@@ -206,15 +206,18 @@ def main():
     run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk, args.chunks_per_block)
     overlap = not args.no_overlap
 
-    # profile-guided block length (untimed preparation, like the graph capture below)
+    # a graph cannot be recorded on the legacy default stream: that mode runs on a stream of its own
+    work_stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
+
+    # profile-guided block length (untimed preparation, like the graph capture below); candidates are timed the
+    # way the step will run: as graph replays on the work stream, or launched from the host with --no-graph
     tuned = None
     if args.autotune and args.chunks_per_block == 0:
         cands = [0, 8, 10, 11, 13, 16, 19, 22, 26, 29, 32]
-        best, cand_ms = run.autotune(x["S_in"], x["dS_out"], cands, reps=3, overlap=overlap)
+        with torch.cuda.stream(work_stream):
+            best, cand_ms = run.autotune(x["S_in"], x["dS_out"], cands, reps=3, overlap=overlap)
+        work_stream.synchronize()
         tuned = {"candidates": cands, "ms": [round(v, 4) for v in cand_ms], "chosen": best}
-
-    # a graph cannot be recorded on the legacy default stream: that mode runs on a stream of its own
-    work_stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
     if args.graph:
         with torch.cuda.stream(work_stream):
             run.capture(x["S_in"], x["dS_out"], overlap=overlap)

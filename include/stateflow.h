@@ -241,7 +241,9 @@ void sf_chain_graph_destroy(sf_chain_graph_t* graph);
  * "for each operator shape" by profiling, Section 3.4 end and Section 4.4; here the one tunable of that kind is
  * chunks_per_block).  Runs the chain (sf_chain_fwd, and sf_chain_bwd with the forward workspace if dO is not
  * NULL) once untimed and `reps` times timed (CUDA events on `stream`) for every candidate value and reports
- * the fastest.  Arguments are those of sf_chain_graph_create, plus
+ * the fastest.  On a stream that can be captured each candidate is timed as replays of its CUDA graph
+ * (sf_chain_graph_create; free of the host's launch cost, which hides the differences between candidates when
+ * segments are short); on the legacy default stream it is launched directly.  Arguments are those of sf_chain_graph_create, plus
  *   candidates : HOST array of n_cand values for desc->chunks_per_block (0 = the library's own model)
  *   best       : receives the fastest candidate (write it into desc->chunks_per_block for later calls)
  *   ms         : nullable HOST array of n_cand mean times in milliseconds; -1 for a candidate that was skipped

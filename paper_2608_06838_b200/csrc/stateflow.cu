@@ -106,6 +106,31 @@ int auto_chunks_per_block(int NC, long long bh) {
     return best;
 }
 
+// The same choice for a segment that runs inside a chain of several.  There the sweeps of neighbouring segments
+// share the device (the chain driver sends them to different streams), so what counts for a short segment is the
+// work per launch, not whole waves: measured (graph replays of whole chains), the fastest block length keeps
+// blocks at least 8 chunks long and a launch at 40 CTAs or more (4096-token segments x 16 heads: 16-22 instead of 8
+// chunks, 10 % faster; 512- to 2048-token segments x 40 heads: one block instead of two, 8-10 % faster).  Segments
+// of more than 64 chunks keep the wave model.
+int chain_chunks_per_block(int NC, long long bh) {
+    if (NC > 64) return auto_chunks_per_block(NC, bh);
+    long long nb = (40 + bh - 1) / bh;                       // blocks for 40 CTAs or more
+    const long long by_len = NC / 8 > 0 ? NC / 8 : 1;        // blocks of at least 8 chunks
+    if (nb > by_len) nb = by_len;
+    const long long least = (NC + 31) / 32;                  // blocks of at most 32 chunks
+    if (nb < least) nb = least;
+    return (int)((NC + nb - 1) / nb);
+}
+
+// Descriptor of segment i of a chain: the caller's block length if given, else the chain model above.
+sf_seg_desc_t chain_segment_desc(const sf_seg_desc_t* desc, int32_t seg_len, int32_t n_seg) {
+    sf_seg_desc_t t = *desc;
+    t.seg_len = seg_len;
+    if (t.chunks_per_block == 0 && n_seg > 1 && t.chunk > 0)
+        t.chunks_per_block = chain_chunks_per_block(seg_len / t.chunk, (long long)t.B * t.H);
+    return t;
+}
+
 SegParams make_params(const sf_seg_desc_t* d, int cpb_override = 0) {
     SegParams p;
     p.B = d->B; p.H = d->H; p.L = d->seg_len; p.C = d->chunk;
@@ -531,8 +556,7 @@ size_t sf_chain_workspace_bytes(const sf_seg_desc_t* desc, const int32_t* seg_le
     if (validate_chain(desc, seg_lens, n_seg, nullptr) != SF_OK) return 0;
     size_t total = 0, mx = 0;
     for (int i = 0; i < n_seg; ++i) {
-        sf_seg_desc_t t = *desc;
-        t.seg_len = seg_lens[i];
+        sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[i], n_seg);
         const size_t b = sf_workspace_bytes(&t, backward);
         total += b;
         mx = b > mx ? b : mx;
@@ -576,8 +600,7 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     size_t ws_off = 0;
     long long tok = 0;
     for (int i = 0; i < n_seg; ++i) {
-        sf_seg_desc_t t = *desc;
-        t.seg_len = seg_lens[i];
+        sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[i], n_seg);
         const Path path = classify(&t);
         const SegParams p = make_params(&t);
         const FwdWs w = fwd_ws(&t, p, static_cast<char*>(workspace) + ws_off);
@@ -662,8 +685,7 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
         size_t fo = 0, bo = 0;
         long long t = 0;
         for (int i = 0; i < n_seg; ++i) {
-            sf_seg_desc_t d1 = *desc;
-            d1.seg_len = seg_lens[i];
+            sf_seg_desc_t d1 = chain_segment_desc(desc, seg_lens[i], n_seg);
             fwd_off[i] = fo; bwd_off[i] = bo; tok0[i] = t;
             fo += sf_workspace_bytes(&d1, 0);
             bo += sf_workspace_bytes(&d1, mode);
@@ -685,8 +707,7 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     if (ov) {
         // all backward aggregates first, in the order the scans will need them
         for (int i = n_seg - 1; i >= 0; --i) {
-            sf_seg_desc_t t = *desc;
-            t.seg_len = seg_lens[i];
+            sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[i], n_seg);
             const Path path = classify(&t);
             const SegParams p = make_params(&t);
             const BwdWs w = bwd_ws(&t, p, seg_base + bwd_off[i]);
@@ -697,8 +718,7 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     }
     const float* dS_next = dS_final;
     for (int i = n_seg - 1; i >= 0; --i) {
-        sf_seg_desc_t t = *desc;
-        t.seg_len = seg_lens[i];
+        sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[i], n_seg);
         const Path path = classify(&t);
         const SegParams p = make_params(&t);
         char* wsi = seg_base + bwd_off[i];
@@ -847,7 +867,12 @@ sf_status_t sf_chain_autotune(const sf_seg_desc_t* desc, const int32_t* seg_lens
         const size_t need_f = sf_chain_workspace_bytes(&d, seg_lens, n_seg, 0);
         const size_t need_b = dO ? sf_chain_workspace_bytes(&d, seg_lens, n_seg, 1) : 0;
         if (need_f == 0 || need_f > fwd_workspace_bytes || need_b > bwd_workspace_bytes) continue;
+        // On a stream that can be captured the candidate is timed as a graph replay (what a tuned caller will most
+        // likely run, and free of the host's launch cost, which hides the differences for short segments);
+        // on the legacy default stream it is launched directly.
+        sf_chain_graph_t* graph = nullptr;
         auto run = [&]() -> sf_status_t {
+            if (graph) return sf_chain_graph_launch(graph, stream);
             SF_TRY(sf_chain_fwd(&d, seg_lens, n_seg, q, k, v, g, S_init, o, S_bounds, fwd_workspace, fwd_workspace_bytes,
                                 overlap, stream));
             if (dO)
@@ -855,9 +880,18 @@ sf_status_t sf_chain_autotune(const sf_seg_desc_t* desc, const int32_t* seg_lens
                                     fwd_workspace, bwd_workspace, bwd_workspace_bytes, overlap, stream));
             return SF_OK;
         };
-        sf_status_t rs = run();                                   // untimed: first-use costs of this shape
+        sf_status_t rs;
+        if (st != nullptr && st != cudaStreamLegacy) {
+            rs = sf_chain_graph_create(&d, seg_lens, n_seg, q, k, v, g, S_init, o, S_bounds, fwd_workspace,
+                                       fwd_workspace_bytes, dO, dS_final, dq, dk, dv, dg, dS_init, bwd_workspace,
+                                       bwd_workspace_bytes, overlap, stream, &graph);       // runs the chain once itself
+            if (rs == SF_OK) rs = run();
+        } else {
+            rs = run();                                           // untimed: first-use costs of this shape
+        }
         if (rs == SF_ERR_UNSUPPORTED || rs == SF_ERR_INVALID_ARG) {  // this value is not available for this shape
             if (result != SF_OK) result = rs;
+            sf_chain_graph_destroy(graph);
             continue;
         }
         bool ok = rs == SF_OK && cudaEventRecord(e0, st) == cudaSuccess;
@@ -865,6 +899,7 @@ sf_status_t sf_chain_autotune(const sf_seg_desc_t* desc, const int32_t* seg_lens
         float t = 0.f;
         ok = ok && cudaEventRecord(e1, st) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess &&
              cudaEventElapsedTime(&t, e0, e1) == cudaSuccess;
+        sf_chain_graph_destroy(graph);
         if (!ok) {
             cudaGetLastError();
             result = rs != SF_OK ? rs : SF_ERR_CUDA;
