@@ -89,7 +89,8 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm),
+                "window": "timed region plus the same steps kept running until 3 samples were taken"}
 
 
 def max_over_ranks(x: float, dist, device) -> float:
@@ -240,10 +241,17 @@ def main():
         for _ in range(args.warmup):
             step()
     barrier()
+    # Clock samples must come from the GPU under this load.  The timed region of a small workload lasts a few
+    # milliseconds, shorter than nvidia-smi's sampling period, so rank 0 waits for the sampler's first line before
+    # the region (the sampler is then running) and keeps the same steps going, untimed, after the region until three
+    # samples have been taken under load.
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
+        t_wait = time.perf_counter()
+        while not sampler.lines and time.perf_counter() - t_wait < 3.0:
+            time.sleep(0.02)
+        sampler.lines.clear()
     n0 = binding.sf_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -255,6 +263,12 @@ def main():
     barrier()
     ms = e0.elapsed_time(e1)
     launches = binding.sf_launch_count() - n0
+    if rank == 0:
+        t_wait = time.perf_counter()
+        while len(sampler.lines) < 3 and time.perf_counter() - t_wait < 3.0:
+            with torch.cuda.stream(work_stream):
+                step()
+            torch.cuda.synchronize()
     assert binding.sf_device_status() == 0, "a bounded device-side wait ran out"
     ms = max_over_ranks(ms, dist, dev)
     clocks = sampler.stop() if rank == 0 else None
