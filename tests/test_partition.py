@@ -104,10 +104,10 @@ def _near_tie(T, N, wt, ws, alpha, multiple):
 
 def test_library_matches_the_oracle_on_the_paper_grid(binding):
     # N and alpha values the paper profiles (Section 3.2), model-like weights
-    for T in (32768, 65536, 131072, 262144):
+    for T in (65536, 262144):
         for N in (2, 4, 6, 8, 16, 32):
             for alpha in (0.0, 0.1, 0.2, 0.3, 0.4, 0.5, 0.6, 0.7, 0.8, 0.9, 1.0, 1.25):
-                for ws in (0.0, 3e-5, 4e-4):
+                for ws in (3e-5, 4e-4):
                     if _near_tie(T, N, 1.0, ws, alpha, 128):
                         continue
                     assert binding.sf_partition_hybrid(T, N, 1.0, ws, alpha, 128) == P.partition(T, N, 1.0, ws, alpha, 128), \
