@@ -1,4 +1,4 @@
-// Inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, no multicast), tcgen05
+// Inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, plain loads into this CTA only), tcgen05
 // (TMEM allocation, MMA, commit, ld/st) and the shared-memory / instruction descriptors.
 #pragma once
 #include <cuda_runtime.h>
