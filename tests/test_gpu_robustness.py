@@ -1,0 +1,80 @@
+"""Checks that stand in for a race detector and a memory checker: run-to-run bit determinism with the stream overlap
+on, guard regions around every output and workspace buffer, and every block length against the oracle."""
+import pytest
+import torch
+
+from paper_2608_06838_b200 import binding, inputs
+from paper_2608_06838_b200.inputs import Workload
+
+from helpers import NAMES, compare, oracle_reference, run_chain, tolerance
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+GUARD = 4096          # bytes on each side
+
+
+def guarded(nbytes, fill=0xA5):
+    """A byte buffer of nbytes between two guard regions; returns (whole, middle view, 256-byte aligned)."""
+    pad = (GUARD + 255) // 256 * 256
+    whole = torch.full((pad + (nbytes + 255) // 256 * 256 + pad,), fill, dtype=torch.uint8, device=DEV)
+    return whole, whole[pad:pad + nbytes]
+
+
+def guards_intact(whole, nbytes, fill=0xA5):
+    pad = (GUARD + 255) // 256 * 256
+    return bool((whole[:pad] == fill).all()) and bool((whole[pad + nbytes:] == fill).all())
+
+
+@pytest.mark.parametrize("dtype,d,chunk", [("bf16", 128, 64), ("f32", 64, 32)])
+def test_nothing_is_written_outside_the_buffers(dtype, d, chunk):
+    w = Workload("guards", 2, 3, d, d, [5 * chunk, 3 * chunk, 8 * chunk], chunk, dtype=dtype, g_scale=0.1, s_in_sigma=0.05,
+                 ds_out_sigma=0.05, seed=21)
+    x = inputs.make_inputs(w, DEV)
+    B, T, H = w.B, w.T, w.H
+    esz = 2 if dtype == "bf16" else 4
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    desc = binding.make_desc(x["q"], x["v"], x["g"], chunk, 2, seg_len=w.seg_lens[0])
+    sizes = dict(o=B * T * H * d * esz, dq=B * T * H * d * esz, dk=B * T * H * d * esz, dv=B * T * H * d * esz,
+                 dg=B * T * H * 4, S_bounds=(len(w.seg_lens) + 1) * B * H * d * d * 4, dS_init=B * H * d * d * 4,
+                 ws_f=binding.sf_chain_workspace_bytes(desc, w.seg_lens, 0),
+                 ws_b=binding.sf_chain_workspace_bytes(desc, w.seg_lens, 1))
+    whole, mid = {}, {}
+    for n, sz in sizes.items():
+        whole[n], mid[n] = guarded(sz)
+    view = lambda n, dt, shape: mid[n].view(dt).view(*shape)
+    o, dv = view("o", tdt, (B, T, H, d)), view("dv", tdt, (B, T, H, d))
+    dq, dk = view("dq", tdt, (B, T, H, d)), view("dk", tdt, (B, T, H, d))
+    dg = view("dg", torch.float32, (B, T, H))
+    S_bounds = view("S_bounds", torch.float32, (len(w.seg_lens) + 1, B, H, d, d))
+    dS_init = view("dS_init", torch.float32, (B, H, d, d))
+    for overlap in (False, True):
+        binding.sf_chain_fwd(desc, w.seg_lens, x["q"], x["k"], x["v"], x["g"], x["S_in"], o, S_bounds, mid["ws_f"], overlap)
+        binding.sf_chain_bwd(desc, w.seg_lens, x["q"], x["k"], x["v"], x["g"], S_bounds, x["dO"], x["dS_out"], dq, dk, dv, dg,
+                             dS_init, mid["ws_f"], mid["ws_b"], overlap)
+        torch.cuda.synchronize()
+        assert binding.sf_device_status() == 0
+        for n, sz in sizes.items():
+            assert guards_intact(whole[n], sz), "guard region of %s was overwritten (overlap=%s)" % (n, overlap)
+    got = dict(o=o, S_out=S_bounds[-1], dq=dq, dk=dk, dv=dv, dg=dg, dS_in=dS_init)
+    compare(got, oracle_reference(x), tolerance(w), label="guards")
+
+
+def test_repeated_runs_with_overlap_are_bit_identical():
+    # a race between the streams or inside a kernel would show as run-to-run differences
+    w = Workload("determinism", 1, 8, 128, 128, [2048, 1024, 512, 512], 64, s_in_sigma=0.02, ds_out_sigma=0.02, seed=22)
+    x = inputs.make_inputs(w, DEV)
+    first, _ = run_chain(w, x, overlap=True)
+    first = {n: first[n].clone() for n in NAMES}
+    for _ in range(5):
+        again, _ = run_chain(w, x, overlap=True)
+        for n in NAMES:
+            assert torch.equal(first[n], again[n]), n
+
+
+@pytest.mark.parametrize("cpb", [1, 2, 3, 5, 7, 8, 13, 16, 31, 32])
+def test_every_block_length_matches_the_oracle(cpb):
+    # 37 chunks: most block lengths leave a ragged last block
+    w = Workload("blocks-%d" % cpb, 1, 2, 128, 128, [37 * 64], 64, g_scale=0.05, s_in_sigma=0.02, ds_out_sigma=0.02, seed=23)
+    x = inputs.make_inputs(w, DEV)
+    got, _ = run_chain(w, x, chunks_per_block=cpb)
+    compare(got, oracle_reference(x), tolerance(w), label=w.name)
