@@ -49,7 +49,7 @@ typedef struct CUstream_st* sf_stream_t;
 
 typedef enum {
     SF_OK = 0,
-    SF_ERR_INVALID_ARG = 1,   /* NULL where required, bad shape, seg_len % chunk != 0, misalignment, aliasing */
+    SF_ERR_INVALID_ARG = 1,   /* NULL where required, bad shape, misalignment, aliasing */
     SF_ERR_UNSUPPORTED = 2,   /* (dtype, d_k, d_v, chunk) outside the supported set */
     SF_ERR_WORKSPACE = 3,     /* workspace NULL or smaller than sf_workspace_bytes() */
     SF_ERR_CUDA = 4,          /* a CUDA runtime/driver call or a launch failed (cudaGetLastError, no sync) */
@@ -63,8 +63,10 @@ typedef enum { SF_BF16 = 0, SF_F32 = 1 } sf_dtype_t;
  *   SF_F32  : d_k, d_v in {32, 64, 128}, chunk in {16, 32, 64}          (CUDA-core kernels)
  *   SF_BF16 : d_k = d_v = 128, chunk = 64                               (tcgen05 / TMEM / TMA kernels)
  *             d_k, d_v in {32, 64}, chunk in {16, 32, 64}               (CUDA-core kernels)
- * seg_len must be a positive multiple of chunk (the paper rounds boundaries to multiples of 128,
- * Section 3.2).  chunks_per_block sets how many chunks form one block, the only granularity
+ * seg_len is any positive number of tokens.  The paper rounds boundaries to multiples of 128 (Section 3.2), so
+ * its workloads never leave a partial chunk; when seg_len is not a multiple of chunk the last chunk simply has
+ * fewer tokens (its missing rows count as zero keys, values and gradients with log-decay 0, and are never
+ * written).  chunks_per_block sets how many chunks form one block, the only granularity
  * whose states are written to the workspace (at most 32 on the tensor-core path); 0 lets the library
  * pick the length in [4, 32] that fills the device's SMs best for this shape.  Heads are independent.
  */
@@ -79,7 +81,7 @@ typedef struct {
 
 const char* sf_status_string(sf_status_t s);
 
-/* Number of blocks of the segment: ceil((seg_len / chunk) / chunks_per_block), with the library's own choice
+/* Number of blocks of the segment: ceil(ceil(seg_len / chunk) / chunks_per_block), with the library's own choice
    of chunks_per_block when the descriptor leaves it 0.  0 on an invalid descriptor. */
 int32_t sf_num_blocks(const sf_seg_desc_t* desc);
 
@@ -171,7 +173,7 @@ sf_status_t sf_state_scan(const sf_seg_desc_t* desc, int32_t chunks_per_block, i
 /*
  * Segment-chaining driver (paper Eq. 5 and Eq. 7; the single-device part of the partial order of
  * Eq. 8: F_{i-1} before F_i, F_i before B_i, B_{i+1} before B_i).  seg_lens is a HOST array of
- * n_seg segment lengths (each a positive multiple of desc->chunk; desc->seg_len is ignored);
+ * n_seg segment lengths (each positive; desc->seg_len is ignored);
  * q, k, v, g, o, ... address token 0 of the whole sequence of T = sum(seg_lens) tokens.
  *
  * sf_chain_fwd runs Fwd on segments 0..n_seg-1 with S_{i+1}^in = S_i^out.

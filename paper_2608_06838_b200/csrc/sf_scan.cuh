@@ -94,13 +94,16 @@ __global__ void __launch_bounds__(DG_NT) dg_epilogue_kernel(SegParams p, int m, 
 
     // per chunk: suffix sums of x_t and the chunk total, one warp per chunk (C <= 64: two tokens per lane)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ntok = min(nch * C, p.L - c0 * C);          // tokens of this block (the segment's last chunk may be partial)
     const float* xqh = xq + bh * p.L;
     const float* xkh = xk + bh * p.L;
     for (int c = warp; c < nch; c += DG_NT / 32) {
         const long long t0 = (long long)(c0 + c) * C;
         const int r0 = 2 * lane, r1 = 2 * lane + 1;
-        const float x0 = (r0 < C) ? xqh[t0 + r0] - xkh[t0 + r0] : 0.f;
-        const float x1 = (r1 < C) ? xqh[t0 + r1] - xkh[t0 + r1] : 0.f;
+        // tokens past the end of the segment (ragged last chunk) contribute nothing
+        const int lim = min(C, ntok - c * C), i0 = min(r0, lim - 1), i1 = min(r1, lim - 1);
+        const float x0 = (xqh[t0 + i0] - xkh[t0 + i0]) * (r0 < lim ? 1.f : 0.f);
+        const float x1 = (xqh[t0 + i1] - xkh[t0 + i1]) * (r1 < lim ? 1.f : 0.f);
         float incl = x0 + x1;                       // inclusive suffix sum over lanes
         for (int off = 1; off < 32; off <<= 1) {
             const float up = __shfl_down_sync(0xffffffffu, incl, off);
@@ -123,7 +126,7 @@ __global__ void __launch_bounds__(DG_NT) dg_epilogue_kernel(SegParams p, int m, 
     float* dgh = dg + (long long)b * p.bg + h;
     for (int idx = threadIdx.x; idx < nch * C; idx += DG_NT) {
         const int c = idx / C, r = idx - c * C;
-        dgh[((long long)(c0 + c) * C + r) * p.tg] = P_next[c] + suffix[c * 64 + r];
+        if (idx < ntok) dgh[((long long)(c0 + c) * C + r) * p.tg] = P_next[c] + suffix[c * 64 + r];
     }
 }
 

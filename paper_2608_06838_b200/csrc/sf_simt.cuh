@@ -24,24 +24,27 @@ constexpr int NT = 256;        // threads per CTA
 constexpr int MAXC = 64;       // largest chunk
 constexpr int MAXR = 64;       // largest chunks_per_block
 
+// A segment need not be a whole number of chunks: the last chunk then has `valid` < C tokens.  Its missing rows
+// are loaded as zeros and their log-decay as 0, which leaves every sum of the chunk algebra unchanged; their
+// outputs are not stored.
 template <typename T>
-__device__ __forceinline__ void load_tile(float* dst, const T* src, long long tok_stride, int rows, int D) {
-    // dst[r*D + i] = src[r*tok_stride + i]
+__device__ __forceinline__ void load_tile(float* dst, const T* src, long long tok_stride, int rows, int D, int valid) {
+    // dst[r*D + i] = src[r*tok_stride + i] for r < valid, else 0
     for (int idx = threadIdx.x; idx < rows * D; idx += NT) {
         const int r = idx / D, i = idx - r * D;
-        dst[idx] = to_f32(src[(long long)r * tok_stride + i]);
+        dst[idx] = r < valid ? to_f32(src[(long long)r * tok_stride + i]) : 0.f;
     }
 }
 
 // Per-chunk decay tables from the chunk's g (token stride tg):
 //   bcum[r] = sum_{u<=r} g_u     wsuf[r] = exp(sum_{u>r} g_u)     ebc[r] = exp(bcum[r])
 // Returns nothing; bcum[C-1] is the chunk total b_C.  Called by all threads; syncs inside.
-__device__ __forceinline__ void chunk_decay(const float* g, long long tg, int C, float* bcum, float* wsuf, float* ebc) {
+__device__ __forceinline__ void chunk_decay(const float* g, long long tg, int C, int valid, float* bcum, float* wsuf, float* ebc) {
     const int r = threadIdx.x;
     if (r < C) {
         float pre = 0.f, suf = 0.f;
-        for (int u = 0; u <= r; ++u) pre += g[(long long)u * tg];
-        for (int u = C - 1; u > r; --u) suf += g[(long long)u * tg];
+        for (int u = 0; u <= r && u < valid; ++u) pre += g[(long long)u * tg];
+        for (int u = valid - 1; u > r; --u) suf += g[(long long)u * tg];
         bcum[r] = pre;
         wsuf[r] = __expf(suf);
         ebc[r] = __expf(pre);
@@ -74,7 +77,8 @@ __global__ void __launch_bounds__(NT) block_aggregate_kernel(SegParams p, const 
     for (int c = threadIdx.x; c < nch; c += NT) {
         float s = 0.f;
         const long long t0 = (long long)(c0 + c) * C;
-        for (int r = 0; r < C; ++r) s += gh[(t0 + r) * p.tg];
+        const int valid = (int)min((long long)C, p.L - t0);
+        for (int r = 0; r < valid; ++r) s += gh[(t0 + r) * p.tg];
         ctot[c] = s;
     }
     __syncthreads();
@@ -96,13 +100,14 @@ __global__ void __launch_bounds__(NT) block_aggregate_kernel(SegParams p, const 
 
     for (int c = 0; c < nch; ++c) {
         const long long t0 = (long long)(c0 + c) * C;
-        load_tile(Xs, Xh + t0 * p.tqk, p.tqk, C, DK);
-        load_tile(Ys, Yh + t0 * p.tv, p.tv, C, DV);
+        const int valid = (int)min((long long)C, p.L - t0);
+        load_tile(Xs, Xh + t0 * p.tqk, p.tqk, C, DK, valid);
+        load_tile(Ys, Yh + t0 * p.tv, p.tv, C, DV, valid);
         if (threadIdx.x < C) {
             const int r = threadIdx.x;
             float e = 0.f;
-            if (mode == 0) { for (int u = C - 1; u > r; --u) e += gh[(t0 + u) * p.tg]; }
-            else           { for (int u = 0; u <= r; ++u)    e += gh[(t0 + u) * p.tg]; }
+            if (mode == 0) { for (int u = valid - 1; u > r; --u) e += gh[(t0 + u) * p.tg]; }
+            else           { for (int u = 0; u <= r && u < valid; ++u) e += gh[(t0 + u) * p.tg]; }
             w[r] = __expf(e + cofs[c]);
         }
         __syncthreads();
@@ -184,10 +189,11 @@ __global__ void __launch_bounds__(NT) fwd_out_kernel(SegParams p, const T* __res
 
     for (int c = 0; c < nch; ++c) {
         const long long t0 = (long long)(c0 + c) * C;
-        load_tile(Qs, q + qk_off + t0 * p.tqk, p.tqk, C, DK);
-        load_tile(Ks, k + qk_off + t0 * p.tqk, p.tqk, C, DK);
-        load_tile(Vs, v + v_off + t0 * p.tv, p.tv, C, DV);
-        chunk_decay(gh + t0 * p.tg, p.tg, C, bcum, wsuf, ebc);     // syncs
+        const int valid = (int)min((long long)C, p.L - t0);
+        load_tile(Qs, q + qk_off + t0 * p.tqk, p.tqk, C, DK, valid);
+        load_tile(Ks, k + qk_off + t0 * p.tqk, p.tqk, C, DK, valid);
+        load_tile(Vs, v + v_off + t0 * p.tv, p.tv, C, DV, valid);
+        chunk_decay(gh + t0 * p.tg, p.tg, C, valid, bcum, wsuf, ebc);     // syncs
         masked_scores<DK>(A, nullptr, Qs, Ks, bcum, C);
         __syncthreads();
         for (int idx = threadIdx.x; idx < C * DV; idx += NT) {
@@ -195,7 +201,7 @@ __global__ void __launch_bounds__(NT) fwd_out_kernel(SegParams p, const T* __res
             float intra = 0.f, inter = 0.f;
             for (int s = 0; s <= r; ++s) intra = fmaf(A[r * C + s], Vs[s * DV + jv], intra);
             for (int i = 0; i < DK; ++i) inter = fmaf(Qs[r * DK + i], S[i * DV + jv], inter);
-            o[v_off + (t0 + r) * p.tv + jv] = from_f32<T>(intra + ebc[r] * inter);
+            if (r < valid) o[v_off + (t0 + r) * p.tv + jv] = from_f32<T>(intra + ebc[r] * inter);
         }
         __syncthreads();
         state_update<DK, DV>(S, Ks, Vs, wsuf, ebc[C - 1], C);
@@ -233,11 +239,12 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(SegParams p, const T* __rest
 
     for (int c = 0; c < nch; ++c) {
         const long long t0 = (long long)(c0 + c) * C;
-        load_tile(Qs, q + qk_off + t0 * p.tqk, p.tqk, C, DK);
-        load_tile(Ks, k + qk_off + t0 * p.tqk, p.tqk, C, DK);
-        load_tile(Vs, v + v_off + t0 * p.tv, p.tv, C, DV);
-        load_tile(Ds, dO + v_off + t0 * p.tv, p.tv, C, DV);
-        chunk_decay(gh + t0 * p.tg, p.tg, C, bcum, wsuf, ebc);     // syncs
+        const int valid = (int)min((long long)C, p.L - t0);
+        load_tile(Qs, q + qk_off + t0 * p.tqk, p.tqk, C, DK, valid);
+        load_tile(Ks, k + qk_off + t0 * p.tqk, p.tqk, C, DK, valid);
+        load_tile(Vs, v + v_off + t0 * p.tv, p.tv, C, DV, valid);
+        load_tile(Ds, dO + v_off + t0 * p.tv, p.tv, C, DV, valid);
+        chunk_decay(gh + t0 * p.tg, p.tg, C, valid, bcum, wsuf, ebc);     // syncs
         masked_scores<DV>(dA, nullptr, Ds, Vs, bcum, C);
         __syncthreads();
         for (int idx = threadIdx.x; idx < C * DK; idx += NT) {
@@ -249,11 +256,11 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(SegParams p, const T* __rest
                 inter = fmaf(Ds[r * DV + jv], S[i * DV + jv], inter);
             }
             const float tot = intra + ebc[r] * inter;
-            dq[qk_off + (t0 + r) * p.tqk + i] = from_f32<T>(tot);
+            if (r < valid) dq[qk_off + (t0 + r) * p.tqk + i] = from_f32<T>(tot);
             Qs[idx] *= tot;                         // q_r[i] * dq_r[i], reduced below
         }
         __syncthreads();
-        if (threadIdx.x < C) {
+        if (threadIdx.x < valid) {
             const int r = threadIdx.x;
             float s = 0.f;
             for (int i0 = 0; i0 < DK; ++i0) s += Qs[r * DK + ((i0 + r) & (DK - 1))];
@@ -295,11 +302,12 @@ __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __re
 
     for (int c = nch - 1; c >= 0; --c) {
         const long long t0 = (long long)(c0 + c) * C;
-        load_tile(Qs, q + qk_off + t0 * p.tqk, p.tqk, C, DK);
-        load_tile(Ks, k + qk_off + t0 * p.tqk, p.tqk, C, DK);
-        load_tile(Vs, v + v_off + t0 * p.tv, p.tv, C, DV);
-        load_tile(Ds, dO + v_off + t0 * p.tv, p.tv, C, DV);
-        chunk_decay(gh + t0 * p.tg, p.tg, C, bcum, wsuf, ebc);     // syncs
+        const int valid = (int)min((long long)C, p.L - t0);
+        load_tile(Qs, q + qk_off + t0 * p.tqk, p.tqk, C, DK, valid);
+        load_tile(Ks, k + qk_off + t0 * p.tqk, p.tqk, C, DK, valid);
+        load_tile(Vs, v + v_off + t0 * p.tv, p.tv, C, DV, valid);
+        load_tile(Ds, dO + v_off + t0 * p.tv, p.tv, C, DV, valid);
+        chunk_decay(gh + t0 * p.tg, p.tg, C, valid, bcum, wsuf, ebc);     // syncs
         masked_scores<DK>(A, nullptr, Qs, Ks, bcum, C);            // A  = (Q K^T) * D
         masked_scores<DV>(dA, nullptr, Ds, Vs, bcum, C);           // dA = (dO V^T) * D
         __syncthreads();
@@ -308,7 +316,7 @@ __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __re
             float intra = 0.f, inter = 0.f;
             for (int r = s; r < C; ++r) intra = fmaf(A[r * C + s], Ds[r * DV + jv], intra);
             for (int i = 0; i < DK; ++i) inter = fmaf(Ks[s * DK + i], G[i * DV + jv], inter);
-            dv[v_off + (t0 + s) * p.tv + jv] = from_f32<T>(intra + wsuf[s] * inter);
+            if (s < valid) dv[v_off + (t0 + s) * p.tv + jv] = from_f32<T>(intra + wsuf[s] * inter);
         }
         __syncthreads();
         for (int idx = threadIdx.x; idx < C * DK; idx += NT) {     // dk
@@ -320,11 +328,11 @@ __global__ void __launch_bounds__(NT) bwd_dkdv_kernel(SegParams p, const T* __re
                 inter = fmaf(Vs[s * DV + jv], G[i * DV + jv], inter);
             }
             const float tot = intra + wsuf[s] * inter;
-            dk[qk_off + (t0 + s) * p.tqk + i] = from_f32<T>(tot);
+            if (s < valid) dk[qk_off + (t0 + s) * p.tqk + i] = from_f32<T>(tot);
             Ks[idx] *= tot;                         // k_s[i] * dk_s[i], reduced below
         }
         __syncthreads();
-        if (threadIdx.x < C) {
+        if (threadIdx.x < valid) {
             const int s = threadIdx.x;
             float kd = 0.f;
             for (int i0 = 0; i0 < DK; ++i0) kd += Ks[s * DK + ((i0 + s) & (DK - 1))];

@@ -91,12 +91,16 @@ __device__ __forceinline__ void tma_tile(void* dst, const CUtensorMap* m, uint64
 // synchronise afterwards.
 //   bloc[t]  = inclusive cumulative log-decay of token t inside ITS chunk  (t = 0 .. nch*64-1)
 //   ctot[c]  = chunk totals
-__device__ __forceinline__ void prep_decay(const float* __restrict__ gh, long long tg, long long t0, int nch, float* bloc, float* ctot,
-                                           int nwarps) {
+// Tokens at or beyond `L` (a last chunk that is not full) get log-decay 0; TMA fills their tile rows with zeros.
+__device__ __forceinline__ void prep_decay(const float* __restrict__ gh, long long tg, long long t0, int nch, int L, float* bloc,
+                                           float* ctot, int nwarps) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lim = L - (int)t0;                            // tokens from the block start to the end of the segment
     for (int c = warp; c < nch; c += nwarps) {
-        const float g0 = gh[(t0 + c * C + 2 * lane) * tg];
-        const float g1 = gh[(t0 + c * C + 2 * lane + 1) * tg];
+        // unconditional loads from clamped (always valid) tokens, zeroed afterwards: keeps both loads in flight together
+        const int r = c * C + 2 * lane;
+        const float g0 = gh[(t0 + min(r, lim - 1)) * tg] * (r < lim ? 1.f : 0.f);
+        const float g1 = gh[(t0 + min(r + 1, lim - 1)) * tg] * (r + 1 < lim ? 1.f : 0.f);
         float incl = g0 + g1;
         for (int off = 1; off < 32; off <<= 1) {
             const float up = __shfl_up_sync(0xffffffffu, incl, off);
@@ -288,7 +292,8 @@ struct NoWait { __device__ __forceinline__ void operator()() const {} };
 template <bool DOT, typename W = NoWait>
 __device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float scaleB, __nv_bfloat16* __restrict__ out_A,
                                               __nv_bfloat16* __restrict__ out_B, const __nv_bfloat16* __restrict__ e_A,
-                                              const __nv_bfloat16* __restrict__ e_B, float& dotA, float& dotB, W ready = W()) {
+                                              const __nv_bfloat16* __restrict__ e_B, float& dotA, float& dotB, bool validA,
+                                              bool validB, W ready = W()) {
     const int q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
     const uint32_t taddr = pair + ((uint32_t)(q * 32) << 16);
     const int c16 = 8 * (lane & 3);                      // first column of this lane's 16-byte pieces
@@ -299,7 +304,7 @@ __device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float
         uint4 va[4], vb[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            va[i] = __ldg(reinterpret_cast<const uint4*>(e_A + 32 * i + c16));
+            va[i] = __ldg(reinterpret_cast<const uint4*>(e_A + 32 * i + c16));      // callers pass rows inside the segment
             vb[i] = __ldg(reinterpret_cast<const uint4*>(e_B + 32 * i + c16));
         }
 #pragma unroll
@@ -331,8 +336,9 @@ __device__ __forceinline__ void pair_epilogue(uint32_t pair, float scaleA, float
             wa[jj] = pack2(a0, a1);
             wb[jj] = pack2(b0, b1);
         }
-        *reinterpret_cast<uint4*>(out_A + 32 * i + c16) = lanes4_transpose(wa[0], wa[1], wa[2], wa[3]);
-        *reinterpret_cast<uint4*>(out_B + 32 * i + c16) = lanes4_transpose(wb[0], wb[1], wb[2], wb[3]);
+        const uint4 ua = lanes4_transpose(wa[0], wa[1], wa[2], wa[3]), ub = lanes4_transpose(wb[0], wb[1], wb[2], wb[3]);
+        if (validA) *reinterpret_cast<uint4*>(out_A + 32 * i + c16) = ua;      // rows past the end of the segment are not stored
+        if (validB) *reinterpret_cast<uint4*>(out_B + 32 * i + c16) = ub;
     }
     if (DOT) {
         dotA += __shfl_xor_sync(0xffffffffu, dotA, 1); dotA += __shfl_xor_sync(0xffffffffu, dotA, 2);
@@ -441,7 +447,7 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
     } else {
         const float* gh = g + (long long)b * p.bg + h;
-        prep_decay(gh, p.tg, t0, nch, sm.bloc, sm.ctot, WT);
+        prep_decay(gh, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, WT);
         ptx::named_bar_sync(1, AGG_COMP);
         if (tid == 0) {
             float acc = 0.f;
@@ -594,7 +600,7 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
         }
     } else if (warp < 16) {
-        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
+        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, 16);
         ptx::named_bar_sync(1, 512);
         const int wg = warp >> 2, t = tid & 127;
         const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
@@ -624,9 +630,15 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 SF_TR(4, c, 0);
             };
             float dotA, dotB;
+            const bool vA = tokA < p.L, vB = tokB < p.L;          // rows past the end of a ragged segment: computed, not stored
+            const long long lastTok = p.L - 1;
             pair_epilogue<DQ>(tmem + T_O + bf * 128, eA, eB, out_h + tokA * out_tok, out_h + tokB * out_tok,
-                              DQ ? e_h + tokA * out_tok : nullptr, DQ ? e_h + tokB * out_tok : nullptr, dotA, dotB, ready);
-            if (DQ && (lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
+                              DQ ? e_h + min(tokA, lastTok) * out_tok : nullptr, DQ ? e_h + min(tokB, lastTok) * out_tok : nullptr,
+                              dotA, dotB, vA, vB, ready);
+            if (DQ && (lane & 3) == 0) {
+                if (vA) xo[tokA] = dotA;
+                if (vB) xo[tokB] = dotB;
+            }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive_warp(&sm.o_free[bf]);
             SF_TR(4, c, 1);
@@ -809,7 +821,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
         }
     } else if (warp < 16) {
-        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, sm.bloc, sm.ctot, 16);
+        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, 16);
         ptx::named_bar_sync(1, 512);
         const int wg = warp >> 2, t = tid & 127;
         const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
@@ -834,6 +846,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const int c = nch - 1 - i;
                 const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
                 const float wA = fast_exp(sm.ctot[c] - sm.bloc[c * C + rA]), wB = fast_exp(sm.ctot[c] - sm.bloc[c * C + rB]);
+                const bool vA = tokA < p.L, vB = tokB < p.L;
                 float dotA, dotB;
                 auto dk_ready = [&]() {
                     SF_TR(4, i, 1);
@@ -846,7 +859,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     SF_WAIT(&sm.dv_done, i & 1, DEV_TIMEOUT_MMA);
                     ptx::tc_fence_after_sync();
                     SF_TR(6, i, 1);
-                    pair_epilogue<false>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, dotA, dotB);
+                    pair_epilogue<false>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, dotA, dotB, vA, vB);
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dv_free);
                     SF_TR(6, i, 2);
@@ -854,8 +867,11 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     SF_TR(6, i, 3);
                 } else {
                     SF_TR(4, i, 0);
-                    pair_epilogue<true>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, k_h + tokA * p.tqk, k_h + tokB * p.tqk, dotA, dotB, dk_ready);
-                    if ((lane & 3) == 0) { xo[tokA] = dotA; xo[tokB] = dotB; }
+                    pair_epilogue<true>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, k_h + min(tokA, (long long)p.L - 1) * p.tqk, k_h + min(tokB, (long long)p.L - 1) * p.tqk, dotA, dotB, vA, vB, dk_ready);
+                    if ((lane & 3) == 0) {
+                        if (vA) xo[tokA] = dotA;
+                        if (vB) xo[tokB] = dotB;
+                    }
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dk_free);
                     SF_TR(4, i, 3);

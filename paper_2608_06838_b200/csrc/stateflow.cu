@@ -57,7 +57,6 @@ enum class Path { Invalid, Unsupported, Simt, Tc };
 Path classify(const sf_seg_desc_t* d) {
     if (!d) return Path::Invalid;
     if (d->B <= 0 || d->H <= 0 || d->d_k <= 0 || d->d_v <= 0 || d->chunk <= 0 || d->seg_len <= 0) return Path::Invalid;
-    if (d->seg_len % d->chunk != 0) return Path::Invalid;
     if (d->chunks_per_block < 0 || d->chunks_per_block > sf::simt::MAXR) return Path::Invalid;
     if (d->dtype != SF_BF16 && d->dtype != SF_F32) return Path::Invalid;
     if (d->tok_stride_qk < (long long)d->H * d->d_k || d->tok_stride_v < (long long)d->H * d->d_v || d->tok_stride_g < d->H)
@@ -127,14 +126,14 @@ sf_seg_desc_t chain_segment_desc(const sf_seg_desc_t* desc, int32_t seg_len, int
     sf_seg_desc_t t = *desc;
     t.seg_len = seg_len;
     if (t.chunks_per_block == 0 && n_seg > 1 && t.chunk > 0)
-        t.chunks_per_block = chain_chunks_per_block(seg_len / t.chunk, (long long)t.B * t.H);
+        t.chunks_per_block = chain_chunks_per_block((seg_len + t.chunk - 1) / t.chunk, (long long)t.B * t.H);
     return t;
 }
 
 SegParams make_params(const sf_seg_desc_t* d, int cpb_override = 0) {
     SegParams p;
     p.B = d->B; p.H = d->H; p.L = d->seg_len; p.C = d->chunk;
-    p.NC = d->seg_len / d->chunk;
+    p.NC = (d->seg_len + d->chunk - 1) / d->chunk;      // the last chunk may be partial
     int r = cpb_override > 0 ? cpb_override : d->chunks_per_block;
     p.R = r > 0 ? r : auto_chunks_per_block(p.NC, (long long)d->B * d->H);
     p.NB = (p.NC + p.R - 1) / p.R;
@@ -418,7 +417,7 @@ sf_status_t validate_chain(const sf_seg_desc_t* d, const int32_t* seg_lens, int3
     if (!d || !seg_lens || n_seg <= 0 || n_seg > 1 << 20) return SF_ERR_INVALID_ARG;
     long long T = 0;
     for (int i = 0; i < n_seg; ++i) {
-        if (seg_lens[i] <= 0 || d->chunk <= 0 || seg_lens[i] % d->chunk) return SF_ERR_INVALID_ARG;
+        if (seg_lens[i] <= 0 || d->chunk <= 0) return SF_ERR_INVALID_ARG;
         T += seg_lens[i];
     }
     sf_seg_desc_t t = *d;

@@ -78,3 +78,43 @@ def test_every_block_length_matches_the_oracle(cpb):
     x = inputs.make_inputs(w, DEV)
     got, _ = run_chain(w, x, chunks_per_block=cpb)
     compare(got, oracle_reference(x), tolerance(w), label=w.name)
+
+
+@pytest.mark.parametrize("dtype,d,chunk,segs", [
+    ("f32", 64, 32, [100, 37, 200]),
+    ("f32", 32, 16, [5]),
+    ("bf16", 128, 64, [1000, 70, 300, 65]),
+    ("bf16", 128, 64, [17]),
+    ("bf16", 64, 64, [130, 63]),
+])
+def test_segments_that_are_not_whole_chunks(dtype, d, chunk, segs):
+    # the last chunk of a segment may be partial; the next segment then starts in the middle of a chunk-sized stretch
+    w = Workload("ragged-%s-%d" % (dtype, sum(segs)), 2, 3, d, d, segs, chunk, dtype=dtype, g_scale=0.1, s_in_sigma=0.05,
+                 ds_out_sigma=0.05, seed=31)
+    x = inputs.make_inputs(w, DEV)
+    for cpb in (2, 0):
+        got, _ = run_chain(w, x, chunks_per_block=cpb)
+        compare(got, oracle_reference(x), tolerance(w), label=w.name)
+    got = {n: got[n].clone() for n in NAMES}                  # the run with the library's own block length
+    # and nothing beyond the last token is touched: the same run on views of tensors with `chunk` more tokens per batch
+    T, pad = w.T, chunk
+    def padded(t, fill):
+        shape = list(t.shape)
+        shape[1] = T + pad
+        big = torch.full(shape, fill, dtype=t.dtype, device=DEV)
+        big[:, :T] = t
+        return big
+    xin = {n: padded(x[n], 3.0) for n in ("q", "k", "v", "g", "dO")}
+    run = binding.ChainRun(xin["q"][:, :T], xin["k"][:, :T], xin["v"][:, :T], xin["g"][:, :T], xin["dO"][:, :T], w.seg_lens, w.chunk)
+    outs = {n: padded(getattr(run, n), 7.0) for n in ("o", "dq", "dk", "dv", "dg")}
+    for n in outs:
+        setattr(run, n, outs[n][:, :T])
+    run.forward(x["S_in"])
+    run.backward(x["dS_out"])
+    torch.cuda.synchronize()
+    assert binding.sf_device_status() == 0
+    for n in outs:
+        assert bool((outs[n][:, T:] == 7.0).all()), "%s was written beyond the last token" % n
+    padded_got = dict(o=run.o, S_out=run.S_bounds[-1], dq=run.dq, dk=run.dk, dv=run.dv, dg=run.dg, dS_in=run.dS_init)
+    for n in NAMES:
+        assert torch.equal(padded_got[n], got[n]), n          # the padding's content (3.0, not zero) must not leak in

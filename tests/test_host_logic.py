@@ -52,7 +52,7 @@ def fwd(lib, d, q=P, k=P, v=P, g=P, S_in=None, o=P, S_out=ctypes.c_void_p(0x2000
 def test_forward_validation_happens_before_any_launch(lib):
     assert fwd(lib, desc(), q=None) == 1
     assert fwd(lib, desc(), S_out=None) == 1
-    assert fwd(lib, desc(seg_len=1000)) == 1                       # not a multiple of the chunk
+    assert fwd(lib, desc(seg_len=0)) == 1 and fwd(lib, desc(seg_len=-64)) == 1     # empty or negative segment
     assert fwd(lib, desc(B=0)) == 1
     assert fwd(lib, desc(d_k=96, d_v=96)) == 2                      # unsupported head width
     assert fwd(lib, desc(chunk=32)) == 2                            # bf16 d=128 needs chunk 64
@@ -89,7 +89,9 @@ def test_workspace_arithmetic(lib):
     assert b1 == 32 * 8 * state + 2 * 32 * 8192 * 4
     assert binding.sf_workspace_bytes(d, 2) == b1 + f + 32 * state
     assert binding.sf_num_blocks(desc(seg_len=17 * 64, chunks_per_block=4)) == 5
-    assert binding.sf_workspace_bytes(desc(seg_len=1000), 0) == 0
+    assert binding.sf_workspace_bytes(desc(seg_len=0), 0) == 0
+    # a ragged segment counts its partial last chunk: 1000 tokens = 16 chunks of 64
+    assert binding.sf_workspace_bytes(desc(seg_len=1000, chunks_per_block=16), 0) == binding.sf_workspace_bytes(desc(seg_len=1024, chunks_per_block=16), 0)
     segs = [12288, 10240, 8192]
     tot = sum(binding.sf_workspace_bytes(desc(H=32, seg_len=s, chunks_per_block=16), 0) for s in segs)
     assert binding.sf_chain_workspace_bytes(d, segs, 0) == tot
@@ -100,7 +102,7 @@ def test_workspace_arithmetic(lib):
     assert binding.sf_num_blocks(auto) == 4                          # 32 chunks per block: 128 CTAs, one wave
     assert binding.sf_num_blocks(desc(H=16, seg_len=4096)) == 8      # 8 chunks per block: 128 CTAs
     assert 1 <= binding.sf_num_blocks(desc(H=1, seg_len=64)) <= 1
-    assert binding.sf_chain_workspace_bytes(d, [100], 0) == 0
+    assert binding.sf_chain_workspace_bytes(d, [0], 0) == 0 and binding.sf_chain_workspace_bytes(d, [100], 0) > 0
 
 
 def test_status_strings(lib):
@@ -179,6 +181,6 @@ def test_autotune_rejects_bad_arguments_before_any_cuda_call(lib):
     assert lib.sf_chain_autotune(*head, cands, 0, 3, 1, None, ctypes.byref(best), None) == 1
     assert lib.sf_chain_autotune(*head, cands, 2, 0, 1, None, ctypes.byref(best), None) == 1       # no repetitions
     assert lib.sf_chain_autotune(*head, cands, 2, 3, 1, None, None, None) == 1                     # nowhere to report
-    bad = (ctypes.c_int32 * 1)(1000)                                                               # not a multiple of the chunk
+    bad = (ctypes.c_int32 * 1)(0)                                                                  # an empty segment
     assert lib.sf_chain_autotune(ctypes.byref(d), bad, 1, *head[3:], cands, 2, 3, 1, None, ctypes.byref(best), None) == 1
     assert best.value == -7
