@@ -43,6 +43,23 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def copy_probe(device, nbytes=1 << 30, reps=5):
+    """Device-to-device copy bandwidth of this machine right now (read + write bytes per second), so that a degraded
+    box shows in the report next to the roofline's fixed denominator.  Uses the driver's copy, none of this library."""
+    import torch
+    a = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    b = torch.empty_like(a)
+    b.copy_(a)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        b.copy_(a)
+    e1.record()
+    torch.cuda.synchronize()
+    return 2.0 * nbytes * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -272,6 +289,7 @@ def main():
     assert binding.sf_device_status() == 0, "a bounded device-side wait ran out"
     ms = max_over_ranks(ms, dist, dev)
     clocks = sampler.stop() if rank == 0 else None
+    probe = copy_probe(dev) if rank == 0 else None
     ms_per_step = ms / args.steps
     tokens = w.B * w.T
     value = replica_throughput(tokens, world, ms_per_step)
@@ -353,7 +371,7 @@ def main():
                    "autotune": tuned, "overlap": overlap, "graph": bool(args.graph),
                    "l2": "inputs (%.0f MB) exceed L2, no flush" % (4 * tokens * w.H * w.d_k * 2 / 1e6),
                    "parallelism": "replicas only"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roof, "path_roofline": path_roof,
+        "clocks": clocks, "copy_probe_gbs": probe, "e2e": e2e, "gpu_launches": launches, "roofline": roof, "path_roofline": path_roof,
         "stages": stage, "cpu_baseline": cpu,
     }
     print(json.dumps(out))
