@@ -188,10 +188,12 @@ sf_status_t sf_state_scan(const sf_seg_desc_t* desc, int32_t chunks_per_block, i
  * overlap != 0 lets the driver run state-independent stages on internal side streams concurrently
  * with the state scans (the split-and-overlap idea of Section 3.4, Eq. 17-18).  Only the scans carry
  * the state from segment to segment, so they alone chain on `stream`: forward, the block aggregates
- * run ahead on one side stream and each segment's sweep starts on another as soon as its own scan is
+ * run ahead on side streams and each segment's sweep starts on another as soon as its own scan is
  * done; backward (with fwd_workspace given), all aggregates run ahead, and each segment's dq sweep and
- * dk/dv sweep (+ dg) start on further streams after its own reverse scan.  Sweeps of consecutive
- * segments go to different streams (round-robin), so short segments share the device.
+ * dk/dv sweep (+ dg) start on further streams after its own reverse scan.  Aggregates and sweeps of
+ * consecutive short segments go to different streams (round-robin), so they share the device, and
+ * up to 8 neighbouring segments of at most 4096 tokens in total are scanned by one kernel that carries
+ * the state from one to the next in registers.
  * The result is bit-identical to overlap == 0.  The side streams are joined back
  * into `stream` before the call returns, so later work on `stream` sees all outputs.
  */

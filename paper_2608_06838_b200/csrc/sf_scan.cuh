@@ -56,6 +56,64 @@ __global__ void __launch_bounds__(SCAN_NT) state_scan_kernel(int n, int m, int r
     *reinterpret_cast<float4*>(final_state + (long long)bh * m + e) = x;
 }
 
+// The same recurrence carried through several consecutive segments in one launch (paper Eq. 5 / Eq. 7: the state
+// leaving one segment enters the next).  With short segments the chain of one small scan kernel per segment is
+// what the hand-off costs (launch and dependency latency, not bytes), so the chaining driver scans a group of
+// segments at once.  Segments are listed in the order they are visited (ascending forward, descending in
+// reverse); the arithmetic per element is the one of state_scan_kernel, so results are bit-identical.
+constexpr int SCAN_GROUP_MAX = 8;
+struct ScanSeg {
+    const float* ld;        // [B*H, n] block totals of the log-decay
+    float* UH;              // [B*H, n, m] aggregates in, states out (in place)
+    float* fin;             // [B*H, m] boundary state leaving the segment in scan direction
+    int n;
+};
+struct ScanGroup {
+    ScanSeg seg[SCAN_GROUP_MAX];
+    int count;
+};
+
+__global__ void __launch_bounds__(SCAN_NT) state_scan_group_kernel(ScanGroup grp, int m, int reverse, const float* __restrict__ init) {
+    const int bh = blockIdx.y;
+    const int e = (blockIdx.x * SCAN_NT + threadIdx.x) * 4;
+    if (e >= m) return;
+    const long long step = m / 4;
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (init) x = *reinterpret_cast<const float4*>(init + (long long)bh * m + e);
+    for (int si = 0; si < grp.count; ++si) {
+        const ScanSeg sg = grp.seg[si];
+        const int n = sg.n;
+        const float* ldh = sg.ld + (long long)bh * n;
+        float4* Sh = reinterpret_cast<float4*>(sg.UH + (long long)bh * n * m + e);
+        for (int s0 = 0; s0 < n; s0 += SCAN_UNROLL) {
+            float4 u[SCAN_UNROLL];
+            float a[SCAN_UNROLL];
+#pragma unroll
+            for (int i = 0; i < SCAN_UNROLL; ++i) {
+                const int s = s0 + i;
+                if (s < n) {
+                    const int j = reverse ? (n - 1 - s) : s;
+                    u[i] = Sh[j * step];
+                    a[i] = __expf(ldh[j]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < SCAN_UNROLL; ++i) {
+                const int s = s0 + i;
+                if (s < n) {
+                    const int j = reverse ? (n - 1 - s) : s;
+                    Sh[j * step] = x;
+                    x.x = fmaf(a[i], x.x, u[i].x);
+                    x.y = fmaf(a[i], x.y, u[i].y);
+                    x.z = fmaf(a[i], x.z, u[i].z);
+                    x.w = fmaf(a[i], x.w, u[i].w);
+                }
+            }
+        }
+        *reinterpret_cast<float4*>(sg.fin + (long long)bh * m + e) = x;
+    }
+}
+
 // Log-decay gradient.  With x_t = q_t.dq_t - k_t.dk_t (the dq and dk/dv passes emit both dot products
 // from their float32 accumulators) the recurrence gives dg_t = dg_{t+1} + x_t, and at a block start
 // dg equals <H, dH> of the block-entering state and its gradient plus the block's x.  So, with

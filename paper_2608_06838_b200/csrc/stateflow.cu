@@ -285,6 +285,31 @@ sf_status_t launch_scan(const sf_seg_desc_t* d, const SegParams& p, int reverse,
     return check_launch();
 }
 
+// Scan of a group of consecutive segments in one launch (the chaining driver's way to shorten the serial chain of
+// small scan kernels).  `grp` lists the segments in visiting order.
+sf_status_t launch_scan_group(const sf_seg_desc_t* d, int BH, const sf::ScanGroup& grp, int reverse, const float* init,
+                              cudaStream_t st) {
+    const int m = d->d_k * d->d_v;
+    StageTimer timer(ST_SCAN, st);
+    dim3 grid((m / 4 + sf::SCAN_NT - 1) / sf::SCAN_NT, BH);
+    sf::state_scan_group_kernel<<<grid, sf::SCAN_NT, 0, st>>>(grp, m, reverse, init);
+    return check_launch();
+}
+
+// Segments i, i+dir, ... that the chaining driver scans together: up to SCAN_GROUP_MAX short segments of at most
+// kScanGroupTokens tokens in total (one long segment is a group of its own).
+constexpr long long kScanGroupTokens = 4096;
+int scan_group_size(const int32_t* seg_lens, int n_seg, int i, int dir) {
+    int count = 1;
+    long long tokens = seg_lens[i];
+    for (int k = i + dir; k >= 0 && k < n_seg && count < sf::SCAN_GROUP_MAX; k += dir) {
+        if (tokens + seg_lens[k] > kScanGroupTokens) break;
+        tokens += seg_lens[k];
+        ++count;
+    }
+    return count;
+}
+
 // ---- one segment -------------------------------------------------------------------------------
 struct FwdPtrs { const void *q, *k, *v; const float* g; const float* S_in; void* o; float* S_out; };
 
@@ -365,8 +390,14 @@ sf_status_t validate_bwd(const sf_seg_desc_t* d, const BwdPtrs& x, const void* s
 // Side streams and events of the chaining driver (host objects only; created once per process).
 // Sweeps of consecutive segments go to different streams: a short segment's sweep does not fill the device.
 constexpr int kSweepStreams = 4;
+// The aggregates of different segments are independent of everything: they go round-robin to their own streams
+// (with short segments one stream of small aggregate kernels is the longest chain of the step).
+constexpr int kAggStreams = 4;
+// ... unless a segment's aggregate kernel fills half the device by itself: those stay in order on one stream
+inline int agg_stream_index(const SegParams& p, int i) { return (long long)p.B * p.H * p.NB >= 74 ? 0 : i % kAggStreams; }
 struct ChainRes {
-    cudaStream_t side[1 + 2 * kSweepStreams] = {};   // 0: aggregates; then two groups of sweep streams, used round-robin by segment
+    cudaStream_t side[1 + 2 * kSweepStreams] = {};   // 0: unused; then two groups of sweep streams, used round-robin by segment
+    cudaStream_t agg[kAggStreams] = {};
     cudaEvent_t ev[64] = {};
     std::vector<cudaEvent_t> pool;          // extra events of the backward driver, grown on demand
     bool ok = false;
@@ -381,6 +412,8 @@ sf_status_t chain_resources(ChainRes** out) {
     if (cudaGetDevice(&dev) != cudaSuccess) return SF_ERR_CUDA;
     if (!g_chain.ok || g_chain.device != dev) {
         for (auto& s : g_chain.side)
+            if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SF_ERR_CUDA;
+        for (auto& s : g_chain.agg)
             if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SF_ERR_CUDA;
         for (auto& e : g_chain.ev)
             if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return SF_ERR_CUDA;
@@ -592,46 +625,74 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     //   side streams 1..: [wait ST(i)] Out(i)             (round-robin, so that the sweeps of short neighbouring
     //                                                      segments, which do not fill the device, run side by side)
     if (overlap) {
-        SF_TRY(chain_events(res, (size_t)n_seg + 2 + kSweepStreams));
+        SF_TRY(chain_events(res, 2 * (size_t)n_seg + 2 + kSweepStreams + kAggStreams));
         SF_CUDA(cudaEventRecord(res->ev[0], st));
         for (int s = 0; s <= kSweepStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->side[s], res->ev[0], 0));
+        for (int s = 0; s < kAggStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->agg[s], res->ev[0], 0));
     }
-    size_t ws_off = 0;
-    long long tok = 0;
-    for (int i = 0; i < n_seg; ++i) {
-        sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[i], n_seg);
-        const Path path = classify(&t);
-        const SegParams p = make_params(&t);
-        const FwdWs w = fwd_ws(&t, p, static_cast<char*>(workspace) + ws_off);
-        ws_off += w.bytes;
-        FwdPtrs x{SeqPtr::at(q, tok, t.tok_stride_qk, esz), SeqPtr::at(k, tok, t.tok_stride_qk, esz),
-                  SeqPtr::at(v, tok, t.tok_stride_v, esz),
-                  static_cast<const float*>(SeqPtr::at(g, tok, t.tok_stride_g, sizeof(float))),
-                  S_bounds + (size_t)i * sN, SeqPtr::at(o, tok, t.tok_stride_v, esz), S_bounds + (size_t)(i + 1) * sN};
-        if (overlap) {
-            cudaEvent_t e = res->ev[1 + (i % 32)];
-            SF_TRY(fwd_pre(path, &t, p, x, w, res->side[0]));
-            SF_CUDA(cudaEventRecord(e, res->side[0]));
-            SF_CUDA(cudaStreamWaitEvent(st, e, 0));
-        } else {
-            SF_TRY(fwd_pre(path, &t, p, x, w, st));
+    struct Seg { sf_seg_desc_t t; Path path; SegParams p; FwdWs w; FwdPtrs x; };
+    std::vector<Seg> segs(n_seg);
+    {
+        size_t ws_off = 0;
+        long long tok = 0;
+        for (int i = 0; i < n_seg; ++i) {
+            Seg& sg = segs[i];
+            sg.t = chain_segment_desc(desc, seg_lens[i], n_seg);
+            sg.path = classify(&sg.t);
+            sg.p = make_params(&sg.t);
+            sg.w = fwd_ws(&sg.t, sg.p, static_cast<char*>(workspace) + ws_off);
+            ws_off += sg.w.bytes;
+            sg.x = FwdPtrs{SeqPtr::at(q, tok, sg.t.tok_stride_qk, esz), SeqPtr::at(k, tok, sg.t.tok_stride_qk, esz),
+                           SeqPtr::at(v, tok, sg.t.tok_stride_v, esz),
+                           static_cast<const float*>(SeqPtr::at(g, tok, sg.t.tok_stride_g, sizeof(float))),
+                           S_bounds + (size_t)i * sN, SeqPtr::at(o, tok, sg.t.tok_stride_v, esz), S_bounds + (size_t)(i + 1) * sN};
+            tok += seg_lens[i];
         }
-        SF_TRY(fwd_scan(&t, p, x, w, st));
-        if (overlap) {
-            cudaStream_t s_out = res->side[1 + (i % kSweepStreams)];
+    }
+    if (!overlap) {
+        for (int i = 0; i < n_seg; ++i) {
+            const Seg& sg = segs[i];
+            SF_TRY(fwd_pre(sg.path, &sg.t, sg.p, sg.x, sg.w, st));
+            SF_TRY(fwd_scan(&sg.t, sg.p, sg.x, sg.w, st));
+            SF_TRY(fwd_out(sg.path, &sg.t, sg.p, sg.x, sg.w, st));
+        }
+    } else {
+        for (int i = 0; i < n_seg;) {
+            // short neighbouring segments are scanned in one launch (the state is carried in registers from one to
+            // the next); their aggregates go first, their sweeps after
+            const int cnt = scan_group_size(seg_lens, n_seg, i, +1);
+            sf::ScanGroup grp{};
+            grp.count = cnt;
+            for (int k = 0; k < cnt; ++k) {
+                const Seg& sg = segs[i + k];
+                cudaStream_t s_agg = res->agg[agg_stream_index(sg.p, i + k)];
+                cudaEvent_t e = res->pool[(size_t)n_seg + (i + k)];
+                SF_TRY(fwd_pre(sg.path, &sg.t, sg.p, sg.x, sg.w, s_agg));
+                SF_CUDA(cudaEventRecord(e, s_agg));
+                SF_CUDA(cudaStreamWaitEvent(st, e, 0));
+                grp.seg[k] = sf::ScanSeg{sg.w.beta, sg.w.UH, sg.x.S_out, sg.p.NB};
+            }
+            SF_TRY(launch_scan_group(desc, desc->B * desc->H, grp, 0, segs[i].x.S_in, st));
             SF_CUDA(cudaEventRecord(res->pool[i], st));
-            SF_CUDA(cudaStreamWaitEvent(s_out, res->pool[i], 0));
-            SF_TRY(fwd_out(path, &t, p, x, w, s_out));
-        } else {
-            SF_TRY(fwd_out(path, &t, p, x, w, st));
+            for (int k = 0; k < cnt; ++k) {
+                const Seg& sg = segs[i + k];
+                cudaStream_t s_out = res->side[1 + ((i + k) % kSweepStreams)];
+                SF_CUDA(cudaStreamWaitEvent(s_out, res->pool[i], 0));
+                SF_TRY(fwd_out(sg.path, &sg.t, sg.p, sg.x, sg.w, s_out));
+            }
+            i += cnt;
         }
-        tok += seg_lens[i];
     }
     if (overlap) {
         // join the sweep streams back into the caller's stream
         for (int s = 1; s <= kSweepStreams; ++s) {
-            cudaEvent_t e = res->pool[(size_t)n_seg + s];
+            cudaEvent_t e = res->pool[2 * (size_t)n_seg + s];
             SF_CUDA(cudaEventRecord(e, res->side[s]));
+            SF_CUDA(cudaStreamWaitEvent(st, e, 0));
+        }
+        for (int s = 0; s < kAggStreams; ++s) {
+            cudaEvent_t e = res->pool[2 * (size_t)n_seg + 1 + kSweepStreams + s];
+            SF_CUDA(cudaEventRecord(e, res->agg[s]));
             SF_CUDA(cudaStreamWaitEvent(st, e, 0));
         }
     }
@@ -661,20 +722,19 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     char* seg_base = base + (size_t)n_seg * sB;
 
     // overlap schedule (Section 3.4, Eq. 18, across segments): only the reverse scans carry the boundary
-    // gradient from segment to segment.  The backward aggregates need no boundary gradient (side stream 0,
+    // gradient from segment to segment.  The backward aggregates need no boundary gradient (their own streams,
     // ahead of everything), the scans chain on the main stream, and the two sweeps of a segment need only
     // its own scan: dq sweeps queue on one group of side streams, dk/dv sweeps and the dg epilogue on another
     // (round-robin by segment, so that neighbouring short segments share the device).
     const bool ov = overlap != 0 && fwd_workspace != nullptr;
     ChainRes* res = nullptr;
-    cudaStream_t s_pre = st;
     if (ov) {
         SF_TRY(chain_resources(&res));
-        SF_TRY(chain_events(res, 3 * (size_t)n_seg + 2 + 2 * kSweepStreams));
-        s_pre = res->side[0];
+        SF_TRY(chain_events(res, 3 * (size_t)n_seg + 2 + 2 * kSweepStreams + kAggStreams));
         cudaEvent_t e0 = res->pool[3 * (size_t)n_seg];
         SF_CUDA(cudaEventRecord(e0, st));
         for (int s = 0; s <= 2 * kSweepStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->side[s], e0, 0));
+        for (int s = 0; s < kAggStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->agg[s], e0, 0));
     }
 
     // per-segment offsets
@@ -711,60 +771,93 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
             const SegParams p = make_params(&t);
             const BwdWs w = bwd_ws(&t, p, seg_base + bwd_off[i]);
             BwdPtrs x = seg_ptrs(i, t, nullptr, nullptr);
-            SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, s_pre));
-            SF_CUDA(cudaEventRecord(res->pool[3 * (size_t)i], s_pre));
+            cudaStream_t s_agg = res->agg[agg_stream_index(p, i)];
+            SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, s_agg));
+            SF_CUDA(cudaEventRecord(res->pool[3 * (size_t)i], s_agg));
         }
     }
     const float* dS_next = dS_final;
-    for (int i = n_seg - 1; i >= 0; --i) {
-        sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[i], n_seg);
-        const Path path = classify(&t);
-        const SegParams p = make_params(&t);
-        char* wsi = seg_base + bwd_off[i];
-        const BwdWs w = bwd_ws(&t, p, wsi);
-        float* dS_here = dS_buf(i);
-        BwdPtrs x = seg_ptrs(i, t, dS_next, dS_here);
-        FwdWs fw;
-        if (fwd_workspace) {
-            fw = fwd_ws(&t, p, const_cast<char*>(static_cast<const char*>(fwd_workspace)) + fwd_off[i]);
-        } else {
-            char* fbase = wsi + w.bytes;
-            fw = fwd_ws(&t, p, fbase);
-            float* sfin = reinterpret_cast<float*>(fbase + fw.bytes);
-            FwdPtrs fx{x.q, x.k, x.v, x.g, x.S_in, nullptr, sfin};
-            SF_TRY(fwd_pre(path, &t, p, fx, fw, st));
-            SF_TRY(fwd_scan(&t, p, fx, fw, st));
-        }
-        if (ov) {
-            SF_CUDA(cudaStreamWaitEvent(st, res->pool[3 * (size_t)i], 0));
-        } else {
-            SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, st));
-        }
-        SF_TRY(bwd_scan(&t, p, x, w, fw.beta, st));
-        if (ov) {
-            cudaEvent_t e_scan = res->pool[3 * (size_t)i + 1], e_dq = res->pool[3 * (size_t)i + 2];
-            // the sweeps of neighbouring segments alternate between two pairs of streams
-            cudaStream_t s_dq = res->side[1 + (i % kSweepStreams)], s_kv = res->side[1 + kSweepStreams + (i % kSweepStreams)];
+    if (ov) {
+        // (ov implies the forward workspace is given)  Groups of short neighbouring segments, visited in descending
+        // order, share one reverse scan; each segment's sweeps start when its group's scan is done.
+        for (int i = n_seg - 1; i >= 0;) {
+            const int cnt = scan_group_size(seg_lens, n_seg, i, -1);
+            struct Seg { sf_seg_desc_t t; Path path; SegParams p; BwdWs w; BwdPtrs x; FwdWs fw; };
+            Seg sg[sf::SCAN_GROUP_MAX];
+            sf::ScanGroup grp{};
+            grp.count = cnt;
+            const float* group_init = dS_next;
+            for (int k = 0; k < cnt; ++k) {
+                const int idx = i - k;
+                Seg& s = sg[k];
+                s.t = chain_segment_desc(desc, seg_lens[idx], n_seg);
+                s.path = classify(&s.t);
+                s.p = make_params(&s.t);
+                s.w = bwd_ws(&s.t, s.p, seg_base + bwd_off[idx]);
+                float* dS_here = dS_buf(idx);
+                s.x = seg_ptrs(idx, s.t, dS_next, dS_here);
+                s.fw = fwd_ws(&s.t, s.p, const_cast<char*>(static_cast<const char*>(fwd_workspace)) + fwd_off[idx]);
+                grp.seg[k] = sf::ScanSeg{s.fw.beta, s.w.GU, dS_here, s.p.NB};
+                dS_next = dS_here;
+            }
+            for (int k = 0; k < cnt; ++k) SF_CUDA(cudaStreamWaitEvent(st, res->pool[3 * (size_t)(i - k)], 0));
+            SF_TRY(launch_scan_group(desc, desc->B * desc->H, grp, 1, group_init, st));
+            cudaEvent_t e_scan = res->pool[3 * (size_t)i + 1];
             SF_CUDA(cudaEventRecord(e_scan, st));
-            SF_CUDA(cudaStreamWaitEvent(s_dq, e_scan, 0));
-            SF_CUDA(cudaStreamWaitEvent(s_kv, e_scan, 0));
-            SF_TRY(bwd_dq(path, &t, p, x, w, fw.UH, s_dq));
-            SF_CUDA(cudaEventRecord(e_dq, s_dq));
-            SF_TRY(bwd_dkdv(path, &t, p, x, w, s_kv));
-            SF_CUDA(cudaStreamWaitEvent(s_kv, e_dq, 0));
-            SF_TRY(bwd_dg(&t, p, x, w, fw.UH, s_kv));
-        } else {
+            for (int k = 0; k < cnt; ++k) {
+                const int idx = i - k;
+                const Seg& s = sg[k];
+                cudaEvent_t e_dq = res->pool[3 * (size_t)idx + 2];
+                // the sweeps of neighbouring segments go round-robin to different streams
+                cudaStream_t s_dq = res->side[1 + (idx % kSweepStreams)], s_kv = res->side[1 + kSweepStreams + (idx % kSweepStreams)];
+                SF_CUDA(cudaStreamWaitEvent(s_dq, e_scan, 0));
+                SF_CUDA(cudaStreamWaitEvent(s_kv, e_scan, 0));
+                SF_TRY(bwd_dq(s.path, &s.t, s.p, s.x, s.w, s.fw.UH, s_dq));
+                SF_CUDA(cudaEventRecord(e_dq, s_dq));
+                SF_TRY(bwd_dkdv(s.path, &s.t, s.p, s.x, s.w, s_kv));
+                SF_CUDA(cudaStreamWaitEvent(s_kv, e_dq, 0));
+                SF_TRY(bwd_dg(&s.t, s.p, s.x, s.w, s.fw.UH, s_kv));
+            }
+            i -= cnt;
+        }
+    } else {
+        for (int i = n_seg - 1; i >= 0; --i) {
+            sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[i], n_seg);
+            const Path path = classify(&t);
+            const SegParams p = make_params(&t);
+            char* wsi = seg_base + bwd_off[i];
+            const BwdWs w = bwd_ws(&t, p, wsi);
+            float* dS_here = dS_buf(i);
+            BwdPtrs x = seg_ptrs(i, t, dS_next, dS_here);
+            FwdWs fw;
+            if (fwd_workspace) {
+                fw = fwd_ws(&t, p, const_cast<char*>(static_cast<const char*>(fwd_workspace)) + fwd_off[i]);
+            } else {
+                char* fbase = wsi + w.bytes;
+                fw = fwd_ws(&t, p, fbase);
+                float* sfin = reinterpret_cast<float*>(fbase + fw.bytes);
+                FwdPtrs fx{x.q, x.k, x.v, x.g, x.S_in, nullptr, sfin};
+                SF_TRY(fwd_pre(path, &t, p, fx, fw, st));
+                SF_TRY(fwd_scan(&t, p, fx, fw, st));
+            }
+            SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, st));
+            SF_TRY(bwd_scan(&t, p, x, w, fw.beta, st));
             SF_TRY(bwd_dq(path, &t, p, x, w, fw.UH, st));
             SF_TRY(bwd_dkdv(path, &t, p, x, w, st));
             SF_TRY(bwd_dg(&t, p, x, w, fw.UH, st));
+            dS_next = dS_here;
         }
-        dS_next = dS_here;
     }
     if (ov) {
         // join the side streams back into the caller's stream
         for (int s = 1; s <= 2 * kSweepStreams; ++s) {
             cudaEvent_t e = res->pool[3 * (size_t)n_seg + s];
             SF_CUDA(cudaEventRecord(e, res->side[s]));
+            SF_CUDA(cudaStreamWaitEvent(st, e, 0));
+        }
+        for (int s = 0; s < kAggStreams; ++s) {
+            cudaEvent_t e = res->pool[3 * (size_t)n_seg + 1 + 2 * kSweepStreams + s];
+            SF_CUDA(cudaEventRecord(e, res->agg[s]));
             SF_CUDA(cudaStreamWaitEvent(st, e, 0));
         }
     }

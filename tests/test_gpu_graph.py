@@ -22,7 +22,9 @@ def test_graph_replay_matches_direct_calls(overlap):
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
         kernels = run.capture(x["S_in"], x["dS_out"], overlap=overlap)
-        assert kernels == 8 * len(w.seg_lens)        # forward: aggregate, scan, sweep; backward: aggregate, scan, dq, dk/dv, dg
+        # per segment: aggregate, sweep; aggregate, dq, dk/dv, dg = 6 kernels, plus the scans (one per group of short
+        # neighbouring segments when the streams overlap, one per segment otherwise)
+        assert 6 * len(w.seg_lens) + 2 <= kernels <= 8 * len(w.seg_lens)
         for t in (run.o, run.dq, run.dk, run.dv, run.dg, run.dS_init, run.S_bounds):
             t.zero_()
         before = binding.sf_launch_count()
