@@ -10,7 +10,7 @@
 // over tokens (ptx::desc_lo).
 #pragma once
 #include <cuda.h>
-#include <cstdio>
+#include <mutex>
 
 #include "../../include/stateflow.h"
 #include "sf_common.cuh"
@@ -20,13 +20,6 @@ namespace sf {
 namespace tc {
 
 __device__ int g_dev_status = 0;
-
-#ifdef SF_TRACE
-__device__ long long g_trace[8][64][4];
-#define SF_TR(role, c, e) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 31) == 0 && ((threadIdx.x >> 5) & 3) == 0) g_trace[role][c][e] = clock64(); } while (0)
-#else
-#define SF_TR(role, c, e) do { } while (0)
-#endif
 
 inline int read_device_status() {
     int v = 0;
@@ -81,6 +74,13 @@ inline bool make_tmap(CUtensorMap* m, const void* base, int B, int L, int H, lon
 }
 
 // ---- device helpers --------------------------------------------------------------------------------
+// First 1024-byte boundary of the dynamic shared memory.  The result is formed by adding an offset to the
+// __shared__ array itself, never by casting an integer back to a pointer: a pointer that went through an integer
+// loses its address space, and every access through it is compiled as a generic load or store.
+__device__ __forceinline__ unsigned char* align1024(unsigned char* smem) {
+    return smem + ((1024u - (ptx::smem_u32(smem) & 1023u)) & 1023u);
+}
+
 // Load one [64 x 128] tile (two boxes) of head h, batch b starting at token t0.
 __device__ __forceinline__ void tma_tile(void* dst, const CUtensorMap* m, uint64_t* bar, int h, int t0, int b) {
     ptx::tma_load_4d(dst, m, bar, 0, h, t0, b);
@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(AGG_THREADS, 1)
 tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, SegParams p,
                     const float* __restrict__ g, int mode, float* __restrict__ U, float* __restrict__ beta_out, int* status) {
     extern __shared__ unsigned char smem_raw[];
-    AggSmem& sm = *reinterpret_cast<AggSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    AggSmem& sm = *reinterpret_cast<AggSmem*>(align1024(smem_raw));
     const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
@@ -486,200 +486,13 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     if (warp == WT) ptx::tmem_dealloc(tmem, 128);
 }
 
-// ==================================================================================================
-// Chunk sweep with a forward-running state (Out + ST of paper Eq. 2; SR + OG of Section 3.4).
-// With tile roles (xq, xk, xv) and the state St[a][b] = sum xk[.][a] * xv[.][b]:
-//     out_r = sum_{s<=r} (xq_r . xk_s) D[r,s] xv_s  +  exp(b_r) * xq_r St_c ;   St_{c+1} = exp(b_C) St_c + xk^T diag(w) xv
-//   forward output pass : (xq, xk, xv) = (q, k, v),  St = H (from Hs[j]),         out = o
-//   dq pass             : (xq, xk, xv) = (dO, v, k), St = H^T (Hs[j] transposed), out = dq, and
-//                         xout[t] = q_t . dq_t (float32), q read from global memory in the epilogue
-// TMEM columns: St 0-127; O pair (intra at lanes +0, inter at lanes +16) double-buffered at 128 / 256;
-// scores double-buffered at 384 / 448.
-constexpr int SW_STAGES = 3;
-struct SweepSmem {
-    alignas(1024) unsigned char tiles[SW_STAGES][3][TILE];
-    alignas(1024) unsigned char xvw[TILE];
-    alignas(1024) unsigned char am[2][BOX];
-    alignas(1024) unsigned char sb[2 * 16384];
-    float bloc[MAXR * C];
-    float ctot[MAXR];
-    uint64_t full[SW_STAGES], sc_done[2], am_ready[2], st_ready, w_ready, st_done, out_done[2], o_free[2];
-    uint32_t tmem_base;
-    int abort_flag;
-};
+}  // namespace tc
+}  // namespace sf
 
-template <bool DQ>
-__global__ void __launch_bounds__(SW_THREADS, 1)
-tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                SegParams p, const float* __restrict__ g, const float* __restrict__ Hs, __nv_bfloat16* __restrict__ out, long long out_tok,
-                long long out_bat, const __nv_bfloat16* __restrict__ e_glob, float* __restrict__ xout, int* status) {
-    extern __shared__ unsigned char smem_raw[];
-    SweepSmem& sm = *reinterpret_cast<SweepSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
-    const long long t0 = (long long)c0 * C;
-    volatile int* abort_flag = &sm.abort_flag;
-    constexpr uint32_t T_ST = 0, T_O = 128, T_SC = 384;
+#include "sf_tc_sweep.cuh"
 
-    if (tid == 0) {
-        sm.abort_flag = 0;
-        for (int s = 0; s < SW_STAGES; ++s) ptx::mbar_init(&sm.full[s], 1);
-        for (int i = 0; i < 2; ++i) {
-            ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 4);
-            ptx::mbar_init(&sm.out_done[i], 1); ptx::mbar_init(&sm.o_free[i], 4);
-        }
-        ptx::mbar_init(&sm.st_ready, 12);
-        ptx::mbar_init(&sm.w_ready, 8);
-        ptx::mbar_init(&sm.st_done, 1);
-        ptx::fence_mbar_init();
-    }
-    if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::tc_fence_after_sync();
-    const uint32_t tmem = sm.tmem_base;
-    // the decay tables are built by the compute warps while the first tiles are already on their way
-
-    if (warp == W_TMA) {
-        if (lane == 0) {
-            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
-            for (int c = 0; c < nch; ++c) {
-                const int s = c % SW_STAGES;
-                // the stage was last used by chunk c-3, complete once all its MMAs retired
-                if (c >= SW_STAGES) SF_WAIT(&sm.out_done[(c - SW_STAGES) & 1], ((c - SW_STAGES) >> 1) & 1, DEV_TIMEOUT_MMA);
-                ptx::mbar_expect_tx(&sm.full[s], 3 * TILE);
-                const int tok = (int)t0 + c * C;
-                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
-            }
-        }
-    } else if (warp == W_MMA) {
-        if (lane == 0) {
-            constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
-            constexpr uint32_t id_o1 = ptx::idesc_bf16(64, 128, 0, 1);
-            constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
-            const uint32_t sb = ptx::smem_u32(sm.sb), xvw = ptx::smem_u32(sm.xvw);
-            auto scores = [&](int c) {
-                const int s = c % SW_STAGES;
-                SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
-                ptx::tc_fence_after_sync();
-                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
-                mma_group<8, DK8, DK8, 0>(tmem + T_SC + (c & 1) * 64, klo(xq), klo(xk), id_sc);
-                ptx::mma_commit(&sm.sc_done[c & 1]);
-            };
-            scores(0);
-            if (nch > 1) scores(1);
-            for (int c = 0; c < nch; ++c) {
-                const int s = c % SW_STAGES, bf = c & 1;
-                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]), xv = ptx::smem_u32(sm.tiles[s][2]);
-                const uint32_t am = ptx::smem_u32(sm.am[bf]);
-                const uint32_t to = tmem + T_O + bf * 128;
-                if (c >= 2) SF_WAIT(&sm.o_free[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
-                SF_TR(7, c, 0);
-                SF_WAIT(&sm.st_ready, c & 1, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-                SF_TR(1, c, 0);
-                // the state-dependent MMAs first: inter-chunk output (lanes +16), then the state update
-                mma_group<8, DK8, DMN, 0>(to + (16u << 16), klo(xq), mlo(sb, 16384), id_o1);
-                SF_TR(7, c, 1);
-                SF_WAIT(&sm.w_ready, c & 1, DEV_TIMEOUT_MMA);        // the weighted tile is written while the MMAs above run
-                ptx::tc_fence_after_sync();
-                SF_TR(7, c, 2);
-                mma_group<4, DMN, DMN, 1>(tmem + T_ST, mlo(xk, BOX), mlo(xvw, BOX), id_st);
-                ptx::mma_commit(&sm.st_done);
-                SF_TR(1, c, 1);
-                SF_WAIT(&sm.am_ready[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-                mma_group<4, DK8, DMN, 0>(to, klo(am), mlo(xv, BOX), id_o1);                // intra
-                ptx::mma_commit(&sm.out_done[bf]);
-                SF_TR(1, c, 2);
-                if (c + 2 < nch) scores(c + 2);          // into the score buffer the mask of chunk c has released
-                SF_TR(1, c, 3);
-            }
-        }
-    } else if (warp < 16) {
-        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, 16);
-        ptx::named_bar_sync(1, 512);
-        const int wg = warp >> 2, t = tid & 127;
-        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
-        const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
-        __nv_bfloat16* out_h = out + (long long)b * out_bat + (long long)h * D;
-        const __nv_bfloat16* e_h = DQ ? e_glob + (long long)b * out_bat + (long long)h * D : nullptr;
-        float* xo = DQ ? xout + ((long long)b * p.H + h) * p.L : nullptr;
-        auto mask = [&](int c) {
-            const int bf = c & 1;
-            SF_WAIT(&sm.sc_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
-            if (c >= 2) SF_WAIT(&sm.out_done[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);      // Am[bf] no longer read
-            ptx::tc_fence_after_sync();
-            SF_TR(3, c, 0);
-            mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], nullptr);
-            ptx::fence_proxy_async();
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive_warp(&sm.am_ready[bf]);
-            SF_TR(3, c, 1);
-        };
-        auto epilogue = [&](int c) {
-            const int bf = c & 1;
-            const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
-            const float eA = fast_exp(sm.bloc[c * C + rA]), eB = fast_exp(sm.bloc[c * C + rB]);
-            auto ready = [&]() {
-                SF_WAIT(&sm.out_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-                SF_TR(4, c, 0);
-            };
-            float dotA, dotB;
-            const bool vA = tokA < p.L, vB = tokB < p.L;          // rows past the end of a ragged segment: computed, not stored
-            const long long lastTok = p.L - 1;
-            pair_epilogue<DQ>(tmem + T_O + bf * 128, eA, eB, out_h + tokA * out_tok, out_h + tokB * out_tok,
-                              DQ ? e_h + min(tokA, lastTok) * out_tok : nullptr, DQ ? e_h + min(tokB, lastTok) * out_tok : nullptr,
-                              dotA, dotB, vA, vB, ready);
-            if (DQ && (lane & 3) == 0) {
-                if (vA) xo[tokA] = dotA;
-                if (vB) xo[tokB] = dotB;
-            }
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive_warp(&sm.o_free[bf]);
-            SF_TR(4, c, 1);
-        };
-        if (wg == 3) {
-            for (int c = 0; c < nch; ++c) epilogue(c);
-        } else {
-            if (wg == 2) mask(0);
-            for (int c = 0; c < nch; ++c) {
-                const int s = c % SW_STAGES;
-                const float* bch = sm.bloc + c * C;
-                const float bC = sm.ctot[c];
-                if (wg < 2) SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
-                SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 0);
-                if (c > 0) SF_WAIT(&sm.st_done, (c - 1) & 1, DEV_TIMEOUT_MMA);
-                ptx::tc_fence_after_sync();
-                SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 1);
-                // 16-column units: WG0 0-2, WG1 3-5, WG2 6-7
-                if (wg < 2) state_pass<3>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 3 * wg);
-                else        state_pass<2>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 6);
-                ptx::fence_proxy_async();
-                ptx::tc_fence_before_sync();
-                ptx::mbar_arrive_warp(&sm.st_ready);
-                SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 2);
-                if (wg < 2) {
-                    scale_box(sm.xvw + wg * BOX, sm.tiles[s][2] + wg * BOX, t, [&](int row) { return fast_exp(bC - bch[row]); });
-                    if (wg == 0) SF_TR(0, c, 1);
-                    ptx::fence_proxy_async();
-                    if (wg == 0) SF_TR(0, c, 2);
-                    ptx::mbar_arrive_warp(&sm.w_ready);
-                    if (wg == 0) SF_TR(0, c, 3);
-                }
-                SF_TR(wg == 0 ? 2 : (wg == 1 ? 5 : 6), c, 3);
-                if (wg == 2 && c + 1 < nch) mask(c + 1);
-            }
-        }
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    if (warp == W_MMA) ptx::tmem_dealloc(tmem, 512);
-}
+namespace sf {
+namespace tc {
 
 // ==================================================================================================
 // dk/dv pass (STB inside the block + PG, Section 3.4): reverse chunk sweep carrying G = dH (the
@@ -713,7 +526,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                const __nv_bfloat16* __restrict__ k_glob, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
                float* __restrict__ xk, int* status) {
     extern __shared__ unsigned char smem_raw[];
-    DkdvSmem& sm = *reinterpret_cast<DkdvSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    DkdvSmem& sm = *reinterpret_cast<DkdvSmem*>(align1024(smem_raw));
     const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
@@ -785,39 +598,29 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
                 const uint32_t xv = ptx::smem_u32(sm.tiles[s][2]), xd = ptx::smem_u32(sm.tiles[s][3]);
                 const uint32_t am = ptx::smem_u32(sm.am[s]), dam = ptx::smem_u32(sm.dam[s]);
-                SF_TR(1, i, 0);
                 SF_WAIT(&sm.st_ready, i & 1, DEV_TIMEOUT_MMA);
-                SF_TR(1, i, 1);
                 if (i >= 1) SF_WAIT(&sm.dv_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                SF_TR(1, i, 2);
                 // Everything that touches the carried gradient goes first, so that its rescaling for the next chunk
                 // runs while the intra-chunk MMAs and the next scores execute:
                 //   dv (lanes +16) = K G,  dk (lanes +16) = V G^T,  G += (diag(exp(b)) Q)^T dO
                 mma_group<8, DK8, DMN, 0>(tmem + T_DV + (16u << 16), klo(xk), mlo(gb, 16384), id_kn);
-                SF_TR(1, i, 3);
                 if (i >= 1) SF_WAIT(&sm.dk_free, (i - 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                SF_TR(7, i, 0);
                 mma_group<8, DK8, DK16, 0>(tmem + T_DK + (16u << 16), klo(xv), klo(gb), id_kk);
                 SF_WAIT(&sm.w_ready, i & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                SF_TR(7, i, 1);
                 mma_group<4, DMN, DMN, 1>(tmem + T_G, mlo(qw, BOX), mlo(xd, BOX), id_st);
                 ptx::mma_commit(&sm.st_done[s]);                 // G, its bf16 copy and qw are free again
-                SF_TR(7, i, 2);
                 // intra-chunk parts: dv (lanes +0) = A^T dO, dk (lanes +0) = dA^T Q
                 SF_WAIT(&sm.am_ready[s], (i >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                SF_TR(7, i, 3);
                 mma_group<4, DMN, DMN, 0>(tmem + T_DV, mlo(am, BOX), mlo(xd, BOX), id_tt);
                 ptx::mma_commit(&sm.dv_done);
                 mma_group<4, DMN, DMN, 0>(tmem + T_DK, mlo(dam, BOX), mlo(xq, BOX), id_tt);
                 ptx::mma_commit(&sm.dk_done);
                 ptx::mma_commit(&sm.it_done[s]);                 // tiles and masks of this iteration are free again
-                SF_TR(0, i, 0);
                 if (i + 1 < nch) scores(i + 1);      // two stages: the next chunk's tiles are already resident
-                SF_TR(0, i, 2);
             }
         }
     } else if (warp < 16) {
@@ -849,24 +652,17 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const bool vA = tokA < p.L, vB = tokB < p.L;
                 float dotA, dotB;
                 auto dk_ready = [&]() {
-                    SF_TR(4, i, 1);
                     SF_WAIT(&sm.dk_done, i & 1, DEV_TIMEOUT_MMA);
                     ptx::tc_fence_after_sync();
-                    SF_TR(4, i, 2);
                 };
                 if (wg == 2) {
-                    SF_TR(6, i, 0);
                     SF_WAIT(&sm.dv_done, i & 1, DEV_TIMEOUT_MMA);
                     ptx::tc_fence_after_sync();
-                    SF_TR(6, i, 1);
                     pair_epilogue<false>(tmem + T_DV, wA, wB, dv_h + tokA * p.tv, dv_h + tokB * p.tv, nullptr, nullptr, dotA, dotB, vA, vB);
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dv_free);
-                    SF_TR(6, i, 2);
                     if (i + 1 < nch) mask(i + 1);
-                    SF_TR(6, i, 3);
                 } else {
-                    SF_TR(4, i, 0);
                     pair_epilogue<true>(tmem + T_DK, wA, wB, dk_h + tokA * p.tqk, dk_h + tokB * p.tqk, k_h + min(tokA, (long long)p.L - 1) * p.tqk, k_h + min(tokB, (long long)p.L - 1) * p.tqk, dotA, dotB, vA, vB, dk_ready);
                     if ((lane & 3) == 0) {
                         if (vA) xo[tokA] = dotA;
@@ -874,7 +670,6 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     }
                     ptx::tc_fence_before_sync();
                     ptx::mbar_arrive_warp(&sm.dk_free);
-                    SF_TR(4, i, 3);
                 }
             }
         } else {
@@ -884,19 +679,15 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 SF_WAIT(&sm.full[s], (i >> 1) & 1, DEV_TIMEOUT_TMA);
                 // G, its bf16 copy and qw are rewritten below; the state update of the previous chunk is committed
                 // after every MMA that read them
-                SF_TR(wg == 0 ? 2 : 5, i, 0);
                 if (i > 0) SF_WAIT(&sm.st_done[(i - 1) & 1], ((i - 1) >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
-                SF_TR(wg == 0 ? 2 : 5, i, 1);
                 state_pass<4>(tmem + T_G, sm.gb, fast_exp(sm.ctot[c]), i == 0 ? G0 : nullptr, false, 4 * wg);
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive_warp(&sm.st_ready);
-                SF_TR(wg == 0 ? 2 : 5, i, 2);
                 scale_box(sm.qw + wg * BOX, sm.tiles[s][0] + wg * BOX, t, [&](int row) { return fast_exp(bch[row]); });
                 ptx::fence_proxy_async();
                 ptx::mbar_arrive_warp(&sm.w_ready);
-                SF_TR(wg == 0 ? 2 : 5, i, 3);
             }
         }
     }
@@ -906,28 +697,45 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 }
 
 // ---- host launch -------------------------------------------------------------------------------------
-template <typename K>
-inline bool opt_in_smem(K kern, size_t bytes) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) { cudaGetLastError(); return false; }
-    return true;
-}
-
-inline int* status_ptr() {
-    static int* ptr = nullptr;
-    if (!ptr) {
+// Per-device host state: the address of the status word and whether the kernels' shared-memory attribute has been
+// set there (both belong to a device, not to the process).
+constexpr int MAX_DEVICES = 64;
+enum { K_AGG = 0, K_FWD, K_DQ, K_DKDV, K_COUNT };
+struct DeviceState {
+    int* status = nullptr;
+    bool attr_done[K_COUNT] = {};
+};
+inline DeviceState* device_state() {
+    static DeviceState table[MAX_DEVICES];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) { cudaGetLastError(); return nullptr; }
+    std::lock_guard<std::mutex> lk(mu);
+    DeviceState* d = &table[dev];
+    if (!d->status) {
         void* sym = nullptr;
         if (cudaGetSymbolAddress(&sym, g_dev_status) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-        ptr = static_cast<int*>(sym);
+        d->status = static_cast<int*>(sym);
     }
-    return ptr;
+    return d;
+}
+template <typename K>
+inline bool opt_in_smem(DeviceState* d, int which, K kern, size_t bytes) {
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lk(mu);
+    if (d->attr_done[which]) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) { cudaGetLastError(); return false; }
+    d->attr_done[which] = true;
+    return true;
 }
 
 // role: 0 aggregate, 1 forward output pass, 2 dq pass, 3 dk/dv pass (same order as the host's Role enum)
 inline sf_status_t launch(int role, const sf_seg_desc_t* d, const SegParams& p, const void* q, const void* k, const void* v,
                           const void* dO, const float* g, int mode, float* U, float* beta, const float* states, void* o,
                           void* dq, void* dk, void* dv, float* xq, float* xk, cudaStream_t st, long long* n_launch) {
-    int* status = status_ptr();
-    if (!status) return SF_ERR_CUDA;
+    DeviceState* ds = device_state();
+    if (!ds) return SF_ERR_CUDA;
+    int* status = ds->status;
     if (p.R > MAXR) return SF_ERR_UNSUPPORTED;
     dim3 grid(p.H, p.NB, p.B);
     auto map_qk = [&](CUtensorMap* m, const void* base) { return make_tmap(m, base, p.B, p.L, p.H, p.tqk, p.bqk); };
@@ -936,45 +744,34 @@ inline sf_status_t launch(int role, const sf_seg_desc_t* d, const SegParams& p, 
         CUtensorMap tmX, tmY;
         if (!map_qk(&tmX, mode == 0 ? k : q) || !map_v(&tmY, mode == 0 ? v : dO)) return SF_ERR_CUDA;
         constexpr size_t smem = sizeof(AggSmem) + 1024;
-        static bool ok = opt_in_smem(tc_aggregate_kernel, smem);
-        if (!ok) return SF_ERR_CUDA;
+        if (!opt_in_smem(ds, K_AGG, tc_aggregate_kernel, smem)) return SF_ERR_CUDA;
         tc_aggregate_kernel<<<grid, AGG_THREADS, smem, st>>>(tmX, tmY, p, g, mode, U, beta, status);
     } else if (role == 1) {
-        CUtensorMap tq, tk, tv;
-        if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v)) return SF_ERR_CUDA;
-        constexpr size_t smem = sizeof(SweepSmem) + 1024;
-        static bool ok = opt_in_smem(tc_sweep_kernel<false>, smem);
-        if (!ok) return SF_ERR_CUDA;
-        tc_sweep_kernel<false><<<grid, SW_THREADS, smem, st>>>(tq, tk, tv, p, g, states, static_cast<__nv_bfloat16*>(o), p.tv, p.bv,
-                                                               nullptr, nullptr, status);
+        CUtensorMap tq, tk, tv, to;
+        if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&to, o)) return SF_ERR_CUDA;
+        constexpr size_t smem = sizeof(FsSmem) + 1024;
+        if (!opt_in_smem(ds, K_FWD, tc_fsweep_kernel<false>, smem)) return SF_ERR_CUDA;
+        tc_fsweep_kernel<false><<<grid, FS_THREADS, smem, st>>>(tq, tk, tv, to, p, g, states, nullptr, 0, 0, nullptr, status);
     } else if (role == 2) {
-        CUtensorMap tk, tv, td;
-        if (!map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;
-        constexpr size_t smem = sizeof(SweepSmem) + 1024;
-        static bool ok = opt_in_smem(tc_sweep_kernel<true>, smem);
-        if (!ok) return SF_ERR_CUDA;
+        CUtensorMap tk, tv, td, to;
+        if (!map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO) || !map_qk(&to, dq)) return SF_ERR_CUDA;
+        constexpr size_t smem = sizeof(FsSmem) + 1024;
+        if (!opt_in_smem(ds, K_DQ, tc_fsweep_kernel<true>, smem)) return SF_ERR_CUDA;
         // roles: xq = dO, xk = v, xv = k; q is read from global memory for the row dot products
-        tc_sweep_kernel<true><<<grid, SW_THREADS, smem, st>>>(td, tv, tk, p, g, states, static_cast<__nv_bfloat16*>(dq), p.tqk, p.bqk,
-                                                              static_cast<const __nv_bfloat16*>(q), xq, status);
+        tc_fsweep_kernel<true><<<grid, FS_THREADS, smem, st>>>(td, tv, tk, to, p, g, states, static_cast<const __nv_bfloat16*>(q),
+                                                               p.tqk, p.bqk, xq, status);
     } else if (role == 3) {
         CUtensorMap tq, tk, tv, td;
         if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;
         constexpr size_t smem = sizeof(DkdvSmem) + 1024;
-        static bool ok = opt_in_smem(tc_dkdv_kernel, smem);
-        if (!ok) return SF_ERR_CUDA;
+        if (!opt_in_smem(ds, K_DKDV, tc_dkdv_kernel, smem)) return SF_ERR_CUDA;
         tc_dkdv_kernel<<<grid, SW_THREADS, smem, st>>>(tq, tk, tv, td, p, g, states, static_cast<const __nv_bfloat16*>(k),
                                                        static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), xk, status);
     } else {
         return SF_ERR_UNSUPPORTED;
     }
     *n_launch += 1;
-    {
-        cudaError_t e = cudaGetLastError();
-#ifdef SF_TRACE
-        if (e != cudaSuccess) fprintf(stderr, "[sf] launch role %d failed: %s\n", role, cudaGetErrorString(e));
-#endif
-        return e == cudaSuccess ? SF_OK : SF_ERR_CUDA;
-    }
+    return cudaGetLastError() == cudaSuccess ? SF_OK : SF_ERR_CUDA;
 }
 
 }  // namespace tc

@@ -1112,10 +1112,6 @@ int32_t sf_device_status(void) { return sf::tc::read_device_status(); }
 void sf_device_status_clear(void) { sf::tc::clear_device_status(); }
 int64_t sf_launch_count(void) { return g_launches.load(); }
 
-#ifdef SF_TRACE
-void sf_debug_trace(long long* out) { cudaMemcpyFromSymbol(out, sf::tc::g_trace, sizeof(long long) * 8 * 64 * 4); }
-#endif
-
 void sf_stage_timing(int32_t enable) {
     std::lock_guard<std::mutex> lk(g_timing_mu);
     g_timing_on = enable != 0;
