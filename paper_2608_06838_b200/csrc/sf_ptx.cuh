@@ -46,9 +46,6 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volati
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-#ifdef SF_WAIT_SLEEP
-        __nanosleep(SF_WAIT_SLEEP);
-#endif
         if ((it & 255u) == 255u) {
             if (*abort_flag) return;
             if (clock64() - t0 > 2000000000LL) {
@@ -80,20 +77,6 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* tmap, ui
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
-
-// 4-D tiled store of a shared-memory box to global memory (bulk-group completion).  Rows of the box that fall
-// outside the tensor map's extents are not written.  c0 must be a multiple of 8 bf16; no coordinate is negative.
-__device__ __forceinline__ void tma_store_4d(const void* tmap, const void* smem_src, int c0, int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
-        ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// all committed stores have finished READING their shared-memory source (it may be overwritten)
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-// all committed stores are complete
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ---- TMEM ------------------------------------------------------------------------------------------
 // One full warp allocates `ncols` (power of two >= 32) columns; the base address lands in *dst_smem.
@@ -217,31 +200,6 @@ __device__ __forceinline__ void mma_lo(uint32_t d_tmem, uint32_t alo, uint32_t b
         "mov.b64 db, {%2, %4};\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, %5;\n\t}"
         ::"r"(d_tmem), "r"(alo), "r"(blo), "r"(idesc), "r"(DESC_HI), "n"(ACC) : "memory");
-}
-// The same with the accumulate flag taken at run time (acc != 0: D += A*B, else D = A*B).
-__device__ __forceinline__ void mma_lo_rt(uint32_t d_tmem, uint32_t alo, uint32_t blo, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
-        "mov.b64 da, {%1, %4};\n\t"
-        "mov.b64 db, {%2, %4};\n\t"
-        "setp.ne.u32 p, %5, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(alo), "r"(blo), "r"(idesc), "r"(DESC_HI), "r"(acc) : "memory");
-}
-// kind::tf32 with the A operand in TMEM: A[m][k] = 32-bit column (a_tmem + k) of lane m, read as tf32 (the upper 19
-// bits of a float32, so a float32 accumulator can be used as it stands); B from shared memory as 32-bit elements,
-// K-major (rows of 32 elements = 128 bytes, SWIZZLE_128B; a K step of 8 elements is +32 B).  float32 accumulation.
-__host__ __device__ constexpr uint32_t idesc_tf32(int M, int N, int b_mn_major) {
-    return (1u << 4) | (2u << 7) | (2u << 10) | (static_cast<uint32_t>(b_mn_major) << 16) |
-           (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
-}
-template <int ACC>
-__device__ __forceinline__ void mma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, uint32_t blo, uint32_t idesc) {
-    asm volatile(
-        "{\n\t.reg .b64 db;\n\t"
-        "mov.b64 db, {%2, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], db, %3, %5;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(blo), "r"(idesc), "r"(DESC_HI), "n"(ACC) : "memory");
 }
 // Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {

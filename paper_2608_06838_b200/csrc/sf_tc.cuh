@@ -486,13 +486,182 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     if (warp == WT) ptx::tmem_dealloc(tmem, 128);
 }
 
-}  // namespace tc
-}  // namespace sf
+// ==================================================================================================
+// Chunk sweep with a forward-running state (Out + ST of paper Eq. 2; SR + OG of Section 3.4).
+// With tile roles (xq, xk, xv) and the state St[a][b] = sum xk[.][a] * xv[.][b]:
+//     out_r = sum_{s<=r} (xq_r . xk_s) D[r,s] xv_s  +  exp(b_r) * xq_r St_c ;   St_{c+1} = exp(b_C) St_c + xk^T diag(w) xv
+//   forward output pass : (xq, xk, xv) = (q, k, v),  St = H (from Hs[j]),         out = o
+//   dq pass             : (xq, xk, xv) = (dO, v, k), St = H^T (Hs[j] transposed), out = dq, and
+//                         xout[t] = q_t . dq_t (float32), q read from global memory in the epilogue
+// TMEM columns: St 0-127; O pair (intra at lanes +0, inter at lanes +16) double-buffered at 128 / 256;
+// scores double-buffered at 384 / 448.
+constexpr int SW_STAGES = 3;
+struct SweepSmem {
+    alignas(1024) unsigned char tiles[SW_STAGES][3][TILE];
+    alignas(1024) unsigned char xvw[TILE];
+    alignas(1024) unsigned char am[2][BOX];
+    alignas(1024) unsigned char sb[2 * 16384];
+    float bloc[MAXR * C];
+    float ctot[MAXR];
+    uint64_t full[SW_STAGES], sc_done[2], am_ready[2], st_ready, w_ready, st_done, out_done[2], o_free[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
 
-#include "sf_tc_sweep.cuh"
+template <bool DQ>
+__global__ void __launch_bounds__(SW_THREADS, 1)
+tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                SegParams p, const float* __restrict__ g, const float* __restrict__ Hs, __nv_bfloat16* __restrict__ out, long long out_tok,
+                long long out_bat, const __nv_bfloat16* __restrict__ e_glob, float* __restrict__ xout, int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    SweepSmem& sm = *reinterpret_cast<SweepSmem*>(align1024(smem_raw));
+    const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
+    const long long t0 = (long long)c0 * C;
+    volatile int* abort_flag = &sm.abort_flag;
+    constexpr uint32_t T_ST = 0, T_O = 128, T_SC = 384;
 
-namespace sf {
-namespace tc {
+    if (tid == 0) {
+        sm.abort_flag = 0;
+        for (int s = 0; s < SW_STAGES; ++s) ptx::mbar_init(&sm.full[s], 1);
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&sm.sc_done[i], 1); ptx::mbar_init(&sm.am_ready[i], 4);
+            ptx::mbar_init(&sm.out_done[i], 1); ptx::mbar_init(&sm.o_free[i], 4);
+        }
+        ptx::mbar_init(&sm.st_ready, 12);
+        ptx::mbar_init(&sm.w_ready, 8);
+        ptx::mbar_init(&sm.st_done, 1);
+        ptx::fence_mbar_init();
+    }
+    if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;
+    // the decay tables are built by the compute warps while the first tiles are already on their way
+
+    if (warp == W_TMA) {
+        if (lane == 0) {
+            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
+            for (int c = 0; c < nch; ++c) {
+                const int s = c % SW_STAGES;
+                // the stage was last used by chunk c-3, complete once all its MMAs retired
+                if (c >= SW_STAGES) SF_WAIT(&sm.out_done[(c - SW_STAGES) & 1], ((c - SW_STAGES) >> 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::mbar_expect_tx(&sm.full[s], 3 * TILE);
+                const int tok = (int)t0 + c * C;
+                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
+            }
+        }
+    } else if (warp == W_MMA) {
+        if (lane == 0) {
+            constexpr uint32_t id_sc = ptx::idesc_bf16(64, 64, 0, 0);
+            constexpr uint32_t id_o1 = ptx::idesc_bf16(64, 128, 0, 1);
+            constexpr uint32_t id_st = ptx::idesc_bf16(128, 128, 1, 1);
+            const uint32_t sb = ptx::smem_u32(sm.sb), xvw = ptx::smem_u32(sm.xvw);
+            auto scores = [&](int c) {
+                const int s = c % SW_STAGES;
+                SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
+                ptx::tc_fence_after_sync();
+                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]);
+                mma_group<8, DK8, DK8, 0>(tmem + T_SC + (c & 1) * 64, klo(xq), klo(xk), id_sc);
+                ptx::mma_commit(&sm.sc_done[c & 1]);
+            };
+            scores(0);
+            if (nch > 1) scores(1);
+            for (int c = 0; c < nch; ++c) {
+                const int s = c % SW_STAGES, bf = c & 1;
+                const uint32_t xq = ptx::smem_u32(sm.tiles[s][0]), xk = ptx::smem_u32(sm.tiles[s][1]), xv = ptx::smem_u32(sm.tiles[s][2]);
+                const uint32_t am = ptx::smem_u32(sm.am[bf]);
+                const uint32_t to = tmem + T_O + bf * 128;
+                if (c >= 2) SF_WAIT(&sm.o_free[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
+                SF_WAIT(&sm.st_ready, c & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                // the state-dependent MMAs first: inter-chunk output (lanes +16), then the state update
+                mma_group<8, DK8, DMN, 0>(to + (16u << 16), klo(xq), mlo(sb, 16384), id_o1);
+                SF_WAIT(&sm.w_ready, c & 1, DEV_TIMEOUT_MMA);        // the weighted tile is written while the MMAs above run
+                ptx::tc_fence_after_sync();
+                mma_group<4, DMN, DMN, 1>(tmem + T_ST, mlo(xk, BOX), mlo(xvw, BOX), id_st);
+                ptx::mma_commit(&sm.st_done);
+                SF_WAIT(&sm.am_ready[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                mma_group<4, DK8, DMN, 0>(to, klo(am), mlo(xv, BOX), id_o1);                // intra
+                ptx::mma_commit(&sm.out_done[bf]);
+                if (c + 2 < nch) scores(c + 2);          // into the score buffer the mask of chunk c has released
+            }
+        }
+    } else if (warp < 16) {
+        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, 16);
+        ptx::named_bar_sync(1, 512);
+        const int wg = warp >> 2, t = tid & 127;
+        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
+        const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
+        __nv_bfloat16* out_h = out + (long long)b * out_bat + (long long)h * D;
+        const __nv_bfloat16* e_h = DQ ? e_glob + (long long)b * out_bat + (long long)h * D : nullptr;
+        float* xo = DQ ? xout + ((long long)b * p.H + h) * p.L : nullptr;
+        auto mask = [&](int c) {
+            const int bf = c & 1;
+            SF_WAIT(&sm.sc_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
+            if (c >= 2) SF_WAIT(&sm.out_done[bf], ((c - 2) >> 1) & 1, DEV_TIMEOUT_MMA);      // Am[bf] no longer read
+            ptx::tc_fence_after_sync();
+            mask_pass(tmem + T_SC + bf * 64, sm.bloc + c * C, sm.am[bf], nullptr);
+            ptx::fence_proxy_async();
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive_warp(&sm.am_ready[bf]);
+        };
+        auto epilogue = [&](int c) {
+            const int bf = c & 1;
+            const long long tokA = t0 + c * C + rA, tokB = tokA + 8;
+            const float eA = fast_exp(sm.bloc[c * C + rA]), eB = fast_exp(sm.bloc[c * C + rB]);
+            auto ready = [&]() {
+                SF_WAIT(&sm.out_done[bf], (c >> 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+            };
+            float dotA, dotB;
+            const bool vA = tokA < p.L, vB = tokB < p.L;          // rows past the end of a ragged segment: computed, not stored
+            const long long lastTok = p.L - 1;
+            pair_epilogue<DQ>(tmem + T_O + bf * 128, eA, eB, out_h + tokA * out_tok, out_h + tokB * out_tok,
+                              DQ ? e_h + min(tokA, lastTok) * out_tok : nullptr, DQ ? e_h + min(tokB, lastTok) * out_tok : nullptr,
+                              dotA, dotB, vA, vB, ready);
+            if (DQ && (lane & 3) == 0) {
+                if (vA) xo[tokA] = dotA;
+                if (vB) xo[tokB] = dotB;
+            }
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive_warp(&sm.o_free[bf]);
+        };
+        if (wg == 3) {
+            for (int c = 0; c < nch; ++c) epilogue(c);
+        } else {
+            if (wg == 2) mask(0);
+            for (int c = 0; c < nch; ++c) {
+                const int s = c % SW_STAGES;
+                const float* bch = sm.bloc + c * C;
+                const float bC = sm.ctot[c];
+                if (wg < 2) SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
+                if (c > 0) SF_WAIT(&sm.st_done, (c - 1) & 1, DEV_TIMEOUT_MMA);
+                ptx::tc_fence_after_sync();
+                // 16-column units: WG0 0-2, WG1 3-5, WG2 6-7
+                if (wg < 2) state_pass<3>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 3 * wg);
+                else        state_pass<2>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 6);
+                ptx::fence_proxy_async();
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive_warp(&sm.st_ready);
+                if (wg < 2) {
+                    scale_box(sm.xvw + wg * BOX, sm.tiles[s][2] + wg * BOX, t, [&](int row) { return fast_exp(bC - bch[row]); });
+                    ptx::fence_proxy_async();
+                    ptx::mbar_arrive_warp(&sm.w_ready);
+                }
+                if (wg == 2 && c + 1 < nch) mask(c + 1);
+            }
+        }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == W_MMA) ptx::tmem_dealloc(tmem, 512);
+}
 
 // ==================================================================================================
 // dk/dv pass (STB inside the block + PG, Section 3.4): reverse chunk sweep carrying G = dH (the
@@ -747,19 +916,20 @@ inline sf_status_t launch(int role, const sf_seg_desc_t* d, const SegParams& p, 
         if (!opt_in_smem(ds, K_AGG, tc_aggregate_kernel, smem)) return SF_ERR_CUDA;
         tc_aggregate_kernel<<<grid, AGG_THREADS, smem, st>>>(tmX, tmY, p, g, mode, U, beta, status);
     } else if (role == 1) {
-        CUtensorMap tq, tk, tv, to;
-        if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&to, o)) return SF_ERR_CUDA;
-        constexpr size_t smem = sizeof(FsSmem) + 1024;
-        if (!opt_in_smem(ds, K_FWD, tc_fsweep_kernel<false>, smem)) return SF_ERR_CUDA;
-        tc_fsweep_kernel<false><<<grid, FS_THREADS, smem, st>>>(tq, tk, tv, to, p, g, states, nullptr, 0, 0, nullptr, status);
+        CUtensorMap tq, tk, tv;
+        if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v)) return SF_ERR_CUDA;
+        constexpr size_t smem = sizeof(SweepSmem) + 1024;
+        if (!opt_in_smem(ds, K_FWD, tc_sweep_kernel<false>, smem)) return SF_ERR_CUDA;
+        tc_sweep_kernel<false><<<grid, SW_THREADS, smem, st>>>(tq, tk, tv, p, g, states, static_cast<__nv_bfloat16*>(o), p.tv, p.bv,
+                                                               nullptr, nullptr, status);
     } else if (role == 2) {
-        CUtensorMap tk, tv, td, to;
-        if (!map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO) || !map_qk(&to, dq)) return SF_ERR_CUDA;
-        constexpr size_t smem = sizeof(FsSmem) + 1024;
-        if (!opt_in_smem(ds, K_DQ, tc_fsweep_kernel<true>, smem)) return SF_ERR_CUDA;
+        CUtensorMap tk, tv, td;
+        if (!map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;
+        constexpr size_t smem = sizeof(SweepSmem) + 1024;
+        if (!opt_in_smem(ds, K_DQ, tc_sweep_kernel<true>, smem)) return SF_ERR_CUDA;
         // roles: xq = dO, xk = v, xv = k; q is read from global memory for the row dot products
-        tc_fsweep_kernel<true><<<grid, FS_THREADS, smem, st>>>(td, tv, tk, to, p, g, states, static_cast<const __nv_bfloat16*>(q),
-                                                               p.tqk, p.bqk, xq, status);
+        tc_sweep_kernel<true><<<grid, SW_THREADS, smem, st>>>(td, tv, tk, p, g, states, static_cast<__nv_bfloat16*>(dq), p.tqk, p.bqk,
+                                                              static_cast<const __nv_bfloat16*>(q), xq, status);
     } else if (role == 3) {
         CUtensorMap tq, tk, tv, td;
         if (!map_qk(&tq, q) || !map_qk(&tk, k) || !map_v(&tv, v) || !map_v(&td, dO)) return SF_ERR_CUDA;

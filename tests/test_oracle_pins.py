@@ -183,6 +183,72 @@ def test_adjoint_identity(decay):
     assert abs((lp - lm) / (2 * eps) - rhs) <= 1e-6 * max(1.0, abs(rhs))
 
 
+# The reverse sweep of the oracle replays states from checkpoints taken every clamp(floor(sqrt(T)), 16, 512) tokens and
+# walks the windows backwards; the last window is shorter when T is not a multiple of the interval.  The shapes above
+# have a single window (T <= 16) or only whole ones.  These have several windows and a short last one:
+# T = 37 -> 16, 16, 5 ; T = 300 -> seventeen windows of 17 and one of 11.  d_k != d_v throughout.
+@pytest.mark.parametrize("decay", DECAYS)
+@pytest.mark.parametrize("ds_out", [False, True])
+def test_gradients_match_central_differences_across_checkpoint_windows(decay, ds_out):
+    q, k, v, g, S_in, dO, dS_out = rand_case(1, 1, 2, 3, 37, decay=decay, ds_out=ds_out, rng=np.random.default_rng(37))
+    if decay == "spike":
+        g = np.maximum(g, -3.0)
+    grads = oracle.segment_bwd(q, k, v, g, S_in, dO, dS_out)
+    args = [q, k, v, g, S_in]
+    h = 1e-6
+    for idx, (x, gx) in enumerate(zip(args, grads)):
+        fd = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            i = it.multi_index
+            old = x[i]
+            x[i] = old + h
+            lp = loss(*args, dO, dS_out)
+            x[i] = old - h
+            lm = loss(*args, dO, dS_out)
+            x[i] = old
+            fd[i] = (lp - lm) / (2 * h)
+        scale = max(np.abs(fd).max(), 1e-3)
+        assert np.abs(fd - gx).max() / scale < 2e-7, "input %d" % idx
+
+
+@pytest.mark.parametrize("T", [37, 300])
+@pytest.mark.parametrize("decay", DECAYS)
+@pytest.mark.parametrize("ds_out", [False, True])
+def test_adjoint_and_directional_derivatives_across_checkpoint_windows(T, decay, ds_out):
+    q, k, v, g, S_in, dO, dS_out = rand_case(1, 2, 3, 5, T, decay=decay, ds_out=ds_out, rng=np.random.default_rng(T))
+    if decay == "spike":
+        g = np.maximum(g, -3.0)
+    dq, dk, dv, dg, dS_in = oracle.segment_bwd(q, k, v, g, S_in, dO, dS_out)
+    r = np.random.default_rng(T + 1)
+    # exact in the linear inputs (v, S_in)
+    d_v, d_S = r.standard_normal(v.shape), r.standard_normal(S_in.shape)
+    o1, S1 = oracle.segment_fwd(q, k, d_v, g, d_S)
+    lhs = np.sum(dO * o1) + (np.sum(dS_out * S1) if ds_out else 0.0)
+    rhs = np.sum(dv * d_v) + np.sum(dS_in * d_S)
+    assert abs(lhs - rhs) <= 1e-10 * max(1.0, abs(lhs))
+    # several random directions of every input, one input at a time (so that an error in one gradient cannot hide
+    # behind another), and directions confined to the last window and to the first one
+    eps = 1e-6
+    ckpt = min(max(int(np.floor(np.sqrt(T))), 16), 512)
+    last0 = (T - 1) // ckpt * ckpt
+    for name, x, gx in (("q", q, dq), ("k", k, dk), ("v", v, dv), ("g", g, dg)):
+        for where in ("all", "last", "first"):
+            d = r.standard_normal(x.shape)
+            if where == "last":
+                d[:, :last0] = 0.0
+            elif where == "first":
+                d[:, ckpt:] = 0.0
+            a = dict(q=q, k=k, v=v, g=g)
+            ap, am = dict(a), dict(a)
+            ap[name] = x + eps * d
+            am[name] = x - eps * d
+            lp = loss(ap["q"], ap["k"], ap["v"], ap["g"], S_in, dO, dS_out)
+            lm = loss(am["q"], am["k"], am["v"], am["g"], S_in, dO, dS_out)
+            want = np.sum(gx * d)
+            assert abs((lp - lm) / (2 * eps) - want) <= 2e-6 * max(1.0, abs(want)), (name, where)
+
+
 def test_zero_decay_backward_closed_form():
     q, k, v, g, _, dO, _ = rand_case(1, 1, 6, 4, 32, decay="zero", s_in=False, ds_out=False)
     dq, dk, dv, dg, dS_in = oracle.segment_bwd(q, k, v, g, None, dO, None)

@@ -5,11 +5,16 @@ are handed only input and output pointers, real-time loops) cannot provide a wor
 keeps a fixed scratch array of its own.  The test calls the entry point through the C ABI twice in a
 row, with different inputs, and checks each result against sf_segment_fwd run with a caller-owned
 workspace: the second call must not be disturbed by what the first one left in the shared scratch.
+The two entry points run the same kernels, so their results must agree bit for bit (which also
+satisfies the tolerance the parity tests use); one case is compared with the fp64 oracle as well, and
+the free device memory must not change across a call.
 This file sorts last so that a run stopping at the first failure has already run every other test.
 """
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2608_06838_b200 import binding, inputs
 from paper_2608_06838_b200.inputs import Workload
 
@@ -26,8 +31,11 @@ def _both(w, x):
     o_ref, S_ref = torch.empty_like(v), torch.empty(B, H, dk, dv, dtype=torch.float32, device=DEV)
     binding.sf_segment_fwd(desc, q, k, v, g, x["S_in"], o_ref, S_ref, ws)
     o, S = torch.empty_like(v), torch.empty_like(S_ref)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     binding.sf_segment_fwd_static(desc, q, k, v, g, x["S_in"], o, S)
     torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the amount of free device memory"
     assert binding.sf_device_status() == 0
     return (o, S), (o_ref, S_ref)
 
@@ -46,6 +54,12 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(dtype, d, chunk, tol
         (o, S), (o_ref, S_ref) = _both(w, x)
         assert torch.isfinite(o.float()).all() and torch.isfinite(S).all()
         assert _close(o, o_ref, tol) and _close(S, S_ref, tol), w.name
+        assert torch.equal(o, o_ref) and torch.equal(S, S_ref), w.name      # same kernels, same bits
+        f = inputs.to_f64
+        o_or, S_or = oracle.segment_fwd(f(x["q"]), f(x["k"]), f(x["v"]), f(x["g"]), f(x["S_in"]))
+        for got, ref in ((o, o_or), (S, S_or)):
+            err = np.abs(f(got) - ref).max() / max(np.abs(ref).max(), 1e-30)
+            assert err <= tol, (w.name, err)
 
 
 def test_shapes_beyond_the_static_scratch_are_rejected():
