@@ -67,7 +67,7 @@ typedef enum { SF_BF16 = 0, SF_F32 = 1 } sf_dtype_t;
  * its workloads never leave a partial chunk; when seg_len is not a multiple of chunk the last chunk simply has
  * fewer tokens (its missing rows count as zero keys, values and gradients with log-decay 0, and are never
  * written).  chunks_per_block sets how many chunks form one block, the only granularity
- * whose states are written to the workspace (at most 32 on the tensor-core path); 0 lets the library
+ * whose states are written to the workspace (at most 64); 0 lets the library
  * pick the length in [4, 32] that fills the device's SMs best for this shape.  Heads are independent.
  */
 typedef struct {

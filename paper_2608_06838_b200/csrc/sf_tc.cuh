@@ -35,7 +35,7 @@ constexpr int C = 64;              // chunk
 constexpr int D = 128;             // d_k = d_v
 constexpr int BOX = 8192;          // bytes of one [64 x 64] bf16 box
 constexpr int TILE = 2 * BOX;      // bytes of one [64 x 128] bf16 tile
-constexpr int MAXR = 32;           // largest chunks_per_block of the tensor-core path
+constexpr int MAXR = 64;           // largest chunks_per_block of the tensor-core path
 constexpr float LOG2E = 1.4426950408889634f;
 
 __device__ __forceinline__ float fast_exp(float x) { return ptx::ex2(x * LOG2E); }
@@ -92,24 +92,43 @@ __device__ __forceinline__ void tma_tile(void* dst, const CUtensorMap* m, uint64
 //   bloc[t]  = inclusive cumulative log-decay of token t inside ITS chunk  (t = 0 .. nch*64-1)
 //   ctot[c]  = chunk totals
 // Tokens at or beyond `L` (a last chunk that is not full) get log-decay 0; TMA fills their tile rows with zeros.
+// `issued`, if given, is an mbarrier (count = nwarps) on which every warp arrives once its loads are on their way: the
+// TMA warp waits for it, so that these small requests do not queue behind the first burst of tile loads that all CTAs
+// of the device send at the same moment.
 __device__ __forceinline__ void prep_decay(const float* __restrict__ gh, long long tg, long long t0, int nch, int L, float* bloc,
-                                           float* ctot, int nwarps) {
+                                           float* ctot, int nwarps, uint64_t* issued = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int lim = L - (int)t0;                            // tokens from the block start to the end of the segment
-    for (int c = warp; c < nch; c += nwarps) {
-        // unconditional loads from clamped (always valid) tokens, zeroed afterwards: keeps both loads in flight together
-        const int r = c * C + 2 * lane;
-        const float g0 = gh[(t0 + min(r, lim - 1)) * tg] * (r < lim ? 1.f : 0.f);
-        const float g1 = gh[(t0 + min(r + 1, lim - 1)) * tg] * (r + 1 < lim ? 1.f : 0.f);
-        float incl = g0 + g1;
-        for (int off = 1; off < 32; off <<= 1) {
-            const float up = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += up;
+    // All loads of this warp's chunks go out before the first scan (one memory round trip for the whole block, not one
+    // per chunk).  Unconditional loads from clamped (always valid) tokens, zeroed afterwards.
+    constexpr int MAXC = 4;                                 // chunks per warp in one round (MAXR / 8 warps)
+    for (int cbase = warp; cbase < nch; cbase += nwarps * MAXC) {
+        float g0[MAXC], g1[MAXC];
+#pragma unroll
+        for (int i = 0; i < MAXC; ++i) {
+            const int c = cbase + i * nwarps;
+            const int r = c * C + 2 * lane;
+            const bool on = c < nch;
+            g0[i] = on ? gh[(t0 + min(r, lim - 1)) * tg] * (r < lim ? 1.f : 0.f) : 0.f;
+            g1[i] = on ? gh[(t0 + min(r + 1, lim - 1)) * tg] * (r + 1 < lim ? 1.f : 0.f) : 0.f;
         }
-        bloc[c * C + 2 * lane] = incl - g1;
-        bloc[c * C + 2 * lane + 1] = incl;
-        if (lane == 31) ctot[c] = incl;
+        if (issued && cbase == warp) { ptx::mbar_arrive_warp(issued); issued = nullptr; }
+#pragma unroll
+        for (int i = 0; i < MAXC; ++i) {
+            const int c = cbase + i * nwarps;
+            if (c < nch) {
+                float incl = g0[i] + g1[i];
+                for (int off = 1; off < 32; off <<= 1) {
+                    const float up = __shfl_up_sync(0xffffffffu, incl, off);
+                    if (lane >= off) incl += up;
+                }
+                bloc[c * C + 2 * lane] = incl - g1[i];
+                bloc[c * C + 2 * lane + 1] = incl;
+                if (lane == 31) ctot[c] = incl;
+            }
+        }
     }
+    if (issued) ptx::mbar_arrive_warp(issued);             // a warp without a chunk of its own has nothing to wait for
 }
 
 __device__ __forceinline__ void st_unit(unsigned char* box, int row, int unit, uint4 v) {
@@ -390,7 +409,7 @@ struct AggSmem {
     float bloc[MAXR * C];
     float ctot[MAXR];
     float cofs[MAXR];
-    uint64_t full[AGG_STAGES], empty[AGG_STAGES], ready[AGG_STAGES], done;
+    uint64_t full[AGG_STAGES], empty[AGG_STAGES], ready[AGG_STAGES], done, g_issued;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -411,6 +430,7 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         sm.abort_flag = 0;
         for (int s = 0; s < AGG_STAGES; ++s) { ptx::mbar_init(&sm.full[s], 1); ptx::mbar_init(&sm.empty[s], 1); ptx::mbar_init(&sm.ready[s], AGG_COMP / 32); }
         ptx::mbar_init(&sm.done, 1);
+        ptx::mbar_init(&sm.g_issued, AGG_COMP / 32);
         ptx::fence_mbar_init();
     }
     if (warp == WT) ptx::tmem_alloc(&sm.tmem_base, 128);
@@ -423,6 +443,7 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         if (lane == 0) {
             ptx::prefetch_tmap(&tmX);
             ptx::prefetch_tmap(&tmY);
+            SF_WAIT(&sm.g_issued, 0, DEV_TIMEOUT_TMA);
             for (int c = 0; c < nch; ++c) {
                 const int s = c % AGG_STAGES, it = c / AGG_STAGES;
                 if (it > 0) SF_WAIT(&sm.empty[s], (it - 1) & 1, DEV_TIMEOUT_MMA);
@@ -447,7 +468,7 @@ tc_aggregate_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
     } else {
         const float* gh = g + (long long)b * p.bg + h;
-        prep_decay(gh, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, WT);
+        prep_decay(gh, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, WT, &sm.g_issued);
         ptx::named_bar_sync(1, AGG_COMP);
         if (tid == 0) {
             float acc = 0.f;
@@ -503,19 +524,19 @@ struct SweepSmem {
     alignas(1024) unsigned char sb[2 * 16384];
     float bloc[MAXR * C];
     float ctot[MAXR];
-    uint64_t full[SW_STAGES], sc_done[2], am_ready[2], st_ready, w_ready, st_done, out_done[2], o_free[2];
+    uint64_t full[SW_STAGES], sc_done[2], am_ready[2], st_ready, w_ready, st_done, out_done[2], o_free[2], g_issued;
     uint32_t tmem_base;
     int abort_flag;
 };
 
 template <bool DQ>
-__global__ void __launch_bounds__(SW_THREADS, 1)
-tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                SegParams p, const float* __restrict__ g, const float* __restrict__ Hs, __nv_bfloat16* __restrict__ out, long long out_tok,
-                long long out_bat, const __nv_bfloat16* __restrict__ e_glob, float* __restrict__ xout, int* status) {
+__device__ __forceinline__ void sweep_body(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV, const SegParams& p,
+                                           const float* __restrict__ g, const float* __restrict__ Hs, __nv_bfloat16* __restrict__ out,
+                                           long long out_tok, long long out_bat, const __nv_bfloat16* __restrict__ e_glob,
+                                           float* __restrict__ xout, int* status, int h) {
     extern __shared__ unsigned char smem_raw[];
     SweepSmem& sm = *reinterpret_cast<SweepSmem*>(align1024(smem_raw));
-    const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
+    const int j = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
     const long long t0 = (long long)c0 * C;
@@ -532,6 +553,7 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ptx::mbar_init(&sm.st_ready, 12);
         ptx::mbar_init(&sm.w_ready, 8);
         ptx::mbar_init(&sm.st_done, 1);
+        ptx::mbar_init(&sm.g_issued, 16);
         ptx::fence_mbar_init();
     }
     if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
@@ -543,16 +565,17 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
     if (warp == W_TMA) {
         if (lane == 0) {
-            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
+            ptx::prefetch_tmap(tmQ); ptx::prefetch_tmap(tmK); ptx::prefetch_tmap(tmV);
+            SF_WAIT(&sm.g_issued, 0, DEV_TIMEOUT_TMA);
             for (int c = 0; c < nch; ++c) {
                 const int s = c % SW_STAGES;
                 // the stage was last used by chunk c-3, complete once all its MMAs retired
                 if (c >= SW_STAGES) SF_WAIT(&sm.out_done[(c - SW_STAGES) & 1], ((c - SW_STAGES) >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::mbar_expect_tx(&sm.full[s], 3 * TILE);
                 const int tok = (int)t0 + c * C;
-                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][0], tmQ, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][1], tmK, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][2], tmV, &sm.full[s], h, tok, b);
             }
         }
     } else if (warp == W_MMA) {
@@ -593,10 +616,11 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
         }
     } else if (warp < 16) {
-        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, 16);
+        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
+        ptx::prefetch_l2(H0 + tid * 32);                 // the block's initial state (512 lines) is on its way while the tables are built
+        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, 16, &sm.g_issued);
         ptx::named_bar_sync(1, 512);
         const int wg = warp >> 2, t = tid & 127;
-        const float* H0 = Hs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
         const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
         __nv_bfloat16* out_h = out + (long long)b * out_bat + (long long)h * D;
         const __nv_bfloat16* e_h = DQ ? e_glob + (long long)b * out_bat + (long long)h * D : nullptr;
@@ -663,6 +687,15 @@ tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == W_MMA) ptx::tmem_dealloc(tmem, 512);
 }
 
+template <bool DQ>
+__global__ void __launch_bounds__(SW_THREADS, 1)
+tc_sweep_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                SegParams p, const float* __restrict__ g, const float* __restrict__ Hs, __nv_bfloat16* __restrict__ out, long long out_tok,
+                long long out_bat, const __nv_bfloat16* __restrict__ e_glob, float* __restrict__ xout, int* status) {
+    // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
+    sweep_body<DQ>(&tmQ, &tmK, &tmV, p, g, Hs, out, out_tok, out_bat, e_glob, xout, status, blockIdx.x);
+}
+
 // ==================================================================================================
 // dk/dv pass (STB inside the block + PG, Section 3.4): reverse chunk sweep carrying G = dH (the
 // gradient w.r.t. the state leaving the chunk, from Gs[j]):
@@ -680,7 +713,7 @@ struct DkdvSmem {
     alignas(1024) unsigned char gb[2 * 16384];
     float bloc[MAXR * C];
     float ctot[MAXR];
-    uint64_t full[2], sc_done[2], am_ready[2], st_ready, w_ready, st_done[2], it_done[2], dv_done, dk_done, dv_free, dk_free;
+    uint64_t full[2], sc_done[2], am_ready[2], st_ready, w_ready, st_done[2], it_done[2], dv_done, dk_done, dv_free, dk_free, g_issued;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -689,14 +722,13 @@ struct DkdvSmem {
 // release barrier.  Per iteration the MMAs that read or update the carried gradient G are issued first and
 // st_done is committed right behind them: the rescaling of G for the next chunk (the serial part of the sweep)
 // then overlaps the intra-chunk MMAs, the epilogues and the next chunk's scores.  it_done closes the iteration.
-__global__ void __launch_bounds__(SW_THREADS, 1)
-tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-               const __grid_constant__ CUtensorMap tmD, SegParams p, const float* __restrict__ g, const float* __restrict__ Gs,
-               const __nv_bfloat16* __restrict__ k_glob, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
-               float* __restrict__ xk, int* status) {
+__device__ __forceinline__ void dkdv_body(const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV, const CUtensorMap* tmD,
+                                          const SegParams& p, const float* __restrict__ g, const float* __restrict__ Gs,
+                                          const __nv_bfloat16* __restrict__ k_glob, __nv_bfloat16* __restrict__ dk,
+                                          __nv_bfloat16* __restrict__ dv, float* __restrict__ xk, int* status, int h) {
     extern __shared__ unsigned char smem_raw[];
     DkdvSmem& sm = *reinterpret_cast<DkdvSmem*>(align1024(smem_raw));
-    const int h = blockIdx.x, j = blockIdx.y, b = blockIdx.z;   // heads fastest: co-resident CTAs read neighbouring 256-byte pieces of the same tokens
+    const int j = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = j * p.R, nch = min(p.R, p.NC - c0);
     const long long t0 = (long long)c0 * C;
@@ -717,6 +749,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         ptx::mbar_init(&sm.dk_done, 1);
         ptx::mbar_init(&sm.dv_free, 4);
         ptx::mbar_init(&sm.dk_free, 4);
+        ptx::mbar_init(&sm.g_issued, 16);
         ptx::fence_mbar_init();
     }
     if (warp == W_MMA) ptx::tmem_alloc(&sm.tmem_base, 512);
@@ -729,17 +762,18 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     // iteration i handles chunk c = nch-1-i
     if (warp == W_TMA) {
         if (lane == 0) {
-            ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV); ptx::prefetch_tmap(&tmD);
+            ptx::prefetch_tmap(tmQ); ptx::prefetch_tmap(tmK); ptx::prefetch_tmap(tmV); ptx::prefetch_tmap(tmD);
+            SF_WAIT(&sm.g_issued, 0, DEV_TIMEOUT_TMA);
             for (int i = 0; i < nch; ++i) {
                 const int s = i & 1;
                 // the stage was last used by iteration i-2; it_done is committed after all of its MMAs
                 if (i >= 2) SF_WAIT(&sm.it_done[s], ((i - 2) >> 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::mbar_expect_tx(&sm.full[s], 4 * TILE);
                 const int tok = (int)t0 + (nch - 1 - i) * C;
-                tma_tile(sm.tiles[s][0], &tmQ, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][1], &tmK, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][2], &tmV, &sm.full[s], h, tok, b);
-                tma_tile(sm.tiles[s][3], &tmD, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][0], tmQ, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][1], tmK, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][2], tmV, &sm.full[s], h, tok, b);
+                tma_tile(sm.tiles[s][3], tmD, &sm.full[s], h, tok, b);
             }
         }
     } else if (warp == W_MMA) {
@@ -793,10 +827,11 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
         }
     } else if (warp < 16) {
-        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, 16);
+        const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
+        ptx::prefetch_l2(G0 + tid * 32);                 // the block's incoming state gradient, on its way while the tables are built
+        prep_decay(g + (long long)b * p.bg + h, p.tg, t0, nch, p.L, sm.bloc, sm.ctot, 16, &sm.g_issued);
         ptx::named_bar_sync(1, 512);
         const int wg = warp >> 2, t = tid & 127;
-        const float* G0 = Gs + (((long long)b * p.H + h) * p.NB + j) * (long long)(D * D);
         const int rA = 16 * (warp & 3) + (lane >> 2), rB = rA + 8;
         __nv_bfloat16* dk_h = dk + (long long)b * p.bqk + (long long)h * D;
         __nv_bfloat16* dv_h = dv + (long long)b * p.bv + (long long)h * D;
@@ -863,6 +898,14 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == W_MMA) ptx::tmem_dealloc(tmem, 512);
+}
+
+__global__ void __launch_bounds__(SW_THREADS, 1)
+tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+               const __grid_constant__ CUtensorMap tmD, SegParams p, const float* __restrict__ g, const float* __restrict__ Gs,
+               const __nv_bfloat16* __restrict__ k_glob, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+               float* __restrict__ xk, int* status) {
+    dkdv_body(&tmQ, &tmK, &tmV, &tmD, p, g, Gs, k_glob, dk, dv, xk, status, blockIdx.x);
 }
 
 // ---- host launch -------------------------------------------------------------------------------------

@@ -62,14 +62,17 @@ Path classify(const sf_seg_desc_t* d) {
     if (d->tok_stride_qk < (long long)d->H * d->d_k || d->tok_stride_v < (long long)d->H * d->d_v || d->tok_stride_g < d->H)
         return Path::Invalid;
     if (d->B > 1 && (d->batch_stride_qk <= 0 || d->batch_stride_v <= 0 || d->batch_stride_g <= 0)) return Path::Invalid;
-    if ((long long)d->B * d->H > 65535LL * 65535LL) return Path::Invalid;
     if (d->H > 65535 || d->B > 65535) return Path::Invalid;
     const bool c_ok = d->chunk == 16 || d->chunk == 32 || d->chunk == 64;
     auto d_ok = [](int x) { return x == 32 || x == 64 || x == 128; };
     if (!c_ok || !d_ok(d->d_k) || !d_ok(d->d_v)) return Path::Unsupported;
+    if ((long long)d->B * d->H > 65535LL) return Path::Invalid;              // grid.y of the scan kernels
     if (d->dtype == SF_BF16) {
         if (d->tok_stride_qk % 8 || d->tok_stride_v % 8 || d->batch_stride_qk % 8 || d->batch_stride_v % 8) return Path::Invalid;
-        if (d->d_k == 128 && d->d_v == 128) return d->chunk == 64 ? Path::Tc : Path::Unsupported;
+        if (d->d_k == 128 && d->d_v == 128) {
+            if (d->chunk != 64 || d->chunks_per_block > sf::tc::MAXR || 2LL * d->H > 65535LL) return Path::Unsupported;
+            return Path::Tc;
+        }
         if (d->d_k == 128 || d->d_v == 128) return Path::Unsupported;
         return d->d_k == d->d_v || (d->d_k == 32 && d->d_v == 64) ? Path::Simt : Path::Unsupported;
     }
@@ -88,17 +91,17 @@ int sm_count() {
 }
 
 // Block length when the caller leaves it open: one CTA per (batch, head, block) and one CTA per SM, so a
-// kernel takes waves * (chunks per block + a fixed per-CTA cost of about three chunk times).  Pick the
-// length in [4, 32] that minimises this; ties go to the longer block (fewer block states in HBM).
+// kernel takes waves * (chunks per block + a fixed per-CTA cost of about six chunk times).  Pick the
+// length in [4, 64] that minimises this; ties go to the longer block (fewer block states in HBM).
 int auto_chunks_per_block(int NC, long long bh) {
     const int sms = sm_count();
     int best = kDefaultChunksPerBlock;
     long long best_cost = -1;
-    for (int r = 4; r <= 32; ++r) {
+    for (int r = 4; r <= 64; ++r) {
         const int reff = r < NC ? r : NC;
         const long long nb = (NC + reff - 1) / reff;
         const long long waves = (nb * bh + sms - 1) / sms;
-        const long long cost = waves * (reff + 3);
+        const long long cost = waves * (reff + 6);
         if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = reff; }
         if (r >= NC) break;
     }
@@ -116,7 +119,7 @@ int chain_chunks_per_block(int NC, long long bh) {
     long long nb = (40 + bh - 1) / bh;                       // blocks for 40 CTAs or more
     const long long by_len = NC / 8 > 0 ? NC / 8 : 1;        // blocks of at least 8 chunks
     if (nb > by_len) nb = by_len;
-    const long long least = (NC + 31) / 32;                  // blocks of at most 32 chunks
+    const long long least = (NC + 63) / 64;                  // blocks of at most 64 chunks
     if (nb < least) nb = least;
     return (int)((NC + nb - 1) / nb);
 }

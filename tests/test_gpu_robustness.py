@@ -71,10 +71,11 @@ def test_repeated_runs_with_overlap_are_bit_identical():
             assert torch.equal(first[n], again[n]), n
 
 
-@pytest.mark.parametrize("cpb", [1, 2, 3, 5, 7, 8, 13, 16, 31, 32])
+@pytest.mark.parametrize("cpb", [1, 2, 3, 5, 7, 8, 13, 16, 31, 32, 33, 47, 64])
 def test_every_block_length_matches_the_oracle(cpb):
-    # 37 chunks: most block lengths leave a ragged last block
-    w = Workload("blocks-%d" % cpb, 1, 2, 128, 128, [37 * 64], 64, g_scale=0.05, s_in_sigma=0.02, ds_out_sigma=0.02, seed=23)
+    # 37 chunks (or 131 for the block lengths beyond 32): most block lengths leave a ragged last block
+    nc = 37 if cpb <= 32 else 131
+    w = Workload("blocks-%d" % cpb, 1, 2, 128, 128, [nc * 64], 64, g_scale=0.05, s_in_sigma=0.02, ds_out_sigma=0.02, seed=23)
     x = inputs.make_inputs(w, DEV)
     got, _ = run_chain(w, x, chunks_per_block=cpb)
     compare(got, oracle_reference(x), tolerance(w), label=w.name)
