@@ -229,7 +229,9 @@ def main():
     run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk, args.chunks_per_block)
     overlap = not args.no_overlap
 
-    # a graph cannot be recorded on the legacy default stream: that mode runs on a stream of its own
+    # a graph cannot be recorded on the legacy default stream: that mode runs on a stream of its own (which does not
+    # wait for the default stream, where the inputs were generated, by itself)
+    torch.cuda.synchronize()
     work_stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
 
     # profile-guided block length (untimed preparation, like the graph capture below); candidates are timed the

@@ -33,6 +33,13 @@
  *    prints or traps the device.
  *  - Pointers must be 16-byte aligned; for SF_BF16 the token and batch strides
  *    must be multiples of 8 elements (16 bytes).
+ *  - Devices and threads: the library's own host state (kernel attributes, the
+ *    status word's address, the chain driver's side streams and events) is kept
+ *    per device and created on first use with that device current, so one process
+ *    may drive several devices.  On ONE device, calls that use the chain driver's
+ *    side streams (sf_chain_* with overlap != 0, graphs recorded from them, the
+ *    tuner) must not run concurrently from several host threads: they share those
+ *    streams and events.  Everything else may be called from any thread.
  */
 #ifndef STATEFLOW_H
 #define STATEFLOW_H
@@ -241,6 +248,31 @@ int64_t sf_chain_graph_kernels(const sf_chain_graph_t* graph);
 void sf_chain_graph_destroy(sf_chain_graph_t* graph);
 
 /*
+ * Schedule of the chaining driver (the paper picks "tile sizes, split points and overlap schedules" per operator
+ * shape by profiling a small set of valid choices, Section 3.4 last paragraph and Section 4.4 / Table 3).  Process-wide;
+ * read at every sf_chain_* call (and so frozen into a graph when it is recorded).  Results do not depend on it.
+ *   sweep_streams     1..4  side streams the sweeps of consecutive segments rotate over (per kind of sweep)
+ *   agg_streams       1..4  side streams the block-aggregate kernels of small segments rotate over
+ *   scan_group_tokens >= 0  neighbouring segments of at most this many tokens in total share one scan launch
+ *   agg_inorder_ctas  >= 1  an aggregate launch of at least this many CTAs stays in order on the first aggregate stream
+ *   agg_ahead         >= 0  how many segments the aggregate kernels may run ahead of the sweeps (0 = no limit);
+ *                           a small value keeps what the aggregates read close to the sweeps that read it again
+ * The block length is part of the descriptor (chunks_per_block); forward and backward share it because the backward
+ * starts its blocks from the block states the forward saved.
+ * sf_set_tuning(NULL) restores the defaults {4, 4, 4096, 74, 0}; out-of-range values give SF_ERR_INVALID_ARG and change
+ * nothing.  Host functions.
+ */
+typedef struct {
+    int32_t sweep_streams;
+    int32_t agg_streams;
+    int32_t scan_group_tokens;
+    int32_t agg_inorder_ctas;
+    int32_t agg_ahead;
+} sf_tuning_t;
+sf_status_t sf_set_tuning(const sf_tuning_t* tuning);
+void sf_get_tuning(sf_tuning_t* tuning);
+
+/*
  * Profile-guided choice of the block length (the paper tunes its kernels' tile sizes and overlap schedules
  * "for each operator shape" by profiling, Section 3.4 end and Section 4.4; here the one tunable of that kind is
  * chunks_per_block).  Runs the chain (sf_chain_fwd, and sf_chain_bwd with the forward workspace if dO is not
@@ -304,9 +336,23 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
  * wait has run out since sf_device_status_clear().  Kernels never spin without a limit; when a
  * limit is hit they record a code here, stop waiting and return normally, leaving their outputs
  * undefined.  No counterpart in the paper.
+ *
+ * Codes: 0 none; 1 a wait for tile data (TMA) ran out; 2 a wait for a tensor-core result or for another warp's
+ * hand-off ran out; 3 the wait of sf_selftest_bounded_wait ran out (as it must); -1 the word could not be read.
+ * sf_device_check() maps the word to a status: SF_OK, SF_ERR_TIMEOUT (any code > 0) or SF_ERR_CUDA.
  */
 int32_t sf_device_status(void);
 void sf_device_status_clear(void);
+sf_status_t sf_device_check(void);
+
+/*
+ * Exercises the bounded wait without touching any product kernel: a one-warp kernel waits on a barrier that nothing
+ * ever completes, gives up after `limit_cycles` clock cycles (1 .. 1e8: at most a few hundredths of a second),
+ * records code 3 in the status word and returns normally; the call waits for it and returns what sf_device_check()
+ * then says, i.e. SF_ERR_TIMEOUT when the mechanism works.  The context stays usable; call sf_device_status_clear()
+ * afterwards.  No counterpart in the paper.
+ */
+sf_status_t sf_selftest_bounded_wait(int64_t limit_cycles, sf_stream_t stream);
 
 /* Number of kernels this library has launched in this process (host counter). No paper counterpart. */
 int64_t sf_launch_count(void);

@@ -258,6 +258,48 @@ def sf_device_status_clear() -> None:
     load().sf_device_status_clear()
 
 
+class Tuning(ctypes.Structure):
+    """sf_tuning_t: schedule of the chaining driver."""
+    _fields_ = [("sweep_streams", ctypes.c_int32), ("agg_streams", ctypes.c_int32), ("scan_group_tokens", ctypes.c_int32),
+                ("agg_inorder_ctas", ctypes.c_int32), ("agg_ahead", ctypes.c_int32)]
+
+
+def sf_set_tuning(tuning=None) -> None:
+    """tuning: None (defaults), a Tuning, or a dict with some of its fields (the others keep their current value)."""
+    lib = load()
+    lib.sf_set_tuning.argtypes = [ctypes.c_void_p]
+    if tuning is None:
+        _check(lib.sf_set_tuning(None), "sf_set_tuning")
+        return
+    if isinstance(tuning, dict):
+        t = sf_get_tuning()
+        for k, v in tuning.items():
+            setattr(t, k, int(v))
+        tuning = t
+    _check(lib.sf_set_tuning(ctypes.byref(tuning)), "sf_set_tuning")
+
+
+def sf_get_tuning() -> Tuning:
+    lib = load()
+    lib.sf_get_tuning.argtypes = [ctypes.c_void_p]
+    lib.sf_get_tuning.restype = None
+    t = Tuning()
+    lib.sf_get_tuning(ctypes.byref(t))
+    return t
+
+
+def sf_device_check() -> int:
+    """Status code for the device status word: 0 ok, 5 a bounded wait ran out, 4 the word could not be read."""
+    return int(load().sf_device_check())
+
+
+def sf_selftest_bounded_wait(limit_cycles: int = 2_000_000, stream=None) -> int:
+    """Runs the wait self-test kernel and returns its status code (5 = SF_ERR_TIMEOUT when the mechanism works)."""
+    lib = load()
+    lib.sf_selftest_bounded_wait.argtypes = [ctypes.c_int64, ctypes.c_void_p]
+    return int(lib.sf_selftest_bounded_wait(int(limit_cycles), _stream(stream)))
+
+
 def sf_launch_count() -> int:
     return int(load().sf_launch_count())
 

@@ -37,10 +37,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: gives up after about a second, records `code` in *status (global) and sets the
-// CTA-wide sticky flag *abort_flag (shared) so that every later wait in this CTA returns at once.
+// Bounded wait: gives up after `limit` clock cycles (about a second by default), records `code` in *status (global)
+// and sets the CTA-wide sticky flag *abort_flag (shared) so that every later wait in this CTA returns at once.
 // The kernel then runs to its end on undefined data and releases its TMEM normally.
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                          long long limit = WAIT_LIMIT_CYCLES) {
     if (mbar_try_wait(bar, parity)) return;
     if (*abort_flag) return;
     const long long t0 = clock64();
@@ -48,7 +50,7 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return;
         if ((it & 255u) == 255u) {
             if (*abort_flag) return;
-            if (clock64() - t0 > 2000000000LL) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 atomicExch(status, code);
                 return;

@@ -908,6 +908,20 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     dkdv_body(&tmQ, &tmK, &tmV, &tmD, p, g, Gs, k_glob, dk, dv, xk, status, blockIdx.x);
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier on which nothing ever arrives, with a short limit given by
+// the caller; the wait gives up, records DEV_TIMEOUT_SELFTEST in the status word and the kernel returns normally.
+__global__ void wait_selftest_kernel(long long limit_cycles, int* status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        ptx::mbar_init(&bar, 1);
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    ptx::mbar_wait(&bar, 0, &abort_flag, status, DEV_TIMEOUT_SELFTEST, limit_cycles);
+}
+
 // ---- host launch -------------------------------------------------------------------------------------
 // Per-device host state: the address of the status word and whether the kernels' shared-memory attribute has been
 // set there (both belong to a device, not to the process).
@@ -939,6 +953,13 @@ inline bool opt_in_smem(DeviceState* d, int which, K kern, size_t bytes) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) { cudaGetLastError(); return false; }
     d->attr_done[which] = true;
     return true;
+}
+
+inline sf_status_t launch_wait_selftest(long long limit_cycles, cudaStream_t st) {
+    DeviceState* ds = device_state();
+    if (!ds) return SF_ERR_CUDA;
+    wait_selftest_kernel<<<1, 32, 0, st>>>(limit_cycles, ds->status);
+    return cudaGetLastError() == cudaSuccess ? SF_OK : SF_ERR_CUDA;
 }
 
 // role: 0 aggregate, 1 forward output pass, 2 dq pass, 3 dk/dv pass (same order as the host's Role enum)

@@ -81,13 +81,14 @@ Path classify(const sf_seg_desc_t* d) {
 }
 
 int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else { cudaGetLastError(); n = 148; }
+    static int table[sf::tc::MAX_DEVICES] = {};          // per device: a process may drive several
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= sf::tc::MAX_DEVICES) { cudaGetLastError(); return 148; }
+    if (table[dev] == 0) {
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) table[dev] = v;
+        else { cudaGetLastError(); table[dev] = 148; }
     }
-    return n;
+    return table[dev];
 }
 
 // Block length when the caller leaves it open: one CTA per (batch, head, block) and one CTA per SM, so a
@@ -299,10 +300,19 @@ sf_status_t launch_scan_group(const sf_seg_desc_t* d, int BH, const sf::ScanGrou
     return check_launch();
 }
 
+// Schedule of the chaining driver (sf_tuning_t; process-wide, read at every chain call).
+constexpr int kMaxSweepStreams = 4, kMaxAggStreams = 4;
+const sf_tuning_t kDefaultTuning = {4, 4, 4096, 74, 0};
+std::mutex g_tuning_mu;
+sf_tuning_t g_tuning = kDefaultTuning;
+sf_tuning_t current_tuning() {
+    std::lock_guard<std::mutex> lk(g_tuning_mu);
+    return g_tuning;
+}
+
 // Segments i, i+dir, ... that the chaining driver scans together: up to SCAN_GROUP_MAX short segments of at most
-// kScanGroupTokens tokens in total (one long segment is a group of its own).
-constexpr long long kScanGroupTokens = 4096;
-int scan_group_size(const int32_t* seg_lens, int n_seg, int i, int dir) {
+// scan_group_tokens tokens in total (one long segment is a group of its own).
+int scan_group_size(const int32_t* seg_lens, int n_seg, int i, int dir, long long kScanGroupTokens) {
     int count = 1;
     long long tokens = seg_lens[i];
     for (int k = i + dir; k >= 0 && k < n_seg && count < sf::SCAN_GROUP_MAX; k += dir) {
@@ -392,12 +402,14 @@ sf_status_t validate_bwd(const sf_seg_desc_t* d, const BwdPtrs& x, const void* s
 
 // Side streams and events of the chaining driver (host objects only; created once per process).
 // Sweeps of consecutive segments go to different streams: a short segment's sweep does not fill the device.
-constexpr int kSweepStreams = 4;
+constexpr int kSweepStreams = kMaxSweepStreams;       // streams that exist; a tuning may use fewer
 // The aggregates of different segments are independent of everything: they go round-robin to their own streams
 // (with short segments one stream of small aggregate kernels is the longest chain of the step).
-constexpr int kAggStreams = 4;
+constexpr int kAggStreams = kMaxAggStreams;
 // ... unless a segment's aggregate kernel fills half the device by itself: those stay in order on one stream
-inline int agg_stream_index(const SegParams& p, int i) { return (long long)p.B * p.H * p.NB >= 74 ? 0 : i % kAggStreams; }
+inline int agg_stream_index(const SegParams& p, int i, const sf_tuning_t& tu) {
+    return (long long)p.B * p.H * p.NB >= tu.agg_inorder_ctas ? 0 : i % tu.agg_streams;
+}
 struct ChainRes {
     cudaStream_t side[1 + 2 * kSweepStreams] = {};   // 0: unused; then two groups of sweep streams, used round-robin by segment
     cudaStream_t agg[kAggStreams] = {};
@@ -407,23 +419,24 @@ struct ChainRes {
     int device = -1;
 };
 std::mutex g_chain_mu;
-ChainRes g_chain;
+ChainRes g_chain[sf::tc::MAX_DEVICES];      // one set of side streams and events per device, created on first use there
 
 sf_status_t chain_resources(ChainRes** out) {
     std::lock_guard<std::mutex> lk(g_chain_mu);
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return SF_ERR_CUDA;
-    if (!g_chain.ok || g_chain.device != dev) {
-        for (auto& s : g_chain.side)
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= sf::tc::MAX_DEVICES) { cudaGetLastError(); return SF_ERR_CUDA; }
+    ChainRes& r = g_chain[dev];
+    if (!r.ok) {
+        for (auto& s : r.side)
             if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SF_ERR_CUDA;
-        for (auto& s : g_chain.agg)
+        for (auto& s : r.agg)
             if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SF_ERR_CUDA;
-        for (auto& e : g_chain.ev)
+        for (auto& e : r.ev)
             if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return SF_ERR_CUDA;
-        g_chain.ok = true;
-        g_chain.device = dev;
+        r.ok = true;
+        r.device = dev;
     }
-    *out = &g_chain;
+    *out = &r;
     return SF_OK;
 }
 
@@ -620,6 +633,7 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     if (S_init) SF_CUDA(cudaMemcpyAsync(S_bounds, S_init, sN * sizeof(float), cudaMemcpyDeviceToDevice, st));
     else        SF_CUDA(cudaMemsetAsync(S_bounds, 0, sN * sizeof(float), st));
 
+    const sf_tuning_t tu = current_tuning();
     ChainRes* res = nullptr;
     if (overlap) SF_TRY(chain_resources(&res));
     // overlap schedule (the forward wavefront of Section 3.4, Eq. 17, across segments):
@@ -628,7 +642,7 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     //   side streams 1..: [wait ST(i)] Out(i)             (round-robin, so that the sweeps of short neighbouring
     //                                                      segments, which do not fill the device, run side by side)
     if (overlap) {
-        SF_TRY(chain_events(res, 2 * (size_t)n_seg + 2 + kSweepStreams + kAggStreams));
+        SF_TRY(chain_events(res, 3 * (size_t)n_seg + 2 + kSweepStreams + kAggStreams));
         SF_CUDA(cudaEventRecord(res->ev[0], st));
         for (int s = 0; s <= kSweepStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->side[s], res->ev[0], 0));
         for (int s = 0; s < kAggStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->agg[s], res->ev[0], 0));
@@ -663,13 +677,17 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
         for (int i = 0; i < n_seg;) {
             // short neighbouring segments are scanned in one launch (the state is carried in registers from one to
             // the next); their aggregates go first, their sweeps after
-            const int cnt = scan_group_size(seg_lens, n_seg, i, +1);
+            const int cnt = scan_group_size(seg_lens, n_seg, i, +1, tu.scan_group_tokens);
             sf::ScanGroup grp{};
             grp.count = cnt;
             for (int k = 0; k < cnt; ++k) {
                 const Seg& sg = segs[i + k];
-                cudaStream_t s_agg = res->agg[agg_stream_index(sg.p, i + k)];
+                cudaStream_t s_agg = res->agg[agg_stream_index(sg.p, i + k, tu)];
                 cudaEvent_t e = res->pool[(size_t)n_seg + (i + k)];
+                // agg_ahead: the aggregate of segment j starts only when the sweep of segment j - agg_ahead is done
+                // (a segment of an earlier group: its sweep has been enqueued already)
+                const int jw = i + k - tu.agg_ahead;
+                if (tu.agg_ahead > 0 && jw >= 0 && jw < i) SF_CUDA(cudaStreamWaitEvent(s_agg, res->pool[2 * (size_t)n_seg + jw], 0));
                 SF_TRY(fwd_pre(sg.path, &sg.t, sg.p, sg.x, sg.w, s_agg));
                 SF_CUDA(cudaEventRecord(e, s_agg));
                 SF_CUDA(cudaStreamWaitEvent(st, e, 0));
@@ -679,9 +697,10 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
             SF_CUDA(cudaEventRecord(res->pool[i], st));
             for (int k = 0; k < cnt; ++k) {
                 const Seg& sg = segs[i + k];
-                cudaStream_t s_out = res->side[1 + ((i + k) % kSweepStreams)];
+                cudaStream_t s_out = res->side[1 + ((i + k) % tu.sweep_streams)];
                 SF_CUDA(cudaStreamWaitEvent(s_out, res->pool[i], 0));
                 SF_TRY(fwd_out(sg.path, &sg.t, sg.p, sg.x, sg.w, s_out));
+                SF_CUDA(cudaEventRecord(res->pool[2 * (size_t)n_seg + (i + k)], s_out));
             }
             i += cnt;
         }
@@ -689,12 +708,12 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     if (overlap) {
         // join the sweep streams back into the caller's stream
         for (int s = 1; s <= kSweepStreams; ++s) {
-            cudaEvent_t e = res->pool[2 * (size_t)n_seg + s];
+            cudaEvent_t e = res->pool[3 * (size_t)n_seg + s];
             SF_CUDA(cudaEventRecord(e, res->side[s]));
             SF_CUDA(cudaStreamWaitEvent(st, e, 0));
         }
         for (int s = 0; s < kAggStreams; ++s) {
-            cudaEvent_t e = res->pool[2 * (size_t)n_seg + 1 + kSweepStreams + s];
+            cudaEvent_t e = res->pool[3 * (size_t)n_seg + 1 + kSweepStreams + s];
             SF_CUDA(cudaEventRecord(e, res->agg[s]));
             SF_CUDA(cudaStreamWaitEvent(st, e, 0));
         }
@@ -730,11 +749,12 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     // its own scan: dq sweeps queue on one group of side streams, dk/dv sweeps and the dg epilogue on another
     // (round-robin by segment, so that neighbouring short segments share the device).
     const bool ov = overlap != 0 && fwd_workspace != nullptr;
+    const sf_tuning_t tu = current_tuning();
     ChainRes* res = nullptr;
     if (ov) {
         SF_TRY(chain_resources(&res));
-        SF_TRY(chain_events(res, 3 * (size_t)n_seg + 2 + 2 * kSweepStreams + kAggStreams));
-        cudaEvent_t e0 = res->pool[3 * (size_t)n_seg];
+        SF_TRY(chain_events(res, 4 * (size_t)n_seg + 2 + 2 * kSweepStreams + kAggStreams));
+        cudaEvent_t e0 = res->pool[4 * (size_t)n_seg];
         SF_CUDA(cudaEventRecord(e0, st));
         for (int s = 0; s <= 2 * kSweepStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->side[s], e0, 0));
         for (int s = 0; s < kAggStreams; ++s) SF_CUDA(cudaStreamWaitEvent(res->agg[s], e0, 0));
@@ -766,25 +786,30 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     };
     auto dS_buf = [&](int i) { return i == 0 ? dS_init : reinterpret_cast<float*>(base + (size_t)i * sB); };
 
-    if (ov) {
-        // all backward aggregates first, in the order the scans will need them
-        for (int i = n_seg - 1; i >= 0; --i) {
-            sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[i], n_seg);
-            const Path path = classify(&t);
-            const SegParams p = make_params(&t);
-            const BwdWs w = bwd_ws(&t, p, seg_base + bwd_off[i]);
-            BwdPtrs x = seg_ptrs(i, t, nullptr, nullptr);
-            cudaStream_t s_agg = res->agg[agg_stream_index(p, i)];
-            SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, s_agg));
-            SF_CUDA(cudaEventRecord(res->pool[3 * (size_t)i], s_agg));
-        }
+    // backward aggregate of segment idx on its aggregate stream; with agg_ahead it first waits for the dk/dv sweep of
+    // segment idx + agg_ahead (visited earlier; only called once that sweep has been enqueued)
+    auto enqueue_agg = [&](int idx, bool throttled) -> sf_status_t {
+        sf_seg_desc_t t = chain_segment_desc(desc, seg_lens[idx], n_seg);
+        const Path path = classify(&t);
+        const SegParams p = make_params(&t);
+        const BwdWs w = bwd_ws(&t, p, seg_base + bwd_off[idx]);
+        BwdPtrs x = seg_ptrs(idx, t, nullptr, nullptr);
+        cudaStream_t s_agg = res->agg[agg_stream_index(p, idx, tu)];
+        if (throttled) SF_CUDA(cudaStreamWaitEvent(s_agg, res->pool[4 * (size_t)(idx + tu.agg_ahead) + 3], 0));
+        SF_TRY(bwd_pre(path, &t, p, x, w, nullptr, s_agg));
+        SF_CUDA(cudaEventRecord(res->pool[4 * (size_t)idx], s_agg));
+        return SF_OK;
+    };
+    if (ov && tu.agg_ahead == 0) {
+        // no limit: all backward aggregates first, in the order the scans will need them
+        for (int i = n_seg - 1; i >= 0; --i) SF_TRY(enqueue_agg(i, false));
     }
     const float* dS_next = dS_final;
     if (ov) {
         // (ov implies the forward workspace is given)  Groups of short neighbouring segments, visited in descending
         // order, share one reverse scan; each segment's sweeps start when its group's scan is done.
         for (int i = n_seg - 1; i >= 0;) {
-            const int cnt = scan_group_size(seg_lens, n_seg, i, -1);
+            const int cnt = scan_group_size(seg_lens, n_seg, i, -1, tu.scan_group_tokens);
             struct Seg { sf_seg_desc_t t; Path path; SegParams p; BwdWs w; BwdPtrs x; FwdWs fw; };
             Seg sg[sf::SCAN_GROUP_MAX];
             sf::ScanGroup grp{};
@@ -803,16 +828,18 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
                 grp.seg[k] = sf::ScanSeg{s.fw.beta, s.w.GU, dS_here, s.p.NB};
                 dS_next = dS_here;
             }
-            for (int k = 0; k < cnt; ++k) SF_CUDA(cudaStreamWaitEvent(st, res->pool[3 * (size_t)(i - k)], 0));
+            if (tu.agg_ahead > 0)
+                for (int k = 0; k < cnt; ++k) SF_TRY(enqueue_agg(i - k, i - k + tu.agg_ahead <= n_seg - 1 && i - k + tu.agg_ahead > i));
+            for (int k = 0; k < cnt; ++k) SF_CUDA(cudaStreamWaitEvent(st, res->pool[4 * (size_t)(i - k)], 0));
             SF_TRY(launch_scan_group(desc, desc->B * desc->H, grp, 1, group_init, st));
-            cudaEvent_t e_scan = res->pool[3 * (size_t)i + 1];
+            cudaEvent_t e_scan = res->pool[4 * (size_t)i + 1];
             SF_CUDA(cudaEventRecord(e_scan, st));
             for (int k = 0; k < cnt; ++k) {
                 const int idx = i - k;
                 const Seg& s = sg[k];
-                cudaEvent_t e_dq = res->pool[3 * (size_t)idx + 2];
+                cudaEvent_t e_dq = res->pool[4 * (size_t)idx + 2];
                 // the sweeps of neighbouring segments go round-robin to different streams
-                cudaStream_t s_dq = res->side[1 + (idx % kSweepStreams)], s_kv = res->side[1 + kSweepStreams + (idx % kSweepStreams)];
+                cudaStream_t s_dq = res->side[1 + (idx % tu.sweep_streams)], s_kv = res->side[1 + kSweepStreams + (idx % tu.sweep_streams)];
                 SF_CUDA(cudaStreamWaitEvent(s_dq, e_scan, 0));
                 SF_CUDA(cudaStreamWaitEvent(s_kv, e_scan, 0));
                 SF_TRY(bwd_dq(s.path, &s.t, s.p, s.x, s.w, s.fw.UH, s_dq));
@@ -820,6 +847,7 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
                 SF_TRY(bwd_dkdv(s.path, &s.t, s.p, s.x, s.w, s_kv));
                 SF_CUDA(cudaStreamWaitEvent(s_kv, e_dq, 0));
                 SF_TRY(bwd_dg(&s.t, s.p, s.x, s.w, s.fw.UH, s_kv));
+                SF_CUDA(cudaEventRecord(res->pool[4 * (size_t)idx + 3], s_kv));
             }
             i -= cnt;
         }
@@ -854,12 +882,12 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     if (ov) {
         // join the side streams back into the caller's stream
         for (int s = 1; s <= 2 * kSweepStreams; ++s) {
-            cudaEvent_t e = res->pool[3 * (size_t)n_seg + s];
+            cudaEvent_t e = res->pool[4 * (size_t)n_seg + s];
             SF_CUDA(cudaEventRecord(e, res->side[s]));
             SF_CUDA(cudaStreamWaitEvent(st, e, 0));
         }
         for (int s = 0; s < kAggStreams; ++s) {
-            cudaEvent_t e = res->pool[3 * (size_t)n_seg + 1 + 2 * kSweepStreams + s];
+            cudaEvent_t e = res->pool[4 * (size_t)n_seg + 1 + 2 * kSweepStreams + s];
             SF_CUDA(cudaEventRecord(e, res->agg[s]));
             SF_CUDA(cudaStreamWaitEvent(st, e, 0));
         }
@@ -1111,7 +1139,35 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
     return SF_OK;
 }
 
+sf_status_t sf_set_tuning(const sf_tuning_t* t) {
+    std::lock_guard<std::mutex> lk(g_tuning_mu);
+    if (!t) { g_tuning = kDefaultTuning; return SF_OK; }
+    if (t->sweep_streams < 1 || t->sweep_streams > kMaxSweepStreams || t->agg_streams < 1 || t->agg_streams > kMaxAggStreams ||
+        t->scan_group_tokens < 0 || t->agg_inorder_ctas < 1 || t->agg_ahead < 0)
+        return SF_ERR_INVALID_ARG;
+    g_tuning = *t;
+    return SF_OK;
+}
+
+void sf_get_tuning(sf_tuning_t* t) {
+    if (t) *t = current_tuning();
+}
+
 int32_t sf_device_status(void) { return sf::tc::read_device_status(); }
+
+sf_status_t sf_device_check(void) {
+    const int v = sf::tc::read_device_status();
+    return v < 0 ? SF_ERR_CUDA : (v == 0 ? SF_OK : SF_ERR_TIMEOUT);
+}
+
+sf_status_t sf_selftest_bounded_wait(int64_t limit_cycles, sf_stream_t stream) {
+    if (limit_cycles < 1 || limit_cycles > 100000000LL) return SF_ERR_INVALID_ARG;     // at most a few hundredths of a second
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    SF_TRY(sf::tc::launch_wait_selftest(limit_cycles, st));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return SF_ERR_CUDA; }
+    return sf_device_check();
+}
 void sf_device_status_clear(void) { sf::tc::clear_device_status(); }
 int64_t sf_launch_count(void) { return g_launches.load(); }
 

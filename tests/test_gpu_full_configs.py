@@ -1,5 +1,7 @@
-"""The benchmark configurations at full size, in the launch configuration bench.py times (overlap on,
-saved block states, default block length), checked on sampled heads against the unsplit fp64 oracle."""
+"""The benchmark configurations at full size, in the launch configurations bench.py times, checked on sampled
+heads against the unsplit fp64 oracle: direct launches with the library's block-length model, and - what the
+benchmark's timed region runs - the chain recorded as a CUDA graph after profile-guided tuning of the block length,
+replayed."""
 import numpy as np
 import pytest
 import torch
@@ -12,8 +14,40 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def sampled_check(w, heads):
+def graph_run(w, x):
+    """The benchmark's way: tune the block length on the caller's buffers, record the chain as a graph, replay it."""
+    run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk)
+    # the inputs were generated on the default stream; the side stream below does not wait for it by itself
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        run.autotune(x["S_in"], x["dS_out"], [0, 22, 32, 64], reps=2)
+        run.capture(x["S_in"], x["dS_out"])
+        for t in (run.o, run.dq, run.dk, run.dv, run.dg, run.dS_init, run.S_bounds):
+            t.zero_()
+        run.replay()
+    stream.synchronize()
+    assert binding.sf_device_status() == 0
+    got = dict(o=run.o, S_out=run.S_bounds[-1], dq=run.dq, dk=run.dk, dv=run.dv, dg=run.dg, dS_in=run.dS_init)
+    return got, run
+
+
+def sampled_check(w, heads, mode="direct"):
     x = inputs.make_inputs(w, DEV)
+    if mode == "graph":
+        got, run = graph_run(w, x)
+        ref = oracle_reference(x, heads=heads)
+        errs = compare(got, ref, tolerance(w), heads=heads, label=w.name + "/graph")
+        print(w.name, "graph, block length", int(run.desc.chunks_per_block), "heads", heads, {k: "%.2e" % v for k, v in errs.items()})
+        first = {n: got[n].clone() for n in ("o", "dg", "dS_in")}
+        with torch.cuda.stream(torch.cuda.Stream()):
+            run.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(first["o"], run.o) and torch.equal(first["dg"], run.dg) and torch.equal(first["dS_in"], run.dS_init)
+        run.release()
+        del run, got, x
+        torch.cuda.empty_cache()
+        return
     got, run = run_chain(w, x)
     ref = oracle_reference(x, heads=heads)
     errs = compare(got, ref, tolerance(w), heads=heads, label=w.name)
@@ -30,16 +64,19 @@ def sampled_check(w, heads):
     torch.cuda.empty_cache()
 
 
-def test_config2_32k():
-    sampled_check(inputs.configs()[1], [0, 15])
+@pytest.mark.parametrize("mode", ["direct", "graph"])
+def test_config2_32k(mode):
+    sampled_check(inputs.configs()[1], [0, 15], mode)
 
 
-def test_config3_64k_nonuniform():
-    sampled_check(inputs.configs()[2], [3, 31])
+@pytest.mark.parametrize("mode", ["direct", "graph"])
+def test_config3_64k_nonuniform(mode):
+    sampled_check(inputs.configs()[2], [3, 31], mode)
 
 
-def test_config4_256k():
-    sampled_check(inputs.configs()[3], [17])
+@pytest.mark.parametrize("mode", ["direct", "graph"])
+def test_config4_256k(mode):
+    sampled_check(inputs.configs()[3], [17], mode)
 
 
 @pytest.mark.parametrize("seg_len", [512, 16384])

@@ -62,3 +62,34 @@ def test_autotune_picks_a_candidate_and_results_stay_correct():
     torch.cuda.synchronize()
     got = dict(o=run.o, S_out=run.S_bounds[-1], dq=run.dq, dk=run.dk, dv=run.dv, dg=run.dg, dS_in=run.dS_init)
     compare(got, oracle_reference(x), tolerance(w), label="autotuned")
+
+
+@pytest.mark.parametrize("tuning", [dict(sweep_streams=1, agg_streams=1), dict(sweep_streams=2, agg_ahead=1),
+                                    dict(agg_ahead=2, scan_group_tokens=0), dict(agg_inorder_ctas=1, agg_ahead=3),
+                                    dict(scan_group_tokens=100000, sweep_streams=3)])
+def test_every_schedule_gives_the_bits_of_the_default_one(tuning):
+    # the schedule (streams, scan grouping, how far the aggregates run ahead) only orders independent work
+    w = Workload("tuning", 1, 3, 128, 128, [1024, 512, 512, 256, 768], 64, s_in_sigma=0.02, ds_out_sigma=0.02, seed=17)
+    x = inputs.make_inputs(w, DEV)
+    binding.sf_set_tuning(None)
+    ref, _ = run_chain(w, x)
+    ref = {n: ref[n].clone() for n in NAMES}
+    try:
+        binding.sf_set_tuning(tuning)
+        got, _ = run_chain(w, x)
+        for n in NAMES:
+            assert torch.equal(got[n], ref[n]), n
+        # and recorded as a graph
+        run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk)
+        torch.cuda.synchronize()
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            run.capture(x["S_in"], x["dS_out"])
+            run.replay()
+        stream.synchronize()
+        assert torch.equal(run.o, ref["o"]) and torch.equal(run.dg, ref["dg"]) and torch.equal(run.dS_init, ref["dS_in"])
+        run.release()
+    finally:
+        binding.sf_set_tuning(None)
+    assert binding.sf_device_status() == 0
+    compare(ref, oracle_reference(x), tolerance(w), label="tuning")

@@ -119,3 +119,19 @@ def test_segments_that_are_not_whole_chunks(dtype, d, chunk, segs):
     padded_got = dict(o=run.o, S_out=run.S_bounds[-1], dq=run.dq, dk=run.dk, dv=run.dv, dg=run.dg, dS_in=run.dS_init)
     for n in NAMES:
         assert torch.equal(padded_got[n], got[n]), n          # the padding's content (3.0, not zero) must not leak in
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    # failure detection without a fault: a self-test kernel waits (about a millisecond) on a barrier nothing completes;
+    # the bounded wait gives up, the status word says so, and after clearing it a normal chain runs and is correct
+    binding.sf_device_status_clear()
+    assert binding.sf_device_check() == 0
+    assert binding.sf_selftest_bounded_wait(2_000_000) == 5            # SF_ERR_TIMEOUT
+    assert binding.sf_device_status() == 3 and binding.sf_device_check() == 5
+    binding.sf_device_status_clear()
+    assert binding.sf_device_status() == 0
+    assert binding.sf_selftest_bounded_wait(0) == 1 and binding.sf_selftest_bounded_wait(10 ** 9) == 1   # limit out of range
+    w = Workload("after-timeout", 1, 2, 128, 128, [640, 320], 64, s_in_sigma=0.02, ds_out_sigma=0.02, seed=31)
+    x = inputs.make_inputs(w, DEV)
+    got, _ = run_chain(w, x)
+    compare(got, oracle_reference(x), tolerance(w), label=w.name)

@@ -184,3 +184,22 @@ def test_autotune_rejects_bad_arguments_before_any_cuda_call(lib):
     bad = (ctypes.c_int32 * 1)(0)                                                                  # an empty segment
     assert lib.sf_chain_autotune(ctypes.byref(d), bad, 1, *head[3:], cands, 2, 3, 1, None, ctypes.byref(best), None) == 1
     assert best.value == -7
+
+
+def test_tuning_is_validated_and_restored(lib):
+    from paper_2608_06838_b200.binding import SfError, Tuning
+    binding.sf_set_tuning(None)
+    d = binding.sf_get_tuning()
+    assert (d.sweep_streams, d.agg_streams, d.scan_group_tokens, d.agg_inorder_ctas, d.agg_ahead) == (4, 4, 4096, 74, 0)
+    binding.sf_set_tuning(dict(sweep_streams=2, agg_ahead=1))
+    t = binding.sf_get_tuning()
+    assert (t.sweep_streams, t.agg_streams, t.agg_ahead) == (2, 4, 1)
+    for bad in (dict(sweep_streams=0), dict(sweep_streams=5), dict(agg_streams=0), dict(agg_streams=9),
+                dict(scan_group_tokens=-1), dict(agg_inorder_ctas=0), dict(agg_ahead=-1)):
+        with pytest.raises(SfError) as e:
+            binding.sf_set_tuning(bad)
+        assert e.value.code == 1
+        t2 = binding.sf_get_tuning()                      # a rejected tuning changes nothing
+        assert (t2.sweep_streams, t2.agg_streams, t2.agg_ahead) == (2, 4, 1)
+    binding.sf_set_tuning(None)
+    assert binding.sf_get_tuning().sweep_streams == 4
