@@ -250,6 +250,15 @@ def main():
             best = 0
         run.desc.chunks_per_block = best
         tuned = {"candidates": cands, "ms": [round(v, 4) for v in cand_ms], "chosen": best, "rule": "model unless > 2 % faster over 10 reps"}
+    if args.autotune and overlap and args.graph:
+        # profile-guided schedule of the chain driver (streams, how far the aggregates run ahead), same margin rule
+        with torch.cuda.stream(work_stream):
+            t, t_ms, d_ms = run.autotune_schedule(x["S_in"], x["dS_out"], reps=10, margin=0.02)
+        work_stream.synchronize()
+        tuned = tuned or {}
+        tuned["schedule"] = {"sweep_streams": t.sweep_streams, "agg_streams": t.agg_streams, "scan_group_tokens": t.scan_group_tokens,
+                             "agg_inorder_ctas": t.agg_inorder_ctas, "agg_ahead": t.agg_ahead, "ms": round(t_ms, 4),
+                             "default_ms": round(d_ms, 4)}
     if args.graph:
         with torch.cuda.stream(work_stream):
             run.capture(x["S_in"], x["dS_out"], overlap=overlap)
@@ -395,7 +404,7 @@ def main():
         "timed_regions": {"repeats": len(region_ms), "ms_per_step_median": ms_per_step,
                           "ms_per_step_min": min(region_ms) / args.steps, "ms_per_step_max": max(region_ms) / args.steps},
         "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d_k, "d_v": w.d_v, "T": w.T, "segments": w.seg_lens,
-                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or (tuned["chosen"] if tuned else "auto"),
+                   "chunk": w.chunk, "chunks_per_block": args.chunks_per_block or (tuned.get("chosen", "auto") if tuned else "auto"),
                    "autotune": tuned, "overlap": overlap, "graph": bool(args.graph),
                    "l2": "inputs (%.0f MB) exceed L2, no flush" % (4 * tokens * w.H * w.d_k * 2 / 1e6),
                    "parallelism": "replicas only"},

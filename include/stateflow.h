@@ -299,6 +299,23 @@ sf_status_t sf_chain_autotune(const sf_seg_desc_t* desc, const int32_t* seg_lens
                               sf_stream_t stream, int32_t* best, float* ms);
 
 /*
+ * Profile-guided choice of the driver's schedule (Section 3.4 last paragraph, Section 4.4 / Table 3: the paper's overlap
+ * schedules are picked per shape from measurements).  Times the chain (as sf_chain_autotune does, with the descriptor's
+ * block length) under a small built-in set of valid sf_tuning_t values - how far the aggregates may run ahead (0, 1,
+ * 2 segments), 2 or 4 sweep streams, aggregates in order or spread over their streams - and installs the fastest with
+ * sf_set_tuning, except that the default stays unless it is beaten by more than `margin` (e.g. 0.02) over `reps`
+ * repetitions.  chosen / chosen_ms / default_ms (the last two nullable, HOST) report the outcome.  Needs the same
+ * buffers as sf_chain_graph_create; synchronises `stream`.
+ */
+sf_status_t sf_chain_autotune_schedule(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg,
+                                       const void* q, const void* k, const void* v, const float* g, const float* S_init,
+                                       void* o, float* S_bounds, void* fwd_workspace, size_t fwd_workspace_bytes,
+                                       const void* dO, const float* dS_final, void* dq, void* dk, void* dv, float* dg,
+                                       float* dS_init, void* bwd_workspace, size_t bwd_workspace_bytes, int32_t reps,
+                                       float margin, sf_stream_t stream, sf_tuning_t* chosen, float* chosen_ms,
+                                       float* default_ms);
+
+/*
  * Hybrid-aware sequence chunking (paper Section 3.2, Eq. 9-11): the segment lengths to hand to the chain
  * driver.  Host code only; no CUDA call.  With boundaries 0 = c_0 < ... < c_N = T and s_i = c_{i+1} - c_i,
  *     Cost_i = w_tok * s_i + w_soft * (c_i * s_i + s_i^2 / 2)                                       (Eq. 9)

@@ -83,6 +83,9 @@ def load() -> ctypes.CDLL:
         lib.sf_chain_autotune.restype = ctypes.c_int
         lib.sf_chain_autotune.argtypes = [dp, ip, i32] + [vp] * 7 + [vp, sz] + [vp] * 7 + [vp, sz, ip, i32, i32, i32, vp, ip,
                                                                                          ctypes.POINTER(ctypes.c_float)]
+        lib.sf_chain_autotune_schedule.restype = ctypes.c_int
+        lib.sf_chain_autotune_schedule.argtypes = [dp, ip, i32] + [vp] * 7 + [vp, sz] + [vp] * 7 + [vp, sz, i32, ctypes.c_float, vp,
+                                                                                                  vp, vp, vp]
         lib.sf_partition_hybrid.restype = ctypes.c_int
         lib.sf_partition_hybrid.argtypes = [ctypes.c_int64, i32, ctypes.c_double, ctypes.c_double, ctypes.c_double, i32, ip]
         lib.sf_device_status.restype = i32
@@ -229,6 +232,21 @@ def sf_chain_autotune(desc: SegDesc, seg_lens, q, k, v, g, S_init, o, S_bounds, 
     return int(best.value), [float(x) for x in ms]
 
 
+def sf_chain_autotune_schedule(desc: SegDesc, seg_lens, q, k, v, g, S_init, o, S_bounds, fwd_workspace, dO, dS_final, dq, dk, dv,
+                               dg, dS_init, bwd_workspace, reps=5, margin=0.02, stream=None):
+    """Searches the built-in set of schedules, installs the choice (sf_set_tuning) and returns
+    (chosen Tuning, chosen ms, default ms)."""
+    t = Tuning()
+    ms, dms = ctypes.c_float(-1.0), ctypes.c_float(-1.0)
+    _check(load().sf_chain_autotune_schedule(ctypes.byref(desc), _seg_array(seg_lens), len(seg_lens), _ptr(q), _ptr(k), _ptr(v),
+                                             _ptr(g), _ptr(S_init), _ptr(o), _ptr(S_bounds), _ptr(fwd_workspace),
+                                             fwd_workspace.numel(), _ptr(dO), _ptr(dS_final), _ptr(dq), _ptr(dk), _ptr(dv),
+                                             _ptr(dg), _ptr(dS_init), _ptr(bwd_workspace), bwd_workspace.numel(), int(reps),
+                                             float(margin), _stream(stream), ctypes.byref(t), ctypes.byref(ms), ctypes.byref(dms)),
+           "sf_chain_autotune_schedule")
+    return t, float(ms.value), float(dms.value)
+
+
 def sf_partition_hybrid(T: int, N: int, w_tok: float, w_soft: float, alpha: float, multiple: int = 128) -> List[int]:
     """Segment lengths of the candidate partition (host only)."""
     out = (ctypes.c_int32 * max(N, 1))()
@@ -373,6 +391,13 @@ class ChainRun:
             self.release()
         except Exception:
             pass
+
+    def autotune_schedule(self, S_init=None, dS_final=None, reps=5, margin=0.02, stream=None):
+        """Profile-guided schedule of the chain driver for these buffers; the choice stays installed process-wide."""
+        self.release()
+        return sf_chain_autotune_schedule(self.desc, self.seg_lens, self.q, self.k, self.v, self.g, S_init, self.o, self.S_bounds,
+                                          self.ws_f, self.dO, dS_final, self.dq, self.dk, self.dv, self.dg, self.dS_init,
+                                          self.ws_b, reps, margin, stream)
 
     def autotune(self, S_init=None, dS_final=None, candidates=(0, 8, 10, 11, 13, 16, 19, 22, 26, 29, 32), reps=3, overlap=True, stream=None):
         """Times the chain for every candidate block length, keeps the fastest in the descriptor and returns

@@ -1038,6 +1038,50 @@ sf_status_t sf_chain_autotune(const sf_seg_desc_t* desc, const int32_t* seg_lens
     return result;
 }
 
+sf_status_t sf_chain_autotune_schedule(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q,
+                                       const void* k, const void* v, const float* g, const float* S_init, void* o,
+                                       float* S_bounds, void* fwd_workspace, size_t fwd_workspace_bytes, const void* dO,
+                                       const float* dS_final, void* dq, void* dk, void* dv, float* dg, float* dS_init,
+                                       void* bwd_workspace, size_t bwd_workspace_bytes, int32_t reps, float margin,
+                                       sf_stream_t stream, sf_tuning_t* chosen, float* chosen_ms, float* default_ms) {
+    if (!desc || reps < 1 || !(margin >= 0.f) || !chosen) return SF_ERR_INVALID_ARG;
+    // a small set of valid schedules, the default first
+    std::vector<sf_tuning_t> grid;
+    grid.push_back(kDefaultTuning);
+    for (int ahead : {0, 1, 2})
+        for (int sweeps : {2, 4})
+            for (int inorder : {1, 74}) {
+                sf_tuning_t t = kDefaultTuning;
+                t.agg_ahead = ahead; t.sweep_streams = sweeps; t.agg_inorder_ctas = inorder;
+                if (ahead == 0 && sweeps == 4 && inorder == 74) continue;       // the default itself
+                grid.push_back(t);
+            }
+    const sf_tuning_t before = current_tuning();
+    const int32_t cand = desc->chunks_per_block;
+    float best_ms = -1.f, def_ms = -1.f;
+    sf_tuning_t best = kDefaultTuning;
+    sf_status_t result = SF_OK;
+    for (size_t i = 0; i < grid.size(); ++i) {
+        if (sf_set_tuning(&grid[i]) != SF_OK) continue;
+        int32_t b = 0;
+        float ms = -1.f;
+        const sf_status_t st = sf_chain_autotune(desc, seg_lens, n_seg, q, k, v, g, S_init, o, S_bounds, fwd_workspace,
+                                                 fwd_workspace_bytes, dO, dS_final, dq, dk, dv, dg, dS_init, bwd_workspace,
+                                                 bwd_workspace_bytes, &cand, 1, reps, 1, stream, &b, &ms);
+        if (st != SF_OK) { result = st; break; }
+        if (i == 0) def_ms = ms;
+        if (best_ms < 0.f || ms < best_ms) { best_ms = ms; best = grid[i]; }
+    }
+    if (result != SF_OK) { sf_set_tuning(&before); return result; }
+    // the default stays unless something beats it by more than the margin (differences below that are noise)
+    if (def_ms > 0.f && def_ms <= (1.f + margin) * best_ms) { best = kDefaultTuning; best_ms = def_ms; }
+    sf_set_tuning(&best);
+    *chosen = best;
+    if (chosen_ms) *chosen_ms = best_ms;
+    if (default_ms) *default_ms = def_ms;
+    return SF_OK;
+}
+
 sf_status_t sf_partition_hybrid(int64_t T, int32_t N, double w_tok, double w_soft, double alpha, int32_t multiple,
                                 int32_t* seg_lens) {
     if (T < 1 || N < 1 || multiple < 1 || !seg_lens) return SF_ERR_INVALID_ARG;

@@ -93,3 +93,30 @@ def test_every_schedule_gives_the_bits_of_the_default_one(tuning):
         binding.sf_set_tuning(None)
     assert binding.sf_device_status() == 0
     compare(ref, oracle_reference(x), tolerance(w), label="tuning")
+
+
+def test_schedule_search_installs_a_valid_choice_and_results_do_not_change():
+    w = Workload("sched", 1, 4, 128, 128, [2048, 1024, 1024, 512], 64, s_in_sigma=0.02, ds_out_sigma=0.02, seed=19)
+    x = inputs.make_inputs(w, DEV)
+    binding.sf_set_tuning(None)
+    ref, _ = run_chain(w, x)
+    ref = {n: ref[n].clone() for n in NAMES}
+    run = binding.ChainRun(x["q"], x["k"], x["v"], x["g"], x["dO"], w.seg_lens, w.chunk)
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    try:
+        with torch.cuda.stream(stream):
+            t, ms, default_ms = run.autotune_schedule(x["S_in"], x["dS_out"], reps=2, margin=0.02)
+        stream.synchronize()
+        assert ms > 0 and default_ms > 0 and ms <= default_ms
+        assert t.sweep_streams in (2, 4) and t.agg_ahead in (0, 1, 2) and t.agg_inorder_ctas in (1, 74)
+        now = binding.sf_get_tuning()
+        assert (now.sweep_streams, now.agg_ahead, now.agg_inorder_ctas) == (t.sweep_streams, t.agg_ahead, t.agg_inorder_ctas)
+        if (t.sweep_streams, t.agg_ahead, t.agg_inorder_ctas) != (4, 0, 74):
+            assert ms < default_ms / 1.02                   # the default is only left for a clear win
+        got, _ = run_chain(w, x)
+        for n in NAMES:
+            assert torch.equal(got[n], ref[n]), n
+    finally:
+        binding.sf_set_tuning(None)
+    assert binding.sf_device_status() == 0
