@@ -33,7 +33,9 @@ FLOPS_PER_TOKEN_HEAD = 344064        # full chunk tiles, d = 128, chunk 64: forw
 KERNEL_BYTES = {"agg_kv": 516, "agg_qdo": 516, "fwd_out": 1028, "dq": 1284, "dkdv": 1540}
 # DRAM bytes per token*head of each kernel from the ncu capture of the small case (profiles/, 262144 token*heads per
 # launch), scaled to a bench launch by the token*heads it processes (traffic grows in proportion)
-KERNEL_NCU_TRAFFIC = {"dkdv": (278.056e6 + 107.461e6) / 262144}
+KERNEL_NCU_TRAFFIC = {"agg_kv": (135.293e6 + 3.755e6) / 262144, "agg_qdo": (135.294e6 + 3.791e6) / 262144,
+                      "fwd_out": (210.929e6 + 43.808e6) / 262144, "dq": (277.988e6 + 49.363e6) / 262144,
+                      "dkdv": (278.094e6 + 106.707e6) / 262144}
 
 
 def peaks():
