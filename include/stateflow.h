@@ -386,6 +386,67 @@ int64_t sf_launch_count(void);
 void sf_stage_timing(int32_t enable);
 int32_t sf_stage_timing_read(float* ms, int64_t* launches, int32_t n);
 
+/*
+ * ---- Extensions of the segment operator to further transition families --------------------------------------------
+ * Paper Section 2.1 lets the transition F_t be diagonal or scalar-plus-low-rank besides the scalar decay that the
+ * entry points above implement; Section 3.1 (footnote on auxiliary boundary states) lets a short-convolution state
+ * travel with S across the segment boundary.  The calls below are those three operators with the same segment
+ * semantics (Eq. 4-7): a forward maps the incoming boundary state to the outgoing one, a backward maps the gradient
+ * of the outgoing boundary state to that of the incoming one, so segments chain exactly as with sf_segment_*.
+ * They are float32 CUDA-core kernels that walk the tokens in order (one CTA per batch x head): correct to float32
+ * rounding, deterministic, and not tuned.  All pointers are DEVICE pointers to float32; nothing is allocated and the
+ * calls do not synchronise.
+ *
+ * Descriptor: dtype must be SF_F32, d_k in {32, 64}, d_v in {32, 64, 128}; chunk and chunks_per_block are ignored.
+ * q, k (and the per-channel g / dg of the diagonal family) use tok_stride_qk / batch_stride_qk, v, o, dO, dv use the
+ * _v strides, the per-head scalars g, beta, dg, dbeta of the delta rule use the _g strides; element (b, t, h, i) sits
+ * at b*batch_stride + t*tok_stride + h*d + i.  States are [B, H, d_k, d_v] dense.
+ * Errors as above: SF_ERR_INVALID_ARG (NULL where required, bad shape, an input state aliasing an output state),
+ * SF_ERR_UNSUPPORTED (shape or dtype outside the set), SF_ERR_WORKSPACE, SF_ERR_CUDA.
+ */
+
+/* Workspace of the two backward calls: one state per 16 tokens plus 16 states, per batch x head (0 on a bad descriptor).
+   256-byte aligned. */
+size_t sf_recurrent_workspace_bytes(const sf_seg_desc_t* desc);
+
+/*
+ * Diagonal transition (Section 2.1): one log-decay per key channel, g [B, T, H, d_k] laid out like q.
+ *   S_t = diag(exp(g_t)) S_{t-1} + k_t^T v_t ,  o_t = q_t S_t
+ * S_in nullable (zero state); S_out required.  Backward: dS_out nullable (zero), dg has the layout of g.
+ */
+sf_status_t sf_channel_segment_fwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
+                                   const float* S_in, float* o, float* S_out, sf_stream_t stream);
+sf_status_t sf_channel_segment_bwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
+                                   const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk, float* dv,
+                                   float* dg, float* dS_in, void* workspace, size_t workspace_bytes, sf_stream_t stream);
+
+/*
+ * Gated delta rule (scalar decay plus a rank-one correction; Section 2.1, Eq. 2 with a non-empty V_new), with
+ * a_t = exp(g_t), g and beta [B, T, H] laid out like the g of sf_segment_fwd:
+ *   u_t = k_t S_{t-1} ;  w_t = beta_t (v_t - a_t u_t) ;  S_t = a_t S_{t-1} + k_t^T w_t ;  o_t = q_t S_t
+ * i.e. S_t = a_t (I - beta_t k_t^T k_t) S_{t-1} + beta_t k_t^T v_t.  Keys are used as given (normalise them upstream).
+ */
+sf_status_t sf_delta_segment_fwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
+                                 const float* beta, const float* S_in, float* o, float* S_out, sf_stream_t stream);
+sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
+                                 const float* beta, const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk,
+                                 float* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
+                                 sf_stream_t stream);
+
+/*
+ * Causal depthwise convolution of width W (1..8) over the tokens of a segment, dense float32:
+ *   x, y [B, L, C] ; w [W, C], w[j] multiplies the input j tokens back ; tails [B, W-1, C]
+ *   ext = [tail_in ; x] ,  y_t = sum_j w[j] * ext[W-1+t-j] ,  tail_out = the last W-1 rows of ext
+ * tail_in NULL means zeros (start of the sequence); tail_out is the boundary state handed to the next segment and
+ * is required when W > 1 (L may be shorter than W-1: old tail rows then move up).  Backward: dtail_out nullable;
+ * dw is overwritten with this segment's contribution (the caller adds the segments' dw), summed in a fixed order.
+ */
+sf_status_t sf_conv_segment_fwd(int32_t B, int32_t L, int32_t C, int32_t W, const float* x, const float* w, const float* tail_in,
+                                float* y, float* tail_out, sf_stream_t stream);
+sf_status_t sf_conv_segment_bwd(int32_t B, int32_t L, int32_t C, int32_t W, const float* x, const float* w, const float* tail_in,
+                                const float* dy, const float* dtail_out, float* dx, float* dw, float* dtail_in,
+                                sf_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -95,6 +95,20 @@ def load() -> ctypes.CDLL:
         lib.sf_stage_timing.argtypes = [i32]
         lib.sf_stage_timing_read.restype = i32
         lib.sf_stage_timing_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64), i32]
+        lib.sf_recurrent_workspace_bytes.restype = sz
+        lib.sf_recurrent_workspace_bytes.argtypes = [dp]
+        lib.sf_channel_segment_fwd.restype = ctypes.c_int
+        lib.sf_channel_segment_fwd.argtypes = [dp] + [vp] * 7 + [vp]
+        lib.sf_channel_segment_bwd.restype = ctypes.c_int
+        lib.sf_channel_segment_bwd.argtypes = [dp] + [vp] * 12 + [vp, sz, vp]
+        lib.sf_delta_segment_fwd.restype = ctypes.c_int
+        lib.sf_delta_segment_fwd.argtypes = [dp] + [vp] * 8 + [vp]
+        lib.sf_delta_segment_bwd.restype = ctypes.c_int
+        lib.sf_delta_segment_bwd.argtypes = [dp] + [vp] * 14 + [vp, sz, vp]
+        lib.sf_conv_segment_fwd.restype = ctypes.c_int
+        lib.sf_conv_segment_fwd.argtypes = [i32] * 4 + [vp] * 5 + [vp]
+        lib.sf_conv_segment_bwd.restype = ctypes.c_int
+        lib.sf_conv_segment_bwd.argtypes = [i32] * 4 + [vp] * 8 + [vp]
         _lib = lib
     return _lib
 
@@ -335,6 +349,47 @@ def sf_stage_timing_read():
     cnt = (ctypes.c_int64 * n)()
     load().sf_stage_timing_read(ms, cnt, n)
     return [{"name": STAGE_NAMES[i], "ms": float(ms[i]), "launches": int(cnt[i])} for i in range(n)]
+
+
+# ---- extension operators: diagonal decay, gated delta rule, short convolution with a carried tail ----
+
+def sf_recurrent_workspace_bytes(desc: SegDesc) -> int:
+    return int(load().sf_recurrent_workspace_bytes(ctypes.byref(desc)))
+
+
+def sf_channel_segment_fwd(desc: SegDesc, q, k, v, g, S_in, o, S_out, stream=None):
+    _check(load().sf_channel_segment_fwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(S_in), _ptr(o),
+                                         _ptr(S_out), _stream(stream)), "sf_channel_segment_fwd")
+
+
+def sf_channel_segment_bwd(desc: SegDesc, q, k, v, g, S_in, dO, dS_out, dq, dk, dv, dg, dS_in, workspace, stream=None):
+    _check(load().sf_channel_segment_bwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(S_in), _ptr(dO),
+                                         _ptr(dS_out), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dg), _ptr(dS_in), _ptr(workspace),
+                                         workspace.numel(), _stream(stream)), "sf_channel_segment_bwd")
+
+
+def sf_delta_segment_fwd(desc: SegDesc, q, k, v, g, beta, S_in, o, S_out, stream=None):
+    _check(load().sf_delta_segment_fwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(S_in), _ptr(o),
+                                       _ptr(S_out), _stream(stream)), "sf_delta_segment_fwd")
+
+
+def sf_delta_segment_bwd(desc: SegDesc, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, workspace, stream=None):
+    _check(load().sf_delta_segment_bwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(S_in), _ptr(dO),
+                                       _ptr(dS_out), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dg), _ptr(dbeta), _ptr(dS_in),
+                                       _ptr(workspace), workspace.numel(), _stream(stream)), "sf_delta_segment_bwd")
+
+
+def sf_conv_segment_fwd(x, w, tail_in, y, tail_out, stream=None):
+    """x, y [B, L, C]; w [W, C]; tails [B, W-1, C]; all dense float32."""
+    B, L, C = x.shape
+    _check(load().sf_conv_segment_fwd(B, L, C, w.shape[0], _ptr(x), _ptr(w), _ptr(tail_in), _ptr(y), _ptr(tail_out),
+                                      _stream(stream)), "sf_conv_segment_fwd")
+
+
+def sf_conv_segment_bwd(x, w, tail_in, dy, dtail_out, dx, dw, dtail_in, stream=None):
+    B, L, C = x.shape
+    _check(load().sf_conv_segment_bwd(B, L, C, w.shape[0], _ptr(x), _ptr(w), _ptr(tail_in), _ptr(dy), _ptr(dtail_out), _ptr(dx),
+                                      _ptr(dw), _ptr(dtail_in), _stream(stream)), "sf_conv_segment_bwd")
 
 
 # ---- conveniences built only from the calls above (allocation + one call each) --------------------

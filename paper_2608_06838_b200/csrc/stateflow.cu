@@ -1236,3 +1236,6 @@ int32_t sf_stage_timing_read(float* ms, int64_t* launches, int32_t n) {
 }
 
 }  // extern "C"
+
+// Launches made by the library's other translation units count too.
+namespace sf { void note_launches(long long n) { g_launches.fetch_add(n, std::memory_order_relaxed); } }

@@ -1,0 +1,156 @@
+// C ABI of the extension operators: diagonal decay, gated delta rule, short convolution with a carried tail.
+// Argument checks happen before any launch; nothing here allocates, synchronises or falls back to the host.
+#include "../../include/stateflow.h"
+#include "sf_recurrent.cuh"
+
+namespace sf { void note_launches(long long n); }
+
+namespace {
+
+using sf::rec::RecParams;
+
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+sf_status_t check_desc(const sf_seg_desc_t* d) {
+    if (!d) return SF_ERR_INVALID_ARG;
+    if (d->B <= 0 || d->H <= 0 || d->seg_len <= 0 || d->d_k <= 0 || d->d_v <= 0) return SF_ERR_INVALID_ARG;
+    if (d->B > 65535) return SF_ERR_INVALID_ARG;                                       // grid.y
+    if (d->tok_stride_qk < (long long)d->H * d->d_k || d->tok_stride_v < (long long)d->H * d->d_v || d->tok_stride_g < d->H)
+        return SF_ERR_INVALID_ARG;
+    if (d->B > 1 && (d->batch_stride_qk <= 0 || d->batch_stride_v <= 0 || d->batch_stride_g <= 0)) return SF_ERR_INVALID_ARG;
+    if (d->dtype != SF_F32) return d->dtype == SF_BF16 ? SF_ERR_UNSUPPORTED : SF_ERR_INVALID_ARG;
+    const bool k_ok = d->d_k == 32 || d->d_k == 64;
+    const bool v_ok = d->d_v == 32 || d->d_v == 64 || d->d_v == 128;
+    return k_ok && v_ok ? SF_OK : SF_ERR_UNSUPPORTED;
+}
+
+RecParams make_params(const sf_seg_desc_t* d) {
+    RecParams p;
+    p.B = d->B; p.H = d->H; p.L = d->seg_len;
+    p.tqk = d->tok_stride_qk; p.tv = d->tok_stride_v; p.tg = d->tok_stride_g;
+    p.bqk = d->batch_stride_qk; p.bv = d->batch_stride_v; p.bg = d->batch_stride_g;
+    return p;
+}
+
+size_t ws_bytes(const sf_seg_desc_t* d) {
+    return (size_t)d->B * d->H * (size_t)sf::rec::ws_states(d->seg_len) * d->d_k * d->d_v * sizeof(float);
+}
+
+sf_status_t launched(int n = 1) {
+    sf::note_launches(n);
+    return cudaGetLastError() == cudaSuccess ? SF_OK : SF_ERR_CUDA;
+}
+
+template <int VAR>
+sf_status_t rec_fwd(const sf_seg_desc_t* d, const float* q, const float* k, const float* v, const float* g, const float* beta,
+                    const float* S_in, float* o, float* S_out, cudaStream_t st) {
+    const sf_status_t c = check_desc(d);
+    if (c != SF_OK) return c;
+    if (!q || !k || !v || !g || !o || !S_out || (VAR == sf::rec::DELTA && !beta)) return SF_ERR_INVALID_ARG;
+    if (S_in == S_out) return SF_ERR_INVALID_ARG;
+    if (!aligned4(q) || !aligned4(k) || !aligned4(v) || !aligned4(g) || !aligned4(o) || !aligned4(S_out)) return SF_ERR_INVALID_ARG;
+    const RecParams p = make_params(d);
+    const dim3 grid(d->H, d->B);
+#define SF_REC_FWD(DK, DV)                                                                                         \
+    if (d->d_k == DK && d->d_v == DV) {                                                                            \
+        sf::rec::rec_fwd_kernel<DK, DV, VAR><<<grid, DV, 0, st>>>(p, q, k, v, g, beta, S_in, o, S_out);            \
+        return launched();                                                                                         \
+    }
+    SF_REC_FWD(32, 32) SF_REC_FWD(32, 64) SF_REC_FWD(32, 128) SF_REC_FWD(64, 32) SF_REC_FWD(64, 64) SF_REC_FWD(64, 128)
+#undef SF_REC_FWD
+    return SF_ERR_UNSUPPORTED;
+}
+
+template <int VAR>
+sf_status_t rec_bwd(const sf_seg_desc_t* d, const float* q, const float* k, const float* v, const float* g, const float* beta,
+                    const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk, float* dv, float* dg,
+                    float* dbeta, float* dS_in, void* ws, size_t bytes, cudaStream_t st) {
+    const sf_status_t c = check_desc(d);
+    if (c != SF_OK) return c;
+    if (!q || !k || !v || !g || !dO || !dq || !dk || !dv || !dg || !dS_in) return SF_ERR_INVALID_ARG;
+    if (VAR == sf::rec::DELTA && (!beta || !dbeta)) return SF_ERR_INVALID_ARG;
+    if (dS_in == dS_out) return SF_ERR_INVALID_ARG;
+    if (!ws || bytes < ws_bytes(d) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return SF_ERR_WORKSPACE;
+    const RecParams p = make_params(d);
+    const dim3 grid(d->H, d->B);
+    float* w = static_cast<float*>(ws);
+#define SF_REC_BWD(DK, DV)                                                                                         \
+    if (d->d_k == DK && d->d_v == DV) {                                                                            \
+        sf::rec::rec_bwd_kernel<DK, DV, VAR><<<grid, DV, 0, st>>>(p, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, \
+                                                                  dg, dbeta, dS_in, w);                            \
+        return launched();                                                                                         \
+    }
+    SF_REC_BWD(32, 32) SF_REC_BWD(32, 64) SF_REC_BWD(32, 128) SF_REC_BWD(64, 32) SF_REC_BWD(64, 64) SF_REC_BWD(64, 128)
+#undef SF_REC_BWD
+    return SF_ERR_UNSUPPORTED;
+}
+
+sf_status_t check_conv(int32_t B, int32_t L, int32_t C, int32_t W) {
+    if (B <= 0 || L <= 0 || C <= 0 || W < 1) return SF_ERR_INVALID_ARG;
+    if (W > sf::rec::CONV_MAXW) return SF_ERR_UNSUPPORTED;
+    return SF_OK;
+}
+
+int conv_grid(long long n) {
+    const long long g = (n + 255) / 256;
+    return (int)(g < 1 ? 1 : (g > 148LL * 16 ? 148LL * 16 : g));
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t sf_recurrent_workspace_bytes(const sf_seg_desc_t* desc) {
+    return check_desc(desc) == SF_OK ? ws_bytes(desc) : 0;
+}
+
+sf_status_t sf_channel_segment_fwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
+                                   const float* S_in, float* o, float* S_out, sf_stream_t stream) {
+    return rec_fwd<sf::rec::CHANNEL>(desc, q, k, v, g, nullptr, S_in, o, S_out, reinterpret_cast<cudaStream_t>(stream));
+}
+
+sf_status_t sf_channel_segment_bwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
+                                   const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk, float* dv,
+                                   float* dg, float* dS_in, void* workspace, size_t workspace_bytes, sf_stream_t stream) {
+    return rec_bwd<sf::rec::CHANNEL>(desc, q, k, v, g, nullptr, S_in, dO, dS_out, dq, dk, dv, dg, nullptr, dS_in, workspace,
+                                     workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+sf_status_t sf_delta_segment_fwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
+                                 const float* beta, const float* S_in, float* o, float* S_out, sf_stream_t stream) {
+    return rec_fwd<sf::rec::DELTA>(desc, q, k, v, g, beta, S_in, o, S_out, reinterpret_cast<cudaStream_t>(stream));
+}
+
+sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
+                                 const float* beta, const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk,
+                                 float* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
+                                 sf_stream_t stream) {
+    return rec_bwd<sf::rec::DELTA>(desc, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, workspace,
+                                   workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+sf_status_t sf_conv_segment_fwd(int32_t B, int32_t L, int32_t C, int32_t W, const float* x, const float* w, const float* tail_in,
+                                float* y, float* tail_out, sf_stream_t stream) {
+    const sf_status_t c = check_conv(B, L, C, W);
+    if (c != SF_OK) return c;
+    if (!x || !w || !y || (W > 1 && !tail_out) || (tail_in && tail_in == tail_out)) return SF_ERR_INVALID_ARG;
+    const long long n = (long long)B * (L + W - 1) * C;
+    sf::rec::conv_fwd_kernel<<<conv_grid(n), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(B, L, C, W, x, w, tail_in, y, tail_out);
+    return launched();
+}
+
+sf_status_t sf_conv_segment_bwd(int32_t B, int32_t L, int32_t C, int32_t W, const float* x, const float* w, const float* tail_in,
+                                const float* dy, const float* dtail_out, float* dx, float* dw, float* dtail_in,
+                                sf_stream_t stream) {
+    const sf_status_t c = check_conv(B, L, C, W);
+    if (c != SF_OK) return c;
+    if (!x || !w || !dy || !dx || !dw || (W > 1 && !dtail_in) || (dtail_out && dtail_out == dtail_in)) return SF_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const long long n = (long long)B * (L + W - 1) * C;
+    sf::rec::conv_bwd_input_kernel<<<conv_grid(n), 256, 0, st>>>(B, L, C, W, w, dy, dtail_out, dx, dtail_in);
+    if (cudaGetLastError() != cudaSuccess) return SF_ERR_CUDA;
+    sf::rec::conv_bwd_weight_kernel<<<dim3((C + 31) / 32, W), dim3(32, 8), 0, st>>>(B, L, C, W, x, tail_in, dy, dw);
+    return launched(2);
+}
+
+}  // extern "C"

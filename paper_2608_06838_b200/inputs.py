@@ -101,6 +101,29 @@ def make_inputs(w: Workload, device="cpu"):
     return out
 
 
+def make_variant_inputs(w: Workload, device="cpu", conv_width: int = 4):
+    """make_inputs plus what the extension operators take (float32 workloads only):
+      g_channel [B,T,H,d_k] : -softplus(N(0,1)) * g_scale, one log-decay per key channel (diagonal family)
+      beta [B,T,H]          : sigmoid(N(0,1)), the write strength of the delta rule
+      conv_x, conv_dy [B,T,C], conv_w [W,C] / sqrt(W), conv_tail, conv_dtail [B,W-1,C] with C = H*d_v: N(0,1)"""
+    out = make_inputs(w, device)
+    dev = torch.device(device)
+    B, T, H = w.B, w.T, w.H
+    C = H * w.d_v
+
+    def randn(tid, *shape):
+        return torch.randn(*shape, generator=_gen(dev, w.seed, tid), device=dev, dtype=torch.float32)
+
+    out["g_channel"] = -torch.nn.functional.softplus(randn(7, B, T, H, w.d_k)) * w.g_scale
+    out["beta"] = torch.sigmoid(randn(8, B, T, H))
+    out["conv_x"] = randn(9, B, T, C)
+    out["conv_dy"] = randn(10, B, T, C)
+    out["conv_w"] = randn(11, conv_width, C) / (conv_width ** 0.5)
+    out["conv_tail"] = randn(12, B, max(conv_width - 1, 0), C)
+    out["conv_dtail"] = randn(13, B, max(conv_width - 1, 0), C)
+    return out
+
+
 def to_f64(t):
     """Widen a tensor (or None) to a float64 numpy array on the host - the exact values the GPU sees."""
     return None if t is None else t.detach().to("cpu", torch.float64).numpy()

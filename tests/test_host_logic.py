@@ -203,3 +203,27 @@ def test_tuning_is_validated_and_restored(lib):
         assert (t2.sweep_streams, t2.agg_streams, t2.agg_ahead) == (2, 4, 1)
     binding.sf_set_tuning(None)
     assert binding.sf_get_tuning().sweep_streams == 4
+
+
+def test_extension_operators_validate_before_any_launch(lib):
+    f32 = dict(dtype=binding.SF_F32, d_k=64, d_v=64, seg_len=100)
+    d = desc(**f32)
+    S1, S2 = ctypes.c_void_p(0x20000), ctypes.c_void_p(0x30000)
+    assert lib.sf_recurrent_workspace_bytes(ctypes.byref(d)) == 1 * 2 * (7 + 16) * 64 * 64 * 4   # ceil(100/16) + 16 states
+    assert lib.sf_recurrent_workspace_bytes(ctypes.byref(desc())) == 0                          # bf16: not offered
+    cf = lambda dd, q=P, S_in=None, S_out=S1: lib.sf_channel_segment_fwd(ctypes.byref(dd), q, P, P, P, S_in, P, S_out, None)
+    assert cf(desc()) == 2 and cf(desc(**dict(f32, d_k=128))) == 2 and cf(desc(**dict(f32, d_v=48))) == 2
+    assert cf(d, q=None) == 1 and cf(d, S_out=None) == 1 and cf(d, S_in=S1) == 1
+    assert cf(desc(**dict(f32, seg_len=0))) == 1 and cf(desc(**dict(f32, B=70000))) == 1
+    df = lambda dd, beta=P: lib.sf_delta_segment_fwd(ctypes.byref(dd), P, P, P, P, beta, None, P, S1, None)
+    assert df(d, beta=None) == 1 and df(desc()) == 2
+    bargs = [P] * 4 + [None, P, None] + [P] * 4 + [S2]
+    assert lib.sf_channel_segment_bwd(ctypes.byref(d), *bargs, ctypes.c_void_p(0x40000), 16, None) == 3
+    assert lib.sf_channel_segment_bwd(ctypes.byref(d), *bargs, None, 1 << 40, None) == 3
+    assert lib.sf_channel_segment_bwd(ctypes.byref(d), *bargs, ctypes.c_void_p(0x40010), 1 << 40, None) == 3
+    dargs = [P] * 5 + [None, P, None] + [P] * 4 + [None, S2]                # dbeta missing
+    assert lib.sf_delta_segment_bwd(ctypes.byref(d), *dargs, ctypes.c_void_p(0x40000), 1 << 40, None) == 1
+    conv = lambda B=1, L=8, C=4, W=4, x=P, tail_out=S1: lib.sf_conv_segment_fwd(B, L, C, W, x, P, None, P, tail_out, None)
+    assert conv(L=0) == 1 and conv(W=0) == 1 and conv(W=9) == 2 and conv(x=None) == 1 and conv(tail_out=None) == 1
+    assert lib.sf_conv_segment_bwd(1, 8, 4, 4, P, P, None, P, S1, P, P, S1, None) == 1       # dtail_out aliases dtail_in
+    assert lib.sf_conv_segment_bwd(1, 8, 4, 4, P, P, None, None, None, P, P, S1, None) == 1  # dy missing
