@@ -62,15 +62,38 @@ inline EncodeTiledFn encode_fn() {
 }
 
 // Map of a [B, L, H, 128] bf16 view: dims (feature, head, token, batch), box = 64 features x 1 x 64 tokens x 1.
+// A map is a pure function of (base, B, L, H, strides) and encoding one never reads device memory, so each host
+// thread keeps the last TMAP_CACHE maps it encoded: a chain that is launched again from the host (no graph) with the
+// same buffers re-encodes nothing.
+constexpr int TMAP_CACHE = 64;
+struct TmapKey {
+    const void* base; int B, L, H; long long tok_stride, batch_stride;
+    bool operator==(const TmapKey& o) const {
+        return base == o.base && B == o.B && L == o.L && H == o.H && tok_stride == o.tok_stride && batch_stride == o.batch_stride;
+    }
+};
+struct TmapCache { TmapKey key[TMAP_CACHE]; CUtensorMap map[TMAP_CACHE]; int used = 0, next = 0; };
+
 inline bool make_tmap(CUtensorMap* m, const void* base, int B, int L, int H, long long tok_stride, long long batch_stride) {
+    thread_local TmapCache cache;
+    const TmapKey key{base, B, L, H, tok_stride, batch_stride};
+    for (int i = 0; i < cache.used; ++i)
+        if (cache.key[i] == key) { *m = cache.map[i]; return true; }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
     cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)tok_stride * 2, (cuuint64_t)(B > 1 ? batch_stride : (long long)L * tok_stride) * 2};
     cuuint32_t box[4] = {64, 1, 64, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    const int slot = cache.next;
+    cache.key[slot] = key;
+    cache.map[slot] = *m;
+    cache.next = (slot + 1) % TMAP_CACHE;
+    if (cache.used < TMAP_CACHE) ++cache.used;
+    return true;
 }
 
 // ---- device helpers --------------------------------------------------------------------------------

@@ -18,6 +18,18 @@ def norm_err(a, r):
     return float(np.abs(a - r).max() / max(np.abs(r).max(), 1e-30))
 
 
+def floored_rel_err(a, r):
+    """Largest element-wise relative error with the denominator floored at 1e-3 of the tensor's largest magnitude
+    (a plain relative error is undefined at the zeros of the reference).  Reported, not gated."""
+    m = max(np.abs(r).max(), 1e-30)
+    return float((np.abs(a - r) / np.maximum(np.abs(r), 1e-3 * m)).max())
+
+
+def rms_err(a, r):
+    """RMS of the error over the RMS of the reference.  Reported, not gated."""
+    return float(np.sqrt(np.mean((a - r) ** 2)) / max(np.sqrt(np.mean(r ** 2)), 1e-30))
+
+
 def oracle_reference(x, heads=None):
     """Unsplit oracle run on the same bits; optionally on a subset of heads."""
     f = inputs.to_f64
@@ -48,6 +60,9 @@ def compare(got, ref, tol, heads=None, label=""):
         a = inputs.to_f64(a)
         assert np.isfinite(a).all(), "%s %s has non-finite values" % (label, n)
         errs[n] = norm_err(a, ref[n])
+        # the gate is the normalised max error; the other two figures are printed for the reader (pytest -s shows them)
+        print("[parity] %-28s %-6s normalised-max %.2e  floored-relative %.2e  rms %.2e"
+              % (label, n, errs[n], floored_rel_err(a, ref[n]), rms_err(a, ref[n])))
     bad = {n: e for n, e in errs.items() if not e <= tol}
     assert not bad, "%s: normalised max error above %.1e: %s (all: %s)" % (label, tol, bad, errs)
     return errs

@@ -135,3 +135,36 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     x = inputs.make_inputs(w, DEV)
     got, _ = run_chain(w, x)
     compare(got, oracle_reference(x), tolerance(w), label=w.name)
+
+
+def test_two_host_threads_on_two_streams_give_the_bits_of_the_serial_run():
+    # Calls without side streams (overlap = 0) may come from any thread; ctypes drops the GIL during a call, so the two
+    # threads really are inside the library at the same time.  Each thread has its own stream, buffers and workspaces.
+    import threading
+    ws = [Workload("thr-%d" % i, 1, 4, 128, 128, [1024, 640, 2048], 64, g_scale=0.1, s_in_sigma=0.1, ds_out_sigma=0.1, seed=40 + i)
+          for i in range(2)]
+    xs = [inputs.make_inputs(w, DEV) for w in ws]
+    serial = [run_chain(w, x, overlap=False)[0] for w, x in zip(ws, xs)]
+    torch.cuda.synchronize()
+    out, errors = [None, None], []
+
+    def work(i):
+        try:
+            torch.cuda.set_device(0)
+            with torch.cuda.stream(torch.cuda.Stream()):
+                for _ in range(3):
+                    out[i] = run_chain(ws[i], xs[i], overlap=False)[0]
+        except Exception as e:                   # surfaced below: an exception in a thread would otherwise be lost
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for i in range(2):
+        for n in NAMES:
+            assert torch.equal(out[i][n], serial[i][n]), (i, n)
+    assert binding.sf_device_status() == 0

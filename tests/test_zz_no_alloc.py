@@ -72,3 +72,26 @@ def test_shapes_beyond_the_static_scratch_are_rejected():
     with pytest.raises(binding.SfError) as e:
         binding.sf_segment_fwd_static(desc, x["q"], x["k"], x["v"], x["g"], None, o, S)
     assert e.value.code == 3
+
+
+def test_a_call_recorded_in_a_stream_capture_replays_to_the_same_bits():
+    # the use the entry point exists for: no allocation, no synchronisation, nothing the capture cannot record
+    w = Workload("na-capture", 1, 4, 128, 128, [16 * 64], 64, g_scale=0.1, s_in_sigma=0.1, seed=24)
+    x = inputs.make_inputs(w, DEV)
+    (_, _), (o_ref, S_ref) = _both(w, x)          # a first call outside any capture resolves the scratch address
+    desc = binding.make_desc(x["q"], x["v"], x["g"], w.chunk)
+    o, S = torch.zeros_like(o_ref), torch.zeros_like(S_ref)
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        binding.sf_segment_fwd_static(desc, x["q"], x["k"], x["v"], x["g"], x["S_in"], o, S)
+    torch.cuda.synchronize()
+    assert not o.any() and not S.any()            # recording runs nothing
+    for _ in range(2):
+        o.zero_()
+        S.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(o, o_ref) and torch.equal(S, S_ref)
+    assert binding.sf_device_status() == 0
