@@ -393,11 +393,12 @@ int32_t sf_stage_timing_read(float* ms, int64_t* launches, int32_t n);
  * travel with S across the segment boundary.  The calls below are those three operators with the same segment
  * semantics (Eq. 4-7): a forward maps the incoming boundary state to the outgoing one, a backward maps the gradient
  * of the outgoing boundary state to that of the incoming one, so segments chain exactly as with sf_segment_*.
- * They are float32 CUDA-core kernels that walk the tokens in order (one CTA per batch x head): correct to float32
- * rounding, deterministic, and not tuned.  All pointers are DEVICE pointers to float32; nothing is allocated and the
- * calls do not synchronise.
+ * They are CUDA-core kernels that walk the tokens in order (one CTA per batch x head) with float32 arithmetic:
+ * deterministic, and not tuned.  All pointers are DEVICE pointers; q, k, v, dO and o, dq, dk, dv have the descriptor's
+ * dtype (float32 or bf16; bf16 only rounds what is stored), log-decays, beta, their gradients and the states are
+ * float32.  Nothing is allocated and the calls do not synchronise.
  *
- * Descriptor: dtype must be SF_F32, d_k in {32, 64}, d_v in {32, 64, 128}; chunk and chunks_per_block are ignored.
+ * Descriptor: d_k in {32, 64}, d_v in {32, 64, 128}; chunk and chunks_per_block are ignored.
  * q, k (and the per-channel g / dg of the diagonal family) use tok_stride_qk / batch_stride_qk, v, o, dO, dv use the
  * _v strides, the per-head scalars g, beta, dg, dbeta of the delta rule use the _g strides; element (b, t, h, i) sits
  * at b*batch_stride + t*tok_stride + h*d + i.  States are [B, H, d_k, d_v] dense.
@@ -414,10 +415,10 @@ size_t sf_recurrent_workspace_bytes(const sf_seg_desc_t* desc);
  *   S_t = diag(exp(g_t)) S_{t-1} + k_t^T v_t ,  o_t = q_t S_t
  * S_in nullable (zero state); S_out required.  Backward: dS_out nullable (zero), dg has the layout of g.
  */
-sf_status_t sf_channel_segment_fwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
-                                   const float* S_in, float* o, float* S_out, sf_stream_t stream);
-sf_status_t sf_channel_segment_bwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
-                                   const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk, float* dv,
+sf_status_t sf_channel_segment_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                   const float* S_in, void* o, float* S_out, sf_stream_t stream);
+sf_status_t sf_channel_segment_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                   const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk, void* dv,
                                    float* dg, float* dS_in, void* workspace, size_t workspace_bytes, sf_stream_t stream);
 
 /*
@@ -426,11 +427,11 @@ sf_status_t sf_channel_segment_bwd(const sf_seg_desc_t* desc, const float* q, co
  *   u_t = k_t S_{t-1} ;  w_t = beta_t (v_t - a_t u_t) ;  S_t = a_t S_{t-1} + k_t^T w_t ;  o_t = q_t S_t
  * i.e. S_t = a_t (I - beta_t k_t^T k_t) S_{t-1} + beta_t k_t^T v_t.  Keys are used as given (normalise them upstream).
  */
-sf_status_t sf_delta_segment_fwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
-                                 const float* beta, const float* S_in, float* o, float* S_out, sf_stream_t stream);
-sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
-                                 const float* beta, const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk,
-                                 float* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
+sf_status_t sf_delta_segment_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                 const float* beta, const float* S_in, void* o, float* S_out, sf_stream_t stream);
+sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                 const float* beta, const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk,
+                                 void* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
                                  sf_stream_t stream);
 
 /*

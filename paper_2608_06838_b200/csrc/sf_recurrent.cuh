@@ -1,4 +1,4 @@
-// Token-recurrent float32 kernels (CUDA cores) of two further transition families (paper Section 2.1):
+// Token-recurrent kernels (CUDA cores, float32 arithmetic; q, k, v, dO and o, dq, dk, dv stored as float32 or bf16) of two further transition families (paper Section 2.1):
 //   CHANNEL : diagonal transition, one log-decay per key channel
 //                 S_t = diag(exp(g_t)) S_{t-1} + k_t^T v_t ,            o_t = q_t S_t
 //   DELTA   : scalar decay plus a rank-one correction (the gated delta rule; Eq. 2 with a non-empty V_new)
@@ -62,14 +62,14 @@ struct Tile {
 };
 
 // Loads tokens [t0, t0+n) of one (batch, head) into the tile; rows past n are left untouched (never read).
-template <int DK, int VAR>
-__device__ __forceinline__ void load_tile(Tile<DK, VAR>& s, const RecParams& p, const float* qh, const float* kh,
+template <int DK, int VAR, typename T>
+__device__ __forceinline__ void load_tile(Tile<DK, VAR>& s, const RecParams& p, const T* qh, const T* kh,
                                           const float* gh, const float* bh, int t0, int n, int nthreads) {
     for (int x = threadIdx.x; x < n * DK; x += nthreads) {
         const int r = x / DK, i = x - r * DK;
         const long long off = (long long)(t0 + r) * p.tqk + i;
-        s.q[r][i] = qh[off];
-        s.k[r][i] = kh[off];
+        s.q[r][i] = to_f32(qh[off]);
+        s.k[r][i] = to_f32(kh[off]);
         if (VAR == CHANNEL) s.a[r * DK + i] = expf(gh[off]);
     }
     if (VAR == DELTA)
@@ -104,17 +104,17 @@ __device__ __forceinline__ float step(float (&S)[DK], const Tile<DK, VAR>& s, in
 }
 
 // Forward of one segment.  grid (H, B), DV threads.  o may be NULL (boundary state only).
-template <int DK, int DV, int VAR>
-__global__ void __launch_bounds__(DV) rec_fwd_kernel(RecParams p, const float* __restrict__ q, const float* __restrict__ k,
-                                                     const float* __restrict__ v, const float* __restrict__ g,
+template <typename T, int DK, int DV, int VAR>
+__global__ void __launch_bounds__(DV) rec_fwd_kernel(RecParams p, const T* __restrict__ q, const T* __restrict__ k,
+                                                     const T* __restrict__ v, const float* __restrict__ g,
                                                      const float* __restrict__ beta, const float* __restrict__ S_in,
-                                                     float* __restrict__ o, float* __restrict__ S_out) {
+                                                     T* __restrict__ o, float* __restrict__ S_out) {
     __shared__ Tile<DK, VAR> s;
     const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
-    const float* qh = q + (long long)b * p.bqk + (long long)h * DK;
-    const float* kh = k + (long long)b * p.bqk + (long long)h * DK;
-    const float* vh = v + (long long)b * p.bv + (long long)h * DV;
-    float* oh = o ? o + (long long)b * p.bv + (long long)h * DV : nullptr;
+    const T* qh = q + (long long)b * p.bqk + (long long)h * DK;
+    const T* kh = k + (long long)b * p.bqk + (long long)h * DK;
+    const T* vh = v + (long long)b * p.bv + (long long)h * DV;
+    T* oh = o ? o + (long long)b * p.bv + (long long)h * DV : nullptr;
     const float* gh = VAR == CHANNEL ? g + (long long)b * p.bqk + (long long)h * DK : g + (long long)b * p.bg + h;
     const float* bh = VAR == DELTA ? beta + (long long)b * p.bg + h : nullptr;
     const long long so = ((long long)b * p.H + h) * DK * DV + j;
@@ -127,8 +127,8 @@ __global__ void __launch_bounds__(DV) rec_fwd_kernel(RecParams p, const float* _
         load_tile<DK, VAR>(s, p, qh, kh, gh, bh, t0, n, DV);
         __syncthreads();
         for (int r = 0; r < n; ++r) {
-            const float ot = step<DK, VAR>(S, s, r, vh[(long long)(t0 + r) * p.tv + j]);
-            if (oh) oh[(long long)(t0 + r) * p.tv + j] = ot;
+            const float ot = step<DK, VAR>(S, s, r, to_f32(vh[(long long)(t0 + r) * p.tv + j]));
+            if (oh) oh[(long long)(t0 + r) * p.tv + j] = from_f32<T>(ot);
         }
     }
 #pragma unroll
@@ -136,12 +136,12 @@ __global__ void __launch_bounds__(DV) rec_fwd_kernel(RecParams p, const float* _
 }
 
 // Backward of one segment.  grid (H, B), DV threads.  ws: per (batch, head) ws_states(L) states of DK*DV floats.
-template <int DK, int DV, int VAR>
-__global__ void __launch_bounds__(DV) rec_bwd_kernel(RecParams p, const float* __restrict__ q, const float* __restrict__ k,
-                                                     const float* __restrict__ v, const float* __restrict__ g,
+template <typename T, int DK, int DV, int VAR>
+__global__ void __launch_bounds__(DV) rec_bwd_kernel(RecParams p, const T* __restrict__ q, const T* __restrict__ k,
+                                                     const T* __restrict__ v, const float* __restrict__ g,
                                                      const float* __restrict__ beta, const float* __restrict__ S_in,
-                                                     const float* __restrict__ dO, const float* __restrict__ dS_out,
-                                                     float* __restrict__ dq, float* __restrict__ dk, float* __restrict__ dv,
+                                                     const T* __restrict__ dO, const float* __restrict__ dS_out,
+                                                     T* __restrict__ dq, T* __restrict__ dk, T* __restrict__ dv,
                                                      float* __restrict__ dg, float* __restrict__ dbeta,
                                                      float* __restrict__ dS_in, float* __restrict__ ws) {
     constexpr int NW = DV / 32;
@@ -150,15 +150,15 @@ __global__ void __launch_bounds__(DV) rec_bwd_kernel(RecParams p, const float* _
     __shared__ float red[2][NW][NRED];
     const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x, warp = j >> 5, lane = j & 31;
     const long long qo = (long long)b * p.bqk + (long long)h * DK, vo = (long long)b * p.bv + (long long)h * DV;
-    const float* qh = q + qo;
-    const float* kh = k + qo;
-    const float* vh = v + vo;
-    const float* doh = dO + vo;
+    const T* qh = q + qo;
+    const T* kh = k + qo;
+    const T* vh = v + vo;
+    const T* doh = dO + vo;
     const float* gh = VAR == CHANNEL ? g + qo : g + (long long)b * p.bg + h;
     const float* bh = VAR == DELTA ? beta + (long long)b * p.bg + h : nullptr;
-    float* dqh = dq + qo;
-    float* dkh = dk + qo;
-    float* dvh = dv + vo;
+    T* dqh = dq + qo;
+    T* dkh = dk + qo;
+    T* dvh = dv + vo;
     float* dgh = VAR == CHANNEL ? dg + qo : dg + (long long)b * p.bg + h;
     float* dbh = VAR == DELTA ? dbeta + (long long)b * p.bg + h : nullptr;
     const int ntile = num_tiles(p.L);
@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(DV) rec_bwd_kernel(RecParams p, const float* _
         __syncthreads();
         load_tile<DK, VAR>(s, p, qh, kh, gh, bh, t0, n, DV);
         __syncthreads();
-        for (int r = 0; r < n; ++r) step<DK, VAR>(S, s, r, vh[(long long)(t0 + r) * p.tv + j]);
+        for (int r = 0; r < n; ++r) step<DK, VAR>(S, s, r, to_f32(vh[(long long)(t0 + r) * p.tv + j]));
     }
 
     float G[DK];
@@ -197,11 +197,11 @@ __global__ void __launch_bounds__(DV) rec_bwd_kernel(RecParams p, const float* _
         for (int r = 0; r < n; ++r) {
 #pragma unroll
             for (int i = 0; i < DK; ++i) scratch[((long long)r * DK + i) * DV] = S[i];
-            if (r + 1 < n) step<DK, VAR>(S, s, r, vh[(long long)(t0 + r) * p.tv + j]);
+            if (r + 1 < n) step<DK, VAR>(S, s, r, to_f32(vh[(long long)(t0 + r) * p.tv + j]));
         }
         for (int r = n - 1; r >= 0; --r) {
             const long long t = t0 + r;
-            const float vj = vh[t * p.tv + j], doj = doh[t * p.tv + j];
+            const float vj = to_f32(vh[t * p.tv + j]), doj = to_f32(doh[t * p.tv + j]);
 #pragma unroll
             for (int i = 0; i < DK; ++i) S[i] = scratch[((long long)r * DK + i) * DV];     // S_{t-1}
             float* rd = red[par][warp];
@@ -223,11 +223,11 @@ __global__ void __launch_bounds__(DV) rec_bwd_kernel(RecParams p, const float* _
                 du = -a * bt * dw;
                 sc0 -= bt * dw * u;
                 sc1 = dw * e;
-                dvh[t * p.tv + j] = bt * dw;
+                dvh[t * p.tv + j] = from_f32<T>(bt * dw);
             } else {
 #pragma unroll
                 for (int i = 0; i < DK; ++i) dw = fmaf(s.k[r][i], G[i], dw);
-                dvh[t * p.tv + j] = dw;
+                dvh[t * p.tv + j] = from_f32<T>(dw);
             }
             // per-channel sums over the value channels, 32 key channels at a time
 #pragma unroll
@@ -273,8 +273,8 @@ __global__ void __launch_bounds__(DV) rec_bwd_kernel(RecParams p, const float* _
                 float acc = 0.f;
 #pragma unroll
                 for (int wv = 0; wv < NW; ++wv) acc += red[par][wv][x];
-                if (x < DK) dqh[t * p.tqk + x] = acc;
-                else if (x < 2 * DK) dkh[t * p.tqk + (x - DK)] = acc;
+                if (x < DK) dqh[t * p.tqk + x] = from_f32<T>(acc);
+                else if (x < 2 * DK) dkh[t * p.tqk + (x - DK)] = from_f32<T>(acc);
                 else if (VAR == CHANNEL) { if (x < 3 * DK) dgh[t * p.tqk + (x - 2 * DK)] = acc; }
                 else if (x == 2 * DK) dgh[t * p.tg] = acc;
                 else dbh[t * p.tg] = acc;

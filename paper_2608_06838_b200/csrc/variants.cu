@@ -10,6 +10,7 @@ namespace {
 using sf::rec::RecParams;
 
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+bool aligned2(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 1u) == 0; }
 
 sf_status_t check_desc(const sf_seg_desc_t* d) {
     if (!d) return SF_ERR_INVALID_ARG;
@@ -18,7 +19,7 @@ sf_status_t check_desc(const sf_seg_desc_t* d) {
     if (d->tok_stride_qk < (long long)d->H * d->d_k || d->tok_stride_v < (long long)d->H * d->d_v || d->tok_stride_g < d->H)
         return SF_ERR_INVALID_ARG;
     if (d->B > 1 && (d->batch_stride_qk <= 0 || d->batch_stride_v <= 0 || d->batch_stride_g <= 0)) return SF_ERR_INVALID_ARG;
-    if (d->dtype != SF_F32) return d->dtype == SF_BF16 ? SF_ERR_UNSUPPORTED : SF_ERR_INVALID_ARG;
+    if (d->dtype != SF_F32 && d->dtype != SF_BF16) return SF_ERR_INVALID_ARG;
     const bool k_ok = d->d_k == 32 || d->d_k == 64;
     const bool v_ok = d->d_v == 32 || d->d_v == 64 || d->d_v == 128;
     return k_ok && v_ok ? SF_OK : SF_ERR_UNSUPPORTED;
@@ -41,19 +42,15 @@ sf_status_t launched(int n = 1) {
     return cudaGetLastError() == cudaSuccess ? SF_OK : SF_ERR_CUDA;
 }
 
-template <int VAR>
-sf_status_t rec_fwd(const sf_seg_desc_t* d, const float* q, const float* k, const float* v, const float* g, const float* beta,
-                    const float* S_in, float* o, float* S_out, cudaStream_t st) {
-    const sf_status_t c = check_desc(d);
-    if (c != SF_OK) return c;
-    if (!q || !k || !v || !g || !o || !S_out || (VAR == sf::rec::DELTA && !beta)) return SF_ERR_INVALID_ARG;
-    if (S_in == S_out) return SF_ERR_INVALID_ARG;
-    if (!aligned4(q) || !aligned4(k) || !aligned4(v) || !aligned4(g) || !aligned4(o) || !aligned4(S_out)) return SF_ERR_INVALID_ARG;
-    const RecParams p = make_params(d);
+template <int VAR, typename T>
+sf_status_t rec_fwd_t(const sf_seg_desc_t* d, const RecParams& p, const void* q, const void* k, const void* v, const float* g,
+                      const float* beta, const float* S_in, void* o, float* S_out, cudaStream_t st) {
     const dim3 grid(d->H, d->B);
+    const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v);
+    T* to = static_cast<T*>(o);
 #define SF_REC_FWD(DK, DV)                                                                                         \
     if (d->d_k == DK && d->d_v == DV) {                                                                            \
-        sf::rec::rec_fwd_kernel<DK, DV, VAR><<<grid, DV, 0, st>>>(p, q, k, v, g, beta, S_in, o, S_out);            \
+        sf::rec::rec_fwd_kernel<T, DK, DV, VAR><<<grid, DV, 0, st>>>(p, tq, tk, tv, g, beta, S_in, to, S_out);     \
         return launched();                                                                                         \
     }
     SF_REC_FWD(32, 32) SF_REC_FWD(32, 64) SF_REC_FWD(32, 128) SF_REC_FWD(64, 32) SF_REC_FWD(64, 64) SF_REC_FWD(64, 128)
@@ -62,8 +59,42 @@ sf_status_t rec_fwd(const sf_seg_desc_t* d, const float* q, const float* k, cons
 }
 
 template <int VAR>
-sf_status_t rec_bwd(const sf_seg_desc_t* d, const float* q, const float* k, const float* v, const float* g, const float* beta,
-                    const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk, float* dv, float* dg,
+sf_status_t rec_fwd(const sf_seg_desc_t* d, const void* q, const void* k, const void* v, const float* g, const float* beta,
+                    const float* S_in, void* o, float* S_out, cudaStream_t st) {
+    const sf_status_t c = check_desc(d);
+    if (c != SF_OK) return c;
+    if (!q || !k || !v || !g || !o || !S_out || (VAR == sf::rec::DELTA && !beta)) return SF_ERR_INVALID_ARG;
+    if (S_in == S_out) return SF_ERR_INVALID_ARG;
+    const bool f32 = d->dtype == SF_F32;
+    auto al = [&](const void* x) { return f32 ? aligned4(x) : aligned2(x); };
+    if (!al(q) || !al(k) || !al(v) || !al(o) || !aligned4(g) || !aligned4(S_out)) return SF_ERR_INVALID_ARG;
+    const RecParams p = make_params(d);
+    return f32 ? rec_fwd_t<VAR, float>(d, p, q, k, v, g, beta, S_in, o, S_out, st)
+               : rec_fwd_t<VAR, __nv_bfloat16>(d, p, q, k, v, g, beta, S_in, o, S_out, st);
+}
+
+template <int VAR, typename T>
+sf_status_t rec_bwd_t(const sf_seg_desc_t* d, const RecParams& p, const void* q, const void* k, const void* v, const float* g,
+                      const float* beta, const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk, void* dv,
+                      float* dg, float* dbeta, float* dS_in, float* w, cudaStream_t st) {
+    const dim3 grid(d->H, d->B);
+    const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v),
+            *tdo = static_cast<const T*>(dO);
+    T *tdq = static_cast<T*>(dq), *tdk = static_cast<T*>(dk), *tdv = static_cast<T*>(dv);
+#define SF_REC_BWD(DK, DV)                                                                                         \
+    if (d->d_k == DK && d->d_v == DV) {                                                                            \
+        sf::rec::rec_bwd_kernel<T, DK, DV, VAR><<<grid, DV, 0, st>>>(p, tq, tk, tv, g, beta, S_in, tdo, dS_out, tdq, tdk, \
+                                                                     tdv, dg, dbeta, dS_in, w);                    \
+        return launched();                                                                                         \
+    }
+    SF_REC_BWD(32, 32) SF_REC_BWD(32, 64) SF_REC_BWD(32, 128) SF_REC_BWD(64, 32) SF_REC_BWD(64, 64) SF_REC_BWD(64, 128)
+#undef SF_REC_BWD
+    return SF_ERR_UNSUPPORTED;
+}
+
+template <int VAR>
+sf_status_t rec_bwd(const sf_seg_desc_t* d, const void* q, const void* k, const void* v, const float* g, const float* beta,
+                    const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk, void* dv, float* dg,
                     float* dbeta, float* dS_in, void* ws, size_t bytes, cudaStream_t st) {
     const sf_status_t c = check_desc(d);
     if (c != SF_OK) return c;
@@ -72,17 +103,10 @@ sf_status_t rec_bwd(const sf_seg_desc_t* d, const float* q, const float* k, cons
     if (dS_in == dS_out) return SF_ERR_INVALID_ARG;
     if (!ws || bytes < ws_bytes(d) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return SF_ERR_WORKSPACE;
     const RecParams p = make_params(d);
-    const dim3 grid(d->H, d->B);
     float* w = static_cast<float*>(ws);
-#define SF_REC_BWD(DK, DV)                                                                                         \
-    if (d->d_k == DK && d->d_v == DV) {                                                                            \
-        sf::rec::rec_bwd_kernel<DK, DV, VAR><<<grid, DV, 0, st>>>(p, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, \
-                                                                  dg, dbeta, dS_in, w);                            \
-        return launched();                                                                                         \
-    }
-    SF_REC_BWD(32, 32) SF_REC_BWD(32, 64) SF_REC_BWD(32, 128) SF_REC_BWD(64, 32) SF_REC_BWD(64, 64) SF_REC_BWD(64, 128)
-#undef SF_REC_BWD
-    return SF_ERR_UNSUPPORTED;
+    return d->dtype == SF_F32
+        ? rec_bwd_t<VAR, float>(d, p, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, w, st)
+        : rec_bwd_t<VAR, __nv_bfloat16>(d, p, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, w, st);
 }
 
 sf_status_t check_conv(int32_t B, int32_t L, int32_t C, int32_t W) {
@@ -104,26 +128,26 @@ size_t sf_recurrent_workspace_bytes(const sf_seg_desc_t* desc) {
     return check_desc(desc) == SF_OK ? ws_bytes(desc) : 0;
 }
 
-sf_status_t sf_channel_segment_fwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
-                                   const float* S_in, float* o, float* S_out, sf_stream_t stream) {
+sf_status_t sf_channel_segment_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                   const float* S_in, void* o, float* S_out, sf_stream_t stream) {
     return rec_fwd<sf::rec::CHANNEL>(desc, q, k, v, g, nullptr, S_in, o, S_out, reinterpret_cast<cudaStream_t>(stream));
 }
 
-sf_status_t sf_channel_segment_bwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
-                                   const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk, float* dv,
+sf_status_t sf_channel_segment_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                   const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk, void* dv,
                                    float* dg, float* dS_in, void* workspace, size_t workspace_bytes, sf_stream_t stream) {
     return rec_bwd<sf::rec::CHANNEL>(desc, q, k, v, g, nullptr, S_in, dO, dS_out, dq, dk, dv, dg, nullptr, dS_in, workspace,
                                      workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
-sf_status_t sf_delta_segment_fwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
-                                 const float* beta, const float* S_in, float* o, float* S_out, sf_stream_t stream) {
+sf_status_t sf_delta_segment_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                 const float* beta, const float* S_in, void* o, float* S_out, sf_stream_t stream) {
     return rec_fwd<sf::rec::DELTA>(desc, q, k, v, g, beta, S_in, o, S_out, reinterpret_cast<cudaStream_t>(stream));
 }
 
-sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const float* q, const float* k, const float* v, const float* g,
-                                 const float* beta, const float* S_in, const float* dO, const float* dS_out, float* dq, float* dk,
-                                 float* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
+sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                 const float* beta, const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk,
+                                 void* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
                                  sf_stream_t stream) {
     return rec_bwd<sf::rec::DELTA>(desc, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, workspace,
                                    workspace_bytes, reinterpret_cast<cudaStream_t>(stream));

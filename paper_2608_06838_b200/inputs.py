@@ -102,7 +102,7 @@ def make_inputs(w: Workload, device="cpu"):
 
 
 def make_variant_inputs(w: Workload, device="cpu", conv_width: int = 4):
-    """make_inputs plus what the extension operators take (float32 workloads only):
+    """make_inputs plus what the extension operators take:
       g_channel [B,T,H,d_k] : -softplus(N(0,1)) * g_scale, one log-decay per key channel (diagonal family)
       beta [B,T,H]          : sigmoid(N(0,1)), the write strength of the delta rule
       conv_x, conv_dy [B,T,C], conv_w [W,C] / sqrt(W), conv_tail, conv_dtail [B,W-1,C] with C = H*d_v: N(0,1)"""

@@ -210,7 +210,7 @@ def test_extension_operators_validate_before_any_launch(lib):
     d = desc(**f32)
     S1, S2 = ctypes.c_void_p(0x20000), ctypes.c_void_p(0x30000)
     assert lib.sf_recurrent_workspace_bytes(ctypes.byref(d)) == 1 * 2 * (7 + 16) * 64 * 64 * 4   # ceil(100/16) + 16 states
-    assert lib.sf_recurrent_workspace_bytes(ctypes.byref(desc())) == 0                          # bf16: not offered
+    assert lib.sf_recurrent_workspace_bytes(ctypes.byref(desc())) == 0                          # d_k = 128: not offered
     cf = lambda dd, q=P, S_in=None, S_out=S1: lib.sf_channel_segment_fwd(ctypes.byref(dd), q, P, P, P, S_in, P, S_out, None)
     assert cf(desc()) == 2 and cf(desc(**dict(f32, d_k=128))) == 2 and cf(desc(**dict(f32, d_v=48))) == 2
     assert cf(d, q=None) == 1 and cf(d, S_out=None) == 1 and cf(d, S_in=S1) == 1
