@@ -337,7 +337,11 @@ sf_status_t sf_partition_hybrid(int64_t T, int32_t N, double w_tok, double w_sof
  * pointer is a HOST pointer (pinned memory recommended).  The call copies the inputs to the device
  * buffers in `dev` (caller-allocated device scratch, sf_e2e_device_bytes() bytes, 256-byte
  * aligned), runs sf_chain_fwd + sf_chain_bwd and copies o, dq, dk, dv, dg, the final state and
- * dS_init back, all on `stream`, then synchronises the stream.  Section 3.1, Eq. 4-7.
+ * dS_init back, then synchronises `stream`; everything is ordered after earlier work on `stream` and is complete
+ * when the call returns.  The upload of dO and the download of o run on two copy streams of the library beside the
+ * forward and backward chains, so that both PCIe directions are busy at once where the dependencies allow (needs
+ * pinned host memory to take effect).  Uses the chain driver's per-device streams: the threading rule of
+ * sf_chain_* with overlap != 0 applies.  Section 3.1, Eq. 4-7.
  */
 size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg);
 

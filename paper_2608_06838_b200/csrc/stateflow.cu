@@ -413,6 +413,7 @@ inline int agg_stream_index(const SegParams& p, int i, const sf_tuning_t& tu) {
 struct ChainRes {
     cudaStream_t side[1 + 2 * kSweepStreams] = {};   // 0: unused; then two groups of sweep streams, used round-robin by segment
     cudaStream_t agg[kAggStreams] = {};
+    cudaStream_t copy[2] = {};              // host-buffer wrapper: second upload stream, download stream
     cudaEvent_t ev[64] = {};
     std::vector<cudaEvent_t> pool;          // extra events of the backward driver, grown on demand
     bool ok = false;
@@ -430,6 +431,8 @@ sf_status_t chain_resources(ChainRes** out) {
         for (auto& s : r.side)
             if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SF_ERR_CUDA;
         for (auto& s : r.agg)
+            if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SF_ERR_CUDA;
+        for (auto& s : r.copy)
             if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SF_ERR_CUDA;
         for (auto& e : r.ev)
             if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return SF_ERR_CUDA;
@@ -1157,28 +1160,45 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
     char* wsf = take(wf);
     char* wsb = take(wb);
 
+    // Copies that nothing waits for yet run beside the compute on two copy streams, so that the two PCIe directions
+    // are busy at the same time where the dependencies allow it:
+    //   caller's stream : up q, k, v, g, S_init -> forward chain -> [wait dO] backward chain -> down dq, dk, dv, dg, dS_init
+    //   upload stream   : up dO, dS_final                      (needed only by the backward)
+    //   download stream : [wait forward] down o, S_final       (overlaps the upload of dO and the backward)
+    ChainRes* res = nullptr;
+    SF_TRY(chain_resources(&res));
+    cudaStream_t up = res->copy[0], down = res->copy[1];
+    cudaEvent_t e_start = res->ev[1], e_dO = res->ev[2], e_fwd = res->ev[3], e_o = res->ev[4];
+    SF_CUDA(cudaEventRecord(e_start, st));
     SF_CUDA(cudaMemcpyAsync(q_, q, bqk, cudaMemcpyHostToDevice, st));
     SF_CUDA(cudaMemcpyAsync(k_, k, bqk, cudaMemcpyHostToDevice, st));
     SF_CUDA(cudaMemcpyAsync(v_, v, bv, cudaMemcpyHostToDevice, st));
     SF_CUDA(cudaMemcpyAsync(g_, g, bg, cudaMemcpyHostToDevice, st));
-    SF_CUDA(cudaMemcpyAsync(dO_, dO, bv, cudaMemcpyHostToDevice, st));
     if (S_init) SF_CUDA(cudaMemcpyAsync(sinit, S_init, sbytes, cudaMemcpyHostToDevice, st));
-    if (dS_final) SF_CUDA(cudaMemcpyAsync(dsfin, dS_final, sbytes, cudaMemcpyHostToDevice, st));
+    SF_CUDA(cudaStreamWaitEvent(up, e_start, 0));
+    SF_CUDA(cudaMemcpyAsync(dO_, dO, bv, cudaMemcpyHostToDevice, up));
+    if (dS_final) SF_CUDA(cudaMemcpyAsync(dsfin, dS_final, sbytes, cudaMemcpyHostToDevice, up));
+    SF_CUDA(cudaEventRecord(e_dO, up));
     // sB is a multiple of 256 but the chain driver indexes bounds densely
     float* bounds_dense = bounds;
     SF_TRY(sf_chain_fwd(&d, seg_lens, n_seg, q_, k_, v_, reinterpret_cast<float*>(g_), S_init ? sinit : nullptr, o_,
                         bounds_dense, wsf, wf, 1, stream));
+    SF_CUDA(cudaEventRecord(e_fwd, st));
+    SF_CUDA(cudaStreamWaitEvent(down, e_fwd, 0));
+    SF_CUDA(cudaMemcpyAsync(o, o_, bv, cudaMemcpyDeviceToHost, down));
+    if (S_final)
+        SF_CUDA(cudaMemcpyAsync(S_final, bounds_dense + (size_t)n_seg * (sbytes / sizeof(float)), sbytes, cudaMemcpyDeviceToHost, down));
+    SF_CUDA(cudaEventRecord(e_o, down));
+    SF_CUDA(cudaStreamWaitEvent(st, e_dO, 0));
     SF_TRY(sf_chain_bwd(&d, seg_lens, n_seg, q_, k_, v_, reinterpret_cast<float*>(g_), bounds_dense, dO_,
                         dS_final ? dsfin : nullptr, dq_, dk_, dv_, reinterpret_cast<float*>(dg_), dsinit, wsf, wsb,
                         wb, 1, stream));
-    SF_CUDA(cudaMemcpyAsync(o, o_, bv, cudaMemcpyDeviceToHost, st));
     SF_CUDA(cudaMemcpyAsync(dq, dq_, bqk, cudaMemcpyDeviceToHost, st));
     SF_CUDA(cudaMemcpyAsync(dk, dk_, bqk, cudaMemcpyDeviceToHost, st));
     SF_CUDA(cudaMemcpyAsync(dv, dv_, bv, cudaMemcpyDeviceToHost, st));
     SF_CUDA(cudaMemcpyAsync(dg, dg_, bg, cudaMemcpyDeviceToHost, st));
-    if (S_final)
-        SF_CUDA(cudaMemcpyAsync(S_final, bounds_dense + (size_t)n_seg * (sbytes / sizeof(float)), sbytes, cudaMemcpyDeviceToHost, st));
     SF_CUDA(cudaMemcpyAsync(dS_init, dsinit, sbytes, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaStreamWaitEvent(st, e_o, 0));
     SF_CUDA(cudaStreamSynchronize(st));
     return SF_OK;
 }
