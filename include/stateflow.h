@@ -439,6 +439,25 @@ sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const
                                  sf_stream_t stream);
 
 /*
+ * The same gated delta rule in its chunkwise form (Section 2.2, Eq. 2 with V_new): per chunk the unit-lower-triangular
+ * system (I + L) W = beta*V - beta*gam*(K H) is solved by substitution (UT transform), Pre builds its state-free parts for
+ * all chunks in parallel, ST carries the state from chunk to chunk and emits V_new = W, Out forms the outputs of all
+ * chunks in parallel; the backward mirrors it (transposed solve, reverse state pass, chunk-parallel gradients).
+ * Same arguments, layouts and results (to rounding) as sf_delta_segment_fwd/bwd.  desc->chunk in {16, 32},
+ * d_k, d_v in {32, 64}, float32 or bf16 storage, float32 arithmetic on CUDA cores.  Workspace:
+ * sf_delta_chunked_workspace_bytes(desc, backward) bytes, 256-byte aligned (U/W and Wk per token, one state per chunk;
+ * the backward rebuilds them and adds Z per token and one state gradient per chunk).
+ */
+size_t sf_delta_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward);
+sf_status_t sf_delta_chunked_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                 const float* beta, const float* S_in, void* o, float* S_out, void* workspace, size_t workspace_bytes,
+                                 sf_stream_t stream);
+sf_status_t sf_delta_chunked_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                 const float* beta, const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk,
+                                 void* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
+                                 sf_stream_t stream);
+
+/*
  * Causal depthwise convolution of width W (1..8) over the tokens of a segment, dense float32:
  *   x, y [B, L, C] ; w [W, C], w[j] multiplies the input j tokens back ; tails [B, W-1, C]
  *   ext = [tail_in ; x] ,  y_t = sum_j w[j] * ext[W-1+t-j] ,  tail_out = the last W-1 rows of ext

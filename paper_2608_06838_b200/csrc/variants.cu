@@ -2,6 +2,7 @@
 // Argument checks happen before any launch; nothing here allocates, synchronises or falls back to the host.
 #include "../../include/stateflow.h"
 #include "sf_recurrent.cuh"
+#include "sf_delta_chunk.cuh"
 
 namespace sf { void note_launches(long long n); }
 
@@ -120,6 +121,70 @@ int conv_grid(long long n) {
     return (int)(g < 1 ? 1 : (g > 148LL * 16 ? 148LL * 16 : g));
 }
 
+// ---- chunkwise delta rule ----------------------------------------------------------------------------------------
+sf_status_t check_chunked(const sf_seg_desc_t* d) {
+    const sf_status_t c = check_desc(d);
+    if (c != SF_OK) return c;
+    if (d->chunk <= 0) return SF_ERR_INVALID_ARG;
+    if ((d->chunk != 16 && d->chunk != 32) || d->d_v == 128) return SF_ERR_UNSUPPORTED;
+    if (d->H > 65535) return SF_ERR_INVALID_ARG;
+    return SF_OK;
+}
+
+sf::gdn::Params chunked_params(const sf_seg_desc_t* d) {
+    sf::gdn::Params p;
+    p.B = d->B; p.H = d->H; p.L = d->seg_len; p.C = d->chunk; p.NC = (d->seg_len + d->chunk - 1) / d->chunk;
+    p.dk = d->d_k; p.dv = d->d_v;
+    p.tqk = d->tok_stride_qk; p.tv = d->tok_stride_v; p.tg = d->tok_stride_g;
+    p.bqk = d->batch_stride_qk; p.bv = d->batch_stride_v; p.bg = d->batch_stride_g;
+    return p;
+}
+
+size_t chunked_ws_bytes(const sf_seg_desc_t* d, bool backward) {
+    return (size_t)d->B * d->H * sf::gdn::ws_floats(chunked_params(d), backward) * sizeof(float);
+}
+
+template <typename K>
+bool opt_in(K kern, size_t bytes) {
+    if (bytes <= 48 * 1024) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) { cudaGetLastError(); return false; }
+    return true;
+}
+
+// Pre + ST (+ Out when o != NULL); the backward calls it with o == NULL to rebuild W and the chunk states.
+template <typename T>
+sf_status_t chunked_forward(const sf_seg_desc_t* d, const sf::gdn::Params& p, const void* q, const void* k, const void* v,
+                            const float* g, const float* beta, const float* S_in, void* o, float* S_out, float* ws, int backward,
+                            cudaStream_t st) {
+    using namespace sf::gdn;
+    const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v);
+    const dim3 chunks(p.NC, p.H, p.B), cols(p.dv / DVS, p.H, p.B);
+    const size_t s1 = smem_pre(p.C, p.dk, p.dv), s2 = smem_state(p.C, p.dk), s3 = smem_out(p.C, p.dk, p.dv);
+    if (!opt_in(pre_kernel<T>, s1) || !opt_in(state_kernel<T>, s2) || !opt_in(out_kernel<T>, s3)) return SF_ERR_CUDA;
+    pre_kernel<T><<<chunks, NT, s1, st>>>(p, tk, tv, g, beta, ws, backward);
+    state_kernel<T><<<cols, NT, s2, st>>>(p, tk, g, S_in, S_out, ws, backward);
+    int n = 2;
+    if (o) { out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, g, static_cast<T*>(o), ws, backward); ++n; }
+    return launched(n);
+}
+
+template <typename T>
+sf_status_t chunked_backward(const sf_seg_desc_t* d, const sf::gdn::Params& p, const void* q, const void* k, const void* v,
+                             const float* g, const float* beta, const float* S_in, const void* dO, const float* dS_out, void* dq,
+                             void* dk, void* dv, float* dg, float* dbeta, float* dS_in, float* ws, cudaStream_t st) {
+    using namespace sf::gdn;
+    const sf_status_t f = chunked_forward<T>(d, p, q, k, v, g, beta, S_in, nullptr, nullptr, ws, 1, st);
+    if (f != SF_OK) return f;
+    const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v), *tdo = static_cast<const T*>(dO);
+    const dim3 chunks(p.NC, p.H, p.B), cols(p.dv / DVS, p.H, p.B);
+    const size_t s1 = smem_bwd_state(p.C, p.dk), s2 = smem_bwd_out(p.C, p.dk, p.dv);
+    if (!opt_in(bwd_state_kernel<T>, s1) || !opt_in(bwd_out_kernel<T>, s2)) return SF_ERR_CUDA;
+    bwd_state_kernel<T><<<cols, NT, s1, st>>>(p, tq, tk, g, beta, tdo, dS_out, dS_in, ws);
+    bwd_out_kernel<T><<<chunks, NT, s2, st>>>(p, tq, tk, tv, g, beta, tdo, static_cast<T*>(dq), static_cast<T*>(dk), static_cast<T*>(dv),
+                                              dg, dbeta, ws);
+    return launched(2);
+}
+
 }  // namespace
 
 extern "C" {
@@ -151,6 +216,40 @@ sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const
                                  sf_stream_t stream) {
     return rec_bwd<sf::rec::DELTA>(desc, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, workspace,
                                    workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+size_t sf_delta_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward) {
+    return check_chunked(desc) == SF_OK ? chunked_ws_bytes(desc, backward != 0) : 0;
+}
+
+sf_status_t sf_delta_chunked_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                 const float* beta, const float* S_in, void* o, float* S_out, void* workspace, size_t workspace_bytes,
+                                 sf_stream_t stream) {
+    const sf_status_t c = check_chunked(desc);
+    if (c != SF_OK) return c;
+    if (!q || !k || !v || !g || !beta || !o || !S_out || S_in == S_out) return SF_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < chunked_ws_bytes(desc, false) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SF_ERR_WORKSPACE;
+    const sf::gdn::Params p = chunked_params(desc);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    float* ws = static_cast<float*>(workspace);
+    return desc->dtype == SF_F32 ? chunked_forward<float>(desc, p, q, k, v, g, beta, S_in, o, S_out, ws, 0, st)
+                                 : chunked_forward<__nv_bfloat16>(desc, p, q, k, v, g, beta, S_in, o, S_out, ws, 0, st);
+}
+
+sf_status_t sf_delta_chunked_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                 const float* beta, const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk,
+                                 void* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
+                                 sf_stream_t stream) {
+    const sf_status_t c = check_chunked(desc);
+    if (c != SF_OK) return c;
+    if (!q || !k || !v || !g || !beta || !dO || !dq || !dk || !dv || !dg || !dbeta || !dS_in || dS_in == dS_out) return SF_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < chunked_ws_bytes(desc, true) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SF_ERR_WORKSPACE;
+    const sf::gdn::Params p = chunked_params(desc);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    float* ws = static_cast<float*>(workspace);
+    return desc->dtype == SF_F32
+        ? chunked_backward<float>(desc, p, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, ws, st)
+        : chunked_backward<__nv_bfloat16>(desc, p, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, ws, st);
 }
 
 sf_status_t sf_conv_segment_fwd(int32_t B, int32_t L, int32_t C, int32_t W, const float* x, const float* w, const float* tail_in,

@@ -40,6 +40,9 @@ def run_recurrent(kind, w, x):
         S_out = torch.empty(B, H, dk, dv, device=DEV)
         if kind == "channel":
             binding.sf_channel_segment_fwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], S[-1], o[:, a:b], S_out)
+        elif kind == "delta_chunked":
+            ws = torch.empty(binding.sf_delta_chunked_workspace_bytes(d, 0), dtype=torch.uint8, device=DEV)
+            binding.sf_delta_chunked_fwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], beta[:, a:b], S[-1], o[:, a:b], S_out, ws)
         else:
             binding.sf_delta_segment_fwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], beta[:, a:b], S[-1], o[:, a:b], S_out)
         S.append(S_out)
@@ -47,9 +50,13 @@ def run_recurrent(kind, w, x):
     for i in range(len(segs) - 1, -1, -1):
         a, b = segs[i]
         d = binding.make_desc(q[:, a:b], v[:, a:b], x["g"][:, a:b], w.chunk)
-        ws = torch.empty(binding.sf_recurrent_workspace_bytes(d), dtype=torch.uint8, device=DEV)
+        nws = binding.sf_delta_chunked_workspace_bytes(d, 1) if kind == "delta_chunked" else binding.sf_recurrent_workspace_bytes(d)
+        ws = torch.empty(nws, dtype=torch.uint8, device=DEV)
         dS_in = torch.empty(B, H, dk, dv, device=DEV)
-        if kind == "channel":
+        if kind == "delta_chunked":
+            binding.sf_delta_chunked_bwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], beta[:, a:b], S[i], dO[:, a:b], G,
+                                         dq[:, a:b], dk_[:, a:b], dv_[:, a:b], dg[:, a:b], dbeta[:, a:b], dS_in, ws)
+        elif kind == "channel":
             binding.sf_channel_segment_bwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], S[i], dO[:, a:b], G,
                                            dq[:, a:b], dk_[:, a:b], dv_[:, a:b], dg[:, a:b], dS_in, ws)
         else:
@@ -58,7 +65,7 @@ def run_recurrent(kind, w, x):
         G = dS_in
     torch.cuda.synchronize()
     out = dict(o=o, S_out=S[-1], dq=dq, dk=dk_, dv=dv_, dg=dg, dS_in=G)
-    if kind == "delta":
+    if kind != "channel":
         out["dbeta"] = dbeta
     return out
 
@@ -71,7 +78,7 @@ def oracle_recurrent(kind, x):
         o, S_out = V.channel_fwd(q, k, v, g, S_in)
         dq, dk, dv, dg, dS_in = V.channel_bwd(q, k, v, g, S_in, dO, dS_out)
         return dict(o=o, S_out=S_out, dq=dq, dk=dk, dv=dv, dg=dg, dS_in=dS_in)
-    g, beta = f64(x["g"]), f64(x["beta"])
+    g, beta = f64(x["g"]), f64(x["beta"])                 # "delta" and "delta_chunked": the same operator
     o, S_out = V.delta_fwd(q, k, v, g, beta, S_in)
     dq, dk, dv, dg, dbeta, dS_in = V.delta_bwd(q, k, v, g, beta, S_in, dO, dS_out)
     return dict(o=o, S_out=S_out, dq=dq, dk=dk, dv=dv, dg=dg, dbeta=dbeta, dS_in=dS_in)
@@ -187,3 +194,40 @@ def test_launches_are_counted():
     n0 = binding.sf_launch_count()
     run_recurrent("delta", w, x)
     assert binding.sf_launch_count() - n0 == 2
+
+
+# ---- chunkwise (UT transform) form of the delta rule: same operator, same oracle -------------------------------------
+
+@pytest.mark.parametrize("chunk", [16, 32])
+@pytest.mark.parametrize("dk,dv", [(32, 32), (64, 64), (32, 64), (64, 32)])
+def test_chunked_delta_rule_matches_the_oracle(chunk, dk, dv):
+    # segments of several chunks with a ragged last one, exactly one chunk, shorter than a chunk, one token
+    w = Workload("chunked-%d-%d-%d" % (chunk, dk, dv), 2, 3, dk, dv, [3 * chunk + 5, chunk, 100, 5, 1], chunk, dtype="f32",
+                 qk_norm="l2", g_scale=0.3, s_in_sigma=0.5, ds_out_sigma=0.5, seed=31)
+    x = inputs.make_variant_inputs(w, DEV)
+    check(run_recurrent("delta_chunked", w, x), oracle_recurrent("delta", x), w.name)
+
+
+@pytest.mark.parametrize("g_scale", [1.0, 0.01, 0.0])
+def test_chunked_delta_rule_decay_regimes_and_absent_boundary_states(g_scale):
+    w = Workload("chunked-g%g" % g_scale, 1, 2, 64, 64, [64, 200], 32, dtype="f32", qk_norm="l2", g_scale=g_scale, seed=32)
+    x = inputs.make_variant_inputs(w, DEV)
+    check(run_recurrent("delta_chunked", w, x), oracle_recurrent("delta", x), w.name)
+
+
+def test_chunked_delta_rule_long_segment_bf16_and_agreement_with_the_token_kernel():
+    w = Workload("chunked-long", 1, 4, 64, 64, [2048], 32, dtype="f32", qk_norm="l2", g_scale=0.1, s_in_sigma=0.3,
+                 ds_out_sigma=0.3, seed=33)
+    x = inputs.make_variant_inputs(w, DEV)
+    a = run_recurrent("delta_chunked", w, x)
+    b = run_recurrent("delta_chunked", w, x)
+    for n in a:
+        assert torch.equal(a[n], b[n]), n                      # deterministic
+    check(a, oracle_recurrent("delta", x), w.name)
+    t = run_recurrent("delta", w, x)                           # the token-recurrent kernel: same operator, other algorithm
+    for n in a:
+        assert norm_err(f64(a[n]), f64(t[n])) <= 2 * TOL, n
+    wb = Workload("chunked-bf16", 2, 3, 64, 32, [37, 16, 100, 5, 1], 16, dtype="bf16", qk_norm="l2", g_scale=0.3, s_in_sigma=0.5,
+                  ds_out_sigma=0.5, seed=34)
+    xb = inputs.make_variant_inputs(wb, DEV)
+    check(run_recurrent("delta_chunked", wb, xb), oracle_recurrent("delta", xb), wb.name, tol=2e-2)

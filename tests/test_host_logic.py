@@ -227,3 +227,23 @@ def test_extension_operators_validate_before_any_launch(lib):
     assert conv(L=0) == 1 and conv(W=0) == 1 and conv(W=9) == 2 and conv(x=None) == 1 and conv(tail_out=None) == 1
     assert lib.sf_conv_segment_bwd(1, 8, 4, 4, P, P, None, P, S1, P, P, S1, None) == 1       # dtail_out aliases dtail_in
     assert lib.sf_conv_segment_bwd(1, 8, 4, 4, P, P, None, None, None, P, P, S1, None) == 1  # dy missing
+
+
+def test_chunked_delta_rule_validates_before_any_launch(lib):
+    f32 = dict(dtype=binding.SF_F32, d_k=64, d_v=64, seg_len=100, chunk=32)
+    d = desc(**f32)
+    lib.sf_delta_chunked_workspace_bytes.restype = ctypes.c_size_t
+    per_bh_fwd = 100 * 64 + 100 * 64 + 4 * 64 * 64                 # U/W, Wk per token, one state per chunk (4 chunks)
+    assert lib.sf_delta_chunked_workspace_bytes(ctypes.byref(d), 0) == 2 * per_bh_fwd * 4
+    assert lib.sf_delta_chunked_workspace_bytes(ctypes.byref(d), 1) == 2 * (per_bh_fwd + 100 * 64 + 4 * 64 * 64) * 4
+    S1, S2, W = ctypes.c_void_p(0x20000), ctypes.c_void_p(0x30000), ctypes.c_void_p(0x40000)
+    cf = lambda dd, q=P, beta=P, S_in=None, ws=W, n=1 << 40: lib.sf_delta_chunked_fwd(ctypes.byref(dd), q, P, P, P, beta, S_in, P, S1, ws, n, None)
+    assert cf(d, q=None) == 1 and cf(d, beta=None) == 1 and cf(d, S_in=S1) == 1
+    assert cf(d, ws=None) == 3 and cf(d, n=16) == 3 and cf(d, ws=ctypes.c_void_p(0x40010)) == 3
+    assert cf(desc(**dict(f32, chunk=64))) == 2 and cf(desc(**dict(f32, d_v=128))) == 2 and cf(desc(**dict(f32, d_k=128))) == 2
+    assert cf(desc(**dict(f32, chunk=0))) == 1 and cf(desc(**dict(f32, seg_len=0))) == 1
+    bargs = [P] * 5 + [None, P, None] + [P] * 5 + [S2]
+    assert lib.sf_delta_chunked_bwd(ctypes.byref(d), *bargs, W, 16, None) == 3
+    bad = list(bargs)
+    bad[12] = None                                                  # dbeta missing
+    assert lib.sf_delta_chunked_bwd(ctypes.byref(d), *bad, W, 1 << 40, None) == 1

@@ -230,3 +230,74 @@ def test_conv_gradients_match_central_differences_and_split():
         np.testing.assert_allclose(np.concatenate([dx1, dx2], 1), grads["x"], rtol=1e-12, atol=1e-13)
         np.testing.assert_allclose(dw1 + dw2, grads["w"], rtol=1e-12, atol=1e-13)
         np.testing.assert_allclose(dt0, grads["tail"], rtol=1e-12, atol=1e-13)
+
+
+# ---- the chunkwise (UT transform) form of the delta rule, written out in numpy: a second algorithm for the same operator ----
+
+def _chunk_fwd(Q, K, Vv, g, beta, H):
+    C = Q.shape[0]
+    b = np.cumsum(g)
+    gam = np.exp(b)
+    M = np.tril(np.exp(b[:, None] - b[None, :]))
+    Ms = np.tril(M, -1)
+    Kk = K @ K.T
+    KH = K @ H
+    # (I + L) W = beta*V - beta*gam*(K H),  L = diag(beta) (Ms * K K^T): the tokens of a chunk solved together
+    W = np.linalg.solve(np.eye(C) + beta[:, None] * (Ms * Kk), beta[:, None] * Vv - (beta * gam)[:, None] * KH)
+    QK = Q @ K.T
+    A = M * QK
+    om = np.exp(b[-1] - b)
+    O = A @ W + gam[:, None] * (Q @ H)
+    Hn = gam[-1] * H + K.T @ (om[:, None] * W)
+    return O, Hn, dict(b=b, gam=gam, M=M, Ms=Ms, Kk=Kk, KH=KH, W=W, QK=QK, A=A, om=om, H=H)
+
+
+def _chunk_bwd(Q, K, Vv, beta, c, dO, dHn):
+    C = Q.shape[0]
+    b, gam, M, Ms, Kk, KH, W, QK, A, om, H = (c[n] for n in ("b", "gam", "M", "Ms", "Kk", "KH", "W", "QK", "A", "om", "H"))
+    KdH = K @ dHn
+    dW = A.T @ dO + om[:, None] * KdH
+    dA = dO @ W.T
+    dQK = dA * M
+    Z = np.linalg.solve((np.eye(C) + beta[:, None] * (Ms * Kk)).T, dW)
+    dL = -np.tril(Z @ W.T, -1)
+    bgZ = (beta * gam)[:, None] * Z
+    P = beta[:, None] * dL * Ms
+    dQ = dQK @ K + gam[:, None] * (dO @ H.T)
+    dK = dQK.T @ Q + om[:, None] * (W @ dHn.T) - bgZ @ H.T + P @ K + P.T @ K
+    dV = beta[:, None] * Z
+    dbeta = np.sum(Z * Vv, axis=1) - gam * np.sum(Z * KH, axis=1) + np.sum(dL * Ms * Kk, axis=1)
+    dH = gam[-1] * dHn + Q.T @ (gam[:, None] * dO) - K.T @ bgZ
+    dgam = np.sum(dO * (Q @ H), axis=1) - beta * np.sum(Z * KH, axis=1)
+    dom = np.sum(W * KdH, axis=1)
+    E = (dA * QK * np.tril(np.ones((C, C))) + beta[:, None] * dL * Kk) * M
+    db = E.sum(axis=1) - E.sum(axis=0) + dgam * gam - dom * om
+    db[-1] += np.sum(dom * om) + np.sum(dHn * H) * gam[-1]
+    return dQ, dK, dV, np.cumsum(db[::-1])[::-1], dbeta, dH
+
+
+@pytest.mark.parametrize("T,C,dk,dv", [(50, 16, 5, 4), (64, 64, 8, 8), (33, 32, 3, 6)])
+def test_delta_oracle_equals_the_chunkwise_ut_form(T, C, dk, dv):
+    # Eq. 2 with V_new: Pre / ST / Out per chunk and their adjoints, against the token-by-token oracle (forward and backward)
+    q, k, v, g, beta, S = make(56, T=T, H=1, dk=dk, dv=dv)
+    k /= np.linalg.norm(k, axis=-1, keepdims=True)
+    dO, dS = rnd(80, *v.shape), rnd(81, *S.shape)
+    o_ref, S_ref = V.delta_fwd(q, k, v, g, beta, S)
+    ref = V.delta_bwd(q, k, v, g, beta, S, dO, dS)
+    sl = [slice(t0, min(T, t0 + C)) for t0 in range(0, T, C)]
+    H, caches, o = S[0, 0].copy(), [], np.zeros((T, dv))
+    for s in sl:
+        o[s], H, c = _chunk_fwd(q[0, s, 0], k[0, s, 0], v[0, s, 0], g[0, s, 0], beta[0, s, 0], H)
+        caches.append(c)
+    np.testing.assert_allclose(o, o_ref[0, :, 0], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(H, S_ref[0, 0], rtol=1e-11, atol=1e-12)
+    dH = dS[0, 0].copy()
+    got = [np.zeros((T, dk)), np.zeros((T, dk)), np.zeros((T, dv)), np.zeros(T), np.zeros(T)]
+    for s, c in zip(sl[::-1], caches[::-1]):
+        res = _chunk_bwd(q[0, s, 0], k[0, s, 0], v[0, s, 0], beta[0, s, 0], c, dO[0, s, 0], dH)
+        for a, x in zip(got, res[:5]):
+            a[s] = x
+        dH = res[5]
+    for a, r in zip(got, ref[:5]):
+        np.testing.assert_allclose(a, r[0, :, 0], rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(dH, ref[5][0, 0], rtol=1e-9, atol=1e-11)
