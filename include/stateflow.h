@@ -445,8 +445,9 @@ sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const
  * chunks in parallel; the backward mirrors it (transposed solve, reverse state pass, chunk-parallel gradients).
  * Same arguments, layouts and results (to rounding) as sf_delta_segment_fwd/bwd.  desc->chunk in {16, 32},
  * d_k, d_v in {32, 64}, float32 or bf16 storage, float32 arithmetic on CUDA cores.  Workspace:
- * sf_delta_chunked_workspace_bytes(desc, backward) bytes, 256-byte aligned (U/W and Wk per token, one state per chunk;
- * the backward rebuilds them and adds Z per token and one state gradient per chunk).
+ * sf_delta_chunked_workspace_bytes(desc, backward) bytes, 256-byte aligned (U/W, Wk and the cumulative decay per
+ * token, one state per chunk; the backward rebuilds them and adds Z per token, one state gradient and two
+ * chunk x chunk matrices per chunk).
  */
 size_t sf_delta_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward);
 sf_status_t sf_delta_chunked_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,

@@ -6,20 +6,21 @@
 // the chunk, unrolling S_{t-1} = gam_{t-1} H + sum_{s<t} (gam_{t-1}/gam_s) k_s^T w_s gives a unit-lower-triangular system
 //     (I + L) W = beta*V - (beta*gam)*(K H),     L[t,s] = beta_t M[t,s] (k_t . k_s)  for s < t
 // so  W = U - Wk H  with  U = (I+L)^-1 (beta*V),  Wk = (I+L)^-1 (beta*gam*K)   (the UT transform; no inverse is formed:
-// the systems are solved by substitution, one thread per right-hand-side column).  Then
+// the systems are solved by substitution, one thread per right-hand-side column; for the backward the identity is solved
+// along with them, which gives (I+L)^-1 for the transposed solve).  Then
 //     Pre : U, Wk per chunk                       (needs no state: all chunks in parallel)
 //     ST  : W = U - Wk H  (this is V_new),  H' = gam_n H + (om*K)^T W          (sequential over chunks, per value column)
 //     Out : O = (M * Q K^T) W + gam * (Q H)        (all chunks in parallel, from the stored chunk states)
 // Backward (hand-derived; checked against the fp64 oracle, which is pinned by finite differences), dH' = gradient of the
 // state leaving the chunk:
-//     dW = A^T dO + om*(K dH'),  A = M * QK^T;   Z = (I+L)^-T dW   (back substitution);
+//     dW = A^T dO + om*(K dH'),  A = M * QK^T;   Z = (I+L)^-T dW;
 //     dH = gam_n dH' + Q^T (gam*dO) - K^T (beta*gam*Z)                           (sequential, reverse, per value column)
 // and, chunk-parallel from the stored W, Z, H, dH':  dA = dO W^T,  dL = -strict_lower(Z W^T),  P = beta*dL*M,
 //     dq = (dA*M) K + gam*(dO H^T)
 //     dk = (dA*M)^T Q + om*(W dH'^T) - (beta*gam*Z) H^T + (P + P^T) K
 //     dv = beta*Z,    dbeta = rowsum(Z*V) - gam*rowsum(Z*KH) + rowsum(dL * M * KK^T)
 //     db_t (gradient of the cumulative log-decay) collects the M, gam, om terms; dg = reverse cumulative sum of db.
-// Chunk length C <= 64, d_k, d_v in {32, 64}; a last chunk with fewer tokens is handled by row counts.
+// Chunk length 16 or 32, d_k, d_v in {32, 64}; a last chunk with fewer tokens is handled by row counts.
 #pragma once
 #include "sf_common.cuh"
 
@@ -27,18 +28,20 @@ namespace sf {
 namespace gdn {
 
 constexpr int NT = 256;
-constexpr int DVS = 32;            // value columns per CTA in the sequential kernels
+constexpr int DVS = 16;            // value columns per CTA in the sequential kernels
 
 struct Params {
     int B, H, L, C, NC, dk, dv;
     long long tqk, tv, tg, bqk, bv, bg;      // token / batch strides in elements
 };
 
-// Workspace per (batch, head), in floats: U/W [L][dv], Wk [L][dk], Z [L][dv], Hc [NC][dk][dv], dHc [NC][dk][dv]
-struct Ws { float *W, *Wk, *Z, *Hc, *dHc; };
+// Workspace per (batch, head), in floats: U/W [L][dv], Wk [L][dk], b [L] (cumulative log-decay inside each chunk),
+// Hc [NC][dk][dv]; the backward adds Z [L][dv],
+// dHc [NC][dk][dv], A [NC][C][C] (the masked Q K^T) and Ti [NC][C][C] (the inverse of I + L, used transposed).
+struct Ws { float *W, *Wk, *b, *Z, *Hc, *dHc, *A, *Ti; };
 __host__ __device__ inline size_t ws_floats(const Params& p, bool backward) {
-    size_t n = (size_t)p.L * p.dv + (size_t)p.L * p.dk + (size_t)p.NC * p.dk * p.dv;
-    if (backward) n += (size_t)p.L * p.dv + (size_t)p.NC * p.dk * p.dv;
+    size_t n = (size_t)p.L * p.dv + (size_t)p.L * p.dk + (size_t)p.L + (size_t)p.NC * p.dk * p.dv;
+    if (backward) n += (size_t)p.L * p.dv + (size_t)p.NC * p.dk * p.dv + 2 * (size_t)p.NC * p.C * p.C;
     return n;
 }
 __host__ __device__ inline Ws ws_of(float* base, const Params& p, long long bh, bool backward) {
@@ -46,20 +49,33 @@ __host__ __device__ inline Ws ws_of(float* base, const Params& p, long long bh, 
     Ws w;
     w.W = c;  c += (size_t)p.L * p.dv;
     w.Wk = c; c += (size_t)p.L * p.dk;
+    w.b = c;  c += (size_t)p.L;
     w.Hc = c; c += (size_t)p.NC * p.dk * p.dv;
-    w.Z = backward ? c : nullptr; if (backward) c += (size_t)p.L * p.dv;
-    w.dHc = backward ? c : nullptr;
+    w.Z = w.dHc = w.A = w.Ti = nullptr;
+    if (backward) {
+        w.Z = c;   c += (size_t)p.L * p.dv;
+        w.dHc = c; c += (size_t)p.NC * p.dk * p.dv;
+        w.A = c;   c += (size_t)p.NC * p.C * p.C;
+        w.Ti = c;
+    }
     return w;
 }
+
+// Shared-memory tiles are stored with an odd leading dimension (columns + 1), so that both row-wise and column-wise
+// walks hit different banks.
+__host__ __device__ constexpr int ldp(int cols) { return cols + 1; }
 
 // out[m][n] = keep*out[m][n] + sign * sum_k A(m,k) B(k,n);  A(m,k) = ta ? A[k*lda+m] : A[m*lda+k], likewise B.
 __device__ __forceinline__ void mm(float* out, int ldo, const float* A, int lda, bool ta, const float* Bm, int ldb, bool tb,
                                    int M, int N, int K, float keep, float sign) {
     for (int idx = threadIdx.x; idx < M * N; idx += NT) {
         const int m = idx / N, n = idx - m * N;
+        const float* a = ta ? A + m : A + m * lda;
+        const float* bq = tb ? Bm + n * ldb : Bm + n;
+        const int sa = ta ? lda : 1, sb = tb ? 1 : ldb;
         float acc = 0.f;
-        for (int k = 0; k < K; ++k)
-            acc = fmaf(ta ? A[k * lda + m] : A[m * lda + k], tb ? Bm[n * ldb + k] : Bm[k * ldb + n], acc);
+#pragma unroll 4
+        for (int k = 0; k < K; ++k) acc = fmaf(a[k * sa], bq[k * sb], acc);
         out[m * ldo + n] = keep != 0.f ? fmaf(keep, out[m * ldo + n], sign * acc) : sign * acc;
     }
 }
@@ -71,8 +87,21 @@ __device__ __forceinline__ void load_rows(float* dst, int ld, const T* src, long
         dst[r * ld + c] = to_f32(src[(long long)r * tok_stride + c]);
     }
 }
+// dense [rows][cols] float block in global memory <-> padded tile
+__device__ __forceinline__ void load_dense(float* dst, int ld, const float* src, int src_ld, int rows, int cols) {
+    for (int idx = threadIdx.x; idx < rows * cols; idx += NT) {
+        const int r = idx / cols, c = idx - r * cols;
+        dst[r * ld + c] = src[(long long)r * src_ld + c];
+    }
+}
+__device__ __forceinline__ void store_dense(float* dst, int dst_ld, const float* src, int ld, int rows, int cols) {
+    for (int idx = threadIdx.x; idx < rows * cols; idx += NT) {
+        const int r = idx / cols, c = idx - r * cols;
+        dst[(long long)r * dst_ld + c] = src[r * ld + c];
+    }
+}
 
-// b[t] = inclusive cumulative log-decay of the chunk's n tokens, beta[t]; one thread, n <= 64.  Syncs.
+// b[t] = inclusive cumulative log-decay of the chunk's n tokens (one thread), bt[t] = beta.  Syncs.
 __device__ __forceinline__ void load_decay(float* b, float* bt, const float* g, const float* beta, long long tg, int n) {
     if (threadIdx.x == 0) {
         float acc = 0.f;
@@ -81,53 +110,71 @@ __device__ __forceinline__ void load_decay(float* b, float* bt, const float* g, 
     if (bt) for (int t = threadIdx.x; t < n; t += NT) bt[t] = beta[(long long)t * tg];
     __syncthreads();
 }
-
-// Lm[t][s] = beta_t exp(b_t - b_s) (k_t . k_s) for s < t, 0 elsewhere.  Kk may alias Lm.
-__device__ __forceinline__ void build_L(float* Lm, const float* Ks, const float* b, const float* bt, int n, int C, int dk) {
-    mm(Lm, C, Ks, dk, false, Ks, dk, true, n, n, dk, 0.f, 1.f);
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < n * n; idx += NT) {
-        const int t = idx / n, s = idx - t * n;
-        Lm[t * C + s] = s < t ? bt[t] * __expf(b[t] - b[s]) * Lm[t * C + s] : 0.f;
+// The sequential kernels take the cumulative log-decay from the workspace, where Pre has left it.  Syncs.
+__device__ __forceinline__ void load_decay_ws(float* b, float* bt, const float* bws, const float* beta, long long tg, int n) {
+    for (int t = threadIdx.x; t < n; t += NT) {
+        b[t] = bws[t];
+        if (bt) bt[t] = beta[(long long)t * tg];
     }
     __syncthreads();
 }
 
-// ---- Pre: U = (I+L)^-1 (beta*V), Wk = (I+L)^-1 (beta*gam*K).  grid (NC, H, B) --------------------------------
+// ---- Pre: U = (I+L)^-1 (beta*V), Wk = (I+L)^-1 (beta*gam*K); for the backward also Ti = (I+L)^-1 and A = M * Q K^T.
+//      grid (NC, H, B) -----------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__ k, const T* __restrict__ v,
+__global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                                                  const float* __restrict__ g, const float* __restrict__ beta, float* ws, int backward) {
     extern __shared__ float sm[];
     const int c = blockIdx.x, h = blockIdx.y, bb = blockIdx.z;
     const int C = p.C, dk = p.dk, dv = p.dv, t0 = c * C, n = min(C, p.L - t0);
+    const int ldk = ldp(dk), ldc = ldp(C), ncol = dv + dk + (backward ? C : 0), ldx = ldp(dv + dk + C);
     float* Ks = sm;                    // [C][dk]
-    float* X = Ks + C * dk;            // [C][dv + dk]   right-hand sides, solved in place
-    float* Lm = X + C * (dv + dk);     // [C][C]
-    float* b = Lm + C * C;             // [C]
+    float* X = Ks + C * ldk;           // [C][dv + dk (+ C)]   right-hand sides, solved in place
+    float* Lm = X + C * ldx;           // [C][C]
+    float* Qs = Lm + C * ldc;          // [C][dk]   (backward only)
+    float* b = Qs + C * ldk;           // [C]
     float* bt = b + C;                 // [C]
-    const int ldx = dv + dk;
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(ws, p, bh, backward != 0);
-    load_rows(Ks, dk, k + (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk, p.tqk, n, dk);
+    const long long oqk = (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk;
+    load_rows(Ks, ldk, k + oqk, p.tqk, n, dk);
+    if (backward) load_rows(Qs, ldk, q + oqk, p.tqk, n, dk);
     load_rows(X, ldx, v + (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv, p.tv, n, dv);
     load_decay(b, bt, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, beta + (long long)bb * p.bg + (long long)t0 * p.tg + h, p.tg, n);
-    for (int idx = threadIdx.x; idx < n * ldx; idx += NT) {
-        const int t = idx / ldx, col = idx - t * ldx;
-        X[idx] = col < dv ? bt[t] * X[idx] : bt[t] * __expf(b[t]) * Ks[t * dk + (col - dv)];
+    for (int idx = threadIdx.x; idx < n * ncol; idx += NT) {
+        const int t = idx / ncol, col = idx - t * ncol;
+        float x;
+        if (col < dv) x = bt[t] * X[t * ldx + col];
+        else if (col < dv + dk) x = bt[t] * __expf(b[t]) * Ks[t * ldk + (col - dv)];
+        else x = (col - dv - dk) == t ? 1.f : 0.f;                      // identity: its solution is the inverse
+        X[t * ldx + col] = x;
     }
-    build_L(Lm, Ks, b, bt, n, C, dk);
+    mm(Lm, ldc, Ks, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);     // K K^T
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < n * n; idx += NT) {
+        const int t = idx / n, s = idx - t * n;
+        Lm[t * ldc + s] = s < t ? bt[t] * __expf(b[t] - b[s]) * Lm[t * ldc + s] : 0.f;
+    }
+    __syncthreads();
     // forward substitution, one thread per column
-    for (int col = threadIdx.x; col < ldx; col += NT)
+    for (int col = threadIdx.x; col < ncol; col += NT)
         for (int t = 1; t < n; ++t) {
             float acc = X[t * ldx + col];
-            for (int s = 0; s < t; ++s) acc = fmaf(-Lm[t * C + s], X[s * ldx + col], acc);
+            for (int s = 0; s < t; ++s) acc = fmaf(-Lm[t * ldc + s], X[s * ldx + col], acc);
             X[t * ldx + col] = acc;
         }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < n * ldx; idx += NT) {
-        const int t = idx / ldx, col = idx - t * ldx;
-        if (col < dv) w.W[(long long)(t0 + t) * dv + col] = X[idx];
-        else w.Wk[(long long)(t0 + t) * dk + (col - dv)] = X[idx];
+    store_dense(w.W + (long long)t0 * dv, dv, X, ldx, n, dv);
+    store_dense(w.Wk + (long long)t0 * dk, dk, X + dv, ldx, n, dk);
+    for (int t = threadIdx.x; t < n; t += NT) w.b[t0 + t] = b[t];
+    if (backward) {
+        store_dense(w.Ti + (long long)c * C * C, C, X + dv + dk, ldx, n, n);
+        mm(Lm, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f); // Q K^T (L is no longer needed)
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < n * n; idx += NT) {
+            const int t = idx / n, s = idx - t * n;
+            w.A[(long long)c * C * C + t * C + s] = s <= t ? Lm[t * ldc + s] * __expf(b[t] - b[s]) : 0.f;
+        }
     }
 }
 
@@ -138,47 +185,36 @@ __global__ void __launch_bounds__(NT) state_kernel(Params p, const T* __restrict
     extern __shared__ float sm[];
     const int j0 = blockIdx.x * DVS, h = blockIdx.y, bb = blockIdx.z;
     const int C = p.C, dk = p.dk, dv = p.dv;
+    const int ldk = ldp(dk), lds = ldp(DVS);
     float* Hs = sm;                    // [dk][DVS]
-    float* Ks = Hs + dk * DVS;         // [C][dk]   (scaled by om in place)
-    float* Wks = Ks + C * dk;          // [C][dk]
-    float* Wc = Wks + C * dk;          // [C][DVS]
-    float* b = Wc + C * DVS;           // [C]
+    float* Ks = Hs + dk * lds;         // [C][dk]   (scaled by om in place)
+    float* Wks = Ks + C * ldk;         // [C][dk]
+    float* Wc = Wks + C * ldk;         // [C][DVS]
+    float* b = Wc + C * lds;           // [C]
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(ws, p, bh, backward != 0);
-    for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) {
-        const int i = idx / DVS, jj = idx - i * DVS;
-        Hs[idx] = S_in ? S_in[(bh * dk + i) * dv + j0 + jj] : 0.f;
-    }
+    if (S_in) load_dense(Hs, lds, S_in + bh * dk * dv + j0, dv, dk, DVS);
+    else for (int idx = threadIdx.x; idx < dk * lds; idx += NT) Hs[idx] = 0.f;
     __syncthreads();
     for (int c = 0; c < p.NC; ++c) {
         const int t0 = c * C, n = min(C, p.L - t0);
-        load_rows(Ks, dk, k + (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk, p.tqk, n, dk);
-        for (int idx = threadIdx.x; idx < n * dk; idx += NT) Wks[idx] = w.Wk[(long long)t0 * dk + idx];
-        for (int idx = threadIdx.x; idx < n * DVS; idx += NT) {
-            const int t = idx / DVS, jj = idx - t * DVS;
-            Wc[idx] = w.W[(long long)(t0 + t) * dv + j0 + jj];
-        }
-        for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) {
-            const int i = idx / DVS, jj = idx - i * DVS;
-            w.Hc[((long long)c * dk + i) * dv + j0 + jj] = Hs[idx];
-        }
+        load_rows(Ks, ldk, k + (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk, p.tqk, n, dk);
+        load_dense(Wks, ldk, w.Wk + (long long)t0 * dk, dk, n, dk);
+        load_dense(Wc, lds, w.W + (long long)t0 * dv + j0, dv, n, DVS);
+        store_dense(w.Hc + (long long)c * dk * dv + j0, dv, Hs, lds, dk, DVS);
         load_decay(b, nullptr, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, nullptr, p.tg, n);
-        mm(Wc, DVS, Wks, dk, false, Hs, DVS, false, n, DVS, dk, 1.f, -1.f);        // W = U - Wk H
+        mm(Wc, lds, Wks, ldk, false, Hs, lds, false, n, DVS, dk, 1.f, -1.f);       // W = U - Wk H
         const float bn = b[n - 1];
-        for (int idx = threadIdx.x; idx < n * dk; idx += NT) Ks[idx] *= __expf(bn - b[idx / dk]);
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < n * DVS; idx += NT) {
-            const int t = idx / DVS, jj = idx - t * DVS;
-            w.W[(long long)(t0 + t) * dv + j0 + jj] = Wc[idx];
+        for (int idx = threadIdx.x; idx < n * dk; idx += NT) {
+            const int t = idx / dk;
+            Ks[t * ldk + (idx - t * dk)] *= __expf(bn - b[t]);
         }
-        mm(Hs, DVS, Ks, dk, true, Wc, DVS, false, dk, DVS, n, __expf(bn), 1.f);    // H = gam_n H + (om*K)^T W
+        __syncthreads();
+        store_dense(w.W + (long long)t0 * dv + j0, dv, Wc, lds, n, DVS);
+        mm(Hs, lds, Ks, ldk, true, Wc, lds, false, dk, DVS, n, __expf(bn), 1.f);   // H = gam_n H + (om*K)^T W
         __syncthreads();
     }
-    if (S_out)
-        for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) {
-            const int i = idx / DVS, jj = idx - i * DVS;
-            S_out[(bh * dk + i) * dv + j0 + jj] = Hs[idx];
-        }
+    if (S_out) store_dense(S_out + bh * dk * dv + j0, dv, Hs, lds, dk, DVS);
 }
 
 // ---- Out: O = (M * Q K^T) W + gam * (Q Hc).  grid (NC, H, B) ------------------------------------------------------
@@ -188,39 +224,44 @@ __global__ void __launch_bounds__(NT) out_kernel(Params p, const T* __restrict__
     extern __shared__ float sm[];
     const int c = blockIdx.x, h = blockIdx.y, bb = blockIdx.z;
     const int C = p.C, dk = p.dk, dv = p.dv, t0 = c * C, n = min(C, p.L - t0);
+    const int ldk = ldp(dk), ldv = ldp(dv), ldc = ldp(C);
     float* Qs = sm;                    // [C][dk]
-    float* Ks = Qs + C * dk;           // [C][dk]
-    float* Wc = Ks + C * dk;           // [C][dv]
-    float* Hs = Wc + C * dv;           // [dk][dv]
-    float* A = Hs + dk * dv;           // [C][C]
-    float* O = A + C * C;              // [C][dv]
-    float* b = O + C * dv;             // [C]
+    float* Ks = Qs + C * ldk;          // [C][dk]
+    float* Wc = Ks + C * ldk;          // [C][dv]
+    float* Hs = Wc + C * ldv;          // [dk][dv]
+    float* A = Hs + dk * ldv;          // [C][C]
+    float* O = A + C * ldc;            // [C][dv]
+    float* b = O + C * ldv;            // [C]
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(const_cast<float*>(ws), p, bh, backward != 0);
-    load_rows(Qs, dk, q + (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk, p.tqk, n, dk);
-    load_rows(Ks, dk, k + (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk, p.tqk, n, dk);
-    for (int idx = threadIdx.x; idx < n * dv; idx += NT) Wc[idx] = w.W[(long long)t0 * dv + idx];
-    for (int idx = threadIdx.x; idx < dk * dv; idx += NT) Hs[idx] = w.Hc[(long long)c * dk * dv + idx];
+    const long long oqk = (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk;
+    load_rows(Qs, ldk, q + oqk, p.tqk, n, dk);
+    load_rows(Ks, ldk, k + oqk, p.tqk, n, dk);
+    load_dense(Wc, ldv, w.W + (long long)t0 * dv, dv, n, dv);
+    load_dense(Hs, ldv, w.Hc + (long long)c * dk * dv, dv, dk, dv);
     load_decay(b, nullptr, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, nullptr, p.tg, n);
-    mm(A, C, Qs, dk, false, Ks, dk, true, n, n, dk, 0.f, 1.f);
-    mm(O, dv, Qs, dk, false, Hs, dv, false, n, dv, dk, 0.f, 1.f);
+    mm(A, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
+    mm(O, ldv, Qs, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
     __syncthreads();
     for (int idx = threadIdx.x; idx < n * n; idx += NT) {
         const int t = idx / n, s = idx - t * n;
-        A[t * C + s] = s <= t ? A[t * C + s] * __expf(b[t] - b[s]) : 0.f;
+        A[t * ldc + s] = s <= t ? A[t * ldc + s] * __expf(b[t] - b[s]) : 0.f;
     }
-    for (int idx = threadIdx.x; idx < n * dv; idx += NT) O[idx] *= __expf(b[idx / dv]);
+    for (int idx = threadIdx.x; idx < n * dv; idx += NT) {
+        const int t = idx / dv;
+        O[t * ldv + (idx - t * dv)] *= __expf(b[t]);
+    }
     __syncthreads();
-    mm(O, dv, A, C, false, Wc, dv, false, n, dv, n, 1.f, 1.f);
+    mm(O, ldv, A, ldc, false, Wc, ldv, false, n, dv, n, 1.f, 1.f);
     __syncthreads();
     T* oh = o + (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv;
     for (int idx = threadIdx.x; idx < n * dv; idx += NT) {
         const int t = idx / dv, jj = idx - t * dv;
-        oh[(long long)t * p.tv + jj] = from_f32<T>(O[idx]);
+        oh[(long long)t * p.tv + jj] = from_f32<T>(O[t * ldv + jj]);
     }
 }
 
-// ---- backward, sequential part (reverse over chunks): dHc[c] = dH';  dW = A^T dO + om*(K dH');  Z = (I+L)^-T dW;
+// ---- backward, sequential part (reverse over chunks): dHc[c] = dH';  dW = A^T dO + om*(K dH');  Z = Ti^T dW;
 //      dH = gam_n dH' + Q^T (gam*dO) - K^T (beta*gam*Z).  grid (dv/DVS, H, B) -------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(NT) bwd_state_kernel(Params p, const T* __restrict__ q, const T* __restrict__ k,
@@ -230,71 +271,63 @@ __global__ void __launch_bounds__(NT) bwd_state_kernel(Params p, const T* __rest
     extern __shared__ float sm[];
     const int j0 = blockIdx.x * DVS, h = blockIdx.y, bb = blockIdx.z;
     const int C = p.C, dk = p.dk, dv = p.dv;
+    const int ldk = ldp(dk), ldc = ldp(C), lds = ldp(DVS);
     float* G = sm;                     // [dk][DVS]  carried state gradient
-    float* G2 = G + dk * DVS;          // [dk][DVS]
-    float* Qs = G2 + dk * DVS;         // [C][dk]
-    float* Ks = Qs + C * dk;           // [C][dk]
-    float* A = Ks + C * dk;            // [C][C]
-    float* Lm = A + C * C;             // [C][C]
-    float* dOs = Lm + C * C;           // [C][DVS]
-    float* Zs = dOs + C * DVS;         // [C][DVS]   dW, then Z
-    float* b = Zs + C * DVS;           // [C]
+    float* G2 = G + dk * lds;          // [dk][DVS]
+    float* Qs = G2 + dk * lds;         // [C][dk]
+    float* Ks = Qs + C * ldk;          // [C][dk]
+    float* A = Ks + C * ldk;           // [C][C]
+    float* Ti = A + C * ldc;           // [C][C]
+    float* dOs = Ti + C * ldc;         // [C][DVS]
+    float* dWs = dOs + C * lds;        // [C][DVS]
+    float* Zs = dWs + C * lds;         // [C][DVS]
+    float* b = Zs + C * lds;           // [C]
     float* bt = b + C;                 // [C]
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(ws, p, bh, true);
-    for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) {
-        const int i = idx / DVS, jj = idx - i * DVS;
-        G[idx] = dS_out ? dS_out[(bh * dk + i) * dv + j0 + jj] : 0.f;
-    }
+    if (dS_out) load_dense(G, lds, dS_out + bh * dk * dv + j0, dv, dk, DVS);
+    else for (int idx = threadIdx.x; idx < dk * lds; idx += NT) G[idx] = 0.f;
     __syncthreads();
     for (int c = p.NC - 1; c >= 0; --c) {
         const int t0 = c * C, n = min(C, p.L - t0);
-        load_rows(Qs, dk, q + (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk, p.tqk, n, dk);
-        load_rows(Ks, dk, k + (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk, p.tqk, n, dk);
-        load_rows(dOs, DVS, dO + (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv + j0, p.tv, n, DVS);
-        for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) {
-            const int i = idx / DVS, jj = idx - i * DVS;
-            w.dHc[((long long)c * dk + i) * dv + j0 + jj] = G[idx];
-        }
-        load_decay(b, bt, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, beta + (long long)bb * p.bg + (long long)t0 * p.tg + h, p.tg, n);
+        const long long oqk = (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk;
+        load_rows(Qs, ldk, q + oqk, p.tqk, n, dk);
+        load_rows(Ks, ldk, k + oqk, p.tqk, n, dk);
+        load_rows(dOs, lds, dO + (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv + j0, p.tv, n, DVS);
+        load_dense(A, ldc, w.A + (long long)c * C * C, C, n, n);
+        load_dense(Ti, ldc, w.Ti + (long long)c * C * C, C, n, n);
+        store_dense(w.dHc + (long long)c * dk * dv + j0, dv, G, lds, dk, DVS);
+        load_decay_ws(b, bt, w.b + t0, beta + (long long)bb * p.bg + (long long)t0 * p.tg + h, p.tg, n);
         const float bn = b[n - 1];
-        mm(A, C, Qs, dk, false, Ks, dk, true, n, n, dk, 0.f, 1.f);
-        mm(Zs, DVS, Ks, dk, false, G, DVS, false, n, DVS, dk, 0.f, 1.f);            // K dH'
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < n * n; idx += NT) {
-            const int t = idx / n, s = idx - t * n;
-            A[t * C + s] = s <= t ? A[t * C + s] * __expf(b[t] - b[s]) : 0.f;
-        }
-        for (int idx = threadIdx.x; idx < n * DVS; idx += NT) Zs[idx] *= __expf(bn - b[idx / DVS]);
-        __syncthreads();
-        mm(Zs, DVS, A, C, true, dOs, DVS, false, n, DVS, n, 1.f, 1.f);              // dW = A^T dO + om*(K dH')
-        build_L(Lm, Ks, b, bt, n, C, dk);                                           // syncs inside
-        // back substitution with L^T, one thread per column
-        for (int col = threadIdx.x; col < DVS; col += NT)
-            for (int t = n - 2; t >= 0; --t) {
-                float acc = Zs[t * DVS + col];
-                for (int s = t + 1; s < n; ++s) acc = fmaf(-Lm[s * C + t], Zs[s * DVS + col], acc);
-                Zs[t * DVS + col] = acc;
-            }
+        mm(dWs, lds, Ks, ldk, false, G, lds, false, n, DVS, dk, 0.f, 1.f);          // K dH'
         __syncthreads();
         for (int idx = threadIdx.x; idx < n * DVS; idx += NT) {
-            const int t = idx / DVS, jj = idx - t * DVS;
-            w.Z[(long long)(t0 + t) * dv + j0 + jj] = Zs[idx];
-            dOs[idx] *= __expf(b[t]);                                               // gam*dO
-            Zs[idx] *= bt[t] * __expf(b[t]);                                        // beta*gam*Z
+            const int t = idx / DVS;
+            dWs[t * lds + (idx - t * DVS)] *= __expf(bn - b[t]);
         }
         __syncthreads();
-        mm(G2, DVS, Qs, dk, true, dOs, DVS, false, dk, DVS, n, 0.f, 1.f);
+        mm(dWs, lds, A, ldc, true, dOs, lds, false, n, DVS, n, 1.f, 1.f);           // dW = A^T dO + om*(K dH')
         __syncthreads();
-        mm(G2, DVS, Ks, dk, true, Zs, DVS, false, dk, DVS, n, 1.f, -1.f);
+        mm(Zs, lds, Ti, ldc, true, dWs, lds, false, n, DVS, n, 0.f, 1.f);           // Z = (I+L)^-T dW
         __syncthreads();
-        for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) G[idx] = fmaf(__expf(bn), G[idx], G2[idx]);
+        store_dense(w.Z + (long long)t0 * dv + j0, dv, Zs, lds, n, DVS);
+        for (int idx = threadIdx.x; idx < n * DVS; idx += NT) {
+            const int t = idx / DVS, a = t * lds + (idx - t * DVS);
+            dOs[a] *= __expf(b[t]);                                                 // gam*dO
+            Zs[a] *= bt[t] * __expf(b[t]);                                          // beta*gam*Z
+        }
+        __syncthreads();
+        mm(G2, lds, Qs, ldk, true, dOs, lds, false, dk, DVS, n, 0.f, 1.f);
+        __syncthreads();
+        mm(G2, lds, Ks, ldk, true, Zs, lds, false, dk, DVS, n, 1.f, -1.f);
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) {
+            const int i = idx / DVS, a = i * lds + (idx - i * DVS);
+            G[a] = fmaf(__expf(bn), G[a], G2[a]);
+        }
         __syncthreads();
     }
-    for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) {
-        const int i = idx / DVS, jj = idx - i * DVS;
-        dS_in[(bh * dk + i) * dv + j0 + jj] = G[idx];
-    }
+    store_dense(dS_in + bh * dk * dv + j0, dv, G, lds, dk, DVS);
 }
 
 // ---- backward, chunk-parallel part: every input gradient of the chunk from the stored W, Z, Hc, dHc.  grid (NC, H, B) ----
@@ -307,16 +340,17 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
     extern __shared__ float sm[];
     const int c = blockIdx.x, h = blockIdx.y, bb = blockIdx.z;
     const int C = p.C, dk = p.dk, dv = p.dv, t0 = c * C, n = min(C, p.L - t0);
-    float* Qs = sm;                     float* Ks = Qs + C * dk;
-    float* Vs = Ks + C * dk;            float* dOs = Vs + C * dv;
-    float* Wc = dOs + C * dv;           float* Zs = Wc + C * dv;
-    float* Hs = Zs + C * dv;            float* dHs = Hs + dk * dv;
-    float* QK = dHs + dk * dv;          float* KK = QK + C * C;
-    float* DA = KK + C * C;             float* ZW = DA + C * C;
-    float* KH = ZW + C * C;             float* KdH = KH + C * dv;
-    float* dQs = KdH + C * dv;          float* dKs = dQs + C * dk;
-    float* T1 = dKs + C * dk;
-    float* b = T1 + C * dk;             float* bt = b + C;
+    const int ldk = ldp(dk), ldv = ldp(dv), ldc = ldp(C);
+    float* Qs = sm;                     float* Ks = Qs + C * ldk;
+    float* Vs = Ks + C * ldk;           float* dOs = Vs + C * ldv;
+    float* Wc = dOs + C * ldv;          float* Zs = Wc + C * ldv;
+    float* Hs = Zs + C * ldv;           float* dHs = Hs + dk * ldv;
+    float* QK = dHs + dk * ldv;         float* KK = QK + C * ldc;
+    float* DA = KK + C * ldc;           float* ZW = DA + C * ldc;
+    float* KH = ZW + C * ldc;           float* KdH = KH + C * ldv;
+    float* dQs = KdH + C * ldv;         float* dKs = dQs + C * ldk;
+    float* T1 = dKs + C * ldk;
+    float* b = T1 + C * ldk;            float* bt = b + C;
     float* rs = bt + C;                 float* cs = rs + C;
     float* rl = cs + C;                 float* zkh = rl + C;
     float* zv = zkh + C;                float* doqh = zv + C;
@@ -327,35 +361,34 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
     const long long oqk = (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk;
     const long long ov = (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv;
     const long long og = (long long)bb * p.bg + (long long)t0 * p.tg + h;
-    load_rows(Qs, dk, q + oqk, p.tqk, n, dk);
-    load_rows(Ks, dk, k + oqk, p.tqk, n, dk);
-    load_rows(Vs, dv, v + ov, p.tv, n, dv);
-    load_rows(dOs, dv, dO + ov, p.tv, n, dv);
-    for (int idx = threadIdx.x; idx < n * dv; idx += NT) { Wc[idx] = w.W[(long long)t0 * dv + idx]; Zs[idx] = w.Z[(long long)t0 * dv + idx]; }
-    for (int idx = threadIdx.x; idx < dk * dv; idx += NT) {
-        Hs[idx] = w.Hc[(long long)c * dk * dv + idx];
-        dHs[idx] = w.dHc[(long long)c * dk * dv + idx];
-    }
+    load_rows(Qs, ldk, q + oqk, p.tqk, n, dk);
+    load_rows(Ks, ldk, k + oqk, p.tqk, n, dk);
+    load_rows(Vs, ldv, v + ov, p.tv, n, dv);
+    load_rows(dOs, ldv, dO + ov, p.tv, n, dv);
+    load_dense(Wc, ldv, w.W + (long long)t0 * dv, dv, n, dv);
+    load_dense(Zs, ldv, w.Z + (long long)t0 * dv, dv, n, dv);
+    load_dense(Hs, ldv, w.Hc + (long long)c * dk * dv, dv, dk, dv);
+    load_dense(dHs, ldv, w.dHc + (long long)c * dk * dv, dv, dk, dv);
     load_decay(b, bt, g + og, beta + og, p.tg, n);
     const float bn = b[n - 1];
-    mm(QK, C, Qs, dk, false, Ks, dk, true, n, n, dk, 0.f, 1.f);
-    mm(KK, C, Ks, dk, false, Ks, dk, true, n, n, dk, 0.f, 1.f);
-    mm(DA, C, dOs, dv, false, Wc, dv, true, n, n, dv, 0.f, 1.f);            // dA = dO W^T
-    mm(ZW, C, Zs, dv, false, Wc, dv, true, n, n, dv, 0.f, 1.f);             // Z W^T  (dL = -strict lower)
-    mm(KH, dv, Ks, dk, false, Hs, dv, false, n, dv, dk, 0.f, 1.f);
-    mm(KdH, dv, Ks, dk, false, dHs, dv, false, n, dv, dk, 0.f, 1.f);
-    mm(dQs, dk, dOs, dv, false, Hs, dv, true, n, dk, dv, 0.f, 1.f);         // dO H^T
-    mm(dKs, dk, Wc, dv, false, dHs, dv, true, n, dk, dv, 0.f, 1.f);         // W dH'^T
-    mm(T1, dk, Zs, dv, false, Hs, dv, true, n, dk, dv, 0.f, 1.f);           // Z H^T
+    mm(QK, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
+    mm(KK, ldc, Ks, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
+    mm(DA, ldc, dOs, ldv, false, Wc, ldv, true, n, n, dv, 0.f, 1.f);            // dA = dO W^T
+    mm(ZW, ldc, Zs, ldv, false, Wc, ldv, true, n, n, dv, 0.f, 1.f);             // Z W^T  (dL = -strict lower)
+    mm(KH, ldv, Ks, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
+    mm(KdH, ldv, Ks, ldk, false, dHs, ldv, false, n, dv, dk, 0.f, 1.f);
+    mm(dQs, ldk, dOs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);          // dO H^T
+    mm(dKs, ldk, Wc, ldv, false, dHs, ldv, true, n, dk, dv, 0.f, 1.f);          // W dH'^T
+    mm(T1, ldk, Zs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);            // Z H^T
     for (int i = threadIdx.x; i < dk; i += NT) {
         float acc = 0.f;
-        for (int jj = 0; jj < dv; ++jj) acc = fmaf(dHs[i * dv + jj], Hs[i * dv + jj], acc);
+        for (int jj = 0; jj < dv; ++jj) acc = fmaf(dHs[i * ldv + jj], Hs[i * ldv + jj], acc);
         part[i] = acc;
     }
     __syncthreads();
     // C x C pass: DA <- dA*M (s <= t),  ZW <- P = beta_t dL M (s < t),  QK <- E = (dA QK + beta_t dL KK) M,  KK <- dL M KK
     for (int idx = threadIdx.x; idx < n * n; idx += NT) {
-        const int t = idx / n, s = idx - t * n, a = t * C + s;
+        const int t = idx / n, s = idx - t * n, a = t * ldc + s;
         const float m = s <= t ? __expf(b[t] - b[s]) : 0.f;
         const float dl = s < t ? -ZW[a] : 0.f;
         const float da = DA[a], qk = QK[a], kk = KK[a];
@@ -367,13 +400,13 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
     __syncthreads();
     for (int t = threadIdx.x; t < n; t += NT) {
         float r = 0.f, cc = 0.f, l = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f, a4 = 0.f;
-        for (int s = 0; s < n; ++s) { r += QK[t * C + s]; cc += QK[s * C + t]; l += KK[t * C + s]; }
+        for (int s = 0; s < n; ++s) { r += QK[t * ldc + s]; cc += QK[s * ldc + t]; l += KK[t * ldc + s]; }
         for (int jj = 0; jj < dv; ++jj) {
-            a1 = fmaf(Zs[t * dv + jj], KH[t * dv + jj], a1);
-            a2 = fmaf(Zs[t * dv + jj], Vs[t * dv + jj], a2);
-            a4 = fmaf(Wc[t * dv + jj], KdH[t * dv + jj], a4);
+            a1 = fmaf(Zs[t * ldv + jj], KH[t * ldv + jj], a1);
+            a2 = fmaf(Zs[t * ldv + jj], Vs[t * ldv + jj], a2);
+            a4 = fmaf(Wc[t * ldv + jj], KdH[t * ldv + jj], a4);
         }
-        for (int i = 0; i < dk; ++i) a3 = fmaf(Qs[t * dk + i], dQs[t * dk + i], a3);
+        for (int i = 0; i < dk; ++i) a3 = fmaf(Qs[t * ldk + i], dQs[t * ldk + i], a3);
         rs[t] = r; cs[t] = cc; rl[t] = l; zkh[t] = a1; zv[t] = a2; doqh[t] = a3; wkdh[t] = a4;
     }
     __syncthreads();
@@ -394,36 +427,45 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
         dbeta[og + (long long)t * p.tg] = zv[t] - __expf(b[t]) * zkh[t] + rl[t];
     // dq = (dA*M) K + gam*(dO H^T);  dk = om*(W dH'^T) - beta*gam*(Z H^T) + (dA*M)^T Q + P K + P^T K
     for (int idx = threadIdx.x; idx < n * dk; idx += NT) {
-        const int t = idx / dk;
-        dQs[idx] *= __expf(b[t]);
-        dKs[idx] = __expf(bn - b[t]) * dKs[idx] - bt[t] * __expf(b[t]) * T1[idx];
+        const int t = idx / dk, a = t * ldk + (idx - t * dk);
+        dQs[a] *= __expf(b[t]);
+        dKs[a] = __expf(bn - b[t]) * dKs[a] - bt[t] * __expf(b[t]) * T1[a];
     }
     __syncthreads();
-    mm(dQs, dk, DA, C, false, Ks, dk, false, n, dk, n, 1.f, 1.f);
-    mm(dKs, dk, DA, C, true, Qs, dk, false, n, dk, n, 1.f, 1.f);
+    mm(dQs, ldk, DA, ldc, false, Ks, ldk, false, n, dk, n, 1.f, 1.f);
+    mm(dKs, ldk, DA, ldc, true, Qs, ldk, false, n, dk, n, 1.f, 1.f);
     __syncthreads();
-    mm(dKs, dk, ZW, C, false, Ks, dk, false, n, dk, n, 1.f, 1.f);
+    mm(dKs, ldk, ZW, ldc, false, Ks, ldk, false, n, dk, n, 1.f, 1.f);
     __syncthreads();
-    mm(dKs, dk, ZW, C, true, Ks, dk, false, n, dk, n, 1.f, 1.f);
+    mm(dKs, ldk, ZW, ldc, true, Ks, ldk, false, n, dk, n, 1.f, 1.f);
     __syncthreads();
     for (int idx = threadIdx.x; idx < n * dk; idx += NT) {
         const int t = idx / dk, i = idx - t * dk;
-        dq[oqk + (long long)t * p.tqk + i] = from_f32<T>(dQs[idx]);
-        dk_out[oqk + (long long)t * p.tqk + i] = from_f32<T>(dKs[idx]);
+        dq[oqk + (long long)t * p.tqk + i] = from_f32<T>(dQs[t * ldk + i]);
+        dk_out[oqk + (long long)t * p.tqk + i] = from_f32<T>(dKs[t * ldk + i]);
     }
     for (int idx = threadIdx.x; idx < n * dv; idx += NT) {
         const int t = idx / dv, jj = idx - t * dv;
-        dv_out[ov + (long long)t * p.tv + jj] = from_f32<T>(bt[t] * Zs[idx]);
+        dv_out[ov + (long long)t * p.tv + jj] = from_f32<T>(bt[t] * Zs[t * ldv + jj]);
     }
 }
 
-// shared memory (bytes) of the kernels for a shape
-__host__ inline size_t smem_pre(int C, int dk, int dv) { return sizeof(float) * ((size_t)C * dk + (size_t)C * (dv + dk) + (size_t)C * C + 2 * C); }
-__host__ inline size_t smem_state(int C, int dk) { return sizeof(float) * ((size_t)dk * DVS + 2 * (size_t)C * dk + (size_t)C * DVS + C); }
-__host__ inline size_t smem_out(int C, int dk, int dv) { return sizeof(float) * (2 * (size_t)C * dk + 2 * (size_t)C * dv + (size_t)dk * dv + (size_t)C * C + C); }
-__host__ inline size_t smem_bwd_state(int C, int dk) { return sizeof(float) * (2 * (size_t)dk * DVS + 2 * (size_t)C * dk + 2 * (size_t)C * C + 2 * (size_t)C * DVS + 2 * C); }
+// shared memory (bytes) of the kernels for a shape (padded tiles)
+__host__ inline size_t smem_pre(int C, int dk, int dv) {
+    return sizeof(float) * (2 * (size_t)C * ldp(dk) + (size_t)C * ldp(dv + dk + C) + (size_t)C * ldp(C) + 2 * C);
+}
+__host__ inline size_t smem_state(int C, int dk) {
+    return sizeof(float) * ((size_t)dk * ldp(DVS) + 2 * (size_t)C * ldp(dk) + (size_t)C * ldp(DVS) + C);
+}
+__host__ inline size_t smem_out(int C, int dk, int dv) {
+    return sizeof(float) * (2 * (size_t)C * ldp(dk) + 2 * (size_t)C * ldp(dv) + (size_t)dk * ldp(dv) + (size_t)C * ldp(C) + C);
+}
+__host__ inline size_t smem_bwd_state(int C, int dk) {
+    return sizeof(float) * (2 * (size_t)dk * ldp(DVS) + 2 * (size_t)C * ldp(dk) + 2 * (size_t)C * ldp(C) + 3 * (size_t)C * ldp(DVS) + 2 * C);
+}
 __host__ inline size_t smem_bwd_out(int C, int dk, int dv) {
-    return sizeof(float) * (2 * (size_t)C * dk + 4 * (size_t)C * dv + 2 * (size_t)dk * dv + 4 * (size_t)C * C + 2 * (size_t)C * dv + 3 * (size_t)C * dk + 10 * (size_t)C + dk);
+    return sizeof(float) * (2 * (size_t)C * ldp(dk) + 4 * (size_t)C * ldp(dv) + 2 * (size_t)dk * ldp(dv) + 4 * (size_t)C * ldp(C) +
+                            2 * (size_t)C * ldp(dv) + 3 * (size_t)C * ldp(dk) + 10 * (size_t)C + dk);
 }
 
 }  // namespace gdn

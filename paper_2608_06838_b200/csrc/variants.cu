@@ -161,7 +161,7 @@ sf_status_t chunked_forward(const sf_seg_desc_t* d, const sf::gdn::Params& p, co
     const dim3 chunks(p.NC, p.H, p.B), cols(p.dv / DVS, p.H, p.B);
     const size_t s1 = smem_pre(p.C, p.dk, p.dv), s2 = smem_state(p.C, p.dk), s3 = smem_out(p.C, p.dk, p.dv);
     if (!opt_in(pre_kernel<T>, s1) || !opt_in(state_kernel<T>, s2) || !opt_in(out_kernel<T>, s3)) return SF_ERR_CUDA;
-    pre_kernel<T><<<chunks, NT, s1, st>>>(p, tk, tv, g, beta, ws, backward);
+    pre_kernel<T><<<chunks, NT, s1, st>>>(p, tq, tk, tv, g, beta, ws, backward);
     state_kernel<T><<<cols, NT, s2, st>>>(p, tk, g, S_in, S_out, ws, backward);
     int n = 2;
     if (o) { out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, g, static_cast<T*>(o), ws, backward); ++n; }
