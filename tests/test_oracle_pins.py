@@ -397,3 +397,23 @@ def test_scan_over_block_aggregates_reproduces_the_segment_state():
     np.testing.assert_allclose(final, S_out.reshape(2, -1), atol=1e-12)
     _, S_mid = oracle.segment_fwd(q[:, :blk], k[:, :blk], v[:, :blk], g[:, :blk], S_in)
     np.testing.assert_allclose(states[:, 1], S_mid.reshape(2, -1), atol=1e-12)
+
+
+def test_oracle_runs_clean_under_the_address_and_undefined_behaviour_sanitizers(tmp_path):
+    # the C oracle with exactly-sized buffers, several checkpoint windows with a short last one, with and without boundary
+    # states, and the scan in both directions: any out-of-range index or undefined operation aborts the driver
+    import os
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("gcc not available")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    exe = str(tmp_path / "oracle_san")
+    build = subprocess.run(["gcc", "-O1", "-g", "-fsanitize=address,undefined", "-fno-sanitize-recover=all", "-fopenmp", "-std=c11",
+                            "-o", exe, os.path.join(root, "tests", "oracle_sanitizer_main.c"),
+                            os.path.join(root, "oracle", "sf_oracle.c"), "-lm"], capture_output=True, text=True)
+    if build.returncode != 0 and "sanitize" in build.stderr.lower():
+        pytest.skip("sanitizer runtime not installed: " + build.stderr[-200:])
+    assert build.returncode == 0, build.stderr
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=300)
+    assert run.returncode == 0 and "clean" in run.stdout, run.stdout + run.stderr
