@@ -441,12 +441,12 @@ sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const
 /*
  * The same gated delta rule in its chunkwise form (Section 2.2, Eq. 2 with V_new): per chunk the unit-lower-triangular
  * system (I + L) W = beta*V - beta*gam*(K H) is solved by substitution (UT transform), Pre builds its state-free parts for
- * all chunks in parallel, ST carries the state from chunk to chunk and emits V_new = W, Out forms the outputs of all
- * chunks in parallel; the backward mirrors it (transposed solve, reverse state pass, chunk-parallel gradients).
+ * all chunks in parallel (including each chunk's affine state map), ST carries the state from chunk to chunk, Out forms
+ * V_new = W and the outputs of all chunks in parallel; the backward mirrors it (transposed solve, reverse state pass, chunk-parallel gradients).
  * Same arguments, layouts and results (to rounding) as sf_delta_segment_fwd/bwd.  desc->chunk in {16, 32},
  * d_k, d_v in {32, 64}, float32 or bf16 storage, float32 arithmetic on CUDA cores.  Workspace:
- * sf_delta_chunked_workspace_bytes(desc, backward) bytes, 256-byte aligned (U/W, Wk and the cumulative decay per
- * token, one state per chunk; the backward rebuilds them and adds Z per token, one state gradient and two
+ * sf_delta_chunked_workspace_bytes(desc, backward) bytes, 256-byte aligned (U and Wk per token, the chunk's state map
+ * and one state per chunk; the backward rebuilds them and adds Z0 per token, Theta, one state gradient and two
  * chunk x chunk matrices per chunk).
  */
 size_t sf_delta_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward);

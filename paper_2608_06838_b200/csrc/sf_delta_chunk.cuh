@@ -8,14 +8,16 @@
 // so  W = U - Wk H  with  U = (I+L)^-1 (beta*V),  Wk = (I+L)^-1 (beta*gam*K)   (the UT transform; no inverse is formed:
 // the systems are solved by substitution, one thread per right-hand-side column; for the backward the identity is solved
 // along with them, which gives (I+L)^-1 for the transposed solve).  Then
-//     Pre : U, Wk per chunk                       (needs no state: all chunks in parallel)
-//     ST  : W = U - Wk H  (this is V_new),  H' = gam_n H + (om*K)^T W          (sequential over chunks, per value column)
-//     Out : O = (M * Q K^T) W + gam * (Q H)        (all chunks in parallel, from the stored chunk states)
+//     Pre : U, Wk and the chunk's affine state map  H' = Phi H + Psi,  Phi = gam_n I - (om*K)^T Wk,  Psi = (om*K)^T U
+//                                                                            (needs no state: all chunks in parallel)
+//     ST  : H' = Phi H + Psi, storing the state entering every chunk        (sequential over chunks, per value column)
+//     Out : W = U - Wk H  (this is V_new),  O = (M * Q K^T) W + gam * (Q H)   (all chunks in parallel, from the stored states)
 // Backward (hand-derived; checked against the fp64 oracle, which is pinned by finite differences), dH' = gradient of the
 // state leaving the chunk:
-//     dW = A^T dO + om*(K dH'),  A = M * QK^T;   Z = (I+L)^-T dW;
-//     dH = gam_n dH' + Q^T (gam*dO) - K^T (beta*gam*Z)                           (sequential, reverse, per value column)
-// and, chunk-parallel from the stored W, Z, H, dH':  dA = dO W^T,  dL = -strict_lower(Z W^T),  P = beta*dL*M,
+//     dW = A^T dO + om*(K dH'),  A = M * QK^T;   Z = (I+L)^-T dW = Z0 + (I+L)^-T (om*(K dH')),  Z0 = (I+L)^-T A^T dO;
+//     dH = gam_n dH' + Q^T (gam*dO) - K^T (beta*gam*Z) = Phi^T dH' + Theta,  Theta = Q^T (gam*dO) - K^T (beta*gam*Z0)
+// so Z0 and Theta come from a chunk-parallel kernel, the reverse pass over the chunks is again one small product per chunk,
+// and, chunk-parallel from the stored H, dH' (W and Z are rebuilt in place):  dA = dO W^T,  dL = -strict_lower(Z W^T),  P = beta*dL*M,
 //     dq = (dA*M) K + gam*(dO H^T)
 //     dk = (dA*M)^T Q + om*(W dH'^T) - (beta*gam*Z) H^T + (P + P^T) K
 //     dv = beta*Z,    dbeta = rowsum(Z*V) - gam*rowsum(Z*KH) + rowsum(dL * M * KK^T)
@@ -35,27 +37,31 @@ struct Params {
     long long tqk, tv, tg, bqk, bv, bg;      // token / batch strides in elements
 };
 
-// Workspace per (batch, head), in floats: U/W [L][dv], Wk [L][dk], b [L] (cumulative log-decay inside each chunk),
-// Hc [NC][dk][dv]; the backward adds Z [L][dv],
-// dHc [NC][dk][dv], A [NC][C][C] (the masked Q K^T) and Ti [NC][C][C] (the inverse of I + L, used transposed).
-struct Ws { float *W, *Wk, *b, *Z, *Hc, *dHc, *A, *Ti; };
+// Workspace per (batch, head), in floats: U [L][dv], Wk [L][dk], Phi [NC][dk][dk], Psi [NC][dk][dv], Hc [NC][dk][dv];
+// the backward adds Z0 [L][dv], Theta [NC][dk][dv], dHc [NC][dk][dv], A [NC][C][C] (the masked Q K^T) and
+// Ti [NC][C][C] (the inverse of I + L, used transposed).
+struct Ws { float *U, *Wk, *Phi, *Psi, *Hc, *Z0, *Theta, *dHc, *A, *Ti; };
 __host__ __device__ inline size_t ws_floats(const Params& p, bool backward) {
-    size_t n = (size_t)p.L * p.dv + (size_t)p.L * p.dk + (size_t)p.L + (size_t)p.NC * p.dk * p.dv;
-    if (backward) n += (size_t)p.L * p.dv + (size_t)p.NC * p.dk * p.dv + 2 * (size_t)p.NC * p.C * p.C;
+    const size_t st = (size_t)p.NC * p.dk * p.dv;
+    size_t n = (size_t)p.L * p.dv + (size_t)p.L * p.dk + (size_t)p.NC * p.dk * p.dk + 2 * st;
+    if (backward) n += (size_t)p.L * p.dv + 2 * st + 2 * (size_t)p.NC * p.C * p.C;
     return n;
 }
 __host__ __device__ inline Ws ws_of(float* base, const Params& p, long long bh, bool backward) {
+    const size_t st = (size_t)p.NC * p.dk * p.dv;
     float* c = base + bh * (long long)ws_floats(p, backward);
     Ws w;
-    w.W = c;  c += (size_t)p.L * p.dv;
-    w.Wk = c; c += (size_t)p.L * p.dk;
-    w.b = c;  c += (size_t)p.L;
-    w.Hc = c; c += (size_t)p.NC * p.dk * p.dv;
-    w.Z = w.dHc = w.A = w.Ti = nullptr;
+    w.U = c;   c += (size_t)p.L * p.dv;
+    w.Wk = c;  c += (size_t)p.L * p.dk;
+    w.Phi = c; c += (size_t)p.NC * p.dk * p.dk;
+    w.Psi = c; c += st;
+    w.Hc = c;  c += st;
+    w.Z0 = w.Theta = w.dHc = w.A = w.Ti = nullptr;
     if (backward) {
-        w.Z = c;   c += (size_t)p.L * p.dv;
-        w.dHc = c; c += (size_t)p.NC * p.dk * p.dv;
-        w.A = c;   c += (size_t)p.NC * p.C * p.C;
+        w.Z0 = c;    c += (size_t)p.L * p.dv;
+        w.Theta = c; c += st;
+        w.dHc = c;   c += st;
+        w.A = c;     c += (size_t)p.NC * p.C * p.C;
         w.Ti = c;
     }
     return w;
@@ -66,17 +72,35 @@ __host__ __device__ inline Ws ws_of(float* base, const Params& p, long long bh, 
 __host__ __device__ constexpr int ldp(int cols) { return cols + 1; }
 
 // out[m][n] = keep*out[m][n] + sign * sum_k A(m,k) B(k,n);  A(m,k) = ta ? A[k*lda+m] : A[m*lda+k], likewise B.
+// Element idx is always computed by the same thread, so a second product may accumulate into `out` (keep = 1) without a
+// barrier in between, also when `out` is global memory.
 __device__ __forceinline__ void mm(float* out, int ldo, const float* A, int lda, bool ta, const float* Bm, int ldb, bool tb,
                                    int M, int N, int K, float keep, float sign) {
-    for (int idx = threadIdx.x; idx < M * N; idx += NT) {
-        const int m = idx / N, n = idx - m * N;
-        const float* a = ta ? A + m : A + m * lda;
-        const float* bq = tb ? Bm + n * ldb : Bm + n;
-        const int sa = ta ? lda : 1, sb = tb ? 1 : ldb;
-        float acc = 0.f;
-#pragma unroll 4
-        for (int k = 0; k < K; ++k) acc = fmaf(a[k * sa], bq[k * sb], acc);
-        out[m * ldo + n] = keep != 0.f ? fmaf(keep, out[m * ldo + n], sign * acc) : sign * acc;
+    // four independent accumulators per thread: the products are small and latency-bound, not throughput-bound
+    const int total = M * N, sa = ta ? lda : 1, sb = tb ? 1 : ldb;
+    for (int base = threadIdx.x; base < total; base += 4 * NT) {
+        const float *a[4], *bq[4];
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = min(base + e * NT, total - 1);            // clamped: a lane past the end computes a value it drops
+            const int m = idx / N, n = idx - m * N;
+            a[e] = ta ? A + m : A + m * lda;
+            bq[e] = tb ? Bm + n * ldb : Bm + n;
+        }
+#pragma unroll 2
+        for (int k = 0; k < K; ++k) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[e] = fmaf(a[e][k * sa], bq[e][k * sb], acc[e]);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = base + e * NT;
+            if (idx < total) {
+                const int m = idx / N, n = idx - m * N;
+                out[m * ldo + n] = keep != 0.f ? fmaf(keep, out[m * ldo + n], sign * acc[e]) : sign * acc[e];
+            }
+        }
     }
 }
 
@@ -100,6 +124,14 @@ __device__ __forceinline__ void store_dense(float* dst, int dst_ld, const float*
         dst[(long long)r * dst_ld + c] = src[r * ld + c];
     }
 }
+// rows of a padded [rows][cols] tile times a per-row factor
+template <typename F>
+__device__ __forceinline__ void scale_rows(float* x, int ld, int rows, int cols, F f) {
+    for (int idx = threadIdx.x; idx < rows * cols; idx += NT) {
+        const int r = idx / cols;
+        x[r * ld + (idx - r * cols)] *= f(r);
+    }
+}
 
 // b[t] = inclusive cumulative log-decay of the chunk's n tokens (one thread), bt[t] = beta.  Syncs.
 __device__ __forceinline__ void load_decay(float* b, float* bt, const float* g, const float* beta, long long tg, int n) {
@@ -110,17 +142,9 @@ __device__ __forceinline__ void load_decay(float* b, float* bt, const float* g, 
     if (bt) for (int t = threadIdx.x; t < n; t += NT) bt[t] = beta[(long long)t * tg];
     __syncthreads();
 }
-// The sequential kernels take the cumulative log-decay from the workspace, where Pre has left it.  Syncs.
-__device__ __forceinline__ void load_decay_ws(float* b, float* bt, const float* bws, const float* beta, long long tg, int n) {
-    for (int t = threadIdx.x; t < n; t += NT) {
-        b[t] = bws[t];
-        if (bt) bt[t] = beta[(long long)t * tg];
-    }
-    __syncthreads();
-}
 
-// ---- Pre: U = (I+L)^-1 (beta*V), Wk = (I+L)^-1 (beta*gam*K); for the backward also Ti = (I+L)^-1 and A = M * Q K^T.
-//      grid (NC, H, B) -----------------------------------------------------------------------------------------------
+// ---- Pre: U = (I+L)^-1 (beta*V), Wk = (I+L)^-1 (beta*gam*K), Phi = gam_n I - (om*K)^T Wk, Psi = (om*K)^T U; for the
+//      backward also Ti = (I+L)^-1 and A = M * Q K^T.  grid (NC, H, B) ------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                                                  const float* __restrict__ g, const float* __restrict__ beta, float* ws, int backward) {
@@ -129,10 +153,11 @@ __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__
     const int C = p.C, dk = p.dk, dv = p.dv, t0 = c * C, n = min(C, p.L - t0);
     const int ldk = ldp(dk), ldc = ldp(C), ncol = dv + dk + (backward ? C : 0), ldx = ldp(dv + dk + C);
     float* Ks = sm;                    // [C][dk]
-    float* X = Ks + C * ldk;           // [C][dv + dk (+ C)]   right-hand sides, solved in place
+    float* Kw = Ks + C * ldk;          // [C][dk]   om * K
+    float* Qs = Kw + C * ldk;          // [C][dk]   (backward only)
+    float* X = Qs + C * ldk;           // [C][dv + dk (+ C)]   right-hand sides, solved in place
     float* Lm = X + C * ldx;           // [C][C]
-    float* Qs = Lm + C * ldc;          // [C][dk]   (backward only)
-    float* b = Qs + C * ldk;           // [C]
+    float* b = Lm + C * ldc;           // [C]
     float* bt = b + C;                 // [C]
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(ws, p, bh, backward != 0);
@@ -141,6 +166,7 @@ __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__
     if (backward) load_rows(Qs, ldk, q + oqk, p.tqk, n, dk);
     load_rows(X, ldx, v + (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv, p.tv, n, dv);
     load_decay(b, bt, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, beta + (long long)bb * p.bg + (long long)t0 * p.tg + h, p.tg, n);
+    const float bn = b[n - 1];
     for (int idx = threadIdx.x; idx < n * ncol; idx += NT) {
         const int t = idx / ncol, col = idx - t * ncol;
         float x;
@@ -148,6 +174,10 @@ __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__
         else if (col < dv + dk) x = bt[t] * __expf(b[t]) * Ks[t * ldk + (col - dv)];
         else x = (col - dv - dk) == t ? 1.f : 0.f;                      // identity: its solution is the inverse
         X[t * ldx + col] = x;
+    }
+    for (int idx = threadIdx.x; idx < n * dk; idx += NT) {
+        const int t = idx / dk, i = idx - t * dk;
+        Kw[t * ldk + i] = __expf(bn - b[t]) * Ks[t * ldk + i];
     }
     mm(Lm, ldc, Ks, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);     // K K^T
     __syncthreads();
@@ -164,60 +194,86 @@ __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__
             X[t * ldx + col] = acc;
         }
     __syncthreads();
-    store_dense(w.W + (long long)t0 * dv, dv, X, ldx, n, dv);
+    store_dense(w.U + (long long)t0 * dv, dv, X, ldx, n, dv);
     store_dense(w.Wk + (long long)t0 * dk, dk, X + dv, ldx, n, dk);
-    for (int t = threadIdx.x; t < n; t += NT) w.b[t0 + t] = b[t];
+    float* Phi = w.Phi + (long long)c * dk * dk;
+    mm(Phi, dk, Kw, ldk, true, X + dv, ldx, false, dk, dk, n, 0.f, -1.f);                 // -(om*K)^T Wk
+    mm(w.Psi + (long long)c * dk * dv, dv, Kw, ldk, true, X, ldx, false, dk, dv, n, 0.f, 1.f);
     if (backward) {
         store_dense(w.Ti + (long long)c * C * C, C, X + dv + dk, ldx, n, n);
         mm(Lm, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f); // Q K^T (L is no longer needed)
-        __syncthreads();
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < dk; i += NT) Phi[i * dk + i] += __expf(bn);
+    if (backward)
         for (int idx = threadIdx.x; idx < n * n; idx += NT) {
             const int t = idx / n, s = idx - t * n;
             w.A[(long long)c * C * C + t * C + s] = s <= t ? Lm[t * ldc + s] * __expf(b[t] - b[s]) : 0.f;
         }
-    }
 }
 
-// ---- ST: per chunk  Hc[c] = H;  W = U - Wk H;  H = gam_n H + (om*K)^T W.  grid (dv/DVS, H, B), sequential over chunks ----
-template <typename T>
-__global__ void __launch_bounds__(NT) state_kernel(Params p, const T* __restrict__ k, const float* __restrict__ g,
-                                                   const float* __restrict__ S_in, float* __restrict__ S_out, float* ws, int backward) {
+// ---- ST (forward) and its adjoint (reverse): X' = F X + R per chunk for DVS columns of the state, where
+//      forward:  F = Phi[c],    R = Psi[c],    chunks ascending,  `states[c]` receives the state entering chunk c
+//      reverse:  F = Phi[c]^T,  R = Theta[c],  chunks descending, `states[c]` receives the gradient of the state leaving it
+//      grid (dv/DVS, H, B) ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(NT) chain_kernel(Params p, int reverse, const float* __restrict__ init, float* __restrict__ fin,
+                                                   float* ws, int backward) {
     extern __shared__ float sm[];
     const int j0 = blockIdx.x * DVS, h = blockIdx.y, bb = blockIdx.z;
-    const int C = p.C, dk = p.dk, dv = p.dv;
+    const int dk = p.dk, dv = p.dv;
     const int ldk = ldp(dk), lds = ldp(DVS);
-    float* Hs = sm;                    // [dk][DVS]
-    float* Ks = Hs + dk * lds;         // [C][dk]   (scaled by om in place)
-    float* Wks = Ks + C * ldk;         // [C][dk]
-    float* Wc = Wks + C * ldk;         // [C][DVS]
-    float* b = Wc + C * lds;           // [C]
+    float* X0 = sm;                    // [dk][DVS]
+    float* X1 = X0 + dk * lds;         // [dk][DVS]
+    float* Fs = X1 + dk * lds;         // [dk][dk]
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(ws, p, bh, backward != 0);
-    if (S_in) load_dense(Hs, lds, S_in + bh * dk * dv + j0, dv, dk, DVS);
-    else for (int idx = threadIdx.x; idx < dk * lds; idx += NT) Hs[idx] = 0.f;
+    const float* Rsrc = reverse ? w.Theta : w.Psi;
+    float* states = reverse ? w.dHc : w.Hc;
+    if (init) load_dense(X0, lds, init + bh * dk * dv + j0, dv, dk, DVS);
+    else for (int idx = threadIdx.x; idx < dk * lds; idx += NT) X0[idx] = 0.f;
     __syncthreads();
-    for (int c = 0; c < p.NC; ++c) {
-        const int t0 = c * C, n = min(C, p.L - t0);
-        load_rows(Ks, ldk, k + (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk, p.tqk, n, dk);
-        load_dense(Wks, ldk, w.Wk + (long long)t0 * dk, dk, n, dk);
-        load_dense(Wc, lds, w.W + (long long)t0 * dv + j0, dv, n, DVS);
-        store_dense(w.Hc + (long long)c * dk * dv + j0, dv, Hs, lds, dk, DVS);
-        load_decay(b, nullptr, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, nullptr, p.tg, n);
-        mm(Wc, lds, Wks, ldk, false, Hs, lds, false, n, DVS, dk, 1.f, -1.f);       // W = U - Wk H
-        const float bn = b[n - 1];
-        for (int idx = threadIdx.x; idx < n * dk; idx += NT) {
-            const int t = idx / dk;
-            Ks[t * ldk + (idx - t * dk)] *= __expf(bn - b[t]);
+    // The map of the next chunk is fetched into registers while the product of the current one runs.
+    constexpr int MAXF = (64 * 64) / NT, MAXR = (64 * DVS) / NT;         // d_k <= 64
+    float fr[MAXF], rr[MAXR];
+    auto fetch = [&](int c) {
+        const float* F = w.Phi + (long long)c * dk * dk;
+        const float* R = Rsrc + (long long)c * dk * dv + j0;
+#pragma unroll
+        for (int e = 0; e < MAXF; ++e) {
+            const int idx = threadIdx.x + e * NT;
+            fr[e] = idx < dk * dk ? F[idx] : 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < MAXR; ++e) {
+            const int idx = threadIdx.x + e * NT;
+            rr[e] = idx < dk * DVS ? R[(long long)(idx / DVS) * dv + (idx % DVS)] : 0.f;
+        }
+    };
+    float *cur = X0, *nxt = X1;
+    fetch(reverse ? p.NC - 1 : 0);
+    for (int s = 0; s < p.NC; ++s) {
+        const int c = reverse ? p.NC - 1 - s : s;
+        store_dense(states + (long long)c * dk * dv + j0, dv, cur, lds, dk, DVS);
+#pragma unroll
+        for (int e = 0; e < MAXF; ++e) {
+            const int idx = threadIdx.x + e * NT;
+            if (idx < dk * dk) Fs[(idx / dk) * ldk + (idx % dk)] = fr[e];
+        }
+#pragma unroll
+        for (int e = 0; e < MAXR; ++e) {
+            const int idx = threadIdx.x + e * NT;
+            if (idx < dk * DVS) nxt[(idx / DVS) * lds + (idx % DVS)] = rr[e];
         }
         __syncthreads();
-        store_dense(w.W + (long long)t0 * dv + j0, dv, Wc, lds, n, DVS);
-        mm(Hs, lds, Ks, ldk, true, Wc, lds, false, dk, DVS, n, __expf(bn), 1.f);   // H = gam_n H + (om*K)^T W
+        if (s + 1 < p.NC) fetch(reverse ? c - 1 : c + 1);
+        mm(nxt, lds, Fs, ldk, reverse != 0, cur, lds, false, dk, DVS, dk, 1.f, 1.f);
         __syncthreads();
+        float* t = cur; cur = nxt; nxt = t;
     }
-    if (S_out) store_dense(S_out + bh * dk * dv + j0, dv, Hs, lds, dk, DVS);
+    if (fin) store_dense(fin + bh * dk * dv + j0, dv, cur, lds, dk, DVS);
 }
 
-// ---- Out: O = (M * Q K^T) W + gam * (Q Hc).  grid (NC, H, B) ------------------------------------------------------
+// ---- Out: W = U - Wk Hc (V_new),  O = (M * Q K^T) W + gam * (Q Hc).  grid (NC, H, B) --------------------------------
 template <typename T>
 __global__ void __launch_bounds__(NT) out_kernel(Params p, const T* __restrict__ q, const T* __restrict__ k, const float* __restrict__ g,
                                                  T* __restrict__ o, const float* ws, int backward) {
@@ -227,7 +283,8 @@ __global__ void __launch_bounds__(NT) out_kernel(Params p, const T* __restrict__
     const int ldk = ldp(dk), ldv = ldp(dv), ldc = ldp(C);
     float* Qs = sm;                    // [C][dk]
     float* Ks = Qs + C * ldk;          // [C][dk]
-    float* Wc = Ks + C * ldk;          // [C][dv]
+    float* Wks = Ks + C * ldk;         // [C][dk]
+    float* Wc = Wks + C * ldk;         // [C][dv]
     float* Hs = Wc + C * ldv;          // [dk][dv]
     float* A = Hs + dk * ldv;          // [C][C]
     float* O = A + C * ldc;            // [C][dv]
@@ -237,9 +294,11 @@ __global__ void __launch_bounds__(NT) out_kernel(Params p, const T* __restrict__
     const long long oqk = (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk;
     load_rows(Qs, ldk, q + oqk, p.tqk, n, dk);
     load_rows(Ks, ldk, k + oqk, p.tqk, n, dk);
-    load_dense(Wc, ldv, w.W + (long long)t0 * dv, dv, n, dv);
+    load_dense(Wks, ldk, w.Wk + (long long)t0 * dk, dk, n, dk);
+    load_dense(Wc, ldv, w.U + (long long)t0 * dv, dv, n, dv);
     load_dense(Hs, ldv, w.Hc + (long long)c * dk * dv, dv, dk, dv);
     load_decay(b, nullptr, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, nullptr, p.tg, n);
+    mm(Wc, ldv, Wks, ldk, false, Hs, ldv, false, n, dv, dk, 1.f, -1.f);         // W = U - Wk H
     mm(A, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
     mm(O, ldv, Qs, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
     __syncthreads();
@@ -247,10 +306,7 @@ __global__ void __launch_bounds__(NT) out_kernel(Params p, const T* __restrict__
         const int t = idx / n, s = idx - t * n;
         A[t * ldc + s] = s <= t ? A[t * ldc + s] * __expf(b[t] - b[s]) : 0.f;
     }
-    for (int idx = threadIdx.x; idx < n * dv; idx += NT) {
-        const int t = idx / dv;
-        O[t * ldv + (idx - t * dv)] *= __expf(b[t]);
-    }
+    scale_rows(O, ldv, n, dv, [&](int t) { return __expf(b[t]); });
     __syncthreads();
     mm(O, ldv, A, ldc, false, Wc, ldv, false, n, dv, n, 1.f, 1.f);
     __syncthreads();
@@ -261,76 +317,48 @@ __global__ void __launch_bounds__(NT) out_kernel(Params p, const T* __restrict__
     }
 }
 
-// ---- backward, sequential part (reverse over chunks): dHc[c] = dH';  dW = A^T dO + om*(K dH');  Z = Ti^T dW;
-//      dH = gam_n dH' + Q^T (gam*dO) - K^T (beta*gam*Z).  grid (dv/DVS, H, B) -------------------------------------------
+// ---- backward, first chunk-parallel part: Z0 = Ti^T (A^T dO),  Theta = Q^T (gam*dO) - K^T (beta*gam*Z0).  grid (NC, H, B) ----
 template <typename T>
-__global__ void __launch_bounds__(NT) bwd_state_kernel(Params p, const T* __restrict__ q, const T* __restrict__ k,
-                                                       const float* __restrict__ g, const float* __restrict__ beta,
-                                                       const T* __restrict__ dO, const float* __restrict__ dS_out,
-                                                       float* __restrict__ dS_in, float* ws) {
+__global__ void __launch_bounds__(NT) bwd_pre_kernel(Params p, const T* __restrict__ q, const T* __restrict__ k,
+                                                     const float* __restrict__ g, const float* __restrict__ beta,
+                                                     const T* __restrict__ dO, float* ws) {
     extern __shared__ float sm[];
-    const int j0 = blockIdx.x * DVS, h = blockIdx.y, bb = blockIdx.z;
-    const int C = p.C, dk = p.dk, dv = p.dv;
-    const int ldk = ldp(dk), ldc = ldp(C), lds = ldp(DVS);
-    float* G = sm;                     // [dk][DVS]  carried state gradient
-    float* G2 = G + dk * lds;          // [dk][DVS]
-    float* Qs = G2 + dk * lds;         // [C][dk]
+    const int c = blockIdx.x, h = blockIdx.y, bb = blockIdx.z;
+    const int C = p.C, dk = p.dk, dv = p.dv, t0 = c * C, n = min(C, p.L - t0);
+    const int ldk = ldp(dk), ldv = ldp(dv), ldc = ldp(C);
+    float* Qs = sm;                    // [C][dk]
     float* Ks = Qs + C * ldk;          // [C][dk]
-    float* A = Ks + C * ldk;           // [C][C]
+    float* dOs = Ks + C * ldk;         // [C][dv]
+    float* T1 = dOs + C * ldv;         // [C][dv]
+    float* Z0 = T1 + C * ldv;          // [C][dv]
+    float* A = Z0 + C * ldv;           // [C][C]
     float* Ti = A + C * ldc;           // [C][C]
-    float* dOs = Ti + C * ldc;         // [C][DVS]
-    float* dWs = dOs + C * lds;        // [C][DVS]
-    float* Zs = dWs + C * lds;         // [C][DVS]
-    float* b = Zs + C * lds;           // [C]
+    float* b = Ti + C * ldc;           // [C]
     float* bt = b + C;                 // [C]
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(ws, p, bh, true);
-    if (dS_out) load_dense(G, lds, dS_out + bh * dk * dv + j0, dv, dk, DVS);
-    else for (int idx = threadIdx.x; idx < dk * lds; idx += NT) G[idx] = 0.f;
+    const long long oqk = (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk;
+    load_rows(Qs, ldk, q + oqk, p.tqk, n, dk);
+    load_rows(Ks, ldk, k + oqk, p.tqk, n, dk);
+    load_rows(dOs, ldv, dO + (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv, p.tv, n, dv);
+    load_dense(A, ldc, w.A + (long long)c * C * C, C, n, n);
+    load_dense(Ti, ldc, w.Ti + (long long)c * C * C, C, n, n);
+    load_decay(b, bt, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, beta + (long long)bb * p.bg + (long long)t0 * p.tg + h, p.tg, n);
+    mm(T1, ldv, A, ldc, true, dOs, ldv, false, n, dv, n, 0.f, 1.f);             // A^T dO
     __syncthreads();
-    for (int c = p.NC - 1; c >= 0; --c) {
-        const int t0 = c * C, n = min(C, p.L - t0);
-        const long long oqk = (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk;
-        load_rows(Qs, ldk, q + oqk, p.tqk, n, dk);
-        load_rows(Ks, ldk, k + oqk, p.tqk, n, dk);
-        load_rows(dOs, lds, dO + (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv + j0, p.tv, n, DVS);
-        load_dense(A, ldc, w.A + (long long)c * C * C, C, n, n);
-        load_dense(Ti, ldc, w.Ti + (long long)c * C * C, C, n, n);
-        store_dense(w.dHc + (long long)c * dk * dv + j0, dv, G, lds, dk, DVS);
-        load_decay_ws(b, bt, w.b + t0, beta + (long long)bb * p.bg + (long long)t0 * p.tg + h, p.tg, n);
-        const float bn = b[n - 1];
-        mm(dWs, lds, Ks, ldk, false, G, lds, false, n, DVS, dk, 0.f, 1.f);          // K dH'
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < n * DVS; idx += NT) {
-            const int t = idx / DVS;
-            dWs[t * lds + (idx - t * DVS)] *= __expf(bn - b[t]);
-        }
-        __syncthreads();
-        mm(dWs, lds, A, ldc, true, dOs, lds, false, n, DVS, n, 1.f, 1.f);           // dW = A^T dO + om*(K dH')
-        __syncthreads();
-        mm(Zs, lds, Ti, ldc, true, dWs, lds, false, n, DVS, n, 0.f, 1.f);           // Z = (I+L)^-T dW
-        __syncthreads();
-        store_dense(w.Z + (long long)t0 * dv + j0, dv, Zs, lds, n, DVS);
-        for (int idx = threadIdx.x; idx < n * DVS; idx += NT) {
-            const int t = idx / DVS, a = t * lds + (idx - t * DVS);
-            dOs[a] *= __expf(b[t]);                                                 // gam*dO
-            Zs[a] *= bt[t] * __expf(b[t]);                                          // beta*gam*Z
-        }
-        __syncthreads();
-        mm(G2, lds, Qs, ldk, true, dOs, lds, false, dk, DVS, n, 0.f, 1.f);
-        __syncthreads();
-        mm(G2, lds, Ks, ldk, true, Zs, lds, false, dk, DVS, n, 1.f, -1.f);
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < dk * DVS; idx += NT) {
-            const int i = idx / DVS, a = i * lds + (idx - i * DVS);
-            G[a] = fmaf(__expf(bn), G[a], G2[a]);
-        }
-        __syncthreads();
-    }
-    store_dense(dS_in + bh * dk * dv + j0, dv, G, lds, dk, DVS);
+    mm(Z0, ldv, Ti, ldc, true, T1, ldv, false, n, dv, n, 0.f, 1.f);             // Z0 = (I+L)^-T A^T dO
+    __syncthreads();
+    store_dense(w.Z0 + (long long)t0 * dv, dv, Z0, ldv, n, dv);
+    scale_rows(dOs, ldv, n, dv, [&](int t) { return __expf(b[t]); });
+    scale_rows(Z0, ldv, n, dv, [&](int t) { return bt[t] * __expf(b[t]); });
+    __syncthreads();
+    float* Th = w.Theta + (long long)c * dk * dv;
+    mm(Th, dv, Qs, ldk, true, dOs, ldv, false, dk, dv, n, 0.f, 1.f);
+    mm(Th, dv, Ks, ldk, true, Z0, ldv, false, dk, dv, n, 1.f, -1.f);
 }
 
-// ---- backward, chunk-parallel part: every input gradient of the chunk from the stored W, Z, Hc, dHc.  grid (NC, H, B) ----
+// ---- backward, second chunk-parallel part: every input gradient of the chunk from the stored Hc, dHc, U, Wk, Z0, Ti.
+//      grid (NC, H, B) ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                                                      const float* __restrict__ g, const float* __restrict__ beta,
@@ -349,13 +377,14 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
     float* DA = KK + C * ldc;           float* ZW = DA + C * ldc;
     float* KH = ZW + C * ldc;           float* KdH = KH + C * ldv;
     float* dQs = KdH + C * ldv;         float* dKs = dQs + C * ldk;
-    float* T1 = dKs + C * ldk;
-    float* b = T1 + C * ldk;            float* bt = b + C;
+    float* T1 = dKs + C * ldk;          // [C][max(dk, dv)]: Wk, then om*(K dH'), then Z H^T
+    float* b = T1 + C * ldp(dk > dv ? dk : dv);   float* bt = b + C;
     float* rs = bt + C;                 float* cs = rs + C;
     float* rl = cs + C;                 float* zkh = rl + C;
     float* zv = zkh + C;                float* doqh = zv + C;
     float* wkdh = doqh + C;             float* db = wkdh + C;
     float* part = db + C;               // [dk]
+    float* Ti = QK;                     // the inverse is needed only before the C x C products are formed
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(const_cast<float*>(ws), p, bh, true);
     const long long oqk = (long long)bb * p.bqk + (long long)t0 * p.tqk + (long long)h * dk;
@@ -365,21 +394,34 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
     load_rows(Ks, ldk, k + oqk, p.tqk, n, dk);
     load_rows(Vs, ldv, v + ov, p.tv, n, dv);
     load_rows(dOs, ldv, dO + ov, p.tv, n, dv);
-    load_dense(Wc, ldv, w.W + (long long)t0 * dv, dv, n, dv);
-    load_dense(Zs, ldv, w.Z + (long long)t0 * dv, dv, n, dv);
+    load_dense(Wc, ldv, w.U + (long long)t0 * dv, dv, n, dv);
+    load_dense(T1, ldk, w.Wk + (long long)t0 * dk, dk, n, dk);
+    load_dense(Zs, ldv, w.Z0 + (long long)t0 * dv, dv, n, dv);
     load_dense(Hs, ldv, w.Hc + (long long)c * dk * dv, dv, dk, dv);
     load_dense(dHs, ldv, w.dHc + (long long)c * dk * dv, dv, dk, dv);
+    load_dense(Ti, ldc, w.Ti + (long long)c * C * C, C, n, n);
     load_decay(b, bt, g + og, beta + og, p.tg, n);
     const float bn = b[n - 1];
+    mm(Wc, ldv, T1, ldk, false, Hs, ldv, false, n, dv, dk, 1.f, -1.f);          // W = U - Wk H
+    mm(KH, ldv, Ks, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
+    mm(KdH, ldv, Ks, ldk, false, dHs, ldv, false, n, dv, dk, 0.f, 1.f);
+    __syncthreads();
+    // Z = Z0 + Ti^T (om * (K dH')): the part of the transposed solve that depends on the incoming state gradient
+    const int ldt = ldp(dk > dv ? dk : dv);
+    for (int idx = threadIdx.x; idx < n * dv; idx += NT) {
+        const int t = idx / dv, jj = idx - t * dv;
+        T1[t * ldt + jj] = __expf(bn - b[t]) * KdH[t * ldv + jj];
+    }
+    __syncthreads();
+    mm(Zs, ldv, Ti, ldc, true, T1, ldt, false, n, dv, n, 1.f, 1.f);
+    __syncthreads();
     mm(QK, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
     mm(KK, ldc, Ks, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
     mm(DA, ldc, dOs, ldv, false, Wc, ldv, true, n, n, dv, 0.f, 1.f);            // dA = dO W^T
     mm(ZW, ldc, Zs, ldv, false, Wc, ldv, true, n, n, dv, 0.f, 1.f);             // Z W^T  (dL = -strict lower)
-    mm(KH, ldv, Ks, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
-    mm(KdH, ldv, Ks, ldk, false, dHs, ldv, false, n, dv, dk, 0.f, 1.f);
     mm(dQs, ldk, dOs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);          // dO H^T
     mm(dKs, ldk, Wc, ldv, false, dHs, ldv, true, n, dk, dv, 0.f, 1.f);          // W dH'^T
-    mm(T1, ldk, Zs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);            // Z H^T
+    mm(T1, ldt, Zs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);            // Z H^T
     for (int i = threadIdx.x; i < dk; i += NT) {
         float acc = 0.f;
         for (int jj = 0; jj < dv; ++jj) acc = fmaf(dHs[i * ldv + jj], Hs[i * ldv + jj], acc);
@@ -427,9 +469,9 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
         dbeta[og + (long long)t * p.tg] = zv[t] - __expf(b[t]) * zkh[t] + rl[t];
     // dq = (dA*M) K + gam*(dO H^T);  dk = om*(W dH'^T) - beta*gam*(Z H^T) + (dA*M)^T Q + P K + P^T K
     for (int idx = threadIdx.x; idx < n * dk; idx += NT) {
-        const int t = idx / dk, a = t * ldk + (idx - t * dk);
+        const int t = idx / dk, i = idx - t * dk, a = t * ldk + i;
         dQs[a] *= __expf(b[t]);
-        dKs[a] = __expf(bn - b[t]) * dKs[a] - bt[t] * __expf(b[t]) * T1[a];
+        dKs[a] = __expf(bn - b[t]) * dKs[a] - bt[t] * __expf(b[t]) * T1[t * ldt + i];
     }
     __syncthreads();
     mm(dQs, ldk, DA, ldc, false, Ks, ldk, false, n, dk, n, 1.f, 1.f);
@@ -452,20 +494,18 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
 
 // shared memory (bytes) of the kernels for a shape (padded tiles)
 __host__ inline size_t smem_pre(int C, int dk, int dv) {
-    return sizeof(float) * (2 * (size_t)C * ldp(dk) + (size_t)C * ldp(dv + dk + C) + (size_t)C * ldp(C) + 2 * C);
+    return sizeof(float) * (3 * (size_t)C * ldp(dk) + (size_t)C * ldp(dv + dk + C) + (size_t)C * ldp(C) + 2 * C);
 }
-__host__ inline size_t smem_state(int C, int dk) {
-    return sizeof(float) * ((size_t)dk * ldp(DVS) + 2 * (size_t)C * ldp(dk) + (size_t)C * ldp(DVS) + C);
-}
+__host__ inline size_t smem_chain(int dk) { return sizeof(float) * (2 * (size_t)dk * ldp(DVS) + (size_t)dk * ldp(dk)); }
 __host__ inline size_t smem_out(int C, int dk, int dv) {
-    return sizeof(float) * (2 * (size_t)C * ldp(dk) + 2 * (size_t)C * ldp(dv) + (size_t)dk * ldp(dv) + (size_t)C * ldp(C) + C);
+    return sizeof(float) * (3 * (size_t)C * ldp(dk) + 2 * (size_t)C * ldp(dv) + (size_t)dk * ldp(dv) + (size_t)C * ldp(C) + C);
 }
-__host__ inline size_t smem_bwd_state(int C, int dk) {
-    return sizeof(float) * (2 * (size_t)dk * ldp(DVS) + 2 * (size_t)C * ldp(dk) + 2 * (size_t)C * ldp(C) + 3 * (size_t)C * ldp(DVS) + 2 * C);
+__host__ inline size_t smem_bwd_pre(int C, int dk, int dv) {
+    return sizeof(float) * (2 * (size_t)C * ldp(dk) + 3 * (size_t)C * ldp(dv) + 2 * (size_t)C * ldp(C) + 2 * C);
 }
 __host__ inline size_t smem_bwd_out(int C, int dk, int dv) {
     return sizeof(float) * (2 * (size_t)C * ldp(dk) + 4 * (size_t)C * ldp(dv) + 2 * (size_t)dk * ldp(dv) + 4 * (size_t)C * ldp(C) +
-                            2 * (size_t)C * ldp(dv) + 3 * (size_t)C * ldp(dk) + 10 * (size_t)C + dk);
+                            2 * (size_t)C * ldp(dv) + 2 * (size_t)C * ldp(dk) + (size_t)C * ldp(dk > dv ? dk : dv) + 10 * (size_t)C + dk);
 }
 
 }  // namespace gdn

@@ -151,7 +151,7 @@ bool opt_in(K kern, size_t bytes) {
     return true;
 }
 
-// Pre + ST (+ Out when o != NULL); the backward calls it with o == NULL to rebuild W and the chunk states.
+// Pre + ST (+ Out when o != NULL); the backward calls it with o == NULL to rebuild the chunk states.
 template <typename T>
 sf_status_t chunked_forward(const sf_seg_desc_t* d, const sf::gdn::Params& p, const void* q, const void* k, const void* v,
                             const float* g, const float* beta, const float* S_in, void* o, float* S_out, float* ws, int backward,
@@ -159,10 +159,10 @@ sf_status_t chunked_forward(const sf_seg_desc_t* d, const sf::gdn::Params& p, co
     using namespace sf::gdn;
     const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v);
     const dim3 chunks(p.NC, p.H, p.B), cols(p.dv / DVS, p.H, p.B);
-    const size_t s1 = smem_pre(p.C, p.dk, p.dv), s2 = smem_state(p.C, p.dk), s3 = smem_out(p.C, p.dk, p.dv);
-    if (!opt_in(pre_kernel<T>, s1) || !opt_in(state_kernel<T>, s2) || !opt_in(out_kernel<T>, s3)) return SF_ERR_CUDA;
+    const size_t s1 = smem_pre(p.C, p.dk, p.dv), s2 = smem_chain(p.dk), s3 = smem_out(p.C, p.dk, p.dv);
+    if (!opt_in(pre_kernel<T>, s1) || !opt_in(chain_kernel, s2) || !opt_in(out_kernel<T>, s3)) return SF_ERR_CUDA;
     pre_kernel<T><<<chunks, NT, s1, st>>>(p, tq, tk, tv, g, beta, ws, backward);
-    state_kernel<T><<<cols, NT, s2, st>>>(p, tk, g, S_in, S_out, ws, backward);
+    chain_kernel<<<cols, NT, s2, st>>>(p, 0, S_in, S_out, ws, backward);
     int n = 2;
     if (o) { out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, g, static_cast<T*>(o), ws, backward); ++n; }
     return launched(n);
@@ -177,12 +177,13 @@ sf_status_t chunked_backward(const sf_seg_desc_t* d, const sf::gdn::Params& p, c
     if (f != SF_OK) return f;
     const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v), *tdo = static_cast<const T*>(dO);
     const dim3 chunks(p.NC, p.H, p.B), cols(p.dv / DVS, p.H, p.B);
-    const size_t s1 = smem_bwd_state(p.C, p.dk), s2 = smem_bwd_out(p.C, p.dk, p.dv);
-    if (!opt_in(bwd_state_kernel<T>, s1) || !opt_in(bwd_out_kernel<T>, s2)) return SF_ERR_CUDA;
-    bwd_state_kernel<T><<<cols, NT, s1, st>>>(p, tq, tk, g, beta, tdo, dS_out, dS_in, ws);
-    bwd_out_kernel<T><<<chunks, NT, s2, st>>>(p, tq, tk, tv, g, beta, tdo, static_cast<T*>(dq), static_cast<T*>(dk), static_cast<T*>(dv),
+    const size_t s1 = smem_bwd_pre(p.C, p.dk, p.dv), s2 = smem_chain(p.dk), s3 = smem_bwd_out(p.C, p.dk, p.dv);
+    if (!opt_in(bwd_pre_kernel<T>, s1) || !opt_in(chain_kernel, s2) || !opt_in(bwd_out_kernel<T>, s3)) return SF_ERR_CUDA;
+    bwd_pre_kernel<T><<<chunks, NT, s1, st>>>(p, tq, tk, g, beta, tdo, ws);
+    chain_kernel<<<cols, NT, s2, st>>>(p, 1, dS_out, dS_in, ws, 1);
+    bwd_out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, tv, g, beta, tdo, static_cast<T*>(dq), static_cast<T*>(dk), static_cast<T*>(dv),
                                               dg, dbeta, ws);
-    return launched(2);
+    return launched(3);
 }
 
 }  // namespace
