@@ -439,6 +439,23 @@ sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const
                                  sf_stream_t stream);
 
 /*
+ * The diagonal-decay operator in its chunkwise form (Section 2.2, Eq. 2 with an empty V_new): per chunk the decay-weighted
+ * scores A[t,s] = sum_i q_t[i] k_s[i] exp(b_t[i] - b_s[i]) and the affine state map H' = diag(gam_n) H + (om*K)^T V are
+ * built for all chunks in parallel, the state is carried from chunk to chunk element by element, and the outputs (and,
+ * in the backward, every gradient, with dg anchored per chunk) are again formed for all chunks in parallel.  Same
+ * arguments, layouts and results (to rounding) as sf_channel_segment_fwd/bwd.  desc->chunk in {16, 32}, d_k, d_v in
+ * {32, 64}, float32 or bf16 storage, float32 arithmetic on CUDA cores.  Workspace:
+ * sf_channel_chunked_workspace_bytes(desc, backward) bytes, 256-byte aligned.
+ */
+size_t sf_channel_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward);
+sf_status_t sf_channel_chunked_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                   const float* S_in, void* o, float* S_out, void* workspace, size_t workspace_bytes,
+                                   sf_stream_t stream);
+sf_status_t sf_channel_chunked_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                   const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk, void* dv,
+                                   float* dg, float* dS_in, void* workspace, size_t workspace_bytes, sf_stream_t stream);
+
+/*
  * The same gated delta rule in its chunkwise form (Section 2.2, Eq. 2 with V_new): per chunk the unit-lower-triangular
  * system (I + L) W = beta*V - beta*gam*(K H) is solved by substitution (UT transform), Pre builds its state-free parts for
  * all chunks in parallel (including each chunk's affine state map), ST carries the state from chunk to chunk, Out forms

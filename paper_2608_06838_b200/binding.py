@@ -105,6 +105,12 @@ def load() -> ctypes.CDLL:
         lib.sf_delta_segment_fwd.argtypes = [dp] + [vp] * 8 + [vp]
         lib.sf_delta_segment_bwd.restype = ctypes.c_int
         lib.sf_delta_segment_bwd.argtypes = [dp] + [vp] * 14 + [vp, sz, vp]
+        lib.sf_channel_chunked_workspace_bytes.restype = sz
+        lib.sf_channel_chunked_workspace_bytes.argtypes = [dp, ctypes.c_int]
+        lib.sf_channel_chunked_fwd.restype = ctypes.c_int
+        lib.sf_channel_chunked_fwd.argtypes = [dp] + [vp] * 7 + [vp, sz, vp]
+        lib.sf_channel_chunked_bwd.restype = ctypes.c_int
+        lib.sf_channel_chunked_bwd.argtypes = [dp] + [vp] * 12 + [vp, sz, vp]
         lib.sf_delta_chunked_workspace_bytes.restype = sz
         lib.sf_delta_chunked_workspace_bytes.argtypes = [dp, ctypes.c_int]
         lib.sf_delta_chunked_fwd.restype = ctypes.c_int
@@ -383,6 +389,21 @@ def sf_delta_segment_bwd(desc: SegDesc, q, k, v, g, beta, S_in, dO, dS_out, dq, 
     _check(load().sf_delta_segment_bwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(S_in), _ptr(dO),
                                        _ptr(dS_out), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dg), _ptr(dbeta), _ptr(dS_in),
                                        _ptr(workspace), workspace.numel(), _stream(stream)), "sf_delta_segment_bwd")
+
+
+def sf_channel_chunked_workspace_bytes(desc: SegDesc, backward: int) -> int:
+    return int(load().sf_channel_chunked_workspace_bytes(ctypes.byref(desc), backward))
+
+
+def sf_channel_chunked_fwd(desc: SegDesc, q, k, v, g, S_in, o, S_out, workspace, stream=None):
+    _check(load().sf_channel_chunked_fwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(S_in), _ptr(o), _ptr(S_out),
+                                         _ptr(workspace), workspace.numel(), _stream(stream)), "sf_channel_chunked_fwd")
+
+
+def sf_channel_chunked_bwd(desc: SegDesc, q, k, v, g, S_in, dO, dS_out, dq, dk, dv, dg, dS_in, workspace, stream=None):
+    _check(load().sf_channel_chunked_bwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(S_in), _ptr(dO), _ptr(dS_out),
+                                         _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dg), _ptr(dS_in), _ptr(workspace), workspace.numel(),
+                                         _stream(stream)), "sf_channel_chunked_bwd")
 
 
 def sf_delta_chunked_workspace_bytes(desc: SegDesc, backward: int) -> int:

@@ -3,6 +3,7 @@
 #include "../../include/stateflow.h"
 #include "sf_recurrent.cuh"
 #include "sf_delta_chunk.cuh"
+#include "sf_channel_chunk.cuh"
 
 namespace sf { void note_launches(long long n); }
 
@@ -186,6 +187,40 @@ sf_status_t chunked_backward(const sf_seg_desc_t* d, const sf::gdn::Params& p, c
     return launched(3);
 }
 
+// ---- chunkwise diagonal decay ----------------------------------------------------------------------------------------
+sf::dcc::Params channel_params(const sf_seg_desc_t* d) {
+    const sf::gdn::Params g = chunked_params(d);
+    sf::dcc::Params p;
+    p.B = g.B; p.H = g.H; p.L = g.L; p.C = g.C; p.NC = g.NC; p.dk = g.dk; p.dv = g.dv;
+    p.tqk = g.tqk; p.tv = g.tv; p.tg = g.tg; p.bqk = g.bqk; p.bv = g.bv; p.bg = g.bg;
+    return p;
+}
+
+size_t channel_chunked_ws_bytes(const sf_seg_desc_t* d, bool backward) {
+    return (size_t)d->B * d->H * sf::dcc::ws_floats(channel_params(d), backward) * sizeof(float);
+}
+
+template <typename T>
+sf_status_t channel_chunked_run(const sf::dcc::Params& p, const void* q, const void* k, const void* v, const float* g,
+                                const float* S_in, void* o, float* S_out, const void* dO, const float* dS_out, void* dq, void* dk,
+                                void* dv, float* dg, float* dS_in, float* ws, cudaStream_t st) {
+    using namespace sf::dcc;
+    const bool backward = dO != nullptr;
+    const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v), *tdo = static_cast<const T*>(dO);
+    const dim3 chunks(p.NC, p.H, p.B), elems((p.dk * p.dv + NT - 1) / NT, p.H, p.B);
+    const size_t s1 = smem_pre(p.C, p.dk, p.dv), s2 = smem_out(p.C, p.dk, p.dv), s3 = smem_bwd_out(p.C, p.dk, p.dv);
+    if (!opt_in(pre_kernel<T>, s1) || !opt_in(out_kernel<T>, s2) || !opt_in(bwd_out_kernel<T>, s3)) return SF_ERR_CUDA;
+    pre_kernel<T><<<chunks, NT, s1, st>>>(p, tq, tk, tv, g, tdo, ws, backward);
+    chain_kernel<<<elems, NT, 0, st>>>(p, 0, S_in, S_out, ws, backward);
+    if (!backward) {
+        out_kernel<T><<<chunks, NT, s2, st>>>(p, tq, tk, tv, g, static_cast<T*>(o), ws, 0);
+        return launched(3);
+    }
+    chain_kernel<<<elems, NT, 0, st>>>(p, 1, dS_out, dS_in, ws, 1);
+    bwd_out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, tv, g, tdo, static_cast<T*>(dq), static_cast<T*>(dk), static_cast<T*>(dv), dg, ws);
+    return launched(4);
+}
+
 }  // namespace
 
 extern "C" {
@@ -217,6 +252,40 @@ sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const
                                  sf_stream_t stream) {
     return rec_bwd<sf::rec::DELTA>(desc, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, workspace,
                                    workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+size_t sf_channel_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward) {
+    return check_chunked(desc) == SF_OK ? channel_chunked_ws_bytes(desc, backward != 0) : 0;
+}
+
+sf_status_t sf_channel_chunked_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                   const float* S_in, void* o, float* S_out, void* workspace, size_t workspace_bytes,
+                                   sf_stream_t stream) {
+    const sf_status_t c = check_chunked(desc);
+    if (c != SF_OK) return c;
+    if (!q || !k || !v || !g || !o || !S_out || S_in == S_out) return SF_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < channel_chunked_ws_bytes(desc, false) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SF_ERR_WORKSPACE;
+    const sf::dcc::Params p = channel_params(desc);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    float* ws = static_cast<float*>(workspace);
+    return desc->dtype == SF_F32
+        ? channel_chunked_run<float>(p, q, k, v, g, S_in, o, S_out, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, ws, st)
+        : channel_chunked_run<__nv_bfloat16>(p, q, k, v, g, S_in, o, S_out, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, ws, st);
+}
+
+sf_status_t sf_channel_chunked_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
+                                   const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk, void* dv,
+                                   float* dg, float* dS_in, void* workspace, size_t workspace_bytes, sf_stream_t stream) {
+    const sf_status_t c = check_chunked(desc);
+    if (c != SF_OK) return c;
+    if (!q || !k || !v || !g || !dO || !dq || !dk || !dv || !dg || !dS_in || dS_in == dS_out) return SF_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < channel_chunked_ws_bytes(desc, true) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SF_ERR_WORKSPACE;
+    const sf::dcc::Params p = channel_params(desc);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    float* ws = static_cast<float*>(workspace);
+    return desc->dtype == SF_F32
+        ? channel_chunked_run<float>(p, q, k, v, g, S_in, nullptr, nullptr, dO, dS_out, dq, dk, dv, dg, dS_in, ws, st)
+        : channel_chunked_run<__nv_bfloat16>(p, q, k, v, g, S_in, nullptr, nullptr, dO, dS_out, dq, dk, dv, dg, dS_in, ws, st);
 }
 
 size_t sf_delta_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward) {

@@ -26,7 +26,7 @@ def bounds(seg_lens):
 def run_recurrent(kind, w, x):
     """Chain of segments through sf_{channel,delta}_segment_{fwd,bwd}; returns the outputs over the whole sequence."""
     q, k, v, dO = x["q"], x["k"], x["v"], x["dO"]
-    g = x["g_channel"] if kind == "channel" else x["g"]
+    g = x["g_channel"] if kind.startswith("channel") else x["g"]
     beta = x["beta"]
     B, T, H, dk = q.shape
     dv = v.shape[-1]
@@ -40,6 +40,9 @@ def run_recurrent(kind, w, x):
         S_out = torch.empty(B, H, dk, dv, device=DEV)
         if kind == "channel":
             binding.sf_channel_segment_fwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], S[-1], o[:, a:b], S_out)
+        elif kind == "channel_chunked":
+            ws = torch.empty(binding.sf_channel_chunked_workspace_bytes(d, 0), dtype=torch.uint8, device=DEV)
+            binding.sf_channel_chunked_fwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], S[-1], o[:, a:b], S_out, ws)
         elif kind == "delta_chunked":
             ws = torch.empty(binding.sf_delta_chunked_workspace_bytes(d, 0), dtype=torch.uint8, device=DEV)
             binding.sf_delta_chunked_fwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], beta[:, a:b], S[-1], o[:, a:b], S_out, ws)
@@ -50,12 +53,16 @@ def run_recurrent(kind, w, x):
     for i in range(len(segs) - 1, -1, -1):
         a, b = segs[i]
         d = binding.make_desc(q[:, a:b], v[:, a:b], x["g"][:, a:b], w.chunk)
-        nws = binding.sf_delta_chunked_workspace_bytes(d, 1) if kind == "delta_chunked" else binding.sf_recurrent_workspace_bytes(d)
+        nws = (binding.sf_delta_chunked_workspace_bytes(d, 1) if kind == "delta_chunked" else
+               binding.sf_channel_chunked_workspace_bytes(d, 1) if kind == "channel_chunked" else binding.sf_recurrent_workspace_bytes(d))
         ws = torch.empty(nws, dtype=torch.uint8, device=DEV)
         dS_in = torch.empty(B, H, dk, dv, device=DEV)
         if kind == "delta_chunked":
             binding.sf_delta_chunked_bwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], beta[:, a:b], S[i], dO[:, a:b], G,
                                          dq[:, a:b], dk_[:, a:b], dv_[:, a:b], dg[:, a:b], dbeta[:, a:b], dS_in, ws)
+        elif kind == "channel_chunked":
+            binding.sf_channel_chunked_bwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], S[i], dO[:, a:b], G,
+                                           dq[:, a:b], dk_[:, a:b], dv_[:, a:b], dg[:, a:b], dS_in, ws)
         elif kind == "channel":
             binding.sf_channel_segment_bwd(d, q[:, a:b], k[:, a:b], v[:, a:b], g[:, a:b], S[i], dO[:, a:b], G,
                                            dq[:, a:b], dk_[:, a:b], dv_[:, a:b], dg[:, a:b], dS_in, ws)
@@ -65,7 +72,7 @@ def run_recurrent(kind, w, x):
         G = dS_in
     torch.cuda.synchronize()
     out = dict(o=o, S_out=S[-1], dq=dq, dk=dk_, dv=dv_, dg=dg, dS_in=G)
-    if kind != "channel":
+    if kind.startswith("delta"):
         out["dbeta"] = dbeta
     return out
 
@@ -231,3 +238,39 @@ def test_chunked_delta_rule_long_segment_bf16_and_agreement_with_the_token_kerne
                   ds_out_sigma=0.5, seed=34)
     xb = inputs.make_variant_inputs(wb, DEV)
     check(run_recurrent("delta_chunked", wb, xb), oracle_recurrent("delta", xb), wb.name, tol=2e-2)
+
+
+# ---- chunkwise form of the diagonal decay: same operator, same oracle -------------------------------------------------
+
+@pytest.mark.parametrize("chunk", [16, 32])
+@pytest.mark.parametrize("dk,dv", [(32, 32), (64, 64), (32, 64), (64, 32)])
+def test_chunked_diagonal_decay_matches_the_oracle(chunk, dk, dv):
+    w = Workload("dchunk-%d-%d-%d" % (chunk, dk, dv), 2, 3, dk, dv, [3 * chunk + 5, chunk, 100, 5, 1], chunk, dtype="f32",
+                 qk_norm="l2", g_scale=0.3, s_in_sigma=0.5, ds_out_sigma=0.5, seed=41)
+    x = inputs.make_variant_inputs(w, DEV)
+    check(run_recurrent("channel_chunked", w, x), oracle_recurrent("channel", x), w.name)
+
+
+@pytest.mark.parametrize("g_scale", [1.0, 0.01, 0.0])
+def test_chunked_diagonal_decay_regimes_and_absent_boundary_states(g_scale):
+    w = Workload("dchunk-g%g" % g_scale, 1, 2, 64, 64, [64, 200], 32, dtype="f32", qk_norm="l2", g_scale=g_scale, seed=42)
+    x = inputs.make_variant_inputs(w, DEV)
+    check(run_recurrent("channel_chunked", w, x), oracle_recurrent("channel", x), w.name)
+
+
+def test_chunked_diagonal_decay_long_segment_bf16_and_agreement_with_the_token_kernel():
+    w = Workload("dchunk-long", 1, 4, 64, 64, [2048], 32, dtype="f32", qk_norm="l2", g_scale=0.1, s_in_sigma=0.3,
+                 ds_out_sigma=0.3, seed=43)
+    x = inputs.make_variant_inputs(w, DEV)
+    a = run_recurrent("channel_chunked", w, x)
+    b = run_recurrent("channel_chunked", w, x)
+    for n in a:
+        assert torch.equal(a[n], b[n]), n
+    check(a, oracle_recurrent("channel", x), w.name)
+    t = run_recurrent("channel", w, x)
+    for n in a:
+        assert norm_err(f64(a[n]), f64(t[n])) <= 2 * TOL, n
+    wb = Workload("dchunk-bf16", 2, 3, 64, 32, [37, 16, 100, 5, 1], 16, dtype="bf16", qk_norm="l2", g_scale=0.3, s_in_sigma=0.5,
+                  ds_out_sigma=0.5, seed=44)
+    xb = inputs.make_variant_inputs(wb, DEV)
+    check(run_recurrent("channel_chunked", wb, xb), oracle_recurrent("channel", xb), wb.name, tol=2e-2)

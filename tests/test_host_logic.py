@@ -248,3 +248,21 @@ def test_chunked_delta_rule_validates_before_any_launch(lib):
     bad = list(bargs)
     bad[12] = None                                                  # dbeta missing
     assert lib.sf_delta_chunked_bwd(ctypes.byref(d), *bad, W, 1 << 40, None) == 1
+
+
+def test_chunked_diagonal_decay_validates_before_any_launch(lib):
+    f32 = dict(dtype=binding.SF_F32, d_k=64, d_v=32, seg_len=100, chunk=32)
+    d = desc(**f32)
+    lib.sf_channel_chunked_workspace_bytes.restype = ctypes.c_size_t
+    per_bh = 4 * 64 * 32 + 4 * 64 + 5 * 64 * 32                     # Psi and gam_n per chunk, NC + 1 states (4 chunks)
+    assert lib.sf_channel_chunked_workspace_bytes(ctypes.byref(d), 0) == 2 * per_bh * 4
+    assert lib.sf_channel_chunked_workspace_bytes(ctypes.byref(d), 1) == 2 * (per_bh + 2 * 4 * 64 * 32) * 4
+    S1, S2, W = ctypes.c_void_p(0x20000), ctypes.c_void_p(0x30000), ctypes.c_void_p(0x40000)
+    cf = lambda dd, q=P, S_in=None, ws=W, n=1 << 40: lib.sf_channel_chunked_fwd(ctypes.byref(dd), q, P, P, P, S_in, P, S1, ws, n, None)
+    assert cf(d, q=None) == 1 and cf(d, S_in=S1) == 1 and cf(d, ws=None) == 3 and cf(d, n=16) == 3
+    assert cf(desc(**dict(f32, chunk=64))) == 2 and cf(desc(**dict(f32, d_v=128))) == 2 and cf(desc(**dict(f32, seg_len=0))) == 1
+    bargs = [P] * 4 + [None, P, None] + [P] * 4 + [S2]
+    assert lib.sf_channel_chunked_bwd(ctypes.byref(d), *bargs, W, 16, None) == 3
+    bad = list(bargs)
+    bad[5] = None                                                    # dO missing
+    assert lib.sf_channel_chunked_bwd(ctypes.byref(d), *bad, W, 1 << 40, None) == 1

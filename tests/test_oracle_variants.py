@@ -301,3 +301,51 @@ def test_delta_oracle_equals_the_chunkwise_ut_form(T, C, dk, dv):
     for a, r in zip(got, ref[:5]):
         np.testing.assert_allclose(a, r[0, :, 0], rtol=1e-9, atol=1e-11)
     np.testing.assert_allclose(dH, ref[5][0, 0], rtol=1e-9, atol=1e-11)
+
+
+# ---- the chunkwise form of the diagonal decay in numpy: a second algorithm for the same operator --------------------
+
+def _dchunk_fwd(Q, K, Vv, g, H):
+    b = np.cumsum(g, axis=0)
+    gam = np.exp(b)
+    D = np.exp(b[:, None, :] - b[None, :, :])
+    A = np.tril(np.einsum("ti,si,tsi->ts", Q, K, D))
+    Kw = K * np.exp(b[-1][None, :] - b)
+    Hn = gam[-1][:, None] * H + Kw.T @ Vv
+    return A @ Vv + (Q * gam) @ H, Hn, dict(b=b, gam=gam, D=D, A=A, Kw=Kw, H=H, Hn=Hn)
+
+
+def _dchunk_bwd(Q, K, Vv, c, dO, dHn):
+    b, gam, D, A, Kw, H, Hn = (c[n] for n in ("b", "gam", "D", "A", "Kw", "H", "Hn"))
+    dA = np.tril(dO @ Vv.T)
+    dQ = np.einsum("ts,si,tsi->ti", dA, K, D) + gam * (dO @ H.T)
+    dK = np.einsum("ts,ti,tsi->si", dA, Q, D) + np.exp(b[-1][None, :] - b) * (Vv @ dHn.T)
+    dV = A.T @ dO + Kw @ dHn
+    # rows of S are independent scalar recurrences: dg_t = dg_{t+1} + q dq - k dk per channel, anchored at the chunk end
+    dg = np.cumsum((Q * dQ - K * dK)[::-1], axis=0)[::-1] + np.sum(dHn * Hn, axis=1)[None, :]
+    return dQ, dK, dV, dg, gam[-1][:, None] * dHn + (Q * gam).T @ dO
+
+
+@pytest.mark.parametrize("T,C,dk,dv", [(50, 16, 5, 4), (33, 32, 3, 6)])
+def test_channel_oracle_equals_the_chunkwise_form(T, C, dk, dv):
+    q, k, v, g, _, S = make(57, T=T, H=1, dk=dk, dv=dv, channel=True)
+    dO, dS = rnd(90, *v.shape), rnd(91, *S.shape)
+    o_ref, S_ref = V.channel_fwd(q, k, v, g, S)
+    ref = V.channel_bwd(q, k, v, g, S, dO, dS)
+    sl = [slice(t0, min(T, t0 + C)) for t0 in range(0, T, C)]
+    H, caches, o = S[0, 0].copy(), [], np.zeros((T, dv))
+    for s in sl:
+        o[s], H, c = _dchunk_fwd(q[0, s, 0], k[0, s, 0], v[0, s, 0], g[0, s, 0], H)
+        caches.append(c)
+    np.testing.assert_allclose(o, o_ref[0, :, 0], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(H, S_ref[0, 0], rtol=1e-11, atol=1e-12)
+    dH = dS[0, 0].copy()
+    got = [np.zeros((T, dk)), np.zeros((T, dk)), np.zeros((T, dv)), np.zeros((T, dk))]
+    for s, c in zip(sl[::-1], caches[::-1]):
+        res = _dchunk_bwd(q[0, s, 0], k[0, s, 0], v[0, s, 0], c, dO[0, s, 0], dH)
+        for a, x in zip(got, res[:4]):
+            a[s] = x
+        dH = res[4]
+    for a, r in zip(got, ref[:4]):
+        np.testing.assert_allclose(a, r[0, :, 0], rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(dH, ref[4][0, 0], rtol=1e-9, atol=1e-11)
