@@ -444,7 +444,8 @@ sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const
  * built for all chunks in parallel, the state is carried from chunk to chunk element by element, and the outputs (and,
  * in the backward, every gradient, with dg anchored per chunk) are again formed for all chunks in parallel.  Same
  * arguments, layouts and results (to rounding) as sf_channel_segment_fwd/bwd.  desc->chunk in {16, 32}, d_k, d_v in
- * {32, 64}, float32 or bf16 storage, float32 arithmetic on CUDA cores.  Workspace:
+ * {32, 64, 128} as far as the kernels' tiles fit into shared memory (128-wide heads need chunk 16; otherwise
+ * SF_ERR_UNSUPPORTED), float32 or bf16 storage, float32 arithmetic on CUDA cores.  Workspace:
  * sf_channel_chunked_workspace_bytes(desc, backward) bytes, 256-byte aligned.
  */
 size_t sf_channel_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward);
@@ -461,7 +462,8 @@ sf_status_t sf_channel_chunked_bwd(const sf_seg_desc_t* desc, const void* q, con
  * all chunks in parallel (including each chunk's affine state map), ST carries the state from chunk to chunk, Out forms
  * V_new = W and the outputs of all chunks in parallel; the backward mirrors it (transposed solve, reverse state pass, chunk-parallel gradients).
  * Same arguments, layouts and results (to rounding) as sf_delta_segment_fwd/bwd.  desc->chunk in {16, 32},
- * d_k, d_v in {32, 64}, float32 or bf16 storage, float32 arithmetic on CUDA cores.  Workspace:
+ * d_k, d_v in {32, 64, 128} as far as the kernels' tiles fit into shared memory (128-wide heads need chunk 16; otherwise
+ * SF_ERR_UNSUPPORTED), float32 or bf16 storage, float32 arithmetic on CUDA cores.  Workspace:
  * sf_delta_chunked_workspace_bytes(desc, backward) bytes, 256-byte aligned (U and Wk per token, the chunk's state map
  * and one state per chunk; the backward rebuilds them and adds Z0 per token, Theta, one state gradient and two
  * chunk x chunk matrices per chunk).

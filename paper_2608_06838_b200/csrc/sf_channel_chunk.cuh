@@ -18,7 +18,8 @@
 //     dk[s,i] = sum_{t>=s} dA[t,s] q_t[i] exp(b_t[i]-b_s[i]) + om_s[i] (V dH'^T)[s,i]
 //     dg_t[i] = sum_{u>=t in the chunk} (q_u[i] dq_u[i] - k_u[i] dk_u[i]) + <dH'[i,:], H'[i,:]>           (rows of S are independent
 //               scalar recurrences, so the per-row identity dg_t = dg_{t+1} + q dq - k dk holds and is anchored per chunk)
-// Chunk length 16 or 32, d_k, d_v in {32, 64}; a last chunk with fewer tokens is handled by row counts.
+// Chunk length 16 or 32, d_k, d_v in {32, 64, 128} as far as the tiles fit into shared memory (128 needs chunk 16); a last
+// chunk with fewer tokens is handled by row counts.
 #pragma once
 #include "sf_delta_chunk.cuh"
 
@@ -218,8 +219,7 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
     float* Vs = dKs + C * ldk;         float* dOs = Vs + C * ldv;
     float* dVs = dOs + C * ldv;
     float* Hs = dVs + C * ldv;         float* dHs = Hs + dk * ldv;        // entering state, gradient of the leaving state
-    float* Hn = dHs + dk * ldv;                                           // leaving state
-    float* A = Hn + dk * ldv;          float* dA = A + C * ldc;
+    float* A = dHs + dk * ldv;         float* dA = A + C * ldc;
     float* anchor = dA + C * ldc;      // [dk]
     const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(const_cast<float*>(ws), p, bh, true);
@@ -231,7 +231,6 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
     load_rows(Vs, ldv, v + ov, p.tv, n, dv);
     load_rows(dOs, ldv, dO + ov, p.tv, n, dv);
     load_dense(Hs, ldv, w.Hc + (long long)c * dk * dv, dv, dk, dv);
-    load_dense(Hn, ldv, w.Hc + (long long)(c + 1) * dk * dv, dv, dk, dv);
     load_dense(dHs, ldv, w.dHc + (long long)c * dk * dv, dv, dk, dv);
     cumsum_channels(Bs, ldk, n, dk);
     decay_scores(A, ldc, Qs, Ks, Bs, ldk, n, dk);
@@ -242,9 +241,10 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
         const int t = idx / dk, i = idx - t * dk;
         Kw[t * ldk + i] = Ks[t * ldk + i] * __expf(Bs[(n - 1) * ldk + i] - Bs[t * ldk + i]);
     }
+    const float* Hn = w.Hc + (long long)(c + 1) * dk * dv;                // the state leaving the chunk, read once from memory
     for (int i = threadIdx.x; i < dk; i += NT) {
         float acc = 0.f;
-        for (int jj = 0; jj < dv; ++jj) acc = fmaf(dHs[i * ldv + jj], Hn[i * ldv + jj], acc);
+        for (int jj = 0; jj < dv; ++jj) acc = fmaf(dHs[i * ldv + jj], Hn[i * dv + jj], acc);
         anchor[i] = acc;
     }
     __syncthreads();
@@ -290,7 +290,12 @@ __host__ inline size_t smem_out(int C, int dk, int dv) {
     return sizeof(float) * (3 * (size_t)C * ldp(dk) + 2 * (size_t)C * ldp(dv) + (size_t)dk * ldp(dv) + (size_t)C * ldp(C));
 }
 __host__ inline size_t smem_bwd_out(int C, int dk, int dv) {
-    return sizeof(float) * (6 * (size_t)C * ldp(dk) + 3 * (size_t)C * ldp(dv) + 3 * (size_t)dk * ldp(dv) + 2 * (size_t)C * ldp(C) + dk);
+    return sizeof(float) * (6 * (size_t)C * ldp(dk) + 3 * (size_t)C * ldp(dv) + 2 * (size_t)dk * ldp(dv) + 2 * (size_t)C * ldp(C) + dk);
+}
+
+__host__ inline size_t smem_max(int C, int dk, int dv) {
+    const size_t a = smem_pre(C, dk, dv), b = smem_out(C, dk, dv), c = smem_bwd_out(C, dk, dv);
+    return a > b ? (a > c ? a : c) : (b > c ? b : c);
 }
 
 }  // namespace dcc

@@ -22,7 +22,8 @@
 //     dk = (dA*M)^T Q + om*(W dH'^T) - (beta*gam*Z) H^T + (P + P^T) K
 //     dv = beta*Z,    dbeta = rowsum(Z*V) - gam*rowsum(Z*KH) + rowsum(dL * M * KK^T)
 //     db_t (gradient of the cumulative log-decay) collects the M, gam, om terms; dg = reverse cumulative sum of db.
-// Chunk length 16 or 32, d_k, d_v in {32, 64}; a last chunk with fewer tokens is handled by row counts.
+// Chunk length 16 or 32, d_k, d_v in {32, 64, 128} as far as the tiles fit into shared memory (128 needs chunk 16); a last
+// chunk with fewer tokens is handled by row counts.
 #pragma once
 #include "sf_common.cuh"
 
@@ -216,6 +217,7 @@ __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__
 //      forward:  F = Phi[c],    R = Psi[c],    chunks ascending,  `states[c]` receives the state entering chunk c
 //      reverse:  F = Phi[c]^T,  R = Theta[c],  chunks descending, `states[c]` receives the gradient of the state leaving it
 //      grid (dv/DVS, H, B) ---------------------------------------------------------------------------------------------
+template <int DKM>      // DKM >= d_k: sizes the register prefetch
 __global__ void __launch_bounds__(NT) chain_kernel(Params p, int reverse, const float* __restrict__ init, float* __restrict__ fin,
                                                    float* ws, int backward) {
     extern __shared__ float sm[];
@@ -233,7 +235,7 @@ __global__ void __launch_bounds__(NT) chain_kernel(Params p, int reverse, const 
     else for (int idx = threadIdx.x; idx < dk * lds; idx += NT) X0[idx] = 0.f;
     __syncthreads();
     // The map of the next chunk is fetched into registers while the product of the current one runs.
-    constexpr int MAXF = (64 * 64) / NT, MAXR = (64 * DVS) / NT;         // d_k <= 64
+    constexpr int MAXF = (DKM * DKM) / NT, MAXR = (DKM * DVS) / NT;
     float fr[MAXF], rr[MAXR];
     auto fetch = [&](int c) {
         const float* F = w.Phi + (long long)c * dk * dk;
@@ -506,6 +508,13 @@ __host__ inline size_t smem_bwd_pre(int C, int dk, int dv) {
 __host__ inline size_t smem_bwd_out(int C, int dk, int dv) {
     return sizeof(float) * (2 * (size_t)C * ldp(dk) + 4 * (size_t)C * ldp(dv) + 2 * (size_t)dk * ldp(dv) + 4 * (size_t)C * ldp(C) +
                             2 * (size_t)C * ldp(dv) + 2 * (size_t)C * ldp(dk) + (size_t)C * ldp(dk > dv ? dk : dv) + 10 * (size_t)C + dk);
+}
+
+__host__ inline size_t smem_max(int C, int dk, int dv) {
+    size_t m = smem_pre(C, dk, dv);
+    const size_t o[4] = {smem_chain(dk), smem_out(C, dk, dv), smem_bwd_pre(C, dk, dv), smem_bwd_out(C, dk, dv)};
+    for (size_t x : o) m = x > m ? x : m;
+    return m;
 }
 
 }  // namespace gdn

@@ -14,7 +14,7 @@ using sf::rec::RecParams;
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 bool aligned2(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 1u) == 0; }
 
-sf_status_t check_desc(const sf_seg_desc_t* d) {
+sf_status_t check_desc(const sf_seg_desc_t* d, bool wide_keys = false) {
     if (!d) return SF_ERR_INVALID_ARG;
     if (d->B <= 0 || d->H <= 0 || d->seg_len <= 0 || d->d_k <= 0 || d->d_v <= 0) return SF_ERR_INVALID_ARG;
     if (d->B > 65535) return SF_ERR_INVALID_ARG;                                       // grid.y
@@ -22,7 +22,7 @@ sf_status_t check_desc(const sf_seg_desc_t* d) {
         return SF_ERR_INVALID_ARG;
     if (d->B > 1 && (d->batch_stride_qk <= 0 || d->batch_stride_v <= 0 || d->batch_stride_g <= 0)) return SF_ERR_INVALID_ARG;
     if (d->dtype != SF_F32 && d->dtype != SF_BF16) return SF_ERR_INVALID_ARG;
-    const bool k_ok = d->d_k == 32 || d->d_k == 64;
+    const bool k_ok = d->d_k == 32 || d->d_k == 64 || (wide_keys && d->d_k == 128);
     const bool v_ok = d->d_v == 32 || d->d_v == 64 || d->d_v == 128;
     return k_ok && v_ok ? SF_OK : SF_ERR_UNSUPPORTED;
 }
@@ -123,13 +123,17 @@ int conv_grid(long long n) {
 }
 
 // ---- chunkwise delta rule ----------------------------------------------------------------------------------------
-sf_status_t check_chunked(const sf_seg_desc_t* d) {
-    const sf_status_t c = check_desc(d);
+constexpr size_t kMaxSmem = 227 * 1024;       // dynamic shared memory a CTA can opt into on this architecture
+
+// `delta`: the delta-rule kernels, else the diagonal-decay ones; the shape is supported if every kernel's tiles fit
+sf_status_t check_chunked(const sf_seg_desc_t* d, bool delta) {
+    const sf_status_t c = check_desc(d, true);
     if (c != SF_OK) return c;
     if (d->chunk <= 0) return SF_ERR_INVALID_ARG;
-    if ((d->chunk != 16 && d->chunk != 32) || d->d_v == 128) return SF_ERR_UNSUPPORTED;
+    if (d->chunk != 16 && d->chunk != 32) return SF_ERR_UNSUPPORTED;
     if (d->H > 65535) return SF_ERR_INVALID_ARG;
-    return SF_OK;
+    const size_t need = delta ? sf::gdn::smem_max(d->chunk, d->d_k, d->d_v) : sf::dcc::smem_max(d->chunk, d->d_k, d->d_v);
+    return need <= kMaxSmem ? SF_OK : SF_ERR_UNSUPPORTED;
 }
 
 sf::gdn::Params chunked_params(const sf_seg_desc_t* d) {
@@ -161,9 +165,11 @@ sf_status_t chunked_forward(const sf_seg_desc_t* d, const sf::gdn::Params& p, co
     const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v);
     const dim3 chunks(p.NC, p.H, p.B), cols(p.dv / DVS, p.H, p.B);
     const size_t s1 = smem_pre(p.C, p.dk, p.dv), s2 = smem_chain(p.dk), s3 = smem_out(p.C, p.dk, p.dv);
-    if (!opt_in(pre_kernel<T>, s1) || !opt_in(chain_kernel, s2) || !opt_in(out_kernel<T>, s3)) return SF_ERR_CUDA;
+    if (!opt_in(pre_kernel<T>, s1) || !opt_in(chain_kernel<64>, s2) || !opt_in(chain_kernel<128>, s2) || !opt_in(out_kernel<T>, s3))
+        return SF_ERR_CUDA;
     pre_kernel<T><<<chunks, NT, s1, st>>>(p, tq, tk, tv, g, beta, ws, backward);
-    chain_kernel<<<cols, NT, s2, st>>>(p, 0, S_in, S_out, ws, backward);
+    if (p.dk <= 64) chain_kernel<64><<<cols, NT, s2, st>>>(p, 0, S_in, S_out, ws, backward);
+    else            chain_kernel<128><<<cols, NT, s2, st>>>(p, 0, S_in, S_out, ws, backward);
     int n = 2;
     if (o) { out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, g, static_cast<T*>(o), ws, backward); ++n; }
     return launched(n);
@@ -179,9 +185,11 @@ sf_status_t chunked_backward(const sf_seg_desc_t* d, const sf::gdn::Params& p, c
     const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v), *tdo = static_cast<const T*>(dO);
     const dim3 chunks(p.NC, p.H, p.B), cols(p.dv / DVS, p.H, p.B);
     const size_t s1 = smem_bwd_pre(p.C, p.dk, p.dv), s2 = smem_chain(p.dk), s3 = smem_bwd_out(p.C, p.dk, p.dv);
-    if (!opt_in(bwd_pre_kernel<T>, s1) || !opt_in(chain_kernel, s2) || !opt_in(bwd_out_kernel<T>, s3)) return SF_ERR_CUDA;
+    if (!opt_in(bwd_pre_kernel<T>, s1) || !opt_in(chain_kernel<64>, s2) || !opt_in(chain_kernel<128>, s2) || !opt_in(bwd_out_kernel<T>, s3))
+        return SF_ERR_CUDA;
     bwd_pre_kernel<T><<<chunks, NT, s1, st>>>(p, tq, tk, g, beta, tdo, ws);
-    chain_kernel<<<cols, NT, s2, st>>>(p, 1, dS_out, dS_in, ws, 1);
+    if (p.dk <= 64) chain_kernel<64><<<cols, NT, s2, st>>>(p, 1, dS_out, dS_in, ws, 1);
+    else            chain_kernel<128><<<cols, NT, s2, st>>>(p, 1, dS_out, dS_in, ws, 1);
     bwd_out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, tv, g, beta, tdo, static_cast<T*>(dq), static_cast<T*>(dk), static_cast<T*>(dv),
                                               dg, dbeta, ws);
     return launched(3);
@@ -255,13 +263,13 @@ sf_status_t sf_delta_segment_bwd(const sf_seg_desc_t* desc, const void* q, const
 }
 
 size_t sf_channel_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward) {
-    return check_chunked(desc) == SF_OK ? channel_chunked_ws_bytes(desc, backward != 0) : 0;
+    return check_chunked(desc, false) == SF_OK ? channel_chunked_ws_bytes(desc, backward != 0) : 0;
 }
 
 sf_status_t sf_channel_chunked_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
                                    const float* S_in, void* o, float* S_out, void* workspace, size_t workspace_bytes,
                                    sf_stream_t stream) {
-    const sf_status_t c = check_chunked(desc);
+    const sf_status_t c = check_chunked(desc, false);
     if (c != SF_OK) return c;
     if (!q || !k || !v || !g || !o || !S_out || S_in == S_out) return SF_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes < channel_chunked_ws_bytes(desc, false) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SF_ERR_WORKSPACE;
@@ -276,7 +284,7 @@ sf_status_t sf_channel_chunked_fwd(const sf_seg_desc_t* desc, const void* q, con
 sf_status_t sf_channel_chunked_bwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
                                    const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk, void* dv,
                                    float* dg, float* dS_in, void* workspace, size_t workspace_bytes, sf_stream_t stream) {
-    const sf_status_t c = check_chunked(desc);
+    const sf_status_t c = check_chunked(desc, false);
     if (c != SF_OK) return c;
     if (!q || !k || !v || !g || !dO || !dq || !dk || !dv || !dg || !dS_in || dS_in == dS_out) return SF_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes < channel_chunked_ws_bytes(desc, true) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SF_ERR_WORKSPACE;
@@ -289,13 +297,13 @@ sf_status_t sf_channel_chunked_bwd(const sf_seg_desc_t* desc, const void* q, con
 }
 
 size_t sf_delta_chunked_workspace_bytes(const sf_seg_desc_t* desc, int backward) {
-    return check_chunked(desc) == SF_OK ? chunked_ws_bytes(desc, backward != 0) : 0;
+    return check_chunked(desc, true) == SF_OK ? chunked_ws_bytes(desc, backward != 0) : 0;
 }
 
 sf_status_t sf_delta_chunked_fwd(const sf_seg_desc_t* desc, const void* q, const void* k, const void* v, const float* g,
                                  const float* beta, const float* S_in, void* o, float* S_out, void* workspace, size_t workspace_bytes,
                                  sf_stream_t stream) {
-    const sf_status_t c = check_chunked(desc);
+    const sf_status_t c = check_chunked(desc, true);
     if (c != SF_OK) return c;
     if (!q || !k || !v || !g || !beta || !o || !S_out || S_in == S_out) return SF_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes < chunked_ws_bytes(desc, false) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SF_ERR_WORKSPACE;
@@ -310,7 +318,7 @@ sf_status_t sf_delta_chunked_bwd(const sf_seg_desc_t* desc, const void* q, const
                                  const float* beta, const float* S_in, const void* dO, const float* dS_out, void* dq, void* dk,
                                  void* dv, float* dg, float* dbeta, float* dS_in, void* workspace, size_t workspace_bytes,
                                  sf_stream_t stream) {
-    const sf_status_t c = check_chunked(desc);
+    const sf_status_t c = check_chunked(desc, true);
     if (c != SF_OK) return c;
     if (!q || !k || !v || !g || !beta || !dO || !dq || !dk || !dv || !dg || !dbeta || !dS_in || dS_in == dS_out) return SF_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes < chunked_ws_bytes(desc, true) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SF_ERR_WORKSPACE;

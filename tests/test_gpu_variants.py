@@ -274,3 +274,16 @@ def test_chunked_diagonal_decay_long_segment_bf16_and_agreement_with_the_token_k
                   ds_out_sigma=0.5, seed=44)
     xb = inputs.make_variant_inputs(wb, DEV)
     check(run_recurrent("channel_chunked", wb, xb), oracle_recurrent("channel", xb), wb.name, tol=2e-2)
+
+
+@pytest.mark.parametrize("kind", ["delta_chunked", "channel_chunked"])
+def test_chunked_operators_with_128_wide_heads(kind):
+    # the head width of the paper's models; the tiles fit into shared memory with 16-token chunks
+    w = Workload("%s-128" % kind, 1, 2, 128, 128, [53, 16, 7], 16, dtype="f32", qk_norm="l2", g_scale=0.3, s_in_sigma=0.5,
+                 ds_out_sigma=0.5, seed=51)
+    x = inputs.make_variant_inputs(w, DEV)
+    check(run_recurrent(kind, w, x), oracle_recurrent("delta" if kind == "delta_chunked" else "channel", x), w.name)
+    wb = Workload("%s-128-bf16" % kind, 2, 2, 128, 128, [40, 9], 16, dtype="bf16", qk_norm="l2", g_scale=0.3, s_in_sigma=0.5,
+                  ds_out_sigma=0.5, seed=52)
+    xb = inputs.make_variant_inputs(wb, DEV)
+    check(run_recurrent(kind, wb, xb), oracle_recurrent("delta" if kind == "delta_chunked" else "channel", xb), wb.name, tol=2e-2)

@@ -241,7 +241,8 @@ def test_chunked_delta_rule_validates_before_any_launch(lib):
     cf = lambda dd, q=P, beta=P, S_in=None, ws=W, n=1 << 40: lib.sf_delta_chunked_fwd(ctypes.byref(dd), q, P, P, P, beta, S_in, P, S1, ws, n, None)
     assert cf(d, q=None) == 1 and cf(d, beta=None) == 1 and cf(d, S_in=S1) == 1
     assert cf(d, ws=None) == 3 and cf(d, n=16) == 3 and cf(d, ws=ctypes.c_void_p(0x40010)) == 3
-    assert cf(desc(**dict(f32, chunk=64))) == 2 and cf(desc(**dict(f32, d_v=128))) == 2 and cf(desc(**dict(f32, d_k=128))) == 2
+    assert cf(desc(**dict(f32, chunk=64))) == 2 and cf(desc(**dict(f32, d_v=128))) == 2 and cf(desc(**dict(f32, d_k=128, d_v=128))) == 2
+    assert lib.sf_delta_chunked_workspace_bytes(ctypes.byref(desc(**dict(f32, d_k=128, d_v=128, chunk=16))), 1) > 0   # 128-wide heads fit at chunk 16
     assert cf(desc(**dict(f32, chunk=0))) == 1 and cf(desc(**dict(f32, seg_len=0))) == 1
     bargs = [P] * 5 + [None, P, None] + [P] * 5 + [S2]
     assert lib.sf_delta_chunked_bwd(ctypes.byref(d), *bargs, W, 16, None) == 3
@@ -260,7 +261,10 @@ def test_chunked_diagonal_decay_validates_before_any_launch(lib):
     S1, S2, W = ctypes.c_void_p(0x20000), ctypes.c_void_p(0x30000), ctypes.c_void_p(0x40000)
     cf = lambda dd, q=P, S_in=None, ws=W, n=1 << 40: lib.sf_channel_chunked_fwd(ctypes.byref(dd), q, P, P, P, S_in, P, S1, ws, n, None)
     assert cf(d, q=None) == 1 and cf(d, S_in=S1) == 1 and cf(d, ws=None) == 3 and cf(d, n=16) == 3
-    assert cf(desc(**dict(f32, chunk=64))) == 2 and cf(desc(**dict(f32, d_v=128))) == 2 and cf(desc(**dict(f32, seg_len=0))) == 1
+    assert cf(desc(**dict(f32, chunk=64))) == 2 and cf(desc(**dict(f32, seg_len=0))) == 1
+    wide = dict(f32, d_k=128, d_v=128)
+    assert cf(desc(**wide)) == 2                                     # 128-wide heads do not fit at chunk 32 ...
+    assert lib.sf_channel_chunked_workspace_bytes(ctypes.byref(desc(**dict(wide, chunk=16))), 1) > 0   # ... but do at chunk 16
     bargs = [P] * 4 + [None, P, None] + [P] * 4 + [S2]
     assert lib.sf_channel_chunked_bwd(ctypes.byref(d), *bargs, W, 16, None) == 3
     bad = list(bargs)
