@@ -398,7 +398,7 @@ def main():
                 "note": "stage timers: second pass of the same steps at the same block length with the stream overlap off"}
         roof["frac"] = roof["achieved"] / peak
     # bounded CPU sample: about 5-10 s of oracle work on the machine's cores (fp64 copies of the sample: a few GB of host memory)
-    cpu = None if args.skip_cpu else cpu_baseline(w, min(w.T, (16384 * 32 // w.H) // w.chunk * w.chunk))
+    cpu = None if args.skip_cpu else cpu_baseline(w, min(w.T, (49152 * 32 // w.H) // w.chunk * w.chunk))   # about 10 s of CPU work
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
