@@ -32,24 +32,27 @@ namespace gdn {
 
 constexpr int NT = 256;
 constexpr int DVS = 16;            // value columns per CTA in the sequential kernels
+constexpr int GR = 16;             // chunks per block of the two-level state pass
 
 struct Params {
     int B, H, L, C, NC, dk, dv;
     long long tqk, tv, tg, bqk, bv, bg;      // token / batch strides in elements
 };
 
-// Workspace per (batch, head), in floats: U [L][dv], Wk [L][dk], Phi [NC][dk][dk], Psi [NC][dk][dv], Hc [NC][dk][dv];
+// Workspace per (batch, head), in floats: U [L][dv], Wk [L][dk], Phi [NC][dk][dk], Psi [NC][dk][dv], Hc [NC][dk][dv],
+// Pb [NB][dk][dk], Sb [NB][dk][dv], Hb [NB][dk][dv] (maps composed over blocks of GR chunks and the states entering them);
 // the backward adds Z0 [L][dv], Theta [NC][dk][dv], dHc [NC][dk][dv], A [NC][C][C] (the masked Q K^T) and
 // Ti [NC][C][C] (the inverse of I + L, used transposed).
-struct Ws { float *U, *Wk, *Phi, *Psi, *Hc, *Z0, *Theta, *dHc, *A, *Ti; };
+struct Ws { float *U, *Wk, *Phi, *Psi, *Hc, *Pb, *Sb, *Hb, *Z0, *Theta, *dHc, *A, *Ti; };
 __host__ __device__ inline size_t ws_floats(const Params& p, bool backward) {
-    const size_t st = (size_t)p.NC * p.dk * p.dv;
+    const size_t st = (size_t)p.NC * p.dk * p.dv, nb = (size_t)((p.NC + GR - 1) / GR);
     size_t n = (size_t)p.L * p.dv + (size_t)p.L * p.dk + (size_t)p.NC * p.dk * p.dk + 2 * st;
+    n += nb * p.dk * p.dk + 2 * nb * p.dk * p.dv;                        // composed maps and entering states of the blocks
     if (backward) n += (size_t)p.L * p.dv + 2 * st + 2 * (size_t)p.NC * p.C * p.C;
     return n;
 }
 __host__ __device__ inline Ws ws_of(float* base, const Params& p, long long bh, bool backward) {
-    const size_t st = (size_t)p.NC * p.dk * p.dv;
+    const size_t st = (size_t)p.NC * p.dk * p.dv, nb = (size_t)((p.NC + GR - 1) / GR);
     float* c = base + bh * (long long)ws_floats(p, backward);
     Ws w;
     w.U = c;   c += (size_t)p.L * p.dv;
@@ -57,6 +60,9 @@ __host__ __device__ inline Ws ws_of(float* base, const Params& p, long long bh, 
     w.Phi = c; c += (size_t)p.NC * p.dk * p.dk;
     w.Psi = c; c += st;
     w.Hc = c;  c += st;
+    w.Pb = c;  c += nb * p.dk * p.dk;
+    w.Sb = c;  c += nb * p.dk * p.dv;
+    w.Hb = c;  c += nb * p.dk * p.dv;
     w.Z0 = w.Theta = w.dHc = w.A = w.Ti = nullptr;
     if (backward) {
         w.Z0 = c;    c += (size_t)p.L * p.dv;
@@ -103,6 +109,45 @@ __device__ __forceinline__ void mm(float* out, int ldo, const float* A, int lda,
             }
         }
     }
+}
+
+// The same product with a 4 x 4 block of outputs per thread (M and N multiples of 4): 8 shared-memory reads for 16
+// multiply-adds instead of 20, for the larger products (the composed maps).  Same rule for `keep`.
+__device__ __forceinline__ void mm4x4(float* out, int ldo, const float* A, int lda, bool ta, const float* Bm, int ldb, bool tb,
+                                      int M, int N, int K, float keep, float sign) {
+    const int tn = N >> 2, total = (M >> 2) * tn, sa = ta ? lda : 1, sb = tb ? 1 : ldb;
+    for (int t = threadIdx.x; t < total; t += NT) {
+        const int m0 = (t / tn) << 2, n0 = (t - (t / tn) * tn) << 2;
+        const float* a = ta ? A + m0 : A + m0 * lda;
+        const float* b = tb ? Bm + n0 * ldb : Bm + n0;
+        const int ra = ta ? 1 : lda, rb = tb ? ldb : 1;               // step to the next of the four rows / columns
+        float acc[4][4] = {};
+#pragma unroll 2
+        for (int k = 0; k < K; ++k) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { av[i] = a[i * ra + k * sa]; bv[i] = b[i * rb + k * sb]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) acc[i][jj] = fmaf(av[i], bv[jj], acc[i][jj]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                float* o = out + (m0 + i) * ldo + n0 + jj;
+                *o = keep != 0.f ? fmaf(keep, *o, sign * acc[i][jj]) : sign * acc[i][jj];
+            }
+    }
+}
+
+// Picks the blocked product when the shape allows it and leaves at least half of the threads busy.  The choice depends on
+// the shape alone, so two products that accumulate into the same output take the same path (same thread, same element).
+__device__ __forceinline__ void mmx(float* out, int ldo, const float* A, int lda, bool ta, const float* Bm, int ldb, bool tb,
+                                    int M, int N, int K, float keep, float sign) {
+    if (((M | N) & 3) == 0 && (M >> 2) * (N >> 2) >= NT / 4) mm4x4(out, ldo, A, lda, ta, Bm, ldb, tb, M, N, K, keep, sign);
+    else mm(out, ldo, A, lda, ta, Bm, ldb, tb, M, N, K, keep, sign);
 }
 
 template <typename T>
@@ -180,7 +225,7 @@ __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__
         const int t = idx / dk, i = idx - t * dk;
         Kw[t * ldk + i] = __expf(bn - b[t]) * Ks[t * ldk + i];
     }
-    mm(Lm, ldc, Ks, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);     // K K^T
+    mmx(Lm, ldc, Ks, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);     // K K^T
     __syncthreads();
     for (int idx = threadIdx.x; idx < n * n; idx += NT) {
         const int t = idx / n, s = idx - t * n;
@@ -198,11 +243,11 @@ __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__
     store_dense(w.U + (long long)t0 * dv, dv, X, ldx, n, dv);
     store_dense(w.Wk + (long long)t0 * dk, dk, X + dv, ldx, n, dk);
     float* Phi = w.Phi + (long long)c * dk * dk;
-    mm(Phi, dk, Kw, ldk, true, X + dv, ldx, false, dk, dk, n, 0.f, -1.f);                 // -(om*K)^T Wk
-    mm(w.Psi + (long long)c * dk * dv, dv, Kw, ldk, true, X, ldx, false, dk, dv, n, 0.f, 1.f);
+    mmx(Phi, dk, Kw, ldk, true, X + dv, ldx, false, dk, dk, n, 0.f, -1.f);                 // -(om*K)^T Wk
+    mmx(w.Psi + (long long)c * dk * dv, dv, Kw, ldk, true, X, ldx, false, dk, dv, n, 0.f, 1.f);
     if (backward) {
         store_dense(w.Ti + (long long)c * C * C, C, X + dv + dk, ldx, n, n);
-        mm(Lm, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f); // Q K^T (L is no longer needed)
+        mmx(Lm, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f); // Q K^T (L is no longer needed)
     }
     __syncthreads();
     for (int i = threadIdx.x; i < dk; i += NT) Phi[i * dk + i] += __expf(bn);
@@ -213,32 +258,46 @@ __global__ void __launch_bounds__(NT) pre_kernel(Params p, const T* __restrict__
         }
 }
 
-// ---- ST (forward) and its adjoint (reverse): X' = F X + R per chunk for DVS columns of the state, where
-//      forward:  F = Phi[c],    R = Psi[c],    chunks ascending,  `states[c]` receives the state entering chunk c
-//      reverse:  F = Phi[c]^T,  R = Theta[c],  chunks descending, `states[c]` receives the gradient of the state leaving it
-//      grid (dv/DVS, H, B) ---------------------------------------------------------------------------------------------
+// ---- ST (forward) and its adjoint (reverse): X' = F X + R step by step for DVS columns of the state.
+//      CHUNKS_FWD  F = Phi[c],    R = Psi[c],    all chunks ascending;  Hc[c]  <- state entering chunk c
+//      CHUNKS_REV  F = Phi[c]^T,  R = Theta[c],  all chunks descending; dHc[c] <- gradient of the state leaving chunk c
+//      The two-level pass shortens the dependency chain from NC steps to about GR + NC/GR + GR: compose_kernel multiplies
+//      the maps of each block of GR chunks together (all blocks in parallel), then
+//      BLOCKS_FWD / BLOCKS_REV  F = Pb[j], R = Sb[j] over the blocks;  Hb[j] <- state (gradient) entering block j
+//      INBLOCK_FWD / INBLOCK_REV  the chunks of block j = blockIdx.y starting from Hb[j] (all blocks in parallel)
+//      grid (dv/DVS, H, B), for INBLOCK_* (dv/DVS, NB, B*H) --------------------------------------------------------------
+enum : int { CHUNKS_FWD = 0, CHUNKS_REV = 1, BLOCKS_FWD = 2, BLOCKS_REV = 3, INBLOCK_FWD = 4, INBLOCK_REV = 5 };
+
 template <int DKM>      // DKM >= d_k: sizes the register prefetch
-__global__ void __launch_bounds__(NT) chain_kernel(Params p, int reverse, const float* __restrict__ init, float* __restrict__ fin,
+__global__ void __launch_bounds__(NT) chain_kernel(Params p, int mode, const float* __restrict__ init, float* __restrict__ fin,
                                                    float* ws, int backward) {
     extern __shared__ float sm[];
-    const int j0 = blockIdx.x * DVS, h = blockIdx.y, bb = blockIdx.z;
-    const int dk = p.dk, dv = p.dv;
+    const bool inblock = mode >= INBLOCK_FWD, blocks = mode == BLOCKS_FWD || mode == BLOCKS_REV;
+    const bool rev = (mode & 1) != 0;
+    const int j0 = blockIdx.x * DVS;
+    const long long bh = inblock ? (long long)blockIdx.z : (long long)blockIdx.z * p.H + blockIdx.y;
+    const int dk = p.dk, dv = p.dv, NB = (p.NC + GR - 1) / GR;
     const int ldk = ldp(dk), lds = ldp(DVS);
     float* X0 = sm;                    // [dk][DVS]
     float* X1 = X0 + dk * lds;         // [dk][DVS]
     float* Fs = X1 + dk * lds;         // [dk][dk]
-    const long long bh = (long long)bb * p.H + h;
     const Ws w = ws_of(ws, p, bh, backward != 0);
-    const float* Rsrc = reverse ? w.Theta : w.Psi;
-    float* states = reverse ? w.dHc : w.Hc;
-    if (init) load_dense(X0, lds, init + bh * dk * dv + j0, dv, dk, DVS);
+    const float* Fsrc = blocks ? w.Pb : w.Phi;
+    const float* Rsrc = blocks ? w.Sb : (rev ? w.Theta : w.Psi);
+    float* states = blocks ? w.Hb : (rev ? w.dHc : w.Hc);
+    const bool transpose = rev && !blocks;                              // composed maps are stored the way they are applied
+    // steps first .. first + count - 1 (ascending) or first + count - 1 .. first (descending)
+    int first = 0, count = blocks ? NB : p.NC;
+    if (inblock) { first = blockIdx.y * GR; count = min(GR, p.NC - first); }
+    const float* start = inblock ? w.Hb + (long long)blockIdx.y * dk * dv : (init ? init + bh * dk * dv : nullptr);
+    if (start) load_dense(X0, lds, start + j0, dv, dk, DVS);
     else for (int idx = threadIdx.x; idx < dk * lds; idx += NT) X0[idx] = 0.f;
     __syncthreads();
-    // The map of the next chunk is fetched into registers while the product of the current one runs.
+    // The map of the next step is fetched into registers while the product of the current one runs.
     constexpr int MAXF = (DKM * DKM) / NT, MAXR = (DKM * DVS) / NT;
     float fr[MAXF], rr[MAXR];
     auto fetch = [&](int c) {
-        const float* F = w.Phi + (long long)c * dk * dk;
+        const float* F = Fsrc + (long long)c * dk * dk;
         const float* R = Rsrc + (long long)c * dk * dv + j0;
 #pragma unroll
         for (int e = 0; e < MAXF; ++e) {
@@ -252,9 +311,9 @@ __global__ void __launch_bounds__(NT) chain_kernel(Params p, int reverse, const 
         }
     };
     float *cur = X0, *nxt = X1;
-    fetch(reverse ? p.NC - 1 : 0);
-    for (int s = 0; s < p.NC; ++s) {
-        const int c = reverse ? p.NC - 1 - s : s;
+    fetch(rev ? first + count - 1 : first);
+    for (int s = 0; s < count; ++s) {
+        const int c = rev ? first + count - 1 - s : first + s;
         store_dense(states + (long long)c * dk * dv + j0, dv, cur, lds, dk, DVS);
 #pragma unroll
         for (int e = 0; e < MAXF; ++e) {
@@ -267,12 +326,45 @@ __global__ void __launch_bounds__(NT) chain_kernel(Params p, int reverse, const 
             if (idx < dk * DVS) nxt[(idx / DVS) * lds + (idx % DVS)] = rr[e];
         }
         __syncthreads();
-        if (s + 1 < p.NC) fetch(reverse ? c - 1 : c + 1);
-        mm(nxt, lds, Fs, ldk, reverse != 0, cur, lds, false, dk, DVS, dk, 1.f, 1.f);
+        if (s + 1 < count) fetch(rev ? c - 1 : c + 1);
+        mm(nxt, lds, Fs, ldk, transpose, cur, lds, false, dk, DVS, dk, 1.f, 1.f);
         __syncthreads();
         float* t = cur; cur = nxt; nxt = t;
     }
-    if (fin) store_dense(fin + bh * dk * dv + j0, dv, cur, lds, dk, DVS);
+    if (fin && !inblock) store_dense(fin + bh * dk * dv + j0, dv, cur, lds, dk, DVS);
+}
+
+// ---- maps of a block of GR chunks multiplied together: X' = P X + S with (forward) P = Phi[last] ... Phi[first] and S the
+//      image of zero, or (reverse) the same with the transposed maps and Theta in descending order.  grid (NB, H, B) --------
+__global__ void __launch_bounds__(NT) compose_kernel(Params p, int reverse, float* ws, int backward) {
+    extern __shared__ float sm[];
+    const int j = blockIdx.x, h = blockIdx.y, bb = blockIdx.z;
+    const int dk = p.dk, dv = p.dv;
+    const int ldk = ldp(dk), ldv = ldp(dv);
+    float* P0 = sm;                    float* P1 = P0 + dk * ldk;        // [dk][dk] each
+    float* S0 = P1 + dk * ldk;         float* S1 = S0 + dk * ldv;        // [dk][dv] each
+    float* Fs = S1 + dk * ldv;                                           // [dk][dk]
+    const long long bh = (long long)bb * p.H + h;
+    const Ws w = ws_of(ws, p, bh, backward != 0);
+    const float* Rsrc = reverse ? w.Theta : w.Psi;
+    const int first = j * GR, count = min(GR, p.NC - first);
+    for (int idx = threadIdx.x; idx < dk * dk; idx += NT) P0[(idx / dk) * ldk + (idx % dk)] = (idx / dk) == (idx % dk) ? 1.f : 0.f;
+    for (int idx = threadIdx.x; idx < dk * ldv; idx += NT) S0[idx] = 0.f;
+    float *Pc = P0, *Pn = P1, *Sc = S0, *Sn = S1;
+    for (int s = 0; s < count; ++s) {
+        const int c = reverse ? first + count - 1 - s : first + s;
+        __syncthreads();
+        load_dense(Fs, ldk, w.Phi + (long long)c * dk * dk, dk, dk, dk);
+        load_dense(Sn, ldv, Rsrc + (long long)c * dk * dv, dv, dk, dv);
+        __syncthreads();
+        mm4x4(Sn, ldv, Fs, ldk, reverse != 0, Sc, ldv, false, dk, dv, dk, 1.f, 1.f);
+        mm4x4(Pn, ldk, Fs, ldk, reverse != 0, Pc, ldk, false, dk, dk, dk, 0.f, 1.f);
+        float* t = Pc; Pc = Pn; Pn = t;
+        t = Sc; Sc = Sn; Sn = t;
+    }
+    __syncthreads();
+    store_dense(w.Pb + (long long)j * dk * dk, dk, Pc, ldk, dk, dk);
+    store_dense(w.Sb + (long long)j * dk * dv, dv, Sc, ldv, dk, dv);
 }
 
 // ---- Out: W = U - Wk Hc (V_new),  O = (M * Q K^T) W + gam * (Q Hc).  grid (NC, H, B) --------------------------------
@@ -300,9 +392,9 @@ __global__ void __launch_bounds__(NT) out_kernel(Params p, const T* __restrict__
     load_dense(Wc, ldv, w.U + (long long)t0 * dv, dv, n, dv);
     load_dense(Hs, ldv, w.Hc + (long long)c * dk * dv, dv, dk, dv);
     load_decay(b, nullptr, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, nullptr, p.tg, n);
-    mm(Wc, ldv, Wks, ldk, false, Hs, ldv, false, n, dv, dk, 1.f, -1.f);         // W = U - Wk H
-    mm(A, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
-    mm(O, ldv, Qs, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
+    mmx(Wc, ldv, Wks, ldk, false, Hs, ldv, false, n, dv, dk, 1.f, -1.f);         // W = U - Wk H
+    mmx(A, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
+    mmx(O, ldv, Qs, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
     __syncthreads();
     for (int idx = threadIdx.x; idx < n * n; idx += NT) {
         const int t = idx / n, s = idx - t * n;
@@ -310,7 +402,7 @@ __global__ void __launch_bounds__(NT) out_kernel(Params p, const T* __restrict__
     }
     scale_rows(O, ldv, n, dv, [&](int t) { return __expf(b[t]); });
     __syncthreads();
-    mm(O, ldv, A, ldc, false, Wc, ldv, false, n, dv, n, 1.f, 1.f);
+    mmx(O, ldv, A, ldc, false, Wc, ldv, false, n, dv, n, 1.f, 1.f);
     __syncthreads();
     T* oh = o + (long long)bb * p.bv + (long long)t0 * p.tv + (long long)h * dv;
     for (int idx = threadIdx.x; idx < n * dv; idx += NT) {
@@ -346,17 +438,17 @@ __global__ void __launch_bounds__(NT) bwd_pre_kernel(Params p, const T* __restri
     load_dense(A, ldc, w.A + (long long)c * C * C, C, n, n);
     load_dense(Ti, ldc, w.Ti + (long long)c * C * C, C, n, n);
     load_decay(b, bt, g + (long long)bb * p.bg + (long long)t0 * p.tg + h, beta + (long long)bb * p.bg + (long long)t0 * p.tg + h, p.tg, n);
-    mm(T1, ldv, A, ldc, true, dOs, ldv, false, n, dv, n, 0.f, 1.f);             // A^T dO
+    mmx(T1, ldv, A, ldc, true, dOs, ldv, false, n, dv, n, 0.f, 1.f);             // A^T dO
     __syncthreads();
-    mm(Z0, ldv, Ti, ldc, true, T1, ldv, false, n, dv, n, 0.f, 1.f);             // Z0 = (I+L)^-T A^T dO
+    mmx(Z0, ldv, Ti, ldc, true, T1, ldv, false, n, dv, n, 0.f, 1.f);             // Z0 = (I+L)^-T A^T dO
     __syncthreads();
     store_dense(w.Z0 + (long long)t0 * dv, dv, Z0, ldv, n, dv);
     scale_rows(dOs, ldv, n, dv, [&](int t) { return __expf(b[t]); });
     scale_rows(Z0, ldv, n, dv, [&](int t) { return bt[t] * __expf(b[t]); });
     __syncthreads();
     float* Th = w.Theta + (long long)c * dk * dv;
-    mm(Th, dv, Qs, ldk, true, dOs, ldv, false, dk, dv, n, 0.f, 1.f);
-    mm(Th, dv, Ks, ldk, true, Z0, ldv, false, dk, dv, n, 1.f, -1.f);
+    mmx(Th, dv, Qs, ldk, true, dOs, ldv, false, dk, dv, n, 0.f, 1.f);
+    mmx(Th, dv, Ks, ldk, true, Z0, ldv, false, dk, dv, n, 1.f, -1.f);
 }
 
 // ---- backward, second chunk-parallel part: every input gradient of the chunk from the stored Hc, dHc, U, Wk, Z0, Ti.
@@ -404,9 +496,9 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
     load_dense(Ti, ldc, w.Ti + (long long)c * C * C, C, n, n);
     load_decay(b, bt, g + og, beta + og, p.tg, n);
     const float bn = b[n - 1];
-    mm(Wc, ldv, T1, ldk, false, Hs, ldv, false, n, dv, dk, 1.f, -1.f);          // W = U - Wk H
-    mm(KH, ldv, Ks, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
-    mm(KdH, ldv, Ks, ldk, false, dHs, ldv, false, n, dv, dk, 0.f, 1.f);
+    mmx(Wc, ldv, T1, ldk, false, Hs, ldv, false, n, dv, dk, 1.f, -1.f);          // W = U - Wk H
+    mmx(KH, ldv, Ks, ldk, false, Hs, ldv, false, n, dv, dk, 0.f, 1.f);
+    mmx(KdH, ldv, Ks, ldk, false, dHs, ldv, false, n, dv, dk, 0.f, 1.f);
     __syncthreads();
     // Z = Z0 + Ti^T (om * (K dH')): the part of the transposed solve that depends on the incoming state gradient
     const int ldt = ldp(dk > dv ? dk : dv);
@@ -415,15 +507,15 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
         T1[t * ldt + jj] = __expf(bn - b[t]) * KdH[t * ldv + jj];
     }
     __syncthreads();
-    mm(Zs, ldv, Ti, ldc, true, T1, ldt, false, n, dv, n, 1.f, 1.f);
+    mmx(Zs, ldv, Ti, ldc, true, T1, ldt, false, n, dv, n, 1.f, 1.f);
     __syncthreads();
-    mm(QK, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
-    mm(KK, ldc, Ks, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
-    mm(DA, ldc, dOs, ldv, false, Wc, ldv, true, n, n, dv, 0.f, 1.f);            // dA = dO W^T
-    mm(ZW, ldc, Zs, ldv, false, Wc, ldv, true, n, n, dv, 0.f, 1.f);             // Z W^T  (dL = -strict lower)
-    mm(dQs, ldk, dOs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);          // dO H^T
-    mm(dKs, ldk, Wc, ldv, false, dHs, ldv, true, n, dk, dv, 0.f, 1.f);          // W dH'^T
-    mm(T1, ldt, Zs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);            // Z H^T
+    mmx(QK, ldc, Qs, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
+    mmx(KK, ldc, Ks, ldk, false, Ks, ldk, true, n, n, dk, 0.f, 1.f);
+    mmx(DA, ldc, dOs, ldv, false, Wc, ldv, true, n, n, dv, 0.f, 1.f);            // dA = dO W^T
+    mmx(ZW, ldc, Zs, ldv, false, Wc, ldv, true, n, n, dv, 0.f, 1.f);             // Z W^T  (dL = -strict lower)
+    mmx(dQs, ldk, dOs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);          // dO H^T
+    mmx(dKs, ldk, Wc, ldv, false, dHs, ldv, true, n, dk, dv, 0.f, 1.f);          // W dH'^T
+    mmx(T1, ldt, Zs, ldv, false, Hs, ldv, true, n, dk, dv, 0.f, 1.f);            // Z H^T
     for (int i = threadIdx.x; i < dk; i += NT) {
         float acc = 0.f;
         for (int jj = 0; jj < dv; ++jj) acc = fmaf(dHs[i * ldv + jj], Hs[i * ldv + jj], acc);
@@ -476,12 +568,12 @@ __global__ void __launch_bounds__(NT) bwd_out_kernel(Params p, const T* __restri
         dKs[a] = __expf(bn - b[t]) * dKs[a] - bt[t] * __expf(b[t]) * T1[t * ldt + i];
     }
     __syncthreads();
-    mm(dQs, ldk, DA, ldc, false, Ks, ldk, false, n, dk, n, 1.f, 1.f);
-    mm(dKs, ldk, DA, ldc, true, Qs, ldk, false, n, dk, n, 1.f, 1.f);
+    mmx(dQs, ldk, DA, ldc, false, Ks, ldk, false, n, dk, n, 1.f, 1.f);
+    mmx(dKs, ldk, DA, ldc, true, Qs, ldk, false, n, dk, n, 1.f, 1.f);
     __syncthreads();
-    mm(dKs, ldk, ZW, ldc, false, Ks, ldk, false, n, dk, n, 1.f, 1.f);
+    mmx(dKs, ldk, ZW, ldc, false, Ks, ldk, false, n, dk, n, 1.f, 1.f);
     __syncthreads();
-    mm(dKs, ldk, ZW, ldc, true, Ks, ldk, false, n, dk, n, 1.f, 1.f);
+    mmx(dKs, ldk, ZW, ldc, true, Ks, ldk, false, n, dk, n, 1.f, 1.f);
     __syncthreads();
     for (int idx = threadIdx.x; idx < n * dk; idx += NT) {
         const int t = idx / dk, i = idx - t * dk;
@@ -499,6 +591,7 @@ __host__ inline size_t smem_pre(int C, int dk, int dv) {
     return sizeof(float) * (3 * (size_t)C * ldp(dk) + (size_t)C * ldp(dv + dk + C) + (size_t)C * ldp(C) + 2 * C);
 }
 __host__ inline size_t smem_chain(int dk) { return sizeof(float) * (2 * (size_t)dk * ldp(DVS) + (size_t)dk * ldp(dk)); }
+__host__ inline size_t smem_compose(int dk, int dv) { return sizeof(float) * (3 * (size_t)dk * ldp(dk) + 2 * (size_t)dk * ldp(dv)); }
 __host__ inline size_t smem_out(int C, int dk, int dv) {
     return sizeof(float) * (3 * (size_t)C * ldp(dk) + 2 * (size_t)C * ldp(dv) + (size_t)dk * ldp(dv) + (size_t)C * ldp(C) + C);
 }

@@ -156,6 +156,29 @@ bool opt_in(K kern, size_t bytes) {
     return true;
 }
 
+// The sequential state pass (forward or reverse) of the chunkwise delta rule: two levels (maps composed over blocks of GR
+// chunks, a pass over the blocks, the chunks of all blocks in parallel) when the segment has more chunks than one block and
+// the composing kernel's tiles fit into shared memory, else one pass over the chunks.  Returns the number of launches.
+int delta_state_pass(const sf::gdn::Params& p, bool reverse, const float* init, float* fin, float* ws, int backward, cudaStream_t st) {
+    using namespace sf::gdn;
+    const dim3 cols(p.dv / DVS, p.H, p.B);
+    const size_t s2 = smem_chain(p.dk), sc = smem_compose(p.dk, p.dv);
+    const int NB = (p.NC + GR - 1) / GR;
+    const bool wide = p.dk > 64;
+    auto chain = [&](dim3 grid, int mode, const float* i0, float* f0) {
+        if (wide) chain_kernel<128><<<grid, NT, s2, st>>>(p, mode, i0, f0, ws, backward);
+        else      chain_kernel<64><<<grid, NT, s2, st>>>(p, mode, i0, f0, ws, backward);
+    };
+    if (p.NC > GR && sc <= kMaxSmem && (long long)p.B * p.H <= 65535) {
+        compose_kernel<<<dim3(NB, p.H, p.B), NT, sc, st>>>(p, reverse ? 1 : 0, ws, backward);
+        chain(cols, reverse ? BLOCKS_REV : BLOCKS_FWD, init, fin);
+        chain(dim3(p.dv / DVS, NB, p.B * p.H), reverse ? INBLOCK_REV : INBLOCK_FWD, nullptr, nullptr);
+        return 3;
+    }
+    chain(cols, reverse ? CHUNKS_REV : CHUNKS_FWD, init, fin);
+    return 1;
+}
+
 // Pre + ST (+ Out when o != NULL); the backward calls it with o == NULL to rebuild the chunk states.
 template <typename T>
 sf_status_t chunked_forward(const sf_seg_desc_t* d, const sf::gdn::Params& p, const void* q, const void* k, const void* v,
@@ -165,12 +188,12 @@ sf_status_t chunked_forward(const sf_seg_desc_t* d, const sf::gdn::Params& p, co
     const T *tq = static_cast<const T*>(q), *tk = static_cast<const T*>(k), *tv = static_cast<const T*>(v);
     const dim3 chunks(p.NC, p.H, p.B), cols(p.dv / DVS, p.H, p.B);
     const size_t s1 = smem_pre(p.C, p.dk, p.dv), s2 = smem_chain(p.dk), s3 = smem_out(p.C, p.dk, p.dv);
-    if (!opt_in(pre_kernel<T>, s1) || !opt_in(chain_kernel<64>, s2) || !opt_in(chain_kernel<128>, s2) || !opt_in(out_kernel<T>, s3))
+    const size_t sc = smem_compose(p.dk, p.dv);
+    if (!opt_in(pre_kernel<T>, s1) || !opt_in(chain_kernel<64>, s2) || !opt_in(chain_kernel<128>, s2) || !opt_in(out_kernel<T>, s3) ||
+        (sc <= kMaxSmem && !opt_in(compose_kernel, sc)))
         return SF_ERR_CUDA;
     pre_kernel<T><<<chunks, NT, s1, st>>>(p, tq, tk, tv, g, beta, ws, backward);
-    if (p.dk <= 64) chain_kernel<64><<<cols, NT, s2, st>>>(p, 0, S_in, S_out, ws, backward);
-    else            chain_kernel<128><<<cols, NT, s2, st>>>(p, 0, S_in, S_out, ws, backward);
-    int n = 2;
+    int n = 1 + delta_state_pass(p, false, S_in, S_out, ws, backward, st);
     if (o) { out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, g, static_cast<T*>(o), ws, backward); ++n; }
     return launched(n);
 }
@@ -188,11 +211,10 @@ sf_status_t chunked_backward(const sf_seg_desc_t* d, const sf::gdn::Params& p, c
     if (!opt_in(bwd_pre_kernel<T>, s1) || !opt_in(chain_kernel<64>, s2) || !opt_in(chain_kernel<128>, s2) || !opt_in(bwd_out_kernel<T>, s3))
         return SF_ERR_CUDA;
     bwd_pre_kernel<T><<<chunks, NT, s1, st>>>(p, tq, tk, g, beta, tdo, ws);
-    if (p.dk <= 64) chain_kernel<64><<<cols, NT, s2, st>>>(p, 1, dS_out, dS_in, ws, 1);
-    else            chain_kernel<128><<<cols, NT, s2, st>>>(p, 1, dS_out, dS_in, ws, 1);
+    const int ns = delta_state_pass(p, true, dS_out, dS_in, ws, 1, st);
     bwd_out_kernel<T><<<chunks, NT, s3, st>>>(p, tq, tk, tv, g, beta, tdo, static_cast<T*>(dq), static_cast<T*>(dk), static_cast<T*>(dv),
                                               dg, dbeta, ws);
-    return launched(3);
+    return launched(2 + ns);
 }
 
 // ---- chunkwise diagonal decay ----------------------------------------------------------------------------------------

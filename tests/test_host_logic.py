@@ -233,7 +233,7 @@ def test_chunked_delta_rule_validates_before_any_launch(lib):
     f32 = dict(dtype=binding.SF_F32, d_k=64, d_v=64, seg_len=100, chunk=32)
     d = desc(**f32)
     lib.sf_delta_chunked_workspace_bytes.restype = ctypes.c_size_t
-    per_bh_fwd = 100 * 64 + 100 * 64 + 3 * 4 * 64 * 64             # U, Wk per token; Phi, Psi and one state per chunk (4 chunks)
+    per_bh_fwd = 100 * 64 + 100 * 64 + 3 * 4 * 64 * 64 + 3 * 64 * 64   # U, Wk per token; Phi, Psi, one state per chunk (4 chunks); the same per block of 16 chunks
     assert lib.sf_delta_chunked_workspace_bytes(ctypes.byref(d), 0) == 2 * per_bh_fwd * 4
     # the backward adds Z0 per token, Theta and one state gradient per chunk and two chunk x chunk matrices per chunk
     assert lib.sf_delta_chunked_workspace_bytes(ctypes.byref(d), 1) == 2 * (per_bh_fwd + 100 * 64 + 2 * 4 * 64 * 64 + 2 * 4 * 32 * 32) * 4
