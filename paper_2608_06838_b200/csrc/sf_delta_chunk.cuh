@@ -327,7 +327,9 @@ __global__ void __launch_bounds__(NT) chain_kernel(Params p, int mode, const flo
         }
         __syncthreads();
         if (s + 1 < count) fetch(rev ? c - 1 : c + 1);
-        mm(nxt, lds, Fs, ldk, transpose, cur, lds, false, dk, DVS, dk, 1.f, 1.f);
+        // many CTAs share an SM in the in-block mode (throughput counts: fewer shared-memory reads); one CTA per SM else
+        if (inblock) mm4x4(nxt, lds, Fs, ldk, transpose, cur, lds, false, dk, DVS, dk, 1.f, 1.f);
+        else         mm(nxt, lds, Fs, ldk, transpose, cur, lds, false, dk, DVS, dk, 1.f, 1.f);
         __syncthreads();
         float* t = cur; cur = nxt; nxt = t;
     }
