@@ -259,7 +259,8 @@ def main():
         work_stream.synchronize()
         tuned = tuned or {}
         tuned["schedule"] = {"sweep_streams": t.sweep_streams, "agg_streams": t.agg_streams, "scan_group_tokens": t.scan_group_tokens,
-                             "agg_inorder_ctas": t.agg_inorder_ctas, "agg_ahead": t.agg_ahead, "ms": round(t_ms, 4),
+                             "agg_inorder_ctas": t.agg_inorder_ctas, "agg_ahead": t.agg_ahead, "merge_launches": t.merge_launches,
+                             "ms": round(t_ms, 4),
                              "default_ms": round(d_ms, 4)}
     if args.graph:
         with torch.cuda.stream(work_stream):

@@ -257,9 +257,16 @@ void sf_chain_graph_destroy(sf_chain_graph_t* graph);
  *   agg_inorder_ctas  >= 1  an aggregate launch of at least this many CTAs stays in order on the first aggregate stream
  *   agg_ahead         >= 0  how many segments the aggregate kernels may run ahead of the sweeps (0 = no limit);
  *                           a small value keeps what the aggregates read close to the sweeps that read it again
+ *   merge_launches    0 / 1 1: when every segment but the last is a whole number of blocks of one common length, each
+ *                           stage runs once over the whole chain (the blocks of all segments in one launch) instead of
+ *                           once per segment; same kernels and, for the same block length, the same blocks and bits
+ *                           (with chunks_per_block = 0 the longest common length is taken, which may differ from the
+ *                           segments' own: results then agree to rounding); chains of another shape run segment by
+ *                           segment as with 0.  The forward workspace is laid out differently, so a
+ *                           backward that reuses it must run under the same value as its forward.
  * The block length is part of the descriptor (chunks_per_block); forward and backward share it because the backward
  * starts its blocks from the block states the forward saved.
- * sf_set_tuning(NULL) restores the defaults {4, 4, 4096, 74, 0}; out-of-range values give SF_ERR_INVALID_ARG and change
+ * sf_set_tuning(NULL) restores the defaults {4, 4, 4096, 74, 0, 0}; out-of-range values give SF_ERR_INVALID_ARG and change
  * nothing.  Host functions.
  */
 typedef struct {
@@ -268,6 +275,7 @@ typedef struct {
     int32_t scan_group_tokens;
     int32_t agg_inorder_ctas;
     int32_t agg_ahead;
+    int32_t merge_launches;
 } sf_tuning_t;
 sf_status_t sf_set_tuning(const sf_tuning_t* tuning);
 void sf_get_tuning(sf_tuning_t* tuning);

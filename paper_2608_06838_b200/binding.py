@@ -305,7 +305,7 @@ def sf_device_status_clear() -> None:
 class Tuning(ctypes.Structure):
     """sf_tuning_t: schedule of the chaining driver."""
     _fields_ = [("sweep_streams", ctypes.c_int32), ("agg_streams", ctypes.c_int32), ("scan_group_tokens", ctypes.c_int32),
-                ("agg_inorder_ctas", ctypes.c_int32), ("agg_ahead", ctypes.c_int32)]
+                ("agg_inorder_ctas", ctypes.c_int32), ("agg_ahead", ctypes.c_int32), ("merge_launches", ctypes.c_int32)]
 
 
 def sf_set_tuning(tuning=None) -> None:

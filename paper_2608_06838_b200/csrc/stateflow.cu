@@ -302,7 +302,7 @@ sf_status_t launch_scan_group(const sf_seg_desc_t* d, int BH, const sf::ScanGrou
 
 // Schedule of the chaining driver (sf_tuning_t; process-wide, read at every chain call).
 constexpr int kMaxSweepStreams = 4, kMaxAggStreams = 4;
-const sf_tuning_t kDefaultTuning = {4, 4, 4096, 74, 0};
+const sf_tuning_t kDefaultTuning = {4, 4, 4096, 74, 0, 0};
 std::mutex g_tuning_mu;
 sf_tuning_t g_tuning = kDefaultTuning;
 sf_tuning_t current_tuning() {
@@ -481,6 +481,92 @@ sf_status_t validate_chain(const sf_seg_desc_t* d, const int32_t* seg_lens, int3
     return SF_OK;
 }
 
+// ---- merged launches (sf_tuning_t.merge_launches) ------------------------------------------------------------------
+// When every segment but the last is a whole number of blocks of one common length R, the blocks of all segments are
+// the blocks of ONE segment that spans the sequence: each stage then runs once over the whole chain (one aggregate launch,
+// one scan, one sweep, ...) instead of once per segment, with the same blocks, the same kernels and the same arithmetic
+// (results are bit-identical).  The boundary states S_bounds[i] are the states entering the first block of each segment.
+// Returns the descriptor of that segment, or false if the chain does not have this shape.
+bool merged_desc(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, long long T, sf_seg_desc_t* out) {
+    if (n_seg < 2 || T > 0x7fffffffLL) return false;
+    const int C = desc->chunk;
+    int R = desc->chunks_per_block;
+    for (int i = 0; i + 1 < n_seg; ++i)
+        if (seg_lens[i] % C) return false;
+    if (R == 0) {
+        // the longest block length (at most 64 chunks) that divides the chunk count of every segment but the last
+        for (R = 64; R >= 1; --R) {
+            bool ok = true;
+            for (int i = 0; i + 1 < n_seg && ok; ++i) ok = (seg_lens[i] / C) % R == 0;
+            if (ok) break;
+        }
+        if (R < 4) return false;
+    } else {
+        for (int i = 0; i + 1 < n_seg; ++i)
+            if ((seg_lens[i] / C) % R) return false;
+    }
+    sf_seg_desc_t t = *desc;
+    t.seg_len = (int32_t)T;
+    t.chunks_per_block = R;
+    const Path path = classify(&t);
+    if (path == Path::Invalid || path == Path::Unsupported) return false;
+    if (make_params(&t).NB > 65535) return false;
+    *out = t;
+    return true;
+}
+
+sf_status_t chain_fwd_merged(const sf_seg_desc_t* vd, const int32_t* seg_lens, int32_t n_seg, const FwdPtrs& x, float* S_bounds,
+                             void* workspace, cudaStream_t st) {
+    const Path path = classify(vd);
+    const SegParams p = make_params(vd);
+    const FwdWs w = fwd_ws(vd, p, workspace);
+    SF_TRY(fwd_pre(path, vd, p, x, w, st));
+    SF_TRY(fwd_scan(vd, p, x, w, st));
+    // S_bounds[i] = state entering the first block of segment i (a strided copy: one state per batch x head)
+    const size_t m = (size_t)vd->d_k * vd->d_v, sN = (size_t)vd->B * vd->H * m;
+    long long blk = 0;
+    for (int i = 1; i < n_seg; ++i) {
+        blk += (seg_lens[i - 1] / vd->chunk) / p.R;
+        SF_CUDA(cudaMemcpy2DAsync(S_bounds + (size_t)i * sN, m * sizeof(float), w.UH + (size_t)blk * m, (size_t)p.NB * m * sizeof(float),
+                                  m * sizeof(float), (size_t)vd->B * vd->H, cudaMemcpyDeviceToDevice, st));
+    }
+    return fwd_out(path, vd, p, x, w, st);
+}
+
+sf_status_t chain_bwd_merged(const sf_seg_desc_t* vd, const BwdPtrs& x, const void* fwd_workspace, void* workspace, bool overlap,
+                             cudaStream_t st) {
+    const Path path = classify(vd);
+    const SegParams p = make_params(vd);
+    const BwdWs w = bwd_ws(vd, p, workspace);
+    FwdWs fw;
+    if (fwd_workspace) {
+        fw = fwd_ws(vd, p, const_cast<void*>(fwd_workspace));
+    } else {
+        char* base = static_cast<char*>(workspace) + w.bytes;
+        fw = fwd_ws(vd, p, base);
+        float* sfin = reinterpret_cast<float*>(base + fw.bytes);
+        FwdPtrs fx{x.q, x.k, x.v, x.g, x.S_in, nullptr, sfin};
+        SF_TRY(fwd_pre(path, vd, p, fx, fw, st));
+        SF_TRY(fwd_scan(vd, p, fx, fw, st));
+    }
+    // the dq sweep needs only the forward states: with overlap it runs on a side stream beside the backward aggregate and
+    // the reverse scan (whose dependent steps leave most of the device idle)
+    ChainRes* res = nullptr;
+    if (overlap) {
+        SF_TRY(chain_resources(&res));
+        SF_CUDA(cudaEventRecord(res->ev[5], st));
+        SF_CUDA(cudaStreamWaitEvent(res->side[1], res->ev[5], 0));
+        SF_TRY(bwd_dq(path, vd, p, x, w, fw.UH, res->side[1]));
+        SF_CUDA(cudaEventRecord(res->ev[6], res->side[1]));
+    }
+    SF_TRY(bwd_pre(path, vd, p, x, w, nullptr, st));
+    SF_TRY(bwd_scan(vd, p, x, w, fw.beta, st));
+    if (!overlap) SF_TRY(bwd_dq(path, vd, p, x, w, fw.UH, st));
+    SF_TRY(bwd_dkdv(path, vd, p, x, w, st));
+    if (overlap) SF_CUDA(cudaStreamWaitEvent(st, res->ev[6], 0));
+    return bwd_dg(vd, p, x, w, fw.UH, st);
+}
+
 }  // namespace
 
 // Scratch of sf_segment_fwd_static: part of the library image, one copy per GPU that loads it.  In host
@@ -615,7 +701,16 @@ size_t sf_chain_workspace_bytes(const sf_seg_desc_t* desc, const int32_t* seg_le
     // forward keeps every segment's block states for the backward; the backward gives every segment its own
     // workspace and boundary-gradient buffer so that the stages of different segments can run concurrently
     (void)mx;
-    return backward == 0 ? total : total + (size_t)n_seg * state_bytes(desc);
+    size_t need = backward == 0 ? total : total + (size_t)n_seg * state_bytes(desc);
+    // enough for the merged-launch mode as well (its common block length may be shorter than the segments' own)
+    long long T = 0;
+    for (int i = 0; i < n_seg; ++i) T += seg_lens[i];
+    sf_seg_desc_t vd;
+    if (merged_desc(desc, seg_lens, n_seg, T, &vd)) {
+        const size_t mb = sf_workspace_bytes(&vd, backward);
+        need = mb > need ? mb : need;
+    }
+    return need;
 }
 
 sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q, const void* k,
@@ -637,6 +732,14 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     else        SF_CUDA(cudaMemsetAsync(S_bounds, 0, sN * sizeof(float), st));
 
     const sf_tuning_t tu = current_tuning();
+    {
+        sf_seg_desc_t vd;
+        if (tu.merge_launches && merged_desc(desc, seg_lens, n_seg, T, &vd) &&
+            sf_workspace_bytes(&vd, 0) <= workspace_bytes) {
+            FwdPtrs x{q, k, v, g, S_bounds, o, S_bounds + (size_t)n_seg * sN};
+            return chain_fwd_merged(&vd, seg_lens, n_seg, x, S_bounds, workspace, st);
+        }
+    }
     ChainRes* res = nullptr;
     if (overlap) SF_TRY(chain_resources(&res));
     // overlap schedule (the forward wavefront of Section 3.4, Eq. 17, across segments):
@@ -742,6 +845,14 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     const size_t esz = desc->dtype == SF_BF16 ? 2 : 4;
     const size_t sN = (size_t)desc->B * desc->H * desc->d_k * desc->d_v;
 
+    {
+        sf_seg_desc_t vd;
+        if (current_tuning().merge_launches && merged_desc(desc, seg_lens, n_seg, T, &vd) &&
+            sf_workspace_bytes(&vd, mode) <= workspace_bytes && (!fwd_workspace || sf_workspace_bytes(&vd, 0) <= sf_chain_workspace_bytes(desc, seg_lens, n_seg, 0))) {
+            BwdPtrs x{q, k, v, g, S_bounds, dO, dS_final, dq, dk, dv, dg, dS_init};
+            return chain_bwd_merged(&vd, x, fwd_workspace, workspace, overlap != 0, st);
+        }
+    }
     // layout: [dS buffers: one state per segment][segment workspaces in order]
     char* base = static_cast<char*>(workspace);
     char* seg_base = base + (size_t)n_seg * sB;
@@ -1059,6 +1170,11 @@ sf_status_t sf_chain_autotune_schedule(const sf_seg_desc_t* desc, const int32_t*
                 if (ahead == 0 && sweeps == 4 && inorder == 74) continue;       // the default itself
                 grid.push_back(t);
             }
+    {
+        sf_tuning_t t = kDefaultTuning;
+        t.merge_launches = 1;                                                    // one launch per stage over the whole chain
+        grid.push_back(t);
+    }
     const sf_tuning_t before = current_tuning();
     const int32_t cand = desc->chunks_per_block;
     float best_ms = -1.f, def_ms = -1.f;
@@ -1207,7 +1323,7 @@ sf_status_t sf_set_tuning(const sf_tuning_t* t) {
     std::lock_guard<std::mutex> lk(g_tuning_mu);
     if (!t) { g_tuning = kDefaultTuning; return SF_OK; }
     if (t->sweep_streams < 1 || t->sweep_streams > kMaxSweepStreams || t->agg_streams < 1 || t->agg_streams > kMaxAggStreams ||
-        t->scan_group_tokens < 0 || t->agg_inorder_ctas < 1 || t->agg_ahead < 0)
+        t->scan_group_tokens < 0 || t->agg_inorder_ctas < 1 || t->agg_ahead < 0 || t->merge_launches < 0 || t->merge_launches > 1)
         return SF_ERR_INVALID_ARG;
     g_tuning = *t;
     return SF_OK;

@@ -112,7 +112,8 @@ def test_schedule_search_installs_a_valid_choice_and_results_do_not_change():
         assert t.sweep_streams in (2, 4) and t.agg_ahead in (0, 1, 2) and t.agg_inorder_ctas in (1, 74)
         now = binding.sf_get_tuning()
         assert (now.sweep_streams, now.agg_ahead, now.agg_inorder_ctas) == (t.sweep_streams, t.agg_ahead, t.agg_inorder_ctas)
-        if (t.sweep_streams, t.agg_ahead, t.agg_inorder_ctas) != (4, 0, 74):
+        assert t.merge_launches in (0, 1) and now.merge_launches == t.merge_launches
+        if (t.sweep_streams, t.agg_ahead, t.agg_inorder_ctas, t.merge_launches) != (4, 0, 74, 0):
             assert ms < default_ms / 1.02                   # the default is only left for a clear win
         got, _ = run_chain(w, x)
         for n in NAMES:
@@ -120,3 +121,80 @@ def test_schedule_search_installs_a_valid_choice_and_results_do_not_change():
     finally:
         binding.sf_set_tuning(None)
     assert binding.sf_device_status() == 0
+
+
+@pytest.mark.parametrize("dtype,d,chunk,segs,cpb", [
+    ("bf16", 128, 64, [1024, 512, 512, 2048, 300], 8),        # blocks of 8 chunks divide every segment but the ragged last one
+    ("bf16", 128, 64, [2048, 2048, 2048], 16),
+    ("f32", 64, 32, [256, 128, 384, 77], 4),                  # CUDA-core path
+])
+@pytest.mark.parametrize("save_states", [True, False])
+def test_merged_launches_give_the_bits_of_the_segment_by_segment_run(dtype, d, chunk, segs, cpb, save_states):
+    # one launch per stage over the whole chain: with the same block length the blocks, the kernels and the arithmetic are
+    # the same, so the bits are; fewer launches
+    w = Workload("merged", 2 if dtype == "f32" else 1, 3, d, d, segs, chunk, dtype=dtype, g_scale=0.1, s_in_sigma=0.02,
+                 ds_out_sigma=0.02, seed=61)
+    x = inputs.make_inputs(w, DEV)
+    torch.cuda.synchronize()
+    binding.sf_set_tuning(None)
+    n0 = binding.sf_launch_count()
+    ref, run_ref = run_chain(w, x, chunks_per_block=cpb, save_states=save_states)
+    per_segment = binding.sf_launch_count() - n0
+    ref = {n: ref[n].clone() for n in NAMES}
+    bounds_ref = run_ref.S_bounds.clone()
+    try:
+        binding.sf_set_tuning(dict(merge_launches=1))
+        n0 = binding.sf_launch_count()
+        got, run = run_chain(w, x, chunks_per_block=cpb, save_states=save_states)
+        merged = binding.sf_launch_count() - n0
+        for n in NAMES:
+            assert torch.equal(got[n], ref[n]), n
+        assert torch.equal(run.S_bounds, bounds_ref)            # every boundary state, not only the last
+        assert merged < per_segment and merged == (8 if save_states else 10)   # 3 forward + 5 backward kernels (+ 2 to replay the states)
+        if save_states:
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                run.capture(x["S_in"], x["dS_out"])
+                run.o.zero_()
+                run.dq.zero_()
+                run.replay()
+            stream.synchronize()
+            assert torch.equal(run.o, ref["o"]) and torch.equal(run.dq, ref["dq"]) and torch.equal(run.dS_init, ref["dS_in"])
+            run.release()
+    finally:
+        binding.sf_set_tuning(None)
+    assert binding.sf_device_status() == 0
+    compare(ref, oracle_reference(x), tolerance(w), label="merged")
+
+
+def test_chains_that_cannot_be_merged_run_segment_by_segment():
+    # a middle segment that is not a whole number of chunks: no common block grid
+    w = Workload("unmerged", 1, 2, 128, 128, [512, 300, 512], 64, g_scale=0.1, s_in_sigma=0.02, ds_out_sigma=0.02, seed=62)
+    x = inputs.make_inputs(w, DEV)
+    torch.cuda.synchronize()
+    binding.sf_set_tuning(None)
+    ref, _ = run_chain(w, x)
+    ref = {n: ref[n].clone() for n in NAMES}
+    try:
+        binding.sf_set_tuning(dict(merge_launches=1))
+        got, _ = run_chain(w, x)
+        for n in NAMES:
+            assert torch.equal(got[n], ref[n]), n
+    finally:
+        binding.sf_set_tuning(None)
+
+
+def test_merged_launches_with_the_library_s_own_block_length_match_the_oracle():
+    # chunks_per_block = 0: the merged run picks the longest common block length, which may differ from the segments' own
+    w = Workload("merged-auto", 1, 3, 128, 128, [1024, 512, 512, 2048, 300], 64, g_scale=0.1, s_in_sigma=0.02, ds_out_sigma=0.02,
+                 seed=63)
+    x = inputs.make_inputs(w, DEV)
+    torch.cuda.synchronize()
+    try:
+        binding.sf_set_tuning(dict(merge_launches=1))
+        n0 = binding.sf_launch_count()
+        got, _ = run_chain(w, x)
+        assert binding.sf_launch_count() - n0 == 8
+        compare(got, oracle_reference(x), tolerance(w), label="merged-auto")
+    finally:
+        binding.sf_set_tuning(None)

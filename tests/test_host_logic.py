@@ -190,12 +190,12 @@ def test_tuning_is_validated_and_restored(lib):
     from paper_2608_06838_b200.binding import SfError, Tuning
     binding.sf_set_tuning(None)
     d = binding.sf_get_tuning()
-    assert (d.sweep_streams, d.agg_streams, d.scan_group_tokens, d.agg_inorder_ctas, d.agg_ahead) == (4, 4, 4096, 74, 0)
+    assert (d.sweep_streams, d.agg_streams, d.scan_group_tokens, d.agg_inorder_ctas, d.agg_ahead, d.merge_launches) == (4, 4, 4096, 74, 0, 0)
     binding.sf_set_tuning(dict(sweep_streams=2, agg_ahead=1))
     t = binding.sf_get_tuning()
     assert (t.sweep_streams, t.agg_streams, t.agg_ahead) == (2, 4, 1)
     for bad in (dict(sweep_streams=0), dict(sweep_streams=5), dict(agg_streams=0), dict(agg_streams=9),
-                dict(scan_group_tokens=-1), dict(agg_inorder_ctas=0), dict(agg_ahead=-1)):
+                dict(scan_group_tokens=-1), dict(agg_inorder_ctas=0), dict(agg_ahead=-1), dict(merge_launches=2), dict(merge_launches=-1)):
         with pytest.raises(SfError) as e:
             binding.sf_set_tuning(bad)
         assert e.value.code == 1
