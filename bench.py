@@ -390,7 +390,8 @@ def main():
         heavy = [st for st in stage if st["name"] in KERNEL_BYTES and st["launches"]]
         dom = max(heavy, key=lambda st: st["ms"])
         per_launch_ms = dom["ms"] / max(dom["launches"], 1)
-        th_per_launch = tokens * w.H / len(w.seg_lens)               # token*heads of the mean launch of this step
+        # token*heads of the mean launch: one launch per segment, or one per step when the launches are merged
+        th_per_launch = tokens * w.H * args.steps / max(dom["launches"], 1)
         alg = KERNEL_BYTES[dom["name"]] * th_per_launch
         traffic = KERNEL_NCU_TRAFFIC[dom["name"]] * th_per_launch if dom["name"] in KERNEL_NCU_TRAFFIC else None
         roof = {"bound": "hbm", "kernel": dom["name"], "achieved": alg / (per_launch_ms * 1e-3) / 1e9,
