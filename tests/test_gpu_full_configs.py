@@ -1,7 +1,7 @@
 """The benchmark configurations at full size, in the launch configurations bench.py times, checked on sampled
 heads against the unsplit fp64 oracle: direct launches with the library's block-length model, and - what the
 benchmark's timed region runs - the chain recorded as a CUDA graph after profile-guided tuning of the block length,
-replayed."""
+replayed, with the default schedule and with the merged-launch schedule the schedule search may install."""
 import numpy as np
 import pytest
 import torch
@@ -33,6 +33,13 @@ def graph_run(w, x):
 
 
 def sampled_check(w, heads, mode="direct"):
+    if mode == "graph-merged":
+        binding.sf_set_tuning(dict(merge_launches=1))
+        try:
+            sampled_check(w, heads, "graph")
+        finally:
+            binding.sf_set_tuning(None)
+        return
     x = inputs.make_inputs(w, DEV)
     if mode == "graph":
         got, run = graph_run(w, x)
@@ -64,21 +71,22 @@ def sampled_check(w, heads, mode="direct"):
     torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("mode", ["direct", "graph"])
+@pytest.mark.parametrize("mode", ["direct", "graph", "graph-merged"])
 def test_config2_32k(mode):
     sampled_check(inputs.configs()[1], [0, 15], mode)
 
 
-@pytest.mark.parametrize("mode", ["direct", "graph"])
+@pytest.mark.parametrize("mode", ["direct", "graph", "graph-merged"])
 def test_config3_64k_nonuniform(mode):
     sampled_check(inputs.configs()[2], [3, 31], mode)
 
 
-@pytest.mark.parametrize("mode", ["direct", "graph"])
+@pytest.mark.parametrize("mode", ["direct", "graph", "graph-merged"])
 def test_config4_256k(mode):
     sampled_check(inputs.configs()[3], [17], mode)
 
 
+@pytest.mark.parametrize("mode", ["direct", "graph-merged"])
 @pytest.mark.parametrize("seg_len", [512, 16384])
-def test_config5_sweep_ends(seg_len):
-    sampled_check(inputs.sweep_config(seg_len), [39])
+def test_config5_sweep_ends(seg_len, mode):
+    sampled_check(inputs.sweep_config(seg_len), [39], mode)
