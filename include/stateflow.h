@@ -250,20 +250,23 @@ void sf_chain_graph_destroy(sf_chain_graph_t* graph);
 /*
  * Schedule of the chaining driver (the paper picks "tile sizes, split points and overlap schedules" per operator
  * shape by profiling a small set of valid choices, Section 3.4 last paragraph and Section 4.4 / Table 3).  Process-wide;
- * read at every sf_chain_* call (and so frozen into a graph when it is recorded).  Results do not depend on it.
+ * read at every sf_chain_* call (and so frozen into a graph when it is recorded).  Results do not depend on it
+ * (merge_launches: up to rounding, see there).
  *   sweep_streams     1..4  side streams the sweeps of consecutive segments rotate over (per kind of sweep)
  *   agg_streams       1..4  side streams the block-aggregate kernels of small segments rotate over
  *   scan_group_tokens >= 0  neighbouring segments of at most this many tokens in total share one scan launch
  *   agg_inorder_ctas  >= 1  an aggregate launch of at least this many CTAs stays in order on the first aggregate stream
  *   agg_ahead         >= 0  how many segments the aggregate kernels may run ahead of the sweeps (0 = no limit);
  *                           a small value keeps what the aggregates read close to the sweeps that read it again
- *   merge_launches    0 / 1 1: when every segment but the last is a whole number of blocks of one common length, each
- *                           stage runs once over the whole chain (the blocks of all segments in one launch) instead of
- *                           once per segment; same kernels and, for the same block length, the same blocks and bits
- *                           (with chunks_per_block = 0 the longest common length is taken, which may differ from the
- *                           segments' own: results then agree to rounding); chains of another shape run segment by
- *                           segment as with 0.  The forward workspace is laid out differently, so a
- *                           backward that reuses it must run under the same value as its forward.
+ *   merge_launches    0 / 1 1: the chain runs as ONE segment spanning the sequence, every stage once (one aggregate launch,
+ *                           one scan, one sweep, ...) instead of once per segment.  Tensor-core path: whenever all segments
+ *                           but the last are whole chunks; the blocks then ignore the segment boundaries (block length =
+ *                           chunks_per_block, else the library's choice for the whole sequence) and the forward sweep
+ *                           itself writes the state entering each segment to S_bounds.  CUDA-core path: when every segment
+ *                           but the last is a whole number of blocks of one common length.  Other chains run segment by
+ *                           segment as with 0.  Same kernels; where the blocks coincide with the segments' own the
+ *                           results are bit-identical, else equal to rounding.  The forward workspace is laid out
+ *                           differently, so a backward that reuses it must run under the same value as its forward.
  * The block length is part of the descriptor (chunks_per_block); forward and backward share it because the backward
  * starts its blocks from the block states the forward saved.
  * sf_set_tuning(NULL) restores the defaults {4, 4, 4096, 74, 0, 0}; out-of-range values give SF_ERR_INVALID_ARG and change

@@ -19,6 +19,12 @@ struct SegParams {
     int NB;       // blocks in the segment
     long long tqk, tv, tg;   // token strides (elements)
     long long bqk, bv, bg;   // batch strides (elements)
+    // Boundary states of a chain whose segments run as one (merged launches): bslot[c] >= 0 marks chunk c as the first
+    // chunk of segment bslot[c]; the forward sweep then stores the state entering that chunk to bbase + bslot[c]*bstride
+    // (one [B,H,d_k,d_v] array per segment).  NULL outside that mode.
+    const int* bslot;
+    float* bbase;
+    long long bstride;
 };
 
 // Error codes written to the device status word by kernels whose bounded waits run out.

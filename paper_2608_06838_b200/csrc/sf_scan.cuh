@@ -123,6 +123,15 @@ __global__ void __launch_bounds__(SCAN_NT) state_scan_group_kernel(ScanGroup grp
 // evaluated chunk by chunk: P_{c+1} = P_c - sum_{t in chunk c} x_t, dg_u = P_{c+1} + sum_{t=u}^{end of c} x_t.
 // Re-anchoring at every block keeps rounding errors of the dot products from accumulating over the
 // segment.  grid = (NB, H, B), 256 threads.  xq, xk: [B,H,L]; dg: [B,L,H] with strides.
+// Marks the first chunk of segments first .. first + count - 1 of a chain in slot[] (see SegParams::bslot); the rest of
+// slot[] has been set to -1 before.  The chunk indices travel as kernel arguments, so the launch can be recorded in a graph.
+constexpr int MARK_MAX = 256;
+struct SegStarts { int chunk[MARK_MAX]; int first, count; };
+__global__ void mark_bounds_kernel(int* __restrict__ slot, SegStarts s) {
+    const int i = threadIdx.x;
+    if (i < s.count) slot[s.chunk[i]] = s.first + i;
+}
+
 constexpr int DG_NT = 256;
 
 __global__ void __launch_bounds__(DG_NT) dg_epilogue_kernel(SegParams p, int m, const float* __restrict__ xq,

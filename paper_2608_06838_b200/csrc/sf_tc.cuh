@@ -234,7 +234,7 @@ __device__ __forceinline__ void mask_pass(uint32_t sc, const float* bch, unsigne
 // init[i*128 + a] when `transposed`) instead of TMEM.
 template <int NU>
 __device__ __forceinline__ void state_pass(uint32_t acc, unsigned char* sb, float decay, const float* __restrict__ init, bool transposed,
-                                           int u0) {
+                                           int u0, float* __restrict__ dump = nullptr) {
     const int a = threadIdx.x & 127, warp = a >> 5;
     const uint32_t taddr = acc + ((uint32_t)(warp * 32) << 16);
     // two units (32 registers) at a time keeps the register footprint small enough for the 96-register budget
@@ -264,6 +264,16 @@ __device__ __forceinline__ void state_pass(uint32_t acc, unsigned char* sb, floa
             for (int k = 0; k < 2; ++k)
                 if (k < nk) ptx::tmem_ld16(taddr + (u0 + k0 + k) * 16, v[k]);
             ptx::tmem_ld_wait();
+        }
+        if (dump) {
+            // the state entering this chunk is a boundary state of the chain: row a, this thread's 16-column units
+#pragma unroll
+            for (int k = 0; k < 2; ++k)
+                if (k < nk) {
+                    float4* o4 = reinterpret_cast<float4*>(dump + a * D + (u0 + k0 + k) * 16);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) o4[i] = make_float4(v[k][4 * i], v[k][4 * i + 1], v[k][4 * i + 2], v[k][4 * i + 3]);
+                }
         }
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
@@ -687,12 +697,17 @@ __device__ __forceinline__ void sweep_body(const CUtensorMap* tmQ, const CUtenso
                 const int s = c % SW_STAGES;
                 const float* bch = sm.bloc + c * C;
                 const float bC = sm.ctot[c];
+                float* dump = nullptr;                   // merged launches: the state entering a segment's first chunk goes out
+                if (!DQ && p.bslot) {
+                    const int slot = __ldg(p.bslot + c0 + c);
+                    if (slot >= 0) dump = p.bbase + slot * p.bstride + ((long long)b * p.H + h) * (long long)(D * D);
+                }
                 if (wg < 2) SF_WAIT(&sm.full[s], (c / SW_STAGES) & 1, DEV_TIMEOUT_TMA);
                 if (c > 0) SF_WAIT(&sm.st_done, (c - 1) & 1, DEV_TIMEOUT_MMA);
                 ptx::tc_fence_after_sync();
                 // 16-column units: WG0 0-2, WG1 3-5, WG2 6-7
-                if (wg < 2) state_pass<3>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 3 * wg);
-                else        state_pass<2>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 6);
+                if (wg < 2) state_pass<3>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 3 * wg, dump);
+                else        state_pass<2>(tmem + T_ST, sm.sb, fast_exp(bC), c == 0 ? H0 : nullptr, DQ, 6, dump);
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive_warp(&sm.st_ready);

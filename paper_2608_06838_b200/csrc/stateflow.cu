@@ -143,6 +143,7 @@ SegParams make_params(const sf_seg_desc_t* d, int cpb_override = 0) {
     p.NB = (p.NC + p.R - 1) / p.R;
     p.tqk = d->tok_stride_qk; p.tv = d->tok_stride_v; p.tg = d->tok_stride_g;
     p.bqk = d->batch_stride_qk; p.bv = d->batch_stride_v; p.bg = d->batch_stride_g;
+    p.bslot = nullptr; p.bbase = nullptr; p.bstride = 0;
     return p;
 }
 
@@ -482,17 +483,34 @@ sf_status_t validate_chain(const sf_seg_desc_t* d, const int32_t* seg_lens, int3
 }
 
 // ---- merged launches (sf_tuning_t.merge_launches) ------------------------------------------------------------------
-// When every segment but the last is a whole number of blocks of one common length R, the blocks of all segments are
-// the blocks of ONE segment that spans the sequence: each stage then runs once over the whole chain (one aggregate launch,
+// When the segments are whole chunks (tensor-core path) or, on the CUDA-core path, every segment but the last is a whole
+// number of blocks of one common length R, the chain is ONE segment that spans the sequence: each stage then runs once over the whole chain (one aggregate launch,
 // one scan, one sweep, ...) instead of once per segment, with the same blocks, the same kernels and the same arithmetic
 // (results are bit-identical).  The boundary states S_bounds[i] are the states entering the first block of each segment.
 // Returns the descriptor of that segment, or false if the chain does not have this shape.
-bool merged_desc(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, long long T, sf_seg_desc_t* out) {
+// `free_grid`: on the tensor-core path the forward sweep itself writes the state entering a segment's first chunk
+// (SegParams::bslot), so the blocks need not respect the segment boundaries: any block length, segments of whole chunks.
+bool merged_desc(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, long long T, sf_seg_desc_t* out,
+                 bool* free_grid = nullptr) {
+    if (free_grid) *free_grid = false;
     if (n_seg < 2 || T > 0x7fffffffLL) return false;
     const int C = desc->chunk;
-    int R = desc->chunks_per_block;
     for (int i = 0; i + 1 < n_seg; ++i)
         if (seg_lens[i] % C) return false;
+    sf_seg_desc_t t = *desc;
+    t.seg_len = (int32_t)T;
+    {
+        sf_seg_desc_t f = t;                             // block length: the caller's, else the library's model for one long segment
+        const Path path = classify(&f);
+        if (path == Path::Tc) {
+            if (make_params(&f).NB > 65535) return false;
+            f.chunks_per_block = make_params(&f).R;
+            *out = f;
+            if (free_grid) *free_grid = true;
+            return true;
+        }
+    }
+    int R = desc->chunks_per_block;
     if (R == 0) {
         // the longest block length (at most 64 chunks) that divides the chunk count of every segment but the last
         for (R = 64; R >= 1; --R) {
@@ -505,8 +523,6 @@ bool merged_desc(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_s
         for (int i = 0; i + 1 < n_seg; ++i)
             if ((seg_lens[i] / C) % R) return false;
     }
-    sf_seg_desc_t t = *desc;
-    t.seg_len = (int32_t)T;
     t.chunks_per_block = R;
     const Path path = classify(&t);
     if (path == Path::Invalid || path == Path::Unsupported) return false;
@@ -515,20 +531,44 @@ bool merged_desc(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_s
     return true;
 }
 
-sf_status_t chain_fwd_merged(const sf_seg_desc_t* vd, const int32_t* seg_lens, int32_t n_seg, const FwdPtrs& x, float* S_bounds,
-                             void* workspace, cudaStream_t st) {
+size_t merged_slot_bytes(const sf_seg_desc_t* vd) { return align_up((size_t)make_params(vd).NC * sizeof(int)); }
+
+sf_status_t chain_fwd_merged(const sf_seg_desc_t* vd, bool free_grid, const int32_t* seg_lens, int32_t n_seg, const FwdPtrs& x,
+                             float* S_bounds, void* workspace, cudaStream_t st) {
     const Path path = classify(vd);
-    const SegParams p = make_params(vd);
+    SegParams p = make_params(vd);
     const FwdWs w = fwd_ws(vd, p, workspace);
+    const size_t m = (size_t)vd->d_k * vd->d_v, sN = (size_t)vd->B * vd->H * m;
+    if (free_grid) {
+        // slot[c] = i for the first chunk c of segment i >= 1, else -1; read by the forward sweep
+        int* slot = reinterpret_cast<int*>(static_cast<char*>(workspace) + w.bytes);
+        SF_CUDA(cudaMemsetAsync(slot, 0xFF, (size_t)p.NC * sizeof(int), st));
+        long long chunk = 0;
+        for (int i0 = 1; i0 < n_seg; i0 += sf::MARK_MAX) {
+            sf::SegStarts s{};
+            s.first = i0;
+            s.count = n_seg - i0 < sf::MARK_MAX ? n_seg - i0 : sf::MARK_MAX;
+            for (int k = 0; k < s.count; ++k) {
+                chunk += seg_lens[i0 + k - 1] / vd->chunk;
+                s.chunk[k] = (int)chunk;
+            }
+            sf::mark_bounds_kernel<<<1, sf::MARK_MAX, 0, st>>>(slot, s);
+            SF_TRY(check_launch());
+        }
+        p.bslot = slot;
+        p.bbase = S_bounds;
+        p.bstride = (long long)sN;
+    }
     SF_TRY(fwd_pre(path, vd, p, x, w, st));
     SF_TRY(fwd_scan(vd, p, x, w, st));
-    // S_bounds[i] = state entering the first block of segment i (a strided copy: one state per batch x head)
-    const size_t m = (size_t)vd->d_k * vd->d_v, sN = (size_t)vd->B * vd->H * m;
-    long long blk = 0;
-    for (int i = 1; i < n_seg; ++i) {
-        blk += (seg_lens[i - 1] / vd->chunk) / p.R;
-        SF_CUDA(cudaMemcpy2DAsync(S_bounds + (size_t)i * sN, m * sizeof(float), w.UH + (size_t)blk * m, (size_t)p.NB * m * sizeof(float),
-                                  m * sizeof(float), (size_t)vd->B * vd->H, cudaMemcpyDeviceToDevice, st));
+    if (!free_grid) {
+        // S_bounds[i] = state entering the first block of segment i (a strided copy: one state per batch x head)
+        long long blk = 0;
+        for (int i = 1; i < n_seg; ++i) {
+            blk += (seg_lens[i - 1] / vd->chunk) / p.R;
+            SF_CUDA(cudaMemcpy2DAsync(S_bounds + (size_t)i * sN, m * sizeof(float), w.UH + (size_t)blk * m, (size_t)p.NB * m * sizeof(float),
+                                      m * sizeof(float), (size_t)vd->B * vd->H, cudaMemcpyDeviceToDevice, st));
+        }
     }
     return fwd_out(path, vd, p, x, w, st);
 }
@@ -707,7 +747,7 @@ size_t sf_chain_workspace_bytes(const sf_seg_desc_t* desc, const int32_t* seg_le
     for (int i = 0; i < n_seg; ++i) T += seg_lens[i];
     sf_seg_desc_t vd;
     if (merged_desc(desc, seg_lens, n_seg, T, &vd)) {
-        const size_t mb = sf_workspace_bytes(&vd, backward);
+        const size_t mb = sf_workspace_bytes(&vd, backward) + (backward == 0 ? merged_slot_bytes(&vd) : 0);
         need = mb > need ? mb : need;
     }
     return need;
@@ -734,10 +774,11 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     const sf_tuning_t tu = current_tuning();
     {
         sf_seg_desc_t vd;
-        if (tu.merge_launches && merged_desc(desc, seg_lens, n_seg, T, &vd) &&
-            sf_workspace_bytes(&vd, 0) <= workspace_bytes) {
+        bool free_grid = false;
+        if (tu.merge_launches && merged_desc(desc, seg_lens, n_seg, T, &vd, &free_grid) &&
+            sf_workspace_bytes(&vd, 0) + merged_slot_bytes(&vd) <= workspace_bytes) {
             FwdPtrs x{q, k, v, g, S_bounds, o, S_bounds + (size_t)n_seg * sN};
-            return chain_fwd_merged(&vd, seg_lens, n_seg, x, S_bounds, workspace, st);
+            return chain_fwd_merged(&vd, free_grid, seg_lens, n_seg, x, S_bounds, workspace, st);
         }
     }
     ChainRes* res = nullptr;
