@@ -236,10 +236,20 @@ def main():
     torch.cuda.synchronize()
     work_stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
 
-    # profile-guided block length (untimed preparation, like the graph capture below); candidates are timed the
-    # way the step will run: as graph replays on the work stream, or launched from the host with --no-graph
+    # Profile-guided tuning (untimed preparation, like the graph capture below), both with the same margin rule.  First the
+    # schedule of the chain driver (streams, how far the aggregates run ahead, merged launches) at the library's own block
+    # length, then the block length under the schedule that was installed: the best block length depends on the schedule.
     tuned = None
+    if args.autotune and overlap and args.graph:
+        with torch.cuda.stream(work_stream):
+            t, t_ms, d_ms = run.autotune_schedule(x["S_in"], x["dS_out"], reps=10, margin=0.02)
+        work_stream.synchronize()
+        tuned = {"schedule": {"sweep_streams": t.sweep_streams, "agg_streams": t.agg_streams, "scan_group_tokens": t.scan_group_tokens,
+                              "agg_inorder_ctas": t.agg_inorder_ctas, "agg_ahead": t.agg_ahead, "merge_launches": t.merge_launches,
+                              "ms": round(t_ms, 4), "default_ms": round(d_ms, 4)}}
     if args.autotune and args.chunks_per_block == 0:
+        # candidates are timed the way the step will run: as graph replays on the work stream, or launched from the host
+        # with --no-graph
         cands = [0, 16, 22, 29, 32, 43, 52, 64]
         with torch.cuda.stream(work_stream):
             best, cand_ms = run.autotune(x["S_in"], x["dS_out"], cands, reps=10, overlap=overlap)
@@ -251,17 +261,9 @@ def main():
         if model_ms > 0 and model_ms <= 1.02 * best_ms:
             best = 0
         run.desc.chunks_per_block = best
-        tuned = {"candidates": cands, "ms": [round(v, 4) for v in cand_ms], "chosen": best, "rule": "model unless > 2 % faster over 10 reps"}
-    if args.autotune and overlap and args.graph:
-        # profile-guided schedule of the chain driver (streams, how far the aggregates run ahead), same margin rule
-        with torch.cuda.stream(work_stream):
-            t, t_ms, d_ms = run.autotune_schedule(x["S_in"], x["dS_out"], reps=10, margin=0.02)
-        work_stream.synchronize()
         tuned = tuned or {}
-        tuned["schedule"] = {"sweep_streams": t.sweep_streams, "agg_streams": t.agg_streams, "scan_group_tokens": t.scan_group_tokens,
-                             "agg_inorder_ctas": t.agg_inorder_ctas, "agg_ahead": t.agg_ahead, "merge_launches": t.merge_launches,
-                             "ms": round(t_ms, 4),
-                             "default_ms": round(d_ms, 4)}
+        tuned.update({"candidates": cands, "ms": [round(v, 4) for v in cand_ms], "chosen": best,
+                      "rule": "model unless > 2 % faster over 10 reps"})
     if args.graph:
         with torch.cuda.stream(work_stream):
             run.capture(x["S_in"], x["dS_out"], overlap=overlap)
