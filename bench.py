@@ -202,6 +202,8 @@ def main():
     ap.add_argument("--no-autotune", dest="autotune", action="store_false",
                     help="keep the library's model for the block length instead of timing the candidates first "
                          "(sf_chain_autotune; only used when --chunks-per-block is 0)")
+    ap.add_argument("--merge-launches", action="store_true",
+                    help="install the merged-launch schedule (every stage once over the whole chain) instead of searching")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     args = ap.parse_args()
@@ -240,7 +242,10 @@ def main():
     # schedule of the chain driver (streams, how far the aggregates run ahead, merged launches) at the library's own block
     # length, then the block length under the schedule that was installed: the best block length depends on the schedule.
     tuned = None
-    if args.autotune and overlap and args.graph:
+    if args.merge_launches:
+        binding.sf_set_tuning(dict(merge_launches=1))
+        tuned = {"schedule": {"merge_launches": 1, "forced": True}}
+    if args.autotune and overlap and args.graph and not args.merge_launches:
         with torch.cuda.stream(work_stream):
             t, t_ms, d_ms = run.autotune_schedule(x["S_in"], x["dS_out"], reps=10, margin=0.02)
         work_stream.synchronize()
