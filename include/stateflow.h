@@ -184,7 +184,7 @@ sf_status_t sf_state_scan(const sf_seg_desc_t* desc, int32_t chunks_per_block, i
  * q, k, v, g, o, ... address token 0 of the whole sequence of T = sum(seg_lens) tokens.
  *
  * sf_chain_fwd runs Fwd on segments 0..n_seg-1 with S_{i+1}^in = S_i^out.
- *   S_init   : nullable = zero
+ *   S_init   : nullable = zero; may be S_bounds itself (the initial state is then taken as already in S_bounds[0])
  *   S_bounds : [n_seg+1][B,H,d_k,d_v] float32; on return S_bounds[i] = S_i^in and
  *              S_bounds[n_seg] = the final state.  Kept by the caller for sf_chain_bwd.
  *   workspace: sf_chain_workspace_bytes(..., 0) bytes; holds every segment's saved block states.
@@ -349,9 +349,12 @@ sf_status_t sf_partition_hybrid(int64_t T, int32_t N, double w_tok, double w_sof
  * buffers in `dev` (caller-allocated device scratch, sf_e2e_device_bytes() bytes, 256-byte
  * aligned), runs sf_chain_fwd + sf_chain_bwd and copies o, dq, dk, dv, dg, the final state and
  * dS_init back, then synchronises `stream`; everything is ordered after earlier work on `stream` and is complete
- * when the call returns.  The upload of dO and the download of o run on two copy streams of the library beside the
- * forward and backward chains, so that both PCIe directions are busy at once where the dependencies allow (needs
- * pinned host memory to take effect).  Uses the chain driver's per-device streams: the threading rule of
+ * when the call returns.  The chain is pipelined segment by segment against the copies on two copy streams of the
+ * library: inputs are uploaded in segment order (dO afterwards, last segment first), a segment's forward runs as soon
+ * as its inputs are there and its o goes back while later inputs still arrive; a segment's backward runs as soon as
+ * its dO is there and its gradients go back while earlier segments' dO still arrive.  Both PCIe directions are busy
+ * for most of the call (needs pinned host memory to take effect).  Each segment runs as a one-segment chain, in
+ * order, on `stream`.  Uses the chain driver's per-device streams: the threading rule of
  * sf_chain_* with overlap != 0 applies.  Section 3.1, Eq. 4-7.
  */
 size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg);

@@ -768,8 +768,9 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     const size_t sN = (size_t)desc->B * desc->H * desc->d_k * desc->d_v;
 
     // S_bounds[0] = S_init (or zero)
-    if (S_init) SF_CUDA(cudaMemcpyAsync(S_bounds, S_init, sN * sizeof(float), cudaMemcpyDeviceToDevice, st));
-    else        SF_CUDA(cudaMemsetAsync(S_bounds, 0, sN * sizeof(float), st));
+    if (S_init == S_bounds) {}              // the state is in place already
+    else if (S_init) SF_CUDA(cudaMemcpyAsync(S_bounds, S_init, sN * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    else             SF_CUDA(cudaMemsetAsync(S_bounds, 0, sN * sizeof(float), st));
 
     const sf_tuning_t tu = current_tuning();
     {
@@ -1270,6 +1271,22 @@ sf_status_t sf_partition_hybrid(int64_t T, int32_t N, double w_tok, double w_sof
     return SF_OK;
 }
 
+namespace {
+// Device-buffer plan of the host wrapper: per-segment forward workspaces (kept for the backward), one backward
+// workspace (the segments' backward passes run one after the other on the caller's stream).
+struct E2ePlan { std::vector<size_t> wf; size_t wf_total = 0, wb = 0; };
+E2ePlan e2e_plan(const sf_seg_desc_t* d, const int32_t* seg_lens, int32_t n_seg) {
+    E2ePlan pl;
+    pl.wf.resize(n_seg);
+    for (int i = 0; i < n_seg; ++i) {
+        pl.wf[i] = align_up(sf_chain_workspace_bytes(d, seg_lens + i, 1, 0));
+        pl.wf_total += pl.wf[i];
+        pl.wb = std::max(pl.wb, align_up(sf_chain_workspace_bytes(d, seg_lens + i, 1, 1)));
+    }
+    return pl;
+}
+}  // namespace
+
 size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg) {
     long long T = 0;
     if (validate_chain(desc, seg_lens, n_seg, &T) != SF_OK) return 0;
@@ -1278,8 +1295,8 @@ size_t sf_e2e_device_bytes(const sf_seg_desc_t* desc, const int32_t* seg_lens, i
     const size_t nv = align_up((size_t)desc->B * T * desc->H * desc->d_v * esz);
     const size_t ng = align_up((size_t)desc->B * T * desc->H * sizeof(float));
     const size_t sB = state_bytes(desc);
-    return 4 * nqk + 4 * nv + 2 * ng + (size_t)(n_seg + 1) * sB + 3 * sB +
-           sf_chain_workspace_bytes(desc, seg_lens, n_seg, 0) + sf_chain_workspace_bytes(desc, seg_lens, n_seg, 1);
+    const E2ePlan pl = e2e_plan(desc, seg_lens, n_seg);
+    return 4 * nqk + 4 * nv + 2 * ng + (size_t)(n_seg + 1) * sB + 3 * sB + pl.wf_total + pl.wb;
 }
 
 sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_lens, int32_t n_seg, const void* q,
@@ -1300,62 +1317,107 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
         return SF_ERR_INVALID_ARG;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const size_t esz = d.dtype == SF_BF16 ? 2 : 4;
-    const size_t bqk = (size_t)d.B * T * d.H * d.d_k * esz, bv = (size_t)d.B * T * d.H * d.d_v * esz;
-    const size_t bg = (size_t)d.B * T * d.H * sizeof(float);
+    const size_t rqk = (size_t)d.H * d.d_k * esz, rv = (size_t)d.H * d.d_v * esz, rg = (size_t)d.H * sizeof(float);   // bytes per token
+    const size_t bqk = (size_t)d.B * T * rqk, bv = (size_t)d.B * T * rv, bg = (size_t)d.B * T * rg;
     const size_t nqk = align_up(bqk), nv = align_up(bv), ng = align_up(bg), sB = state_bytes(&d);
-    const size_t sbytes = (size_t)d.B * d.H * d.d_k * d.d_v * sizeof(float);
+    const size_t sN = (size_t)d.B * d.H * d.d_k * d.d_v, sbytes = sN * sizeof(float);
+    const E2ePlan pl = e2e_plan(&d, seg_lens, n_seg);
     char* c = static_cast<char*>(dev);
     auto take = [&](size_t n) { char* r = c; c += n; return r; };
     char *dq_ = take(nqk), *dk_ = take(nqk), *q_ = take(nqk), *k_ = take(nqk);
     char *v_ = take(nv), *dO_ = take(nv), *o_ = take(nv), *dv_ = take(nv);
     char *g_ = take(ng), *dg_ = take(ng);
-    float* bounds = reinterpret_cast<float*>(take((size_t)(n_seg + 1) * sB));
-    float* sinit = reinterpret_cast<float*>(take(sB));
+    float* bounds = reinterpret_cast<float*>(take((size_t)(n_seg + 1) * sB));      // indexed densely (sN floats apart)
     float* dsfin = reinterpret_cast<float*>(take(sB));
-    float* dsinit = reinterpret_cast<float*>(take(sB));
-    const size_t wf = sf_chain_workspace_bytes(&d, seg_lens, n_seg, 0), wb = sf_chain_workspace_bytes(&d, seg_lens, n_seg, 1);
-    char* wsf = take(wf);
-    char* wsb = take(wb);
+    float* dsbuf[2] = {reinterpret_cast<float*>(take(sB)), nullptr};
+    dsbuf[1] = reinterpret_cast<float*>(take(sB));
+    char* wsf = take(pl.wf_total);
+    char* wsb = take(pl.wb);
 
-    // Copies that nothing waits for yet run beside the compute on two copy streams, so that the two PCIe directions
-    // are busy at the same time where the dependencies allow it:
-    //   caller's stream : up q, k, v, g, S_init -> forward chain -> [wait dO] backward chain -> down dq, dk, dv, dg, dS_init
-    //   upload stream   : up dO, dS_final                      (needed only by the backward)
-    //   download stream : [wait forward] down o, S_final       (overlaps the upload of dO and the backward)
+    // The chain is pipelined segment by segment against the copies, so that both PCIe directions carry data for most
+    // of the call (a step moves far more bytes over PCIe than the kernels take time for):
+    //   upload stream   : q, k, v, g of segment 0, 1, ... n-1, then dO of segment n-1, n-2, ... 0
+    //   caller's stream : [wait inputs(i)] forward(i) ...          then [wait dO(i)] backward(i) for i = n-1 ... 0
+    //   download stream : [wait forward(i)] o(i) ...               then [wait backward(i)] dq, dk, dv, dg of segment i
+    // Segment i is one time slice of every [B, T, H, d] tensor: B rows of len*H*d elements, T*H*d apart (a 2-D copy).
     ChainRes* res = nullptr;
     SF_TRY(chain_resources(&res));
     cudaStream_t up = res->copy[0], down = res->copy[1];
-    cudaEvent_t e_start = res->ev[1], e_dO = res->ev[2], e_fwd = res->ev[3], e_o = res->ev[4];
+    std::vector<cudaEvent_t> ev(4 * (size_t)n_seg + 2, nullptr);
+    struct EventGuard {
+        std::vector<cudaEvent_t>& e;
+        ~EventGuard() { for (cudaEvent_t x : e) if (x) cudaEventDestroy(x); }
+    } guard{ev};
+    for (auto& e : ev) SF_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    cudaEvent_t* e_in = ev.data();                   // inputs of segment i on the device
+    cudaEvent_t* e_dO = ev.data() + n_seg;           // dO of segment i on the device
+    cudaEvent_t* e_f = ev.data() + 2 * (size_t)n_seg;   // forward of segment i done
+    cudaEvent_t* e_b = ev.data() + 3 * (size_t)n_seg;   // backward of segment i done
+    cudaEvent_t e_start = ev[4 * (size_t)n_seg], e_end = ev[4 * (size_t)n_seg + 1];
+    auto slice = [&](void* dst, const void* src, size_t row, long long tok, long long len, cudaMemcpyKind kind, cudaStream_t s) {
+        const size_t pitch = (size_t)T * row;
+        return cudaMemcpy2DAsync(static_cast<char*>(dst) + (size_t)tok * row, pitch, static_cast<const char*>(src) + (size_t)tok * row,
+                                 pitch, (size_t)len * row, (size_t)d.B, kind, s);
+    };
+    std::vector<long long> tok0(n_seg + 1, 0);
+    for (int i = 0; i < n_seg; ++i) tok0[i + 1] = tok0[i] + seg_lens[i];
+
     SF_CUDA(cudaEventRecord(e_start, st));
-    SF_CUDA(cudaMemcpyAsync(q_, q, bqk, cudaMemcpyHostToDevice, st));
-    SF_CUDA(cudaMemcpyAsync(k_, k, bqk, cudaMemcpyHostToDevice, st));
-    SF_CUDA(cudaMemcpyAsync(v_, v, bv, cudaMemcpyHostToDevice, st));
-    SF_CUDA(cudaMemcpyAsync(g_, g, bg, cudaMemcpyHostToDevice, st));
-    if (S_init) SF_CUDA(cudaMemcpyAsync(sinit, S_init, sbytes, cudaMemcpyHostToDevice, st));
     SF_CUDA(cudaStreamWaitEvent(up, e_start, 0));
-    SF_CUDA(cudaMemcpyAsync(dO_, dO, bv, cudaMemcpyHostToDevice, up));
+    SF_CUDA(cudaStreamWaitEvent(down, e_start, 0));
+    if (S_init) SF_CUDA(cudaMemcpyAsync(bounds, S_init, sbytes, cudaMemcpyHostToDevice, up));
+    else        SF_CUDA(cudaMemsetAsync(bounds, 0, sbytes, up));
+    for (int i = 0; i < n_seg; ++i) {
+        SF_CUDA(slice(q_, q, rqk, tok0[i], seg_lens[i], cudaMemcpyHostToDevice, up));
+        SF_CUDA(slice(k_, k, rqk, tok0[i], seg_lens[i], cudaMemcpyHostToDevice, up));
+        SF_CUDA(slice(v_, v, rv, tok0[i], seg_lens[i], cudaMemcpyHostToDevice, up));
+        SF_CUDA(slice(g_, g, rg, tok0[i], seg_lens[i], cudaMemcpyHostToDevice, up));
+        SF_CUDA(cudaEventRecord(e_in[i], up));
+    }
     if (dS_final) SF_CUDA(cudaMemcpyAsync(dsfin, dS_final, sbytes, cudaMemcpyHostToDevice, up));
-    SF_CUDA(cudaEventRecord(e_dO, up));
-    // sB is a multiple of 256 but the chain driver indexes bounds densely
-    float* bounds_dense = bounds;
-    SF_TRY(sf_chain_fwd(&d, seg_lens, n_seg, q_, k_, v_, reinterpret_cast<float*>(g_), S_init ? sinit : nullptr, o_,
-                        bounds_dense, wsf, wf, 1, stream));
-    SF_CUDA(cudaEventRecord(e_fwd, st));
-    SF_CUDA(cudaStreamWaitEvent(down, e_fwd, 0));
-    SF_CUDA(cudaMemcpyAsync(o, o_, bv, cudaMemcpyDeviceToHost, down));
-    if (S_final)
-        SF_CUDA(cudaMemcpyAsync(S_final, bounds_dense + (size_t)n_seg * (sbytes / sizeof(float)), sbytes, cudaMemcpyDeviceToHost, down));
-    SF_CUDA(cudaEventRecord(e_o, down));
-    SF_CUDA(cudaStreamWaitEvent(st, e_dO, 0));
-    SF_TRY(sf_chain_bwd(&d, seg_lens, n_seg, q_, k_, v_, reinterpret_cast<float*>(g_), bounds_dense, dO_,
-                        dS_final ? dsfin : nullptr, dq_, dk_, dv_, reinterpret_cast<float*>(dg_), dsinit, wsf, wsb,
-                        wb, 1, stream));
-    SF_CUDA(cudaMemcpyAsync(dq, dq_, bqk, cudaMemcpyDeviceToHost, st));
-    SF_CUDA(cudaMemcpyAsync(dk, dk_, bqk, cudaMemcpyDeviceToHost, st));
-    SF_CUDA(cudaMemcpyAsync(dv, dv_, bv, cudaMemcpyDeviceToHost, st));
-    SF_CUDA(cudaMemcpyAsync(dg, dg_, bg, cudaMemcpyDeviceToHost, st));
-    SF_CUDA(cudaMemcpyAsync(dS_init, dsinit, sbytes, cudaMemcpyDeviceToHost, st));
-    SF_CUDA(cudaStreamWaitEvent(st, e_o, 0));
+    for (int i = n_seg - 1; i >= 0; --i) {
+        SF_CUDA(slice(dO_, dO, rv, tok0[i], seg_lens[i], cudaMemcpyHostToDevice, up));
+        SF_CUDA(cudaEventRecord(e_dO[i], up));
+    }
+    // forward, segment by segment as the inputs arrive; the boundary state of segment i is already in bounds[i]
+    {
+        size_t off = 0;
+        for (int i = 0; i < n_seg; ++i) {
+            float* b_i = bounds + (size_t)i * sN;
+            SF_CUDA(cudaStreamWaitEvent(st, e_in[i], 0));
+            SF_TRY(sf_chain_fwd(&d, seg_lens + i, 1, q_ + tok0[i] * rqk, k_ + tok0[i] * rqk, v_ + tok0[i] * rv,
+                                reinterpret_cast<float*>(g_ + tok0[i] * rg), b_i, o_ + tok0[i] * rv, b_i, wsf + off, pl.wf[i], 0, stream));
+            SF_CUDA(cudaEventRecord(e_f[i], st));
+            SF_CUDA(cudaStreamWaitEvent(down, e_f[i], 0));
+            SF_CUDA(slice(o, o_, rv, tok0[i], seg_lens[i], cudaMemcpyDeviceToHost, down));
+            off += pl.wf[i];
+        }
+        if (S_final) SF_CUDA(cudaMemcpyAsync(S_final, bounds + (size_t)n_seg * sN, sbytes, cudaMemcpyDeviceToHost, down));
+    }
+    // backward, last segment first as its dO arrives; dS ping-pongs between two buffers
+    {
+        size_t off = pl.wf_total;
+        const float* ds_out = dS_final ? dsfin : nullptr;
+        for (int i = n_seg - 1; i >= 0; --i) {
+            off -= pl.wf[i];
+            float* ds_in = dsbuf[i & 1];
+            SF_CUDA(cudaStreamWaitEvent(st, e_dO[i], 0));
+            SF_TRY(sf_chain_bwd(&d, seg_lens + i, 1, q_ + tok0[i] * rqk, k_ + tok0[i] * rqk, v_ + tok0[i] * rv,
+                                reinterpret_cast<float*>(g_ + tok0[i] * rg), bounds + (size_t)i * sN, dO_ + tok0[i] * rv, ds_out,
+                                dq_ + tok0[i] * rqk, dk_ + tok0[i] * rqk, dv_ + tok0[i] * rv, reinterpret_cast<float*>(dg_ + tok0[i] * rg),
+                                ds_in, wsf + off, wsb, pl.wb, 0, stream));
+            SF_CUDA(cudaEventRecord(e_b[i], st));
+            SF_CUDA(cudaStreamWaitEvent(down, e_b[i], 0));
+            SF_CUDA(slice(dq, dq_, rqk, tok0[i], seg_lens[i], cudaMemcpyDeviceToHost, down));
+            SF_CUDA(slice(dk, dk_, rqk, tok0[i], seg_lens[i], cudaMemcpyDeviceToHost, down));
+            SF_CUDA(slice(dv, dv_, rv, tok0[i], seg_lens[i], cudaMemcpyDeviceToHost, down));
+            SF_CUDA(slice(dg, dg_, rg, tok0[i], seg_lens[i], cudaMemcpyDeviceToHost, down));
+            ds_out = ds_in;
+        }
+        SF_CUDA(cudaMemcpyAsync(dS_init, dsbuf[0], sbytes, cudaMemcpyDeviceToHost, down));
+    }
+    SF_CUDA(cudaEventRecord(e_end, down));
+    SF_CUDA(cudaStreamWaitEvent(st, e_end, 0));
     SF_CUDA(cudaStreamSynchronize(st));
     return SF_OK;
 }

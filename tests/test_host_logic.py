@@ -271,3 +271,28 @@ def test_chunked_diagonal_decay_validates_before_any_launch(lib):
     bad = list(bargs)
     bad[5] = None                                                    # dO missing
     assert lib.sf_channel_chunked_bwd(ctypes.byref(d), *bad, W, 1 << 40, None) == 1
+
+
+def test_host_wrapper_scratch_size_and_validation(lib):
+    d = desc()
+    segs = (ctypes.c_int32 * 3)(1024, 512, 2048)
+    T = 3584
+    need = lib.sf_e2e_device_bytes(ctypes.byref(d), segs, 3)
+    # eight [T, H, 128] bf16 tensors, g and dg, four + three boundary-state buffers, per-segment forward workspaces
+    # kept for the backward, one backward workspace (the largest segment's)
+    state = 2 * 128 * 128 * 4
+    one = lambda i, bwd: lib.sf_chain_workspace_bytes(ctypes.byref(d), (ctypes.c_int32 * 1)(segs[i]), 1, bwd)
+    up = lambda n: (n + 255) // 256 * 256
+    want = 8 * T * 2 * 128 * 2 + 2 * T * 2 * 4 + 7 * state + sum(up(one(i, 0)) for i in range(3)) + max(up(one(i, 1)) for i in range(3))
+    assert need == want
+    assert lib.sf_e2e_device_bytes(ctypes.byref(d), segs, 0) == 0
+    call = lambda dev, nbytes, dq=P: lib.sf_chain_fwd_bwd_host(ctypes.byref(d), segs, 3, P, P, P, P, None, P, None, P, None, dq, P, P, P,
+                                                              P, dev, nbytes, None)
+    assert call(ctypes.c_void_p(0x40000), need - 1) == 3          # SF_ERR_WORKSPACE
+    assert call(None, need) == 3
+    assert call(ctypes.c_void_p(0x40000), need, dq=None) == 1     # SF_ERR_INVALID_ARG
+    assert call(ctypes.c_void_p(0x40010), need) == 1              # scratch not 256-byte aligned
+    strided = desc()
+    strided.tok_stride_qk = 2 * 2 * 128                            # the wrapper wants densely packed host tensors
+    assert lib.sf_chain_fwd_bwd_host(ctypes.byref(strided), segs, 3, P, P, P, P, None, P, None, P, None, P, P, P, P, P,
+                                     ctypes.c_void_p(0x40000), 1 << 40, None) == 1
