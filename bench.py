@@ -371,8 +371,20 @@ def main():
         nb = lambda t: 0 if t is None else t.numel() * t.element_size()
         h2d = sum(nb(host[n]) for n in ("q", "k", "v", "g", "dO", "S_in", "dS_out"))
         d2h = sum(nb(t) for t in outs.values()) + nb(S_final) + nb(dS_init)
+        # the host-buffer results against the device chain's results on the same inputs (first and last 4096 tokens of
+        # every output, both boundary results); the two runs may use different block lengths, hence a tolerance: twice the parity bound
+        worst = 0.0
+        pairs = [(outs["o"], run.o), (outs["dq"], run.dq), (outs["dk"], run.dk), (outs["dv"], run.dv), (outs["dg"], run.dg)]
+        for h, dres in pairs:
+            for sl in (slice(0, 4096), slice(-4096, None)):
+                a, b = h[:, sl].float(), dres[:, sl].float().cpu()
+                worst = max(worst, float((a - b).abs().max() / b.abs().max().clamp_min(1e-30)))
+        for h, dres in ((S_final, run.S_bounds[-1]), (dS_init, run.dS_init)):
+            b = dres.float().cpu()
+            worst = max(worst, float((h - b).abs().max() / b.abs().max().clamp_min(1e-30)))
+        assert worst <= 4e-2, "host-buffer entry point disagrees with the device chain: %.3e" % worst
         e2e = {"value": world * tokens * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "ms_per_step": 1e3 * dt / n_e2e}
+               "ms_per_step": 1e3 * dt / n_e2e, "max_norm_diff_vs_device_chain": worst}
         del scratch
 
     if rank != 0:

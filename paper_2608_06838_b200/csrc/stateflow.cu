@@ -1339,7 +1339,7 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
     //   upload stream   : q, k, v, g of segment 0, 1, ... n-1, then dO of segment n-1, n-2, ... 0
     //   caller's stream : [wait inputs(i)] forward(i) ...          then [wait dO(i)] backward(i) for i = n-1 ... 0
     //   download stream : [wait forward(i)] o(i) ...               then [wait backward(i)] dq, dk, dv, dg of segment i
-    // Segment i is one time slice of every [B, T, H, d] tensor: B rows of len*H*d elements, T*H*d apart (a 2-D copy).
+    // Segment i is one time slice of every [B, T, H, d] tensor: B rows of len*H*d elements, T*H*d apart.
     ChainRes* res = nullptr;
     SF_TRY(chain_resources(&res));
     cudaStream_t up = res->copy[0], down = res->copy[1];
@@ -1355,9 +1355,13 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
     cudaEvent_t* e_b = ev.data() + 3 * (size_t)n_seg;   // backward of segment i done
     cudaEvent_t e_start = ev[4 * (size_t)n_seg], e_end = ev[4 * (size_t)n_seg + 1];
     auto slice = [&](void* dst, const void* src, size_t row, long long tok, long long len, cudaMemcpyKind kind, cudaStream_t s) {
-        const size_t pitch = (size_t)T * row;
-        return cudaMemcpy2DAsync(static_cast<char*>(dst) + (size_t)tok * row, pitch, static_cast<const char*>(src) + (size_t)tok * row,
-                                 pitch, (size_t)len * row, (size_t)d.B, kind, s);
+        const size_t pitch = (size_t)T * row;        // one plain copy per batch row (a 2-D copy would cap the pitch at 2 GB)
+        for (int b = 0; b < d.B; ++b) {
+            const size_t off = (size_t)b * pitch + (size_t)tok * row;
+            const cudaError_t e = cudaMemcpyAsync(static_cast<char*>(dst) + off, static_cast<const char*>(src) + off, (size_t)len * row, kind, s);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
     };
     std::vector<long long> tok0(n_seg + 1, 0);
     for (int i = 0; i < n_seg; ++i) tok0[i + 1] = tok0[i] + seg_lens[i];

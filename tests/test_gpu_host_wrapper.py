@@ -32,7 +32,7 @@ def run_host(w, x, pinned=True, want_final=True, chunks_per_block=0):
 
 @pytest.mark.parametrize("pinned", [True, False])
 def test_host_wrapper_fp32_batched_nonuniform_segments(pinned):
-    # B = 2: a segment is two separate slices of every tensor (2-D copies)
+    # B = 2: a segment is two separate slices of every tensor
     w = Workload("host-f32", 2, 3, 32, 64, [128, 224, 32, 96], 32, dtype="f32", g_scale=0.2, s_in_sigma=0.4, ds_out_sigma=0.4, seed=21)
     x = inputs.make_inputs(w, DEV)
     got, _ = run_host(w, x, pinned=pinned)
