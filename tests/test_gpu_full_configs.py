@@ -90,3 +90,28 @@ def test_config4_256k(mode):
 @pytest.mark.parametrize("seg_len", [512, 16384])
 def test_config5_sweep_ends(seg_len, mode):
     sampled_check(inputs.sweep_config(seg_len), [39], mode)
+
+
+@pytest.mark.parametrize("H,d", [(256, 128), (512, 64)])
+def test_tensors_beyond_two_to_the_31_elements(H, d):
+    """Maximum sizes: every [T, H, d] tensor holds more than 2^31 elements (4.4 GB in bf16), so element and byte
+    offsets that were kept in 32 bits anywhere would wrap.  Many heads keep the per-head oracle run short; the last
+    head sits at the largest offsets of every token row, the last segment at the largest of the sequence.  d = 128
+    runs on the tensor-core kernels, d = 64 on the CUDA-core ones."""
+    w = inputs.Workload("beyond-2^31-d%d" % d, 1, H, d, d, [16384, 16384, 16384, 16512], 64, s_in_sigma=0.02, ds_out_sigma=0.02, seed=31)
+    assert w.T * w.H * w.d_k > 2 ** 31
+    heads = [0, H - 1]
+    x = inputs.make_inputs(w, DEV)
+    ref = oracle_reference(x, heads=heads)
+    for merged in (0, 1):
+        binding.sf_set_tuning(dict(merge_launches=merged))
+        try:
+            got, run = run_chain(w, x)
+        finally:
+            binding.sf_set_tuning(None)
+        compare(got, ref, tolerance(w), heads=heads, label="%s/merged=%d" % (w.name, merged))
+        for n in ("o", "dq", "dk", "dv"):
+            tail = got[n][:, -4096:]                           # cheap whole-width look at the far end of the buffers
+            assert torch.isfinite(tail.float()).all() and float(tail.float().abs().max()) > 0, n
+        del run, got
+        torch.cuda.empty_cache()
