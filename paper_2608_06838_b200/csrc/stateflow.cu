@@ -51,6 +51,17 @@ constexpr size_t kAlign = 256;
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+// A chain call made by the host-buffer wrapper on one segment of its own (aligned) buffers: g and dg of a segment
+// that starts at an odd token are only 4-byte aligned, exactly as for an inner segment of a chain.
+thread_local bool tl_segment_of_chain = false;
+struct SegmentOfChain {
+    SegmentOfChain() { tl_segment_of_chain = true; }
+    ~SegmentOfChain() { tl_segment_of_chain = false; }
+};
+inline bool chain_ptr_ok(const void* p, const void* g, const void* dg) {
+    if (tl_segment_of_chain && (p == g || p == dg)) return (reinterpret_cast<uintptr_t>(p) & 3u) == 0;
+    return aligned16(p);
+}
 
 enum class Path { Invalid, Unsupported, Simt, Tc };
 
@@ -762,7 +773,7 @@ sf_status_t sf_chain_fwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     if (!workspace || workspace_bytes < sf_chain_workspace_bytes(desc, seg_lens, n_seg, 0)) return SF_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return SF_ERR_INVALID_ARG;
     const void* ptrs[] = {q, k, v, g, S_init, o, S_bounds};
-    for (const void* ptr : ptrs) if (ptr && !aligned16(ptr)) return SF_ERR_INVALID_ARG;
+    for (const void* ptr : ptrs) if (ptr && !chain_ptr_ok(ptr, g, nullptr)) return SF_ERR_INVALID_ARG;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const size_t esz = desc->dtype == SF_BF16 ? 2 : 4;
     const size_t sN = (size_t)desc->B * desc->H * desc->d_k * desc->d_v;
@@ -882,7 +893,7 @@ sf_status_t sf_chain_bwd(const sf_seg_desc_t* desc, const int32_t* seg_lens, int
     if (!workspace || workspace_bytes < need) return SF_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return SF_ERR_INVALID_ARG;
     const void* ptrs[] = {q, k, v, g, S_bounds, dO, dS_final, dq, dk, dv, dg, dS_init, fwd_workspace};
-    for (const void* ptr : ptrs) if (ptr && !aligned16(ptr)) return SF_ERR_INVALID_ARG;
+    for (const void* ptr : ptrs) if (ptr && !chain_ptr_ok(ptr, g, dg)) return SF_ERR_INVALID_ARG;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const size_t esz = desc->dtype == SF_BF16 ? 2 : 4;
     const size_t sN = (size_t)desc->B * desc->H * desc->d_k * desc->d_v;
@@ -1366,6 +1377,7 @@ sf_status_t sf_chain_fwd_bwd_host(const sf_seg_desc_t* desc, const int32_t* seg_
     std::vector<long long> tok0(n_seg + 1, 0);
     for (int i = 0; i < n_seg; ++i) tok0[i + 1] = tok0[i] + seg_lens[i];
 
+    SegmentOfChain sub_calls;
     SF_CUDA(cudaEventRecord(e_start, st));
     SF_CUDA(cudaStreamWaitEvent(up, e_start, 0));
     SF_CUDA(cudaStreamWaitEvent(down, e_start, 0));

@@ -47,6 +47,16 @@ def test_host_wrapper_bf16_tensor_core_path(segs):
     compare(got, oracle_reference(x), tolerance(w), label=w.name)
 
 
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 32)])
+def test_host_wrapper_segments_that_start_at_odd_tokens(dtype, d):
+    # inner segments of 87, 1 and 15 tokens with one head: the later segments' g and dg start at addresses that are
+    # only 4-byte aligned, as inside any chain
+    w = Workload("host-odd-%s" % dtype, 2, 1, d, d, [512, 87, 1, 320, 15], 64, dtype=dtype, g_scale=0.1, s_in_sigma=0.3, ds_out_sigma=0.3, seed=26)
+    x = inputs.make_inputs(w, DEV)
+    got, _ = run_host(w, x)
+    compare(got, oracle_reference(x), tolerance(w), label=w.name)
+
+
 def test_host_wrapper_without_boundary_inputs_and_without_final_state():
     w = Workload("host-noinit", 1, 2, 64, 64, [192, 128], 32, dtype="f32", g_scale=0.1, seed=23)
     x = inputs.make_inputs(w, DEV)
