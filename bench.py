@@ -7,6 +7,7 @@ configuration 4 (256K tokens in 16 segments of 16384, H = 32), the largest singl
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config {2,3,4,5}] [--seg-len L]
   python bench.py --impl reference ...      times the fp64 CPU oracle on a bounded sample instead
+  python bench.py --op {delta_chunked,channel_chunked,delta,channel,conv}   one extension operator instead of the chain
 
 Multi-GPU: the path does not shard (replicas only): with --gpus N each rank runs the same workload on
 its own GPU, no data-path collective; value = N * tokens / max-over-ranks time.
@@ -33,9 +34,9 @@ FLOPS_PER_TOKEN_HEAD = 344064        # full chunk tiles, d = 128, chunk 64: forw
 KERNEL_BYTES = {"agg_kv": 516, "agg_qdo": 516, "fwd_out": 1028, "dq": 1284, "dkdv": 1540}
 # DRAM bytes per token*head of each kernel from the ncu capture of the small case (profiles/, 262144 token*heads per
 # launch), scaled to a bench launch by the token*heads it processes (traffic grows in proportion)
-KERNEL_NCU_TRAFFIC = {"agg_kv": (135.293e6 + 3.755e6) / 262144, "agg_qdo": (135.294e6 + 3.791e6) / 262144,
-                      "fwd_out": (210.929e6 + 43.808e6) / 262144, "dq": (277.988e6 + 49.363e6) / 262144,
-                      "dkdv": (278.094e6 + 106.707e6) / 262144}
+KERNEL_NCU_TRAFFIC = {"agg_kv": (135.293e6 + 4.131e6) / 262144, "agg_qdo": (135.293e6 + 4.964e6) / 262144,
+                      "fwd_out": (210.914e6 + 43.968e6) / 262144, "dq": (278.050e6 + 49.405e6) / 262144,
+                      "dkdv": (278.054e6 + 106.869e6) / 262144}
 
 
 def peaks():
@@ -182,6 +183,157 @@ def run_reference(args):
     }))
 
 
+# ---- extension operators (diagonal decay, gated delta rule, short convolution): their own measured line ------------
+EXT_OPS = ["delta_chunked", "channel_chunked", "delta", "channel", "conv"]
+
+
+def extension_workload(op):
+    """One 16384-token segment, H = 16, d_k = d_v = 64, float32 (268 MB of q, k, v, dO: larger than L2); chunk 32 for
+    the chunkwise operators.  The convolution runs over the same tokens with H*d_v = 1024 channels, width 4."""
+    from paper_2608_06838_b200 import inputs
+    return inputs.Workload("ext-16k-h16-d64", 1, 16, 64, 64, [16384], 32, dtype="f32", qk_norm="l2", g_scale=0.1,
+                           s_in_sigma=0.02, ds_out_sigma=0.02, seed=7)
+
+
+def extension_bytes(op, w):
+    """Algorithmic bytes per token*head, fwd + bwd: every input read once per direction, every output written once."""
+    e = 4
+    if op == "conv":                     # per token*head: d_v channels; x, y, dy, dx float32 (x is read in both directions)
+        return 5 * w.d_v * e
+    qk, vv = w.d_k * e, w.d_v * e
+    gate = (w.d_k * e if op.startswith("channel") else e) + (e if op.startswith("delta") else 0)      # g (+ beta)
+    fwd = 2 * qk + vv + gate + vv
+    bwd = 2 * qk + 2 * vv + gate + 2 * qk + vv + gate
+    return fwd + bwd
+
+
+def extension_step_fn(op, w, x, dev):
+    """Allocates outputs and workspaces once; returns a function that runs one fwd + bwd of the operator."""
+    import torch
+    from paper_2608_06838_b200 import binding
+    q, k, v, dO = x["q"], x["k"], x["v"], x["dO"]
+    if op == "conv":
+        cx, cw, cdy = x["conv_x"], x["conv_w"], x["conv_dy"]
+        y, dx, dw = torch.empty_like(cx), torch.empty_like(cx), torch.empty_like(cw)
+        tail_out, dtail_in = torch.empty_like(x["conv_tail"]), torch.empty_like(x["conv_tail"])
+
+        def step():
+            binding.sf_conv_segment_fwd(cx, cw, x["conv_tail"], y, tail_out)
+            binding.sf_conv_segment_bwd(cx, cw, x["conv_tail"], cdy, x["conv_dtail"], dx, dw, dtail_in)
+        return step, 2
+    g = x["g_channel"] if op.startswith("channel") else x["g"]
+    beta = x["beta"]
+    d = binding.make_desc(q, v, x["g"], w.chunk)
+    o, dq, dk, dv, dg, dbeta = (torch.empty_like(t) for t in (v, q, k, v, g, beta))
+    S_out = torch.empty(w.B, w.H, w.d_k, w.d_v, device=dev)
+    dS_in = torch.empty_like(S_out)
+    nbytes = {"delta_chunked": lambda b: binding.sf_delta_chunked_workspace_bytes(d, b),
+              "channel_chunked": lambda b: binding.sf_channel_chunked_workspace_bytes(d, b)}.get(
+                  op, lambda b: binding.sf_recurrent_workspace_bytes(d) if b else 16)
+    ws_f = torch.empty(max(nbytes(0), 16), dtype=torch.uint8, device=dev)
+    ws_b = torch.empty(max(nbytes(1), 16), dtype=torch.uint8, device=dev)
+    S_in, dS_out = x["S_in"], x["dS_out"]
+    if op == "delta_chunked":
+        def step():
+            binding.sf_delta_chunked_fwd(d, q, k, v, g, beta, S_in, o, S_out, ws_f)
+            binding.sf_delta_chunked_bwd(d, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, ws_b)
+    elif op == "channel_chunked":
+        def step():
+            binding.sf_channel_chunked_fwd(d, q, k, v, g, S_in, o, S_out, ws_f)
+            binding.sf_channel_chunked_bwd(d, q, k, v, g, S_in, dO, dS_out, dq, dk, dv, dg, dS_in, ws_b)
+    elif op == "delta":
+        def step():
+            binding.sf_delta_segment_fwd(d, q, k, v, g, beta, S_in, o, S_out)
+            binding.sf_delta_segment_bwd(d, q, k, v, g, beta, S_in, dO, dS_out, dq, dk, dv, dg, dbeta, dS_in, ws_b)
+    else:
+        def step():
+            binding.sf_channel_segment_fwd(d, q, k, v, g, S_in, o, S_out)
+            binding.sf_channel_segment_bwd(d, q, k, v, g, S_in, dO, dS_out, dq, dk, dv, dg, dS_in, ws_b)
+    return step, None
+
+
+def extension_cpu_baseline(op, w, tokens=8192):
+    """The numpy fp64 oracle of the operator on the first `tokens` tokens (all heads)."""
+    import dataclasses
+    from oracle import variants as V
+    from paper_2608_06838_b200 import inputs
+    ws = dataclasses.replace(w, seg_lens=[tokens])
+    x = inputs.make_variant_inputs(ws, "cpu")
+    f = inputs.to_f64
+    t0 = time.perf_counter()
+    if op == "conv":
+        V.conv_fwd(f(x["conv_x"]), f(x["conv_w"]), f(x["conv_tail"]))
+        V.conv_bwd(f(x["conv_x"]), f(x["conv_w"]), f(x["conv_tail"]), f(x["conv_dy"]), f(x["conv_dtail"]))
+    elif op.startswith("channel"):
+        a = [f(x[n]) for n in ("q", "k", "v", "g_channel", "S_in")]
+        V.channel_fwd(*a)
+        V.channel_bwd(*a, f(x["dO"]), f(x["dS_out"]))
+    else:
+        a = [f(x[n]) for n in ("q", "k", "v", "g", "beta", "S_in")]
+        V.delta_fwd(*a)
+        V.delta_bwd(*a, f(x["dO"]), f(x["dS_out"]))
+    dt = time.perf_counter() - t0
+    return {"value": ws.B * tokens / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "first %d tokens, all %d heads, fwd+bwd, %.1f s (numpy, one thread drives it)" % (tokens, w.H, dt)}
+
+
+def run_extension(args):
+    """fwd + bwd of one extension operator on its stated workload: device time, HBM roofline fraction, oracle timing."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import torch
+    from paper_2608_06838_b200 import binding, inputs
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    binding.load()
+    op = args.op
+    w = extension_workload(op)
+    x = inputs.make_variant_inputs(w, dev)
+    step, fixed_launches = extension_step_fn(op, w, x, dev)
+    torch.cuda.synchronize()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    regions = []
+    n0 = binding.sf_launch_count()
+    for _ in range(args.repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        regions.append(e0.elapsed_time(e1) / args.steps)
+    launches = binding.sf_launch_count() - n0
+    t_end = time.time() + 0.7
+    while time.time() < t_end:              # keep the same load up until the clock sampler has a few samples
+        step()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    assert binding.sf_device_status() == 0
+    ms = statistics.median(regions)
+    tokens = w.B * w.T
+    hbm, _, src = peaks()
+    bth = extension_bytes(op, w)
+    achieved = bth * tokens * w.H / (ms * 1e-3) / 1e9
+    out = {"metric": "fwd+bwd tokens/s, extension operator %s" % op, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "timed_regions": {"repeats": args.repeats, "ms_per_step_min": min(regions), "ms_per_step_max": max(regions)},
+           "config": {"workload": w.name, "operator": op, "B": w.B, "H": w.H, "d_k": w.d_k, "d_v": w.d_v, "T": w.T,
+                      "chunk": w.chunk if op.endswith("chunked") else None, "conv_width": 4 if op == "conv" else None,
+                      "l2": "inputs (268 MB) exceed L2, no flush", "parallelism": "replicas only"},
+           "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+           "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "peak_source": src, "frac": achieved / hbm,
+                        "traffic": None, "note": "whole operator, fwd + bwd: %d algorithmic bytes per token*head / step time; "
+                                                 "float32 CUDA-core kernels, not bound by HBM" % bth}}
+    if not args.skip_cpu:
+        out["cpu_baseline"] = extension_cpu_baseline(op, w)
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -204,6 +356,9 @@ def main():
                          "(sf_chain_autotune; only used when --chunks-per-block is 0)")
     ap.add_argument("--merge-launches", action="store_true",
                     help="install the merged-launch schedule (every stage once over the whole chain) instead of searching")
+    ap.add_argument("--op", default="chain", choices=["chain"] + EXT_OPS,
+                    help="chain (default): the segment chain of the main path; else fwd+bwd of one extension operator on a "
+                         "16384-token, H = 16, d = 64 float32 segment")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     args = ap.parse_args()
@@ -212,6 +367,9 @@ def main():
         args.skip_e2e = args.skip_cpu = True
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.op != "chain":
+        run_extension(args)
         return
 
     import torch

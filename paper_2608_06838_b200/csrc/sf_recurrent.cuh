@@ -298,59 +298,154 @@ __device__ __forceinline__ float conv_ext(const float* x, const float* tail_in, 
     return x[((long long)b * L + (e - (W - 1))) * C + c];
 }
 
-__global__ void conv_fwd_kernel(int B, int L, int C, int W, const float* __restrict__ x, const float* __restrict__ w,
-                                const float* __restrict__ tail_in, float* __restrict__ y, float* __restrict__ tail_out) {
-    const long long n = (long long)B * (L + W - 1) * C;
-    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)(idx % C);
-        const long long bt = idx / C;
-        const int e = (int)(bt % (L + W - 1)), b = (int)(bt / (L + W - 1));
-        if (e < L) {                                     // output token t = e
-            float acc = 0.f;
-            for (int jj = 0; jj < W; ++jj) acc = fmaf(w[jj * C + c], conv_ext(x, tail_in, b, W - 1 + e - jj, c, L, C, W), acc);
-            y[((long long)b * L + e) * C + c] = acc;
-        } else {                                         // tail_out row e - L = ext row L + (e - L)
-            const int r = e - L;
-            tail_out[((long long)b * (W - 1) + r) * C + c] = conv_ext(x, tail_in, b, L + r, c, L, C, W);
+// Both elementwise kernels walk the token axis: a thread owns V consecutive channels (V = 4: 16-byte accesses) and
+// CONV_TS consecutive rows, keeps the last W rows in registers, so every input row is read once (plus W-1 rows of
+// overlap per 16).  block (32 channel groups, 8 row slices); grid (channel groups / 32, row slices / 8, B).
+constexpr int CONV_TS = 16;
+template <int V> struct ConvVec;
+template <> struct ConvVec<1> {
+    float v[1];
+    __device__ __forceinline__ void load(const float* p) { v[0] = *p; }
+    __device__ __forceinline__ void store(float* p) const { *p = v[0]; }
+};
+template <> struct ConvVec<4> {
+    float v[4];
+    __device__ __forceinline__ void load(const float* p) { const float4 t = *reinterpret_cast<const float4*>(p); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+    __device__ __forceinline__ void store(float* p) const { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
+};
+
+// y_t = sum_j w[j] ext[W-1+t-j]; the window holds ext rows t .. t+W-1 (the newest one is x_t).  The width is a
+// template parameter: weights and window then live in exactly W registers per channel.
+template <int V, int W>
+__global__ void __launch_bounds__(256)
+conv_fwd_kernel(int B, int L, int C, const float* __restrict__ x, const float* __restrict__ w,
+                const float* __restrict__ tail_in, float* __restrict__ y, float* __restrict__ tail_out) {
+    const int c = (blockIdx.x * 32 + threadIdx.x) * V, b = blockIdx.z;
+    if (c >= C) return;
+    // wr[i] multiplies ext[t + i] (window element i): tap W-1-i; the newest row x_t is element W-1
+    ConvVec<V> wr[W], win[W];
+#pragma unroll
+    for (int i = 0; i < W; ++i) wr[i].load(w + (long long)(W - 1 - i) * C + c);
+    const int t0 = (blockIdx.y * 8 + threadIdx.y) * CONV_TS, t1 = min(L, t0 + CONV_TS);
+    auto ext_row = [&](ConvVec<V>& dst, int e) {           // row e of ext = [tail_in ; x]
+        if (e >= W - 1) dst.load(x + ((long long)b * L + (e - (W - 1))) * C + c);
+        else if (tail_in) dst.load(tail_in + ((long long)b * (W - 1) + e) * C + c);
+        else {
+#pragma unroll
+            for (int i = 0; i < V; ++i) dst.v[i] = 0.f;
         }
+    };
+    if (t0 < t1) {
+#pragma unroll
+        for (int i = 0; i < W - 1; ++i) ext_row(win[i], t0 + i);
+#pragma unroll 4
+        for (int t = t0; t < t1; ++t) {
+            ConvVec<V> acc;
+            win[W - 1].load(x + ((long long)b * L + t) * C + c);
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc.v[i] = 0.f;
+#pragma unroll
+            for (int k = 0; k < W; ++k)
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc.v[i] = fmaf(wr[k].v[i], win[k].v[i], acc.v[i]);
+            acc.store(y + ((long long)b * L + t) * C + c);
+#pragma unroll
+            for (int k = 0; k < W - 1; ++k) win[k] = win[k + 1];
+        }
+    }
+    if (blockIdx.y == 0 && tail_out)                     // the last W-1 rows of ext go to the next segment
+        for (int r = threadIdx.y; r < W - 1; r += 8) {
+            ConvVec<V> row;
+            ext_row(row, L + r);
+            row.store(tail_out + ((long long)b * (W - 1) + r) * C + c);
+        }
+}
+
+// dext[e] = sum_j w[j] dy[e-(W-1)+j] (+ dtail_out[e-L] for e >= L); dx = dext[W-1:], dtail_in = dext[:W-1].
+// The window holds dy rows e-(W-1) .. e (zero outside [0, L)); rows e run over [0, L+W-1).
+template <int V, int W>
+__global__ void __launch_bounds__(256)
+conv_bwd_input_kernel(int B, int L, int C, const float* __restrict__ w, const float* __restrict__ dy,
+                      const float* __restrict__ dtail_out, float* __restrict__ dx, float* __restrict__ dtail_in) {
+    const int c = (blockIdx.x * 32 + threadIdx.x) * V, b = blockIdx.z;
+    if (c >= C) return;
+    ConvVec<V> wt[W], win[W];
+#pragma unroll
+    for (int j = 0; j < W; ++j) wt[j].load(w + (long long)j * C + c);
+    const int E = L + W - 1;
+    const int e0 = (blockIdx.y * 8 + threadIdx.y) * CONV_TS, e1 = min(E, e0 + CONV_TS);
+    auto dy_row = [&](ConvVec<V>& dst, int t) {
+        if (t >= 0 && t < L) dst.load(dy + ((long long)b * L + t) * C + c);
+        else {
+#pragma unroll
+            for (int i = 0; i < V; ++i) dst.v[i] = 0.f;
+        }
+    };
+    if (e0 >= e1) return;
+#pragma unroll
+    for (int j = 0; j < W - 1; ++j) dy_row(win[j], e0 - (W - 1) + j);
+#pragma unroll 4
+    for (int e = e0; e < e1; ++e) {
+        ConvVec<V> acc;
+        dy_row(win[W - 1], e);
+        if (e >= L && dtail_out) acc.load(dtail_out + ((long long)b * (W - 1) + (e - L)) * C + c);
+        else {
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc.v[i] = 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < W; ++j)
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc.v[i] = fmaf(wt[j].v[i], win[j].v[i], acc.v[i]);
+        if (e < W - 1) acc.store(dtail_in + ((long long)b * (W - 1) + e) * C + c);
+        else acc.store(dx + ((long long)b * L + (e - (W - 1))) * C + c);
+#pragma unroll
+        for (int k = 0; k < W - 1; ++k) win[k] = win[k + 1];
     }
 }
 
-// dext[e] = sum_j w[j] dy[e-(W-1)+j] (+ dtail_out[e-L] for e >= L); dx = dext[W-1:], dtail_in = dext[:W-1]
-__global__ void conv_bwd_input_kernel(int B, int L, int C, int W, const float* __restrict__ w, const float* __restrict__ dy,
-                                      const float* __restrict__ dtail_out, float* __restrict__ dx, float* __restrict__ dtail_in) {
-    const long long n = (long long)B * (L + W - 1) * C;
-    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)(idx % C);
-        const long long bt = idx / C;
-        const int e = (int)(bt % (L + W - 1)), b = (int)(bt / (L + W - 1));
-        float acc = (e >= L && dtail_out) ? dtail_out[((long long)b * (W - 1) + (e - L)) * C + c] : 0.f;
-        for (int jj = 0; jj < W; ++jj) {
-            const int t = e - (W - 1) + jj;
-            if (t >= 0 && t < L) acc = fmaf(w[jj * C + c], dy[((long long)b * L + t) * C + c], acc);
+// dw[j][c] = sum_b sum_t dy[b,t,c] ext[b, W-1+t-j, c].  grid ceil(C/8), block (8 channels, 128 token lanes): a thread
+// walks one contiguous 1/128 of the tokens once, keeps the last W inputs of its channel in registers and adds into one
+// double-precision sum per tap (x and dy are read once); the 128 partial sums of a tap are added in a fixed order.
+constexpr int CONV_WC = 8, CONV_WT = 128;
+template <int W>
+__global__ void __launch_bounds__(CONV_WC * CONV_WT, 1)
+conv_bwd_weight_kernel(int B, int L, int C, const float* __restrict__ x, const float* __restrict__ tail_in,
+                       const float* __restrict__ dy, float* __restrict__ dw) {
+    __shared__ double part[CONV_WT][CONV_WC + 1];
+    const int cx = threadIdx.x, ty = threadIdx.y, c = blockIdx.x * CONV_WC + cx;
+    const int len = (L + CONV_WT - 1) / CONV_WT, t0 = min(L, ty * len), t1 = min(L, t0 + len);
+    double acc[W];
+#pragma unroll
+    for (int j = 0; j < W; ++j) acc[j] = 0.0;
+    if (c < C && t0 < t1) {
+        for (int b = 0; b < B; ++b) {
+            float win[W];                                // win[j] = ext[b, W-1+t-j, c]
+#pragma unroll
+            for (int j = 1; j < W; ++j) win[j] = conv_ext(x, tail_in, b, W - 1 + t0 - j, c, L, C, W);
+            const float* xr = x + ((long long)b * L) * C + c;
+            const float* dr = dy + ((long long)b * L) * C + c;
+#pragma unroll 4
+            for (int t = t0; t < t1; ++t) {
+                win[0] = xr[(long long)t * C];
+                const double d = (double)dr[(long long)t * C];
+#pragma unroll
+                for (int j = 0; j < W; ++j) acc[j] = fma(d, (double)win[j], acc[j]);
+#pragma unroll
+                for (int j = W - 1; j >= 1; --j) win[j] = win[j - 1];
+            }
         }
-        if (e < W - 1) dtail_in[((long long)b * (W - 1) + e) * C + c] = acc;
-        else dx[((long long)b * L + (e - (W - 1))) * C + c] = acc;
     }
-}
-
-// dw[j][c] = sum_b sum_t dy[b,t,c] ext[b, W-1+t-j, c].  grid (ceil(C/32), W), block (32, 8): each thread sums a fixed
-// subset of the tokens in double precision, the 8 partial sums are added in a fixed order.
-__global__ void conv_bwd_weight_kernel(int B, int L, int C, int W, const float* __restrict__ x, const float* __restrict__ tail_in,
-                                       const float* __restrict__ dy, float* __restrict__ dw) {
-    __shared__ double part[8][32];
-    const int c = blockIdx.x * 32 + threadIdx.x, jj = blockIdx.y;
-    double acc = 0.0;
-    if (c < C)
-        for (int b = 0; b < B; ++b)
-            for (int t = threadIdx.y; t < L; t += 8)
-                acc += (double)dy[((long long)b * L + t) * C + c] * (double)conv_ext(x, tail_in, b, W - 1 + t - jj, c, L, C, W);
-    part[threadIdx.y][threadIdx.x] = acc;
-    __syncthreads();
-    if (threadIdx.y == 0 && c < C) {
-        double sum = 0.0;
-        for (int r = 0; r < 8; ++r) sum += part[r][threadIdx.x];
-        dw[jj * C + c] = (float)sum;
+#pragma unroll
+    for (int j = 0; j < W; ++j) {
+        part[ty][cx] = acc[j];
+        __syncthreads();
+        if (ty == 0 && c < C) {
+            double sum = 0.0;
+            for (int r = 0; r < CONV_WT; ++r) sum += part[r][cx];
+            dw[j * C + c] = (float)sum;
+        }
+        __syncthreads();
     }
 }
 

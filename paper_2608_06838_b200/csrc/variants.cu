@@ -1,5 +1,6 @@
 // C ABI of the extension operators: diagonal decay, gated delta rule, short convolution with a carried tail.
 // Argument checks happen before any launch; nothing here allocates, synchronises or falls back to the host.
+#include <type_traits>
 #include "../../include/stateflow.h"
 #include "sf_recurrent.cuh"
 #include "sf_delta_chunk.cuh"
@@ -113,13 +114,34 @@ sf_status_t rec_bwd(const sf_seg_desc_t* d, const void* q, const void* k, const 
 
 sf_status_t check_conv(int32_t B, int32_t L, int32_t C, int32_t W) {
     if (B <= 0 || L <= 0 || C <= 0 || W < 1) return SF_ERR_INVALID_ARG;
-    if (W > sf::rec::CONV_MAXW) return SF_ERR_UNSUPPORTED;
+    if (W > sf::rec::CONV_MAXW || B > 65535) return SF_ERR_UNSUPPORTED;       // B is a grid dimension
     return SF_OK;
 }
 
-int conv_grid(long long n) {
-    const long long g = (n + 255) / 256;
-    return (int)(g < 1 ? 1 : (g > 148LL * 16 ? 148LL * 16 : g));
+// Launch shape of the row-walking convolution kernels over `rows` rows: V channels per thread (4 when the channel
+// count and every pointer allow 16-byte accesses).
+bool conv_vec4(int C, std::initializer_list<const void*> ptrs) {
+    if (C % 4) return false;
+    for (const void* p : ptrs) if (p && (reinterpret_cast<uintptr_t>(p) & 15u)) return false;
+    return true;
+}
+// Calls f with the convolution width as a compile-time constant (1 .. CONV_MAXW, checked before).
+template <class F>
+void conv_width_switch(int W, F&& f) {
+    switch (W) {
+        case 1: f(std::integral_constant<int, 1>{}); break;
+        case 2: f(std::integral_constant<int, 2>{}); break;
+        case 3: f(std::integral_constant<int, 3>{}); break;
+        case 4: f(std::integral_constant<int, 4>{}); break;
+        case 5: f(std::integral_constant<int, 5>{}); break;
+        case 6: f(std::integral_constant<int, 6>{}); break;
+        case 7: f(std::integral_constant<int, 7>{}); break;
+        default: f(std::integral_constant<int, 8>{}); break;
+    }
+}
+dim3 conv_grid(int B, long long rows, int C, int V) {
+    const int groups = (C + V - 1) / V;
+    return dim3((unsigned)((groups + 31) / 32), (unsigned)((rows + 8LL * sf::rec::CONV_TS - 1) / (8LL * sf::rec::CONV_TS)), (unsigned)B);
 }
 
 // ---- chunkwise delta rule ----------------------------------------------------------------------------------------
@@ -357,8 +379,14 @@ sf_status_t sf_conv_segment_fwd(int32_t B, int32_t L, int32_t C, int32_t W, cons
     const sf_status_t c = check_conv(B, L, C, W);
     if (c != SF_OK) return c;
     if (!x || !w || !y || (W > 1 && !tail_out) || (tail_in && tail_in == tail_out)) return SF_ERR_INVALID_ARG;
-    const long long n = (long long)B * (L + W - 1) * C;
-    sf::rec::conv_fwd_kernel<<<conv_grid(n), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(B, L, C, W, x, w, tail_in, y, tail_out);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const bool v4 = conv_vec4(C, {x, w, tail_in, y, tail_out});
+    const dim3 grid = conv_grid(B, L, C, v4 ? 4 : 1), block(32, 8);
+    conv_width_switch(W, [&](auto wc) {
+        constexpr int Wc = decltype(wc)::value;
+        if (v4) sf::rec::conv_fwd_kernel<4, Wc><<<grid, block, 0, st>>>(B, L, C, x, w, tail_in, y, tail_out);
+        else    sf::rec::conv_fwd_kernel<1, Wc><<<grid, block, 0, st>>>(B, L, C, x, w, tail_in, y, tail_out);
+    });
     return launched();
 }
 
@@ -369,10 +397,19 @@ sf_status_t sf_conv_segment_bwd(int32_t B, int32_t L, int32_t C, int32_t W, cons
     if (c != SF_OK) return c;
     if (!x || !w || !dy || !dx || !dw || (W > 1 && !dtail_in) || (dtail_out && dtail_out == dtail_in)) return SF_ERR_INVALID_ARG;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const long long n = (long long)B * (L + W - 1) * C;
-    sf::rec::conv_bwd_input_kernel<<<conv_grid(n), 256, 0, st>>>(B, L, C, W, w, dy, dtail_out, dx, dtail_in);
+    const long long rows = (long long)L + W - 1;
+    const bool v4 = conv_vec4(C, {w, dy, dtail_out, dx, dtail_in});
+    const dim3 grid = conv_grid(B, rows, C, v4 ? 4 : 1), block(32, 8);
+    conv_width_switch(W, [&](auto wc) {
+        constexpr int Wc = decltype(wc)::value;
+        if (v4) sf::rec::conv_bwd_input_kernel<4, Wc><<<grid, block, 0, st>>>(B, L, C, w, dy, dtail_out, dx, dtail_in);
+        else    sf::rec::conv_bwd_input_kernel<1, Wc><<<grid, block, 0, st>>>(B, L, C, w, dy, dtail_out, dx, dtail_in);
+    });
     if (cudaGetLastError() != cudaSuccess) return SF_ERR_CUDA;
-    sf::rec::conv_bwd_weight_kernel<<<dim3((C + 31) / 32, W), dim3(32, 8), 0, st>>>(B, L, C, W, x, tail_in, dy, dw);
+    conv_width_switch(W, [&](auto wc) {
+        sf::rec::conv_bwd_weight_kernel<decltype(wc)::value><<<dim3((C + sf::rec::CONV_WC - 1) / sf::rec::CONV_WC),
+                                                                 dim3(sf::rec::CONV_WC, sf::rec::CONV_WT), 0, st>>>(B, L, C, x, tail_in, dy, dw);
+    });
     return launched(2);
 }
 

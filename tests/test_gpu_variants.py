@@ -156,9 +156,11 @@ def test_delta_rule_with_beta_zero_only_decays():
     assert norm_err(f64(got["S_out"]), c[:, -1][..., None, None] * f64(x["S_in"])) <= TOL
 
 
-@pytest.mark.parametrize("W,seg_lens", [(4, [37, 2, 1, 88]), (2, [5, 123]), (1, [64, 64]), (8, [3, 300, 7])])
-def test_conv_chain_matches_the_oracle(W, seg_lens):
-    w = Workload("conv-%d" % W, 2, 3, 32, 32, seg_lens, 64, dtype="f32", seed=25)
+# channel counts: 96 and 260 (16-byte accesses, the second with a partly filled last group of threads), 7 (scalar path)
+@pytest.mark.parametrize("H,dv", [(3, 32), (5, 52), (1, 7)])
+@pytest.mark.parametrize("W,seg_lens", [(4, [37, 2, 1, 88]), (2, [5, 123]), (1, [64, 64]), (8, [3, 300, 7]), (4, [700, 257, 32])])
+def test_conv_chain_matches_the_oracle(W, seg_lens, H, dv):
+    w = Workload("conv-%d" % W, 2, H, 32, dv, seg_lens, 64, dtype="f32", seed=25)
     x = inputs.make_variant_inputs(w, DEV, conv_width=W)
     X, Wt, dY = x["conv_x"], x["conv_w"], x["conv_dy"]
     B, T, C = X.shape
