@@ -497,7 +497,10 @@ sf_status_t sf_delta_chunked_bwd(const sf_seg_desc_t* desc, const void* q, const
  *   ext = [tail_in ; x] ,  y_t = sum_j w[j] * ext[W-1+t-j] ,  tail_out = the last W-1 rows of ext
  * tail_in NULL means zeros (start of the sequence); tail_out is the boundary state handed to the next segment and
  * is required when W > 1 (L may be shorter than W-1: old tail rows then move up).  Backward: dtail_out nullable;
- * dw is overwritten with this segment's contribution (the caller adds the segments' dw), summed in a fixed order.
+ * dw is overwritten with this segment's contribution (the caller adds the segments' dw), summed in a fixed order in
+ * double precision.  Channels are processed four at a time with 16-byte accesses when C is a multiple of 4 and every
+ * pointer is 16-byte aligned, one at a time otherwise (same results).  Errors: non-positive B, L, C or W < 1 or a missing
+ * required pointer SF_ERR_INVALID_ARG; W > 8 or B > 65535 SF_ERR_UNSUPPORTED; nothing is launched then.
  */
 sf_status_t sf_conv_segment_fwd(int32_t B, int32_t L, int32_t C, int32_t W, const float* x, const float* w, const float* tail_in,
                                 float* y, float* tail_out, sf_stream_t stream);

@@ -226,6 +226,7 @@ def test_extension_operators_validate_before_any_launch(lib):
     assert lib.sf_delta_segment_bwd(ctypes.byref(d), *dargs, ctypes.c_void_p(0x40000), 1 << 40, None) == 1
     conv = lambda B=1, L=8, C=4, W=4, x=P, tail_out=S1: lib.sf_conv_segment_fwd(B, L, C, W, x, P, None, P, tail_out, None)
     assert conv(L=0) == 1 and conv(W=0) == 1 and conv(W=9) == 2 and conv(x=None) == 1 and conv(tail_out=None) == 1
+    assert conv(B=65536) == 2                                                              # B is a grid dimension
     assert lib.sf_conv_segment_bwd(1, 8, 4, 4, P, P, None, P, S1, P, P, S1, None) == 1       # dtail_out aliases dtail_in
     assert lib.sf_conv_segment_bwd(1, 8, 4, 4, P, P, None, None, None, P, P, S1, None) == 1  # dy missing
 
